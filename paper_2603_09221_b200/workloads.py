@@ -1,0 +1,99 @@
+"""Seeded synthetic inputs shaped like TTC-layer LQR workloads.
+
+This module only draws random numbers and assembles input tensors; it contains none
+of the solver's arithmetic and is the one module that both the CUDA path's callers
+(tests, bench) and the CPU oracle's callers may use.
+
+Batch layout is ``[seq][head][token]``; instance index ``i = (s*heads + h)*tokens + k``.
+Operands shared by a head have size-1 ``seq`` and ``token`` dimensions.
+
+Recipe (one seed per configuration, ``260309221 + c``):
+  A = G * rho / rho(G), G_ij ~ N(0,1), rho(G) = max |eigenvalue|   (float64 on the host)
+  B_ij ~ N(0, 1/n)            R = M M'/m + 0.1 I  (M m x m Gaussian)
+  Q = L L'/n + 0.1 I  (L n x n Gaussian)        x0 ~ N(0, I)
+  configuration 4: Q = U U'/8 + diag(d), U n x 8 Gaussian, d_i ~ U[0.05, 0.2]
+A, B, R are float32.  Q and x0 are float32, or rounded to bfloat16 (round to nearest
+even, element-wise, which keeps Q symmetric) where the configuration says so.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+SEED0 = 260309221
+
+CONFIGS = {
+    0: dict(name="cfg0_tiny_n8_H8", batch=(1, 1, 64), n=8, m=8, H=8, rho=0.9,
+            per_instance_system=True, q_dtype="f32", q_kind="full", first_only=False, tol=1e-4),
+    1: dict(name="cfg1_small_n16_H16", batch=(4, 8, 128), n=16, m=16, H=16, rho=0.9,
+            per_instance_system=False, q_dtype="f32", q_kind="full", first_only=False, tol=1e-4),
+    2: dict(name="cfg2_medium_n64_H8_bf16", batch=(4, 8, 2048), n=64, m=64, H=8, rho=0.9,
+            per_instance_system=False, q_dtype="bf16", q_kind="full", first_only=False, tol=2e-2),
+    3: dict(name="cfg3_long_n32_H64", batch=(1, 16, 1024), n=32, m=32, H=64, rho=0.98,
+            per_instance_system=False, q_dtype="f32", q_kind="full", first_only=False, tol=1e-4),
+    4: dict(name="cfg4_large_n64_H16_bf16_first", batch=(2, 16, 4096), n=64, m=64, H=16, rho=0.9,
+            per_instance_system=False, q_dtype="bf16", q_kind="lowrank8", first_only=True, tol=2e-2),
+}
+
+
+def _system(rng, n, m, rho):
+    G = rng.standard_normal((n, n))
+    A = G * (rho / np.max(np.abs(np.linalg.eigvals(G))))
+    B = rng.standard_normal((n, m)) / np.sqrt(n)
+    M = rng.standard_normal((m, m))
+    R = M @ M.T / m + 0.1 * np.eye(m)
+    return A, B, 0.5 * (R + R.T)
+
+
+def make_workload(cfg_id, device="cpu", batch=None, seed=None, chunk=8192):
+    """Build the inputs of configuration ``cfg_id`` (optionally with a smaller/larger
+    ``batch = (seqs, heads, tokens)``).
+
+    Returns a dict: ``A [*,n,n]``, ``B [*,n,m]``, ``R [*,m,m]`` (float32), ``Q [S,Hd,T,n,n]`` and
+    ``x0 [S,Hd,T,n]`` (float32 or bfloat16) as torch tensors on ``device``, plus the
+    configuration fields (``n, m, H, batch, first_only, tol, name``).
+    """
+    c = dict(CONFIGS[cfg_id])
+    if batch is not None:
+        c["batch"] = tuple(int(b) for b in batch)
+    S, Hd, T = c["batch"]
+    n, m = c["n"], c["m"]
+    seed = SEED0 + cfg_id if seed is None else seed
+    rng = np.random.default_rng(seed)
+
+    if c["per_instance_system"]:
+        sys_shape = (S, Hd, T)
+    else:
+        sys_shape = (1, Hd, 1)
+    nsys = int(np.prod(sys_shape))
+    As, Bs, Rs = zip(*[_system(rng, n, m, c["rho"]) for _ in range(nsys)])
+    to32 = lambda lst, shp: torch.from_numpy(
+        np.stack(lst).astype(np.float32).reshape(sys_shape + shp)).to(device)
+    A, B, R = to32(As, (n, n)), to32(Bs, (n, m)), to32(Rs, (m, m))
+
+    gen = torch.Generator(device=device)
+    gen.manual_seed(seed)
+    N = S * Hd * T
+    qdt = torch.bfloat16 if c["q_dtype"] == "bf16" else torch.float32
+    Q = torch.empty((N, n, n), dtype=qdt, device=device)
+    eye = torch.eye(n, device=device)
+    for s0 in range(0, N, chunk):
+        cnt = min(chunk, N - s0)
+        if c["q_kind"] == "full":
+            L = torch.randn((cnt, n, n), generator=gen, device=device)
+            q = L @ L.transpose(1, 2) / n + 0.1 * eye
+        else:
+            U = torch.randn((cnt, n, 8), generator=gen, device=device)
+            d = 0.05 + 0.15 * torch.rand((cnt, n), generator=gen, device=device)
+            q = U @ U.transpose(1, 2) / 8 + torch.diag_embed(d)
+        q = 0.5 * (q + q.transpose(1, 2))
+        Q[s0:s0 + cnt] = q.to(qdt)
+    x0 = torch.randn((N, n), generator=gen, device=device).to(qdt)
+    c.update(A=A, B=B, R=R, Q=Q.reshape(S, Hd, T, n, n), x0=x0.reshape(S, Hd, T, n),
+             seed=seed, cfg_id=cfg_id)
+    return c
+
+
+def to_float64_numpy(w):
+    """Widen a workload's tensors exactly to float64 numpy arrays (what the oracle reads)."""
+    return {k: w[k].detach().to("cpu").to(torch.float64).numpy() for k in ("A", "B", "Q", "R", "x0")}
