@@ -1,0 +1,337 @@
+#!/usr/bin/env python
+"""Benchmark of the batched LQR solve (one "step" = one ttc_lqr_solve over the whole workload).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg4] [--method auto|riccati|scan]
+    python bench.py --impl reference ...      # the float64 CPU oracle on the host cores
+
+Prints ONE JSON line.  `value` is instances/s with the inputs resident in HBM, timed with CUDA
+events on the launching stream (max over ranks).  `e2e` is the same metric through
+ttc_lqr_solve_host with pinned host buffers, copies inside the timed region.  `roofline`
+describes the dominant kernel; `cpu_baseline` is the oracle, as it stands, on a bounded sample.
+With N > 1 (torchrun) every rank solves its own copy of the workload (instances are independent:
+weak scaling, no collective on the data path).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2603_09221_b200 import workloads  # noqa: E402
+
+SM_COUNT = 148
+FP32_LANES_PER_SM = 128
+TF32_TO_BF16_RATIO = 0.5     # nominal dense tensor ratio tf32 : bf16 on B200 (1.1 : 2.25 PFLOP/s)
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return dict(hbm_gbs=d["hbm_gbs"], bf16_tflops=d["bf16_tflops"],
+                    bf16_tflops_sustained=d["bf16_tflops_sustained"], sm_max_mhz=d.get("sm_max_mhz", 1965.0),
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, sm_max_mhz=1965.0,
+                source="fallback")
+
+
+def algorithmic_counts(c):
+    """Per-instance algorithmic flops (symmetry-exploiting Riccati count) and HBM bytes
+    (inputs once + requested fp32 outputs once)."""
+    n, m, H = c["n"], c["m"], c["H"]
+    flops = (3 * n**3 + 5 * n * n * m + 3 * n * m * m + m**3 / 3.0 + 2 * n * n + 4 * n * m) * H
+    esz = 2 if c["q_dtype"] == "bf16" else 4
+    bytes_in = (n * n + n) * esz
+    if c["first_only"]:
+        bytes_out = 4 * (n * n + m)
+    else:
+        bytes_out = 4 * (H * m * n + (H + 1) * n * n + (H + 1) * n + H * m)
+    return flops, bytes_in, bytes_out
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks / throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.rows = []
+        self._stop = threading.Event()
+        self._t = None
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                out = subprocess.run(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                      "--format=csv,noheader,nounits"], capture_output=True, text=True, timeout=5).stdout
+                parts = [p.strip() for p in out.strip().split(",")]
+                if len(parts) >= 8:
+                    self.rows.append(parts)
+            except Exception:
+                pass
+            self._stop.wait(0.1)
+
+    def start(self):
+        self._t = threading.Thread(target=self._run, daemon=True)
+        self._t.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._t:
+            self._t.join(timeout=6)
+        sm = [float(r[0]) for r in self.rows if r[0].replace(".", "").isdigit()]
+        mx = [float(r[1]) for r in self.rows if r[1].replace(".", "").isdigit()]
+        reasons = set()
+        for r in self.rows:
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(self.rows)}
+
+
+def oracle_sample(w, count):
+    """Stratified sample of instance indices covering every (seq, head)."""
+    S, Hd, T = w["batch"]
+    per = max(1, count // (S * Hd))
+    toks = np.unique(np.linspace(0, T - 1, per).astype(np.int64))
+    idx = (np.arange(S * Hd)[:, None] * T + toks[None, :]).reshape(-1)
+    return idx
+
+
+def time_oracle(w, idx, first_only):
+    from tests import parity_util as pu
+    t0 = time.perf_counter()
+    ref = pu.run_oracle(w, idx=idx, first_only=first_only)
+    dt = time.perf_counter() - t0
+    return ref, dt
+
+
+def run_reference(args, cid):
+    """--impl reference: the float64 oracle on the host cores, bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    c = workloads.CONFIGS[cid]
+    S, Hd, T = c["batch"]
+    tok = max(1, min(T, args.ref_instances // (S * Hd)))
+    w = workloads.make_workload(cid, device="cpu", batch=(S, Hd, tok))
+    n_inst = S * Hd * tok
+    from oracle import lqr_oracle as orc
+    from paper_2603_09221_b200.workloads import to_float64_numpy
+    d = to_float64_numpy(w)
+    want = ("P", "u") if c["first_only"] else ("K", "P", "x", "u")
+    times, threads = [], 0
+    for it in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
+        out = orc.solve_batch(d["A"], d["B"], d["Q"], d["R"], d["x0"], c["H"], batch=(S, Hd, tok),
+                              first_only=c["first_only"], want=want)
+        dt = time.perf_counter() - t0
+        threads = out["threads"]
+        if it >= args.warmup:
+            times.append(dt)
+    ms = 1e3 * sum(times) / len(times)
+    val = n_inst / (ms * 1e-3)
+    line = {"impl": "reference", "metric": "lqr_instances_per_sec", "value": val, "unit": "instances/s",
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": c["name"], "n": c["n"], "m": c["m"], "H": c["H"],
+                       "instances_per_step": n_inst, "note": "bounded sample of the workload per step"},
+            "cpu_baseline": {"value": val, "unit": "instances/s", "cores": threads, "kind": "oracle",
+                             "sample": "%d instances (%dx%dx%d tokens) per step" % (n_inst, S, Hd, tok)},
+            "e2e": {"value": val, "unit": "instances/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg4")
+    ap.add_argument("--method", default="auto", choices=["auto", "riccati", "scan"])
+    ap.add_argument("--math", default="auto", choices=["auto", "fp32", "tf32"])
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--cpu-sample", type=int, default=256, help="instances the oracle is timed on")
+    ap.add_argument("--ref-instances", type=int, default=256)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    cid = int(args.workload.replace("cfg", ""))
+    if args.impl == "reference":
+        run_reference(args, cid)
+        return
+    args.warmup = max(args.warmup, 3)
+
+    from paper_2603_09221_b200 import lqr
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the solver has no CPU path")
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = world > 1
+    if dist:
+        import torch.distributed as td
+        td.init_process_group("nccl", device_id=torch.device("cuda", local))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    peaks = measured_peaks()
+
+    c = workloads.CONFIGS[cid]
+    w = workloads.make_workload(cid, device=dev, seed=workloads.SEED0 + cid + 1000 * rank)
+    n, m, H = c["n"], c["m"], c["H"]
+    N = int(np.prod(c["batch"]))
+    first = c["first_only"]
+    method = {"auto": lqr.TTC_AUTO, "riccati": lqr.TTC_RICCATI, "scan": lqr.TTC_SCAN}[args.method]
+    math = {"auto": lqr.TTC_MATH_AUTO, "fp32": lqr.TTC_MATH_FP32, "tf32": lqr.TTC_MATH_TF32}[args.math]
+    solver = lqr.LqrSolver(n, m, H, c["batch"], device=local, method=method, math=math)
+    want = ("P", "u", "info") if first else ("K", "P", "x", "u", "info")
+    out = lqr.alloc_outputs(n, m, H, N, dev, first_only=first, want=want)
+    flags = lqr.TTC_OUT_FIRST_ONLY if first else 0
+
+    def step():
+        solver.solve(w["A"], w["B"], w["Q"], w["R"], w["x0"], H, K=out.get("K"), P=out.get("P"), x=out.get("x"),
+                     u=out.get("u"), info=out.get("info"), flags=flags)
+
+    def barrier():
+        if dist:
+            td.barrier()
+        torch.cuda.synchronize(dev)
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    launches0 = solver.query(lqr.TTC_QUERY_TOTAL_LAUNCHES)
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    barrier()
+    evs[0].record()
+    for i in range(args.steps):
+        step()
+        evs[i + 1].record()
+    barrier()
+    launches = solver.query(lqr.TTC_QUERY_TOTAL_LAUNCHES) - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    total_ms = evs[0].elapsed_time(evs[-1])
+    per_step = [evs[i].elapsed_time(evs[i + 1]) for i in range(args.steps)]
+    kernel_id = solver.query(lqr.TTC_QUERY_LAST_KERNEL)
+    t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+    if dist:
+        td.all_reduce(t, op=td.ReduceOp.MAX)
+    total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * N / (ms_per_step * 1e-3)
+
+    # ---- end to end through the host-buffer entry point (pinned host memory, copies timed)
+    e2e = None
+    if not args.no_e2e:
+        hin = {k: w[k].cpu().pin_memory() for k in ("A", "B", "Q", "R", "x0")}
+        hout = lqr.alloc_outputs(n, m, H, N, "cpu", first_only=first, want=want, pin=True)
+        h2d = sum(v.numel() * v.element_size() for v in hin.values())
+        d2h = sum(v.numel() * v.element_size() for v in hout.values())
+
+        def host_step():
+            solver.solve_host(hin["A"], hin["B"], hin["Q"], hin["R"], hin["x0"], H, K=hout.get("K"), P=hout.get("P"),
+                              x=hout.get("x"), u=hout.get("u"), info=hout.get("info"), flags=flags)
+
+        host_step()
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(args.e2e_steps):
+            host_step()
+        barrier()
+        e2e_ms = 1e3 * (time.perf_counter() - t0) / args.e2e_steps
+        te = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
+        if dist:
+            td.all_reduce(te, op=td.ReduceOp.MAX)
+        e2e = {"value": world * N / (float(te.item()) * 1e-3), "unit": "instances/s",
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": float(te.item())}
+        del hin, hout
+
+    if rank != 0:
+        if dist:
+            td.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel (one launch per step does the whole backward pass)
+    flops_i, bin_i, bout_i = algorithmic_counts(c)
+    kname = lqr.KERNEL_NAMES.get(kernel_id, str(kernel_id))
+    launches_per_step = launches / args.steps
+    kernel_ms = statistics.median(per_step)       # dominant kernel ~ the whole step (events per step)
+    alg_bytes = N * (bin_i + bout_i)
+    alg_flops = N * flops_i
+    t_hbm = alg_bytes / (peaks["hbm_gbs"] * 1e9)
+    fp32_peak = SM_COUNT * FP32_LANES_PER_SM * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12
+    tf32_peak = peaks["bf16_tflops_sustained"] * TF32_TO_BF16_RATIO
+    if kname == "riccati_mma":
+        bound, peak, unit, ach = "tensor", tf32_peak, "TFLOP/s", alg_flops / (kernel_ms * 1e-3) / 1e12
+        peak_note = "tf32 = measured sustained bf16 x 0.5 (nominal ratio), of %s" % peaks["source"]
+    else:
+        t_alu = alg_flops / (fp32_peak * 1e12)
+        if t_hbm >= t_alu:
+            bound, peak, unit, ach = "hbm", peaks["hbm_gbs"], "GB/s", alg_bytes / (kernel_ms * 1e-3) / 1e9
+            peak_note = "copy bandwidth, of %s" % peaks["source"]
+        else:
+            bound, peak, unit, ach = "alu", fp32_peak, "TFLOP/s", alg_flops / (kernel_ms * 1e-3) / 1e12
+            peak_note = "148 SMs x 128 FP32 lanes x 2 x %.0f MHz (derived)" % peaks["sm_max_mhz"]
+    roofline = {"bound": bound, "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak, "traffic": None,
+                "kernel": kname, "kernel_ms": kernel_ms, "peak_note": peak_note,
+                "algorithmic_flops_per_launch": alg_flops, "algorithmic_bytes_per_launch": alg_bytes,
+                "hbm_frac": (alg_bytes / (kernel_ms * 1e-3) / 1e9) / peaks["hbm_gbs"]}
+    traffic_path = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(traffic_path):
+        with open(traffic_path) as f:
+            tr = json.load(f).get("%s/%s" % (c["name"], kname))
+        if tr:
+            roofline["traffic"] = tr["dram_bytes_per_instance"] * N
+            roofline["traffic_note"] = tr.get("note")
+
+    cpu = None
+    if not args.no_cpu_baseline and world == 1:
+        idx = oracle_sample(w, args.cpu_sample)
+        ref, dt = time_oracle(w, idx, first)
+        # parity of the timed configuration on the sampled instances
+        from tests import parity_util as pu
+        errs = pu.compare(out, ref, idx, c["tol"], names=("P", "u") if first else ("K", "P", "x", "u"))
+        cpu = {"value": len(idx) / dt, "unit": "instances/s", "cores": int(ref["threads"]), "kind": "oracle",
+               "sample": "%d instances of the same workload, every (seq, head) covered" % len(idx),
+               "seconds": dt, "parity_max_rel_err": errs, "speedup_gpu_over_cpu": value / (len(idx) / dt)}
+
+    line = {"metric": "lqr_instances_per_sec", "value": value, "unit": "instances/s", "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "tf32" if kname == "riccati_mma" else "f32",
+            "data": "synthetic",
+            "config": {"workload": c["name"], "n": n, "m": m, "H": H, "instances": N, "batch": list(c["batch"]),
+                       "q_x0_dtype": c["q_dtype"], "outputs": list(want), "method": args.method, "kernel": kname,
+                       "l2": "inputs+outputs per step exceed L2 (%.2f GB)" % (alg_bytes / 1e9)
+                       if alg_bytes > 126e6 else "workload fits L2: latency-bound case"},
+            "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches),
+            "launches_per_step": launches_per_step, "clocks": clocks,
+            "ms_per_step_percentiles": {"p20": float(np.percentile(per_step, 20)), "p50": float(np.percentile(per_step, 50)),
+                                        "p80": float(np.percentile(per_step, 80))}}
+    print(json.dumps(line))
+    solver.close()
+    if dist:
+        td.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

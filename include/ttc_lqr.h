@@ -1,0 +1,171 @@
+/*
+ * ttc_lqr.h -- C ABI of the batched finite-horizon LQR solver (the hot path of a
+ * Test-Time Control layer), NVIDIA B200 (sm_100a) only.
+ *
+ * Problem solved, independently for each of N = batch[0]*batch[1]*batch[2] instances
+ * (the paper's Eq. 3 / Definition A.1 with time-invariant parameters, written with the
+ * usual control indexing):
+ *
+ *     minimise   sum_{t=0}^{H-1} ( x_t' Q x_t + u_t' R u_t ) + x_H' Q x_H
+ *     subject to x_{t+1} = A x_t + B u_t ,  x_0 given
+ *
+ *     A: n x n,  B: n x m,  Q: n x n symmetric PSD,  R: m x m symmetric PD,  x_0: n.
+ *
+ * Results (Prop. 3.1 and Alg. 1 of the paper):
+ *     P_H = Q ;  for t = H-1..0:
+ *         K_t = -(R + B' P_{t+1} B)^{-1} B' P_{t+1} A
+ *         P_t = Q + A' P_{t+1} A + (B' P_{t+1} A)' K_t
+ *     u_t = K_t x_t ;  x_{t+1} = A x_t + B u_t .
+ * Relation to the paper's indexing (h_t = A h_{t-1} + B u_t, t = 1..T, Q_0 = 0):
+ * x_t = h_t, u_t = paper's u_{t+1}, K_t = paper's K_{t+1}, P_t = paper's P_t for t >= 1,
+ * P_0 = paper's P_0 + Q.  The optimal cost is x_0' P_0 x_0.
+ *
+ * Two methods compute the same P_t: the sequential Riccati recursion, and a scan over
+ * the horizon whose element is the symplectic transition matrix of Thm A.2 stored
+ * inverse-free as the triple (A, C = B R^{-1} B', J = Q) (TTC_SCAN).
+ *
+ * All matrices are row-major and contiguous (leading dimension = number of columns).
+ * Instance index i = (i0*batch[1] + i1)*batch[2] + i2; an input operand of instance i
+ * starts at element  i0*bstride[0] + i1*bstride[1] + i2*bstride[2]  of its array; a
+ * stride of 0 shares the operand along that batch dimension (e.g. per-head A, B, R).
+ * Outputs are dense in i.
+ *
+ * Every function returns a status (0 = TTC_OK, negative = error, nothing enqueued).
+ * No function aborts the process; device code never traps and has no unbounded wait.
+ */
+#ifndef TTC_LQR_H_
+#define TTC_LQR_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* status codes */
+#define TTC_OK                        0
+#define TTC_STATUS_INVALID_ARGUMENT  (-1)
+#define TTC_STATUS_CUDA_ERROR        (-2)
+#define TTC_STATUS_ALLOC_FAILED      (-3)
+#define TTC_STATUS_UNSUPPORTED       (-4)
+
+/* element types of input operands */
+#define TTC_F32   0
+#define TTC_BF16  1
+
+/* ttc_lqr_config.method */
+#define TTC_AUTO     0   /* library picks                                            */
+#define TTC_RICCATI  1   /* sequential backward recursion (Prop. 3.1, Alg. 1)        */
+#define TTC_SCAN     2   /* symplectic-pair scan over the horizon (Thm A.2 element)  */
+
+/* ttc_lqr_config.math : arithmetic of the n x n contractions */
+#define TTC_MATH_AUTO  0  /* FP32 when every input is F32, TF32 when Q or x0 is BF16  */
+#define TTC_MATH_FP32  1  /* FFMA, fp32 throughout                                    */
+#define TTC_MATH_TF32  2  /* tensor cores, tf32 operands, fp32 accumulate (n = m = 64)*/
+
+/* ttc_lqr_solve flags */
+#define TTC_OUT_FIRST_ONLY  1u  /* P is [N][n][n] = P_0 and u is [N][m] = u_0          */
+
+/* ttc_lqr_query keys */
+#define TTC_QUERY_LAST_LAUNCHES    1  /* kernels launched by the last solve            */
+#define TTC_QUERY_WORKSPACE_BYTES  2  /* device bytes currently owned by the handle    */
+#define TTC_QUERY_LAST_KERNEL      3  /* id of the main kernel of the last solve       */
+#define TTC_QUERY_TOTAL_LAUNCHES   4  /* kernels launched since create                 */
+
+/* ids returned by TTC_QUERY_LAST_KERNEL */
+#define TTC_KERNEL_NONE           0
+#define TTC_KERNEL_RICCATI_CTA    1  /* generic: one CTA per instance, FFMA            */
+#define TTC_KERNEL_RICCATI_WARP   2  /* register-tiled FFMA, several instances per CTA */
+#define TTC_KERNEL_RICCATI_MMA    3  /* tensor-core contractions, n = m = 64           */
+#define TTC_KERNEL_SCAN           4  /* symplectic-pair scan + gain/rollout kernel     */
+
+typedef struct ttc_lqr_handle ttc_lqr_handle; /* opaque; owned by the library */
+
+/* One input operand.  `ptr` is owned by the caller and only read.  For ttc_lqr_solve it
+ * is a DEVICE pointer (on the handle's device), for ttc_lqr_solve_host a HOST pointer.
+ * It must be aligned to 16 bytes. */
+typedef struct {
+    const void* ptr;
+    int32_t     dtype;       /* TTC_F32 or TTC_BF16 (BF16 only for Q and x0)            */
+    int32_t     reserved;    /* set to 0                                                */
+    int64_t     bstride[3];  /* element stride per batch dimension; 0 = shared          */
+} ttc_operand;
+
+typedef struct {
+    int32_t n;               /* state dimension, 1..64                                  */
+    int32_t m;               /* control dimension, 1..64                                */
+    int32_t max_horizon;     /* largest H that will be passed to solve, >= 1            */
+    int32_t device;          /* CUDA device ordinal                                     */
+    int64_t batch[3];        /* e.g. {sequences, heads, tokens}; each >= 1              */
+    int32_t method;          /* TTC_AUTO | TTC_RICCATI | TTC_SCAN                       */
+    int32_t math;            /* TTC_MATH_*                                              */
+} ttc_lqr_config;
+
+/*
+ * Create a solver for a fixed problem shape (the paper's problem statement, Eq. 3 and
+ * Definition A.1, fixes what a "problem" is: {A,B,Q,R}, h_0 and a horizon).
+ * Validates cfg, selects the device, returns an opaque handle in *out.  The handle owns
+ * only its device workspace, which is allocated on first need inside a solve call (such
+ * a call synchronises the device once) and freed by ttc_lqr_destroy.
+ * Errors: INVALID_ARGUMENT (null pointers, sizes out of range), UNSUPPORTED (method/math
+ * not available for this shape), CUDA_ERROR (no such device / not an sm_100 device).
+ */
+int ttc_lqr_create(const ttc_lqr_config* cfg, ttc_lqr_handle** out);
+
+/*
+ * Solve all N instances (Prop. 3.1 / Alg. 1; or the symplectic scan built on Thm A.2's
+ * transition matrices when the method is TTC_SCAN).  Asynchronous: kernels are enqueued
+ * on `cuda_stream` (a cudaStream_t; NULL = the default stream) and the call returns;
+ * outputs are valid once the stream reaches that point.  One handle serves one stream at
+ * a time.
+ *
+ * Inputs (device):  A [n][n], B [n][m], R [m][m] as F32;  Q [n][n], x0 [n] as F32 or BF16.
+ *                   x0 may be NULL when neither x nor u is requested.
+ * Outputs (device, F32, written completely, each may be NULL = not wanted):
+ *     K    [N][H][m][n]
+ *     P    [N][H+1][n][n]    (or [N][n][n] = P_0   with TTC_OUT_FIRST_ONLY)
+ *     x    [N][H+1][n]
+ *     u    [N][H][m]         (or [N][m]    = u_0   with TTC_OUT_FIRST_ONLY)
+ *     info [N] int32: 0 = solved; t*m + j + 1 > 0 = pivot j (0-based) of R + B'P_{t+1}B at
+ *          time index t was not positive (R not positive definite, Q indefinite, or NaN
+ *          input).  All requested outputs of such an instance are filled with quiet NaN;
+ *          other instances are unaffected.
+ * Output pointers must be 16-byte aligned.
+ * Errors: INVALID_ARGUMENT (null handle/operand, H < 1 or H > max_horizon, bad dtype,
+ * misaligned pointer), ALLOC_FAILED (workspace), CUDA_ERROR (launch failure).
+ */
+int ttc_lqr_solve(ttc_lqr_handle* h,
+                  const ttc_operand* A, const ttc_operand* B, const ttc_operand* Q,
+                  const ttc_operand* R, const ttc_operand* x0, int32_t H,
+                  float* K, float* P, float* x, float* u, int32_t* info,
+                  uint32_t flags, void* cuda_stream);
+
+/*
+ * Same computation with HOST buffers (same problem statement as ttc_lqr_solve): operand
+ * pointers and all outputs are host memory (pinned memory makes the copies faster but is
+ * not required).  The call copies the inputs to device staging buffers owned by the handle,
+ * runs ttc_lqr_solve on an internal stream, copies the requested outputs back and returns
+ * after everything has completed (synchronous).  Strides have the same meaning.
+ */
+int ttc_lqr_solve_host(ttc_lqr_handle* h,
+                       const ttc_operand* A, const ttc_operand* B, const ttc_operand* Q,
+                       const ttc_operand* R, const ttc_operand* x0, int32_t H,
+                       float* K, float* P, float* x, float* u, int32_t* info,
+                       uint32_t flags);
+
+/* Free the handle and its workspace (synchronises the handle's device).  NULL is OK. */
+int ttc_lqr_destroy(ttc_lqr_handle* h);
+
+/* Small integer facts about the handle (TTC_QUERY_*); returns INVALID_ARGUMENT on a bad key. */
+int ttc_lqr_query(const ttc_lqr_handle* h, int32_t key, int64_t* value);
+
+/* Static, human-readable name of a status code. */
+const char* ttc_lqr_status_string(int status);
+
+/* Detail of the last error raised on this thread (empty string if none). */
+const char* ttc_lqr_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TTC_LQR_H_ */

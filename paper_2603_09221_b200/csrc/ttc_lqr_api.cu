@@ -1,0 +1,388 @@
+// Host side of the C ABI declared in include/ttc_lqr.h: argument validation, kernel
+// selection, workspace ownership, launches on the caller's stream, and the host-buffer
+// convenience entry point.  No torch types, no CPU fallback: without a CUDA device of
+// compute capability 10.x every call fails with TTC_STATUS_CUDA_ERROR.
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "common.cuh"
+#include "riccati_cta.cuh"
+#include "scan_pair.cuh"
+
+using namespace ttc;
+
+namespace {
+
+thread_local char g_err[512] = "";
+
+int fail(int status, const char* fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    return status;
+}
+
+#define TTC_CUDA(call)                                                                   \
+    do {                                                                                 \
+        cudaError_t e_ = (call);                                                         \
+        if (e_ != cudaSuccess)                                                           \
+            return fail(TTC_STATUS_CUDA_ERROR, "%s: %s", #call, cudaGetErrorString(e_)); \
+    } while (0)
+
+struct DevBuf {
+    void* ptr = nullptr;
+    size_t bytes = 0;
+};
+
+} // namespace
+
+struct ttc_lqr_handle {
+    ttc_lqr_config cfg;
+    long long N;
+    int sm_count;
+    DevBuf ws_K, ws_P, ws_E;       // scratch used by kernels
+    DevBuf st_in[5], st_out[5];    // device staging of ttc_lqr_solve_host
+    cudaStream_t host_stream;
+    long long last_launches, total_launches;
+    int last_kernel;
+};
+
+namespace {
+
+int ensure(DevBuf& b, size_t bytes)
+{
+    if (bytes <= b.bytes)
+        return TTC_OK;
+    if (b.ptr) {
+        cudaDeviceSynchronize();
+        cudaFree(b.ptr);
+        b.ptr = nullptr;
+        b.bytes = 0;
+    }
+    cudaError_t e = cudaMalloc(&b.ptr, bytes);
+    if (e != cudaSuccess) {
+        b.ptr = nullptr;
+        cudaGetLastError();
+        return fail(TTC_STATUS_ALLOC_FAILED, "cudaMalloc(%zu bytes): %s", bytes, cudaGetErrorString(e));
+    }
+    b.bytes = bytes;
+    return TTC_OK;
+}
+
+void release(DevBuf& b)
+{
+    if (b.ptr)
+        cudaFree(b.ptr);
+    b.ptr = nullptr;
+    b.bytes = 0;
+}
+
+size_t workspace_bytes(const ttc_lqr_handle* h)
+{
+    size_t s = h->ws_K.bytes + h->ws_P.bytes + h->ws_E.bytes;
+    for (int i = 0; i < 5; ++i)
+        s += h->st_in[i].bytes + h->st_out[i].bytes;
+    return s;
+}
+
+int check_operand(const char* name, const ttc_operand* o, bool allow_bf16, bool allow_null)
+{
+    if (!o || !o->ptr) {
+        if (allow_null)
+            return TTC_OK;
+        return fail(TTC_STATUS_INVALID_ARGUMENT, "operand %s is null", name);
+    }
+    if (o->dtype != TTC_F32 && !(allow_bf16 && o->dtype == TTC_BF16))
+        return fail(TTC_STATUS_INVALID_ARGUMENT, "operand %s: dtype %d not supported", name, o->dtype);
+    if (reinterpret_cast<uintptr_t>(o->ptr) & 15u)
+        return fail(TTC_STATUS_INVALID_ARGUMENT, "operand %s is not 16-byte aligned", name);
+    for (int d = 0; d < 3; ++d)
+        if (o->bstride[d] < 0)
+            return fail(TTC_STATUS_INVALID_ARGUMENT, "operand %s: negative stride", name);
+    return TTC_OK;
+}
+
+OperandDev to_dev(const ttc_operand* o)
+{
+    OperandDev d;
+    if (!o || !o->ptr) {
+        d.ptr = nullptr;
+        d.dtype = TTC_F32;
+        d.s0 = d.s1 = d.s2 = 0;
+        return d;
+    }
+    d.ptr = o->ptr;
+    d.dtype = o->dtype;
+    d.s0 = o->bstride[0];
+    d.s1 = o->bstride[1];
+    d.s2 = o->bstride[2];
+    return d;
+}
+
+int validate_common(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, const ttc_operand* Q,
+                    const ttc_operand* R, const ttc_operand* x0, int H, const float* K, const float* P,
+                    const float* x, const float* u, const int32_t* info, uint32_t flags)
+{
+    if (!h)
+        return fail(TTC_STATUS_INVALID_ARGUMENT, "null handle");
+    if (H < 1 || H > h->cfg.max_horizon)
+        return fail(TTC_STATUS_INVALID_ARGUMENT, "H=%d outside [1, max_horizon=%d]", H, h->cfg.max_horizon);
+    if (flags & ~TTC_OUT_FIRST_ONLY)
+        return fail(TTC_STATUS_INVALID_ARGUMENT, "unknown flag bits 0x%x", flags);
+    int s;
+    if ((s = check_operand("A", A, false, false))) return s;
+    if ((s = check_operand("B", B, false, false))) return s;
+    if ((s = check_operand("Q", Q, true, false))) return s;
+    if ((s = check_operand("R", R, false, false))) return s;
+    const bool need_x0 = (x != nullptr) || (u != nullptr);
+    if ((s = check_operand("x0", x0, true, !need_x0))) return s;
+    const void* outs[5] = {K, P, x, u, info};
+    const char* names[5] = {"K", "P", "x", "u", "info"};
+    for (int i = 0; i < 5; ++i)
+        if (outs[i] && (reinterpret_cast<uintptr_t>(outs[i]) & 15u))
+            return fail(TTC_STATUS_INVALID_ARGUMENT, "output %s is not 16-byte aligned", names[i]);
+    return TTC_OK;
+}
+
+int pick_method(const ttc_lqr_handle* h)
+{
+    if (h->cfg.method == TTC_SCAN)
+        return TTC_SCAN;
+    return TTC_RICCATI;
+}
+
+} // namespace
+
+extern "C" {
+
+const char* ttc_lqr_status_string(int status)
+{
+    switch (status) {
+    case TTC_OK: return "TTC_OK";
+    case TTC_STATUS_INVALID_ARGUMENT: return "TTC_STATUS_INVALID_ARGUMENT";
+    case TTC_STATUS_CUDA_ERROR: return "TTC_STATUS_CUDA_ERROR";
+    case TTC_STATUS_ALLOC_FAILED: return "TTC_STATUS_ALLOC_FAILED";
+    case TTC_STATUS_UNSUPPORTED: return "TTC_STATUS_UNSUPPORTED";
+    default: return "TTC_STATUS_UNKNOWN";
+    }
+}
+
+const char* ttc_lqr_last_error(void) { return g_err; }
+
+int ttc_lqr_create(const ttc_lqr_config* cfg, ttc_lqr_handle** out)
+{
+    if (!cfg || !out)
+        return fail(TTC_STATUS_INVALID_ARGUMENT, "null cfg/out");
+    *out = nullptr;
+    if (cfg->n < 1 || cfg->n > 64 || cfg->m < 1 || cfg->m > 64)
+        return fail(TTC_STATUS_INVALID_ARGUMENT, "n=%d, m=%d outside [1, 64]", cfg->n, cfg->m);
+    if (cfg->max_horizon < 1 || cfg->max_horizon > 65536)
+        return fail(TTC_STATUS_INVALID_ARGUMENT, "max_horizon=%d outside [1, 65536]", cfg->max_horizon);
+    long long N = 1;
+    for (int d = 0; d < 3; ++d) {
+        if (cfg->batch[d] < 1 || cfg->batch[d] > (1ll << 31))
+            return fail(TTC_STATUS_INVALID_ARGUMENT, "batch[%d]=%lld out of range", d, (long long)cfg->batch[d]);
+        N *= cfg->batch[d];
+        if (N > (1ll << 31))
+            return fail(TTC_STATUS_INVALID_ARGUMENT, "more than 2^31 instances");
+    }
+    if (cfg->method < TTC_AUTO || cfg->method > TTC_SCAN)
+        return fail(TTC_STATUS_INVALID_ARGUMENT, "unknown method %d", cfg->method);
+    if (cfg->math < TTC_MATH_AUTO || cfg->math > TTC_MATH_TF32)
+        return fail(TTC_STATUS_INVALID_ARGUMENT, "unknown math mode %d", cfg->math);
+    if (cfg->math == TTC_MATH_TF32 && !(cfg->n == 64 && cfg->m == 64))
+        return fail(TTC_STATUS_UNSUPPORTED, "TTC_MATH_TF32 needs n = m = 64");
+    int ndev = 0;
+    TTC_CUDA(cudaGetDeviceCount(&ndev));
+    if (cfg->device < 0 || cfg->device >= ndev)
+        return fail(TTC_STATUS_CUDA_ERROR, "device %d not present (%d devices)", cfg->device, ndev);
+    cudaDeviceProp prop;
+    TTC_CUDA(cudaGetDeviceProperties(&prop, cfg->device));
+    if (prop.major != 10)
+        return fail(TTC_STATUS_CUDA_ERROR, "device %d is sm_%d%d; this library is built for sm_100a only",
+                    cfg->device, prop.major, prop.minor);
+    TTC_CUDA(cudaSetDevice(cfg->device));
+    ttc_lqr_handle* h = new (std::nothrow) ttc_lqr_handle();
+    if (!h)
+        return fail(TTC_STATUS_ALLOC_FAILED, "host allocation failed");
+    h->cfg = *cfg;
+    h->N = N;
+    h->sm_count = prop.multiProcessorCount;
+    h->host_stream = nullptr;
+    h->last_launches = h->total_launches = 0;
+    h->last_kernel = TTC_KERNEL_NONE;
+    *out = h;
+    g_err[0] = 0;
+    return TTC_OK;
+}
+
+int ttc_lqr_destroy(ttc_lqr_handle* h)
+{
+    if (!h)
+        return TTC_OK;
+    cudaSetDevice(h->cfg.device);
+    cudaDeviceSynchronize();
+    release(h->ws_K);
+    release(h->ws_P);
+    release(h->ws_E);
+    for (int i = 0; i < 5; ++i) {
+        release(h->st_in[i]);
+        release(h->st_out[i]);
+    }
+    if (h->host_stream)
+        cudaStreamDestroy(h->host_stream);
+    delete h;
+    return TTC_OK;
+}
+
+int ttc_lqr_query(const ttc_lqr_handle* h, int32_t key, int64_t* value)
+{
+    if (!h || !value)
+        return fail(TTC_STATUS_INVALID_ARGUMENT, "null handle/value");
+    switch (key) {
+    case TTC_QUERY_LAST_LAUNCHES: *value = h->last_launches; return TTC_OK;
+    case TTC_QUERY_WORKSPACE_BYTES: *value = (int64_t)workspace_bytes(h); return TTC_OK;
+    case TTC_QUERY_LAST_KERNEL: *value = h->last_kernel; return TTC_OK;
+    case TTC_QUERY_TOTAL_LAUNCHES: *value = h->total_launches; return TTC_OK;
+    default: return fail(TTC_STATUS_INVALID_ARGUMENT, "unknown query key %d", key);
+    }
+}
+
+int ttc_lqr_solve(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, const ttc_operand* Q,
+                  const ttc_operand* R, const ttc_operand* x0, int32_t H, float* K, float* P, float* x,
+                  float* u, int32_t* info, uint32_t flags, void* cuda_stream)
+{
+    int s = validate_common(h, A, B, Q, R, x0, H, K, P, x, u, info, flags);
+    if (s)
+        return s;
+    TTC_CUDA(cudaSetDevice(h->cfg.device));
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const int n = h->cfg.n, m = h->cfg.m;
+
+    SolveParams p;
+    p.n = n; p.m = m; p.H = H;
+    p.b0 = h->cfg.batch[0]; p.b1 = h->cfg.batch[1]; p.b2 = h->cfg.batch[2]; p.N = h->N;
+    p.A = to_dev(A); p.B = to_dev(B); p.Q = to_dev(Q); p.R = to_dev(R); p.x0 = to_dev(x0);
+    p.K = K; p.P = P; p.x = x; p.u = u; p.info = info;
+    p.Kws = nullptr;
+    p.first_only = (flags & TTC_OUT_FIRST_ONLY) ? 1 : 0;
+    h->last_launches = 0;
+
+    const int method = pick_method(h);
+    // The rollout reads every K_t in forward order after the backward pass produced them in
+    // reverse order; when the caller does not want K they live in the workspace.
+    const bool rollout_needs_all_K = (x != nullptr) || (u != nullptr && !p.first_only);
+
+    if (method == TTC_SCAN) {
+        // Full mode keeps every P_t (in the caller's P or in the workspace); when only P_0 / u_0
+        // are wanted the scan keeps a single value matrix (P_1) per instance.
+        const int pfull = !(p.first_only && !K && !x);
+        float* Pbuf;
+        if (pfull && P && !p.first_only) {
+            Pbuf = P;
+        } else {
+            const size_t per = pfull ? (size_t)(H + 1) * n * n : (size_t)n * n;
+            if ((s = ensure(h->ws_P, sizeof(float) * (size_t)h->N * per))) return s;
+            Pbuf = static_cast<float*>(h->ws_P.ptr);
+        }
+        if ((s = ensure(h->ws_E, sizeof(int) * (size_t)h->N))) return s;
+        int launches = 0;
+        cudaError_t e = launch_scan_path(p, Pbuf, static_cast<int*>(h->ws_E.ptr), pfull, h->sm_count, st, &launches);
+        if (e != cudaSuccess)
+            return fail(TTC_STATUS_CUDA_ERROR, "scan path launch: %s", cudaGetErrorString(e));
+        h->last_launches = launches;
+        h->last_kernel = TTC_KERNEL_SCAN;
+    } else {
+        if (!K && rollout_needs_all_K) {
+            if ((s = ensure(h->ws_K, sizeof(float) * (size_t)h->N * H * m * n))) return s;
+            p.Kws = static_cast<float*>(h->ws_K.ptr);
+        }
+        const size_t smem = riccati_cta_smem_bytes(n, m);
+        TTC_CUDA(cudaFuncSetAttribute(riccati_cta_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        int per_sm = 1;
+        TTC_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, riccati_cta_kernel, 256, smem));
+        if (per_sm < 1) per_sm = 1;
+        long long grid = (long long)h->sm_count * per_sm;
+        if (grid > h->N) grid = h->N;
+        riccati_cta_kernel<<<(unsigned)grid, 256, smem, st>>>(p);
+        TTC_CUDA(cudaGetLastError());
+        h->last_launches = 1;
+        h->last_kernel = TTC_KERNEL_RICCATI_CTA;
+    }
+    h->total_launches += h->last_launches;
+    return TTC_OK;
+}
+
+int ttc_lqr_solve_host(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, const ttc_operand* Q,
+                       const ttc_operand* R, const ttc_operand* x0, int32_t H, float* K, float* P, float* x,
+                       float* u, int32_t* info, uint32_t flags)
+{
+    if (!h)
+        return fail(TTC_STATUS_INVALID_ARGUMENT, "null handle");
+    // alignment of host pointers is irrelevant; validate the rest through a relaxed copy
+    if (H < 1 || H > h->cfg.max_horizon)
+        return fail(TTC_STATUS_INVALID_ARGUMENT, "H=%d outside [1, max_horizon=%d]", H, h->cfg.max_horizon);
+    TTC_CUDA(cudaSetDevice(h->cfg.device));
+    if (!h->host_stream)
+        TTC_CUDA(cudaStreamCreateWithFlags(&h->host_stream, cudaStreamNonBlocking));
+    const int n = h->cfg.n, m = h->cfg.m;
+    const long long N = h->N;
+    const bool first = (flags & TTC_OUT_FIRST_ONLY) != 0;
+    const ttc_operand* in[5] = {A, B, Q, R, x0};
+    const char* names[5] = {"A", "B", "Q", "R", "x0"};
+    const size_t elems[5] = {(size_t)n * n, (size_t)n * m, (size_t)n * n, (size_t)m * m, (size_t)n};
+    ttc_operand dev[5];
+    for (int i = 0; i < 5; ++i) {
+        dev[i].ptr = nullptr; dev[i].dtype = TTC_F32; dev[i].reserved = 0;
+        dev[i].bstride[0] = dev[i].bstride[1] = dev[i].bstride[2] = 0;
+        if (!in[i] || !in[i]->ptr) {
+            if (i == 4 && !x && !u)
+                continue;
+            return fail(TTC_STATUS_INVALID_ARGUMENT, "operand %s is null", names[i]);
+        }
+        if (in[i]->dtype != TTC_F32 && in[i]->dtype != TTC_BF16)
+            return fail(TTC_STATUS_INVALID_ARGUMENT, "operand %s: dtype %d not supported", names[i], in[i]->dtype);
+        size_t extent = elems[i];
+        for (int d = 0; d < 3; ++d) {
+            if (in[i]->bstride[d] < 0)
+                return fail(TTC_STATUS_INVALID_ARGUMENT, "operand %s: negative stride", names[i]);
+            extent += (size_t)(h->cfg.batch[d] - 1) * (size_t)in[i]->bstride[d];
+        }
+        const size_t bytes = extent * (in[i]->dtype == TTC_BF16 ? 2 : 4);
+        int s = ensure(h->st_in[i], bytes);
+        if (s) return s;
+        TTC_CUDA(cudaMemcpyAsync(h->st_in[i].ptr, in[i]->ptr, bytes, cudaMemcpyHostToDevice, h->host_stream));
+        dev[i] = *in[i];
+        dev[i].ptr = h->st_in[i].ptr;
+    }
+    void* host_out[5] = {K, P, x, u, info};
+    const size_t out_bytes[5] = {
+        sizeof(float) * (size_t)N * H * m * n,
+        sizeof(float) * (size_t)N * (first ? 1 : H + 1) * n * n,
+        sizeof(float) * (size_t)N * (H + 1) * n,
+        sizeof(float) * (size_t)N * (first ? 1 : H) * m,
+        sizeof(int32_t) * (size_t)N};
+    void* dev_out[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+    for (int i = 0; i < 5; ++i)
+        if (host_out[i]) {
+            int s = ensure(h->st_out[i], out_bytes[i]);
+            if (s) return s;
+            dev_out[i] = h->st_out[i].ptr;
+        }
+    int s = ttc_lqr_solve(h, &dev[0], &dev[1], &dev[2], &dev[3], dev[4].ptr ? &dev[4] : nullptr, H,
+                          (float*)dev_out[0], (float*)dev_out[1], (float*)dev_out[2], (float*)dev_out[3],
+                          (int32_t*)dev_out[4], flags, h->host_stream);
+    if (s)
+        return s;
+    for (int i = 0; i < 5; ++i)
+        if (host_out[i])
+            TTC_CUDA(cudaMemcpyAsync(host_out[i], dev_out[i], out_bytes[i], cudaMemcpyDeviceToHost, h->host_stream));
+    TTC_CUDA(cudaStreamSynchronize(h->host_stream));
+    return TTC_OK;
+}
+
+} // extern "C"

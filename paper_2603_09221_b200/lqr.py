@@ -1,0 +1,201 @@
+"""Thin ctypes binding of the C ABI in ``include/ttc_lqr.h``.
+
+Argument marshalling only: every step of the solve runs in the CUDA kernels behind
+``libttc_lqr.so``.  There is no CPU fallback; if the library is missing or no sm_100 device
+is present, the calls raise.
+PyTorch is used by callers for device memory and streams; this module only reads
+``data_ptr()``, ``dtype``, ``shape`` and ``stride()`` of the tensors it is given.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+from . import build as _build
+
+TTC_F32, TTC_BF16 = 0, 1
+TTC_AUTO, TTC_RICCATI, TTC_SCAN = 0, 1, 2
+TTC_MATH_AUTO, TTC_MATH_FP32, TTC_MATH_TF32 = 0, 1, 2
+TTC_OUT_FIRST_ONLY = 1
+TTC_QUERY_LAST_LAUNCHES, TTC_QUERY_WORKSPACE_BYTES, TTC_QUERY_LAST_KERNEL, TTC_QUERY_TOTAL_LAUNCHES = 1, 2, 3, 4
+KERNEL_NAMES = {0: "none", 1: "riccati_cta", 2: "riccati_warp", 3: "riccati_mma", 4: "scan"}
+
+EXPORTS = (
+    "ttc_lqr_create", "ttc_lqr_solve", "ttc_lqr_solve_host", "ttc_lqr_destroy", "ttc_lqr_query",
+    "ttc_lqr_status_string", "ttc_lqr_last_error",
+)
+
+
+class ttc_operand(ctypes.Structure):
+    _fields_ = [("ptr", ctypes.c_void_p), ("dtype", ctypes.c_int32), ("reserved", ctypes.c_int32),
+                ("bstride", ctypes.c_int64 * 3)]
+
+
+class ttc_lqr_config(ctypes.Structure):
+    _fields_ = [("n", ctypes.c_int32), ("m", ctypes.c_int32), ("max_horizon", ctypes.c_int32),
+                ("device", ctypes.c_int32), ("batch", ctypes.c_int64 * 3), ("method", ctypes.c_int32),
+                ("math", ctypes.c_int32)]
+
+
+class TtcError(RuntimeError):
+    pass
+
+
+_lib = None
+
+
+def library_path() -> str:
+    return _build.LIB
+
+
+def load_library():
+    """Load ``libttc_lqr.so`` (building it first if a source is newer).  Raises if that fails."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = _build.LIB
+    if not os.path.exists(path) or os.environ.get("TTC_LQR_REBUILD"):
+        path = _build.build_library()
+    lib = ctypes.CDLL(path)
+    P = ctypes.POINTER
+    lib.ttc_lqr_create.restype = ctypes.c_int
+    lib.ttc_lqr_create.argtypes = [P(ttc_lqr_config), P(ctypes.c_void_p)]
+    opp = P(ttc_operand)
+    lib.ttc_lqr_solve.restype = ctypes.c_int
+    lib.ttc_lqr_solve.argtypes = [ctypes.c_void_p, opp, opp, opp, opp, opp, ctypes.c_int32] + \
+        [ctypes.c_void_p] * 5 + [ctypes.c_uint32, ctypes.c_void_p]
+    lib.ttc_lqr_solve_host.restype = ctypes.c_int
+    lib.ttc_lqr_solve_host.argtypes = [ctypes.c_void_p, opp, opp, opp, opp, opp, ctypes.c_int32] + \
+        [ctypes.c_void_p] * 5 + [ctypes.c_uint32]
+    lib.ttc_lqr_destroy.restype = ctypes.c_int
+    lib.ttc_lqr_destroy.argtypes = [ctypes.c_void_p]
+    lib.ttc_lqr_query.restype = ctypes.c_int
+    lib.ttc_lqr_query.argtypes = [ctypes.c_void_p, ctypes.c_int32, P(ctypes.c_int64)]
+    lib.ttc_lqr_status_string.restype = ctypes.c_char_p
+    lib.ttc_lqr_status_string.argtypes = [ctypes.c_int]
+    lib.ttc_lqr_last_error.restype = ctypes.c_char_p
+    lib.ttc_lqr_last_error.argtypes = []
+    _lib = lib
+    return lib
+
+
+def _check(status):
+    if status != 0:
+        lib = load_library()
+        raise TtcError("%s: %s" % (lib.ttc_lqr_status_string(status).decode(), lib.ttc_lqr_last_error().decode()))
+
+
+def _operand(t, tail_ndim, batch):
+    """Describe tensor ``t`` (leading dims broadcastable to ``batch``, trailing ``tail_ndim``
+    matrix/vector dims contiguous) as a ``ttc_operand``."""
+    if t is None:
+        return None
+    if t.dtype == torch.float32:
+        dt = TTC_F32
+    elif t.dtype == torch.bfloat16:
+        dt = TTC_BF16
+    else:
+        raise TypeError("operand dtype must be float32 or bfloat16, got %s" % t.dtype)
+    lead = t.dim() - tail_ndim
+    if lead > 3:
+        raise ValueError("at most 3 batch dimensions")
+    shape = (1,) * (3 - lead) + tuple(t.shape[:lead])
+    strides = (0,) * (3 - lead) + tuple(t.stride()[:lead])
+    exp = 1
+    for d in range(t.dim() - 1, lead - 1, -1):
+        if t.shape[d] != 1 and t.stride(d) != exp:
+            raise ValueError("matrix dimensions of an operand must be contiguous (row-major)")
+        exp *= t.shape[d]
+    op = ttc_operand()
+    op.ptr = t.data_ptr()
+    op.dtype = dt
+    op.reserved = 0
+    for d in range(3):
+        if shape[d] == batch[d]:
+            op.bstride[d] = strides[d] if shape[d] > 1 else 0
+        elif shape[d] == 1:
+            op.bstride[d] = 0
+        else:
+            raise ValueError("operand batch shape %s does not broadcast to %s" % (shape, tuple(batch)))
+    return op
+
+
+class LqrSolver:
+    """Owns one ``ttc_lqr_handle``.  ``batch`` is ``(seqs, heads, tokens)`` (shorter tuples are
+    left-padded with 1)."""
+
+    def __init__(self, n, m, max_horizon, batch, device=0, method=TTC_AUTO, math=TTC_MATH_AUTO):
+        lib = load_library()
+        batch = tuple(int(b) for b in batch)
+        batch = (1,) * (3 - len(batch)) + batch
+        cfg = ttc_lqr_config()
+        cfg.n, cfg.m, cfg.max_horizon, cfg.device = n, m, max_horizon, device
+        for d in range(3):
+            cfg.batch[d] = batch[d]
+        cfg.method, cfg.math = method, math
+        self._h = ctypes.c_void_p()
+        _check(lib.ttc_lqr_create(ctypes.byref(cfg), ctypes.byref(self._h)))
+        self.n, self.m, self.batch, self.device = n, m, batch, device
+        self.N = batch[0] * batch[1] * batch[2]
+
+    def close(self):
+        if getattr(self, "_h", None) is not None and self._h.value:
+            load_library().ttc_lqr_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def query(self, key):
+        v = ctypes.c_int64()
+        _check(load_library().ttc_lqr_query(self._h, key, ctypes.byref(v)))
+        return v.value
+
+    def _ops(self, A, B, Q, R, x0):
+        ops = [_operand(A, 2, self.batch), _operand(B, 2, self.batch), _operand(Q, 2, self.batch),
+               _operand(R, 2, self.batch), _operand(x0, 1, self.batch)]
+        return [ctypes.byref(o) if o is not None else None for o in ops], ops
+
+    @staticmethod
+    def _ptr(t):
+        return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+    def solve(self, A, B, Q, R, x0, H, K=None, P=None, x=None, u=None, info=None, flags=0, stream=None):
+        """Enqueue ``ttc_lqr_solve`` on ``stream`` (a ``torch.cuda.Stream``; default: current)."""
+        refs, keep = self._ops(A, B, Q, R, x0)
+        if stream is None:
+            stream = torch.cuda.current_stream(self.device)
+        _check(load_library().ttc_lqr_solve(
+            self._h, *refs, int(H), self._ptr(K), self._ptr(P), self._ptr(x), self._ptr(u), self._ptr(info),
+            int(flags), ctypes.c_void_p(stream.cuda_stream)))
+
+    def solve_host(self, A, B, Q, R, x0, H, K=None, P=None, x=None, u=None, info=None, flags=0):
+        """``ttc_lqr_solve_host``: all tensors live in host memory; returns when the results are there."""
+        refs, keep = self._ops(A, B, Q, R, x0)
+        _check(load_library().ttc_lqr_solve_host(
+            self._h, *refs, int(H), self._ptr(K), self._ptr(P), self._ptr(x), self._ptr(u), self._ptr(info),
+            int(flags)))
+
+
+def alloc_outputs(n, m, H, N, device, first_only=False, want=("K", "P", "x", "u", "info"), pin=False):
+    """Allocate output tensors of the documented shapes (torch owns the memory)."""
+    kw = dict(device=device)
+    if pin and str(device) == "cpu":
+        kw["pin_memory"] = True
+    out = {}
+    if "K" in want:
+        out["K"] = torch.empty((N, H, m, n), dtype=torch.float32, **kw)
+    if "P" in want:
+        out["P"] = torch.empty((N, n, n) if first_only else (N, H + 1, n, n), dtype=torch.float32, **kw)
+    if "x" in want:
+        out["x"] = torch.empty((N, H + 1, n), dtype=torch.float32, **kw)
+    if "u" in want:
+        out["u"] = torch.empty((N, m) if first_only else (N, H, m), dtype=torch.float32, **kw)
+    if "info" in want:
+        out["info"] = torch.empty((N,), dtype=torch.int32, **kw)
+    return out

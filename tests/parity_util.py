@@ -1,0 +1,100 @@
+"""Helpers shared by the GPU parity tests: run the CUDA library, run the oracle on the same
+inputs (all or a sample of instances), and the error measure.
+
+Error measure ("max relative error" of the target statement, made precise): for one output
+tensor, per instance and per time block t,
+    err = max|gpu - ref| / max( max|ref block|, 1e-6 * max over t of max|ref| ),
+and the reported figure is the maximum over instances and t.
+"""
+import numpy as np
+import torch
+
+from oracle import lqr_oracle as orc
+from paper_2603_09221_b200 import lqr
+
+
+def block_rel_err(gpu, ref, block_ndim):
+    """gpu/ref: [M, T, ...block...] (or [M, ...block...] when there is no time axis)."""
+    gpu = np.asarray(gpu, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    assert gpu.shape == ref.shape, (gpu.shape, ref.shape)
+    if gpu.ndim == 1 + block_ndim:
+        gpu, ref = gpu[:, None], ref[:, None]
+    M, T = ref.shape[:2]
+    g = gpu.reshape(M, T, -1)
+    r = ref.reshape(M, T, -1)
+    if not np.all(np.isfinite(g)):
+        return float("inf")
+    diff = np.abs(g - r).max(axis=2)
+    blk = np.abs(r).max(axis=2)
+    floor = 1e-6 * blk.max(axis=1, keepdims=True)
+    return float((diff / np.maximum(np.maximum(blk, floor), 1e-300)).max())
+
+
+def run_gpu(w, method=lqr.TTC_RICCATI, want=("K", "P", "x", "u", "info"), first_only=None, math=lqr.TTC_MATH_AUTO,
+            H=None, solver=None):
+    """Solve workload ``w`` (tensors already on the GPU) through the C ABI."""
+    n, m = w["n"], w["m"]
+    H = w["H"] if H is None else H
+    first_only = w["first_only"] if first_only is None else first_only
+    N = int(np.prod(w["batch"]))
+    dev = w["Q"].device
+    own = solver is None
+    if own:
+        solver = lqr.LqrSolver(n, m, H, w["batch"], device=dev.index or 0, method=method, math=math)
+    out = lqr.alloc_outputs(n, m, H, N, dev, first_only=first_only, want=want)
+    for v in out.values():
+        if v.dtype == torch.float32:
+            v.fill_(123456.0)          # canary: every element must be overwritten
+        else:
+            v.fill_(-7)
+    solver.solve(w["A"], w["B"], w["Q"], w["R"], w["x0"] if ("x" in want or "u" in want) else None, H,
+                 K=out.get("K"), P=out.get("P"), x=out.get("x"), u=out.get("u"), info=out.get("info"),
+                 flags=lqr.TTC_OUT_FIRST_ONLY if first_only else 0)
+    torch.cuda.synchronize(dev)
+    out["kernel"] = solver.query(lqr.TTC_QUERY_LAST_KERNEL)
+    out["launches"] = solver.query(lqr.TTC_QUERY_LAST_LAUNCHES)
+    if own:
+        solver.close()
+    return out
+
+
+def gather_inputs(w, idx):
+    """float64 numpy inputs of the instances ``idx`` (flat indices), one per row."""
+    S, Hd, T = w["batch"]
+    n, m = w["n"], w["m"]
+    idx_t = torch.as_tensor(idx, device=w["Q"].device, dtype=torch.long)
+
+    def sel(t, tail):
+        full = t.expand((S, Hd, T) + tuple(tail)).reshape((S * Hd * T,) + tuple(tail))
+        return full[idx_t].to(torch.float64).cpu().numpy()
+
+    return (sel(w["A"], (n, n)), sel(w["B"], (n, m)), sel(w["Q"], (n, n)), sel(w["R"], (m, m)), sel(w["x0"], (n,)))
+
+
+def run_oracle(w, idx=None, first_only=None, H=None, nthreads=0):
+    N = int(np.prod(w["batch"]))
+    if idx is None:
+        idx = np.arange(N)
+    A, B, Q, R, x0 = gather_inputs(w, idx)
+    H = w["H"] if H is None else H
+    first_only = w["first_only"] if first_only is None else first_only
+    return orc.solve_batch(A, B, Q, R, x0, H, batch=(len(idx),), first_only=first_only, nthreads=nthreads)
+
+
+def compare(gpu, ref, idx, tol, names=("K", "P", "x", "u")):
+    """Returns {name: err}; asserts every requested output is within tol and info == 0."""
+    n_dims = {"K": 2, "P": 2, "x": 1, "u": 1}
+    errs = {}
+    sel = torch.as_tensor(idx, dtype=torch.long)
+    for k in names:
+        if k not in gpu or k not in ref:
+            continue
+        g = gpu[k].cpu()[sel].numpy()
+        errs[k] = block_rel_err(g, ref[k], n_dims[k])
+    if "info" in gpu:
+        assert int(gpu["info"].cpu()[sel].abs().max()) == 0, "GPU reported failures on valid inputs"
+    assert int(np.abs(ref["info"]).max()) == 0
+    bad = {k: v for k, v in errs.items() if not (v <= tol)}
+    assert not bad, "relative error above %g: %s (all: %s)" % (tol, bad, errs)
+    return errs

@@ -1,0 +1,169 @@
+"""GPU parity: the CUDA library (through the C ABI) against the float64 oracle, element by element.
+
+Tolerances (relative, measure in parity_util.block_rel_err): 1e-4 when every input is fp32,
+2e-2 when Q and x0 are bf16 (the oracle reads the same rounded values).
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2603_09221_b200 import lqr, workloads
+from tests import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+METHODS = {"riccati": lqr.TTC_RICCATI, "scan": lqr.TTC_SCAN}
+
+
+def small_workload(n, m, H, batch, seed, bf16=False, rho=0.9):
+    """Generic-shape workload built from the same recipe as configuration 1."""
+    rng = np.random.default_rng(seed)
+    S, Hd, T = batch
+    sysm = [workloads._system(rng, n, m, rho) for _ in range(Hd)]
+    to = lambda k, shp: torch.from_numpy(np.stack([s[k] for s in sysm]).astype(np.float32).reshape((1, Hd, 1) + shp)).to(DEV)
+    g = torch.Generator(device=DEV)
+    g.manual_seed(seed)
+    L = torch.randn((S, Hd, T, n, n), generator=g, device=DEV)
+    Q = L @ L.transpose(-1, -2) / n + 0.1 * torch.eye(n, device=DEV)
+    Q = 0.5 * (Q + Q.transpose(-1, -2))
+    x0 = torch.randn((S, Hd, T, n), generator=g, device=DEV)
+    dt = torch.bfloat16 if bf16 else torch.float32
+    return dict(A=to(0, (n, n)), B=to(1, (n, m)), R=to(2, (m, m)), Q=Q.to(dt).contiguous(), x0=x0.to(dt).contiguous(),
+                n=n, m=m, H=H, batch=batch, first_only=False, tol=2e-2 if bf16 else 1e-4)
+
+
+SHAPES = [(1, 1, 1), (1, 1, 5), (2, 1, 3), (3, 2, 2), (5, 7, 4), (8, 8, 8), (12, 5, 9), (16, 16, 16), (17, 13, 6),
+          (32, 32, 12), (33, 20, 5), (64, 64, 4), (64, 48, 3), (48, 64, 3)]
+
+
+@pytest.mark.parametrize("method", ["riccati", "scan"])
+@pytest.mark.parametrize("n,m,H", SHAPES)
+def test_small_shapes_all_outputs(n, m, H, method):
+    w = small_workload(n, m, H, (2, 3, 5), seed=1000 + 17 * n + 3 * m + H)
+    gpu = pu.run_gpu(w, method=METHODS[method])
+    ref = pu.run_oracle(w)
+    pu.compare(gpu, ref, np.arange(30), 1e-4)
+    for k in ("K", "P", "x", "u"):
+        assert not torch.any(gpu[k] == 123456.0), "canary left in %s" % k
+
+
+@pytest.mark.parametrize("method", ["riccati", "scan"])
+@pytest.mark.parametrize("n,m,H", [(4, 3, 7), (16, 16, 9), (32, 32, 5), (64, 64, 3)])
+def test_first_only_and_partial_outputs(n, m, H, method):
+    w = small_workload(n, m, H, (1, 2, 7), seed=77 + n + H, bf16=True)
+    ref_full = pu.run_oracle(w, first_only=False)
+    ref_first = pu.run_oracle(w, first_only=True)
+    idx = np.arange(14)
+    g = pu.run_gpu(w, method=METHODS[method], want=("P", "u", "info"), first_only=True)
+    pu.compare(g, ref_first, idx, 2e-2)
+    g = pu.run_gpu(w, method=METHODS[method], want=("K", "P", "x", "u", "info"), first_only=True)
+    pu.compare(g, dict(ref_full, P=ref_first["P"], u=ref_first["u"]), idx, 2e-2)
+    g = pu.run_gpu(w, method=METHODS[method], want=("x", "u", "info"), first_only=False)   # K, P not requested
+    pu.compare(g, ref_full, idx, 2e-2)
+    g = pu.run_gpu(w, method=METHODS[method], want=("P",), first_only=False)
+    pu.compare(g, ref_full, idx, 2e-2)
+    g = pu.run_gpu(w, method=METHODS[method], want=("K", "info"), first_only=False)
+    pu.compare(g, ref_full, idx, 2e-2)
+
+
+@pytest.mark.parametrize("cfg", [0, 1])
+@pytest.mark.parametrize("method", ["riccati", "scan"])
+def test_config_full(cfg, method):
+    w = workloads.make_workload(cfg, device=DEV)
+    gpu = pu.run_gpu(w, method=METHODS[method])
+    ref = pu.run_oracle(w)
+    errs = pu.compare(gpu, ref, np.arange(int(np.prod(w["batch"]))), w["tol"])
+    print("cfg", cfg, method, errs)
+
+
+@pytest.mark.parametrize("cfg,tokens", [(2, 24), (3, 40), (4, 24)])
+@pytest.mark.parametrize("method", ["riccati", "scan"])
+def test_config_reduced_batch(cfg, tokens, method):
+    c = workloads.CONFIGS[cfg]
+    w = workloads.make_workload(cfg, device=DEV, batch=(c["batch"][0], c["batch"][1], tokens))
+    gpu = pu.run_gpu(w, method=METHODS[method])
+    ref = pu.run_oracle(w)
+    errs = pu.compare(gpu, ref, np.arange(int(np.prod(w["batch"]))), w["tol"])
+    print("cfg", cfg, method, errs)
+
+
+def test_horizon_below_max_and_handle_reuse():
+    w = small_workload(16, 16, 12, (1, 2, 9), seed=5)
+    s = lqr.LqrSolver(16, 16, 12, w["batch"], method=lqr.TTC_RICCATI)
+    for H in (12, 3, 1, 7):
+        gpu = pu.run_gpu(w, H=H, solver=s)
+        ref = pu.run_oracle(w, H=H)
+        pu.compare(gpu, ref, np.arange(18), 1e-4)
+    s.close()
+
+
+def test_per_instance_systems_and_strides():
+    # every instance its own A, B, R (configuration 0 layout) and a non-trivial token stride for Q
+    w = workloads.make_workload(0, device=DEV)
+    Qpad = torch.zeros((1, 1, 64, 2, 8, 8), device=DEV)
+    Qpad[:, :, :, 0] = w["Q"]
+    w["Q"] = Qpad[:, :, :, 0]            # token stride = 128 elements
+    gpu = pu.run_gpu(w)
+    ref = pu.run_oracle(w)
+    pu.compare(gpu, ref, np.arange(64), 1e-4)
+
+
+@pytest.mark.parametrize("method", ["riccati", "scan"])
+def test_not_positive_definite_instance_is_isolated(method):
+    w = small_workload(8, 8, 6, (1, 1, 6), seed=9)
+    R_ok = w["R"].expand(1, 1, 6, 8, 8).clone()
+    R = R_ok.clone()
+    R[0, 0, 2] = -10.0 * R[0, 0, 2]               # instance 2: R negative definite
+    Q = w["Q"].clone()
+    Q[0, 0, 4, 0, 0] = float("nan")               # instance 4: NaN input
+    w = dict(w, R=R.contiguous(), Q=Q)
+    gpu = pu.run_gpu(w, method=METHODS[method])
+    info = gpu["info"].cpu().numpy()
+    assert info[2] > 0 and info[4] > 0 and np.all(info[[0, 1, 3, 5]] == 0)
+    if method == "riccati":
+        assert info[2] == (6 - 1) * 8 + 1          # first step t = H-1, first pivot
+    for k in ("K", "P", "x", "u"):
+        assert torch.isnan(gpu[k][2]).all() and torch.isnan(gpu[k][4]).all()
+        assert torch.isfinite(gpu[k][[0, 1, 3, 5]]).all()
+    good = np.array([0, 1, 3, 5])
+    w_ok = dict(w, Q=torch.nan_to_num(Q, nan=1.0), R=R_ok)
+    ref = pu.run_oracle(dict(w_ok), idx=good)
+    gsel = {k: gpu[k] for k in ("K", "P", "x", "u")}
+    pu.compare(gsel, ref, good, 1e-4)
+
+
+def test_invalid_arguments_are_rejected():
+    w = small_workload(8, 8, 4, (1, 1, 4), seed=3)
+    with pytest.raises(lqr.TtcError):
+        lqr.LqrSolver(0, 8, 4, (1, 1, 4))
+    with pytest.raises(lqr.TtcError):
+        lqr.LqrSolver(8, 65, 4, (1, 1, 4))
+    with pytest.raises(lqr.TtcError):
+        lqr.LqrSolver(8, 8, 4, (1, 1, 4), math=lqr.TTC_MATH_TF32)
+    s = lqr.LqrSolver(8, 8, 4, (1, 1, 4))
+    out = lqr.alloc_outputs(8, 8, 4, 4, DEV)
+    with pytest.raises(lqr.TtcError):   # H above max_horizon
+        s.solve(w["A"], w["B"], w["Q"], w["R"], w["x0"], 5, **{k: out[k] for k in ("K", "P", "x", "u", "info")})
+    with pytest.raises(lqr.TtcError):   # H = 0
+        s.solve(w["A"], w["B"], w["Q"], w["R"], w["x0"], 0, P=out["P"])
+    with pytest.raises(lqr.TtcError):   # x0 missing while u requested
+        s.solve(w["A"], w["B"], w["Q"], w["R"], None, 4, u=out["u"])
+    with pytest.raises(lqr.TtcError):   # misaligned output
+        s.solve(w["A"], w["B"], w["Q"], w["R"], w["x0"], 4, P=out["P"].view(-1)[1:])
+    with pytest.raises(lqr.TtcError):   # bf16 A is not supported
+        s.solve(w["A"].to(torch.bfloat16), w["B"], w["Q"], w["R"], w["x0"], 4, P=out["P"])
+    s.solve(w["A"], w["B"], w["Q"], w["R"], w["x0"], 4, P=out["P"])     # still usable afterwards
+    torch.cuda.synchronize()
+    s.close()
+
+
+def test_host_buffer_entry_point_matches_device_entry_point():
+    w = small_workload(16, 16, 6, (1, 2, 11), seed=21, bf16=True)
+    gpu = pu.run_gpu(w)
+    s = lqr.LqrSolver(16, 16, 6, w["batch"])
+    host = {k: w[k].cpu() for k in ("A", "B", "Q", "R", "x0")}
+    out = lqr.alloc_outputs(16, 16, 6, 22, "cpu")
+    s.solve_host(host["A"], host["B"], host["Q"], host["R"], host["x0"], 6, **out)
+    s.close()
+    for k in ("K", "P", "x", "u", "info"):
+        assert torch.equal(out[k], gpu[k].cpu()), k
