@@ -153,6 +153,43 @@ int ttc_lqr_solve_host(ttc_lqr_handle* h,
                        float* K, float* P, float* x, float* u, int32_t* info,
                        uint32_t flags);
 
+/*
+ * Allocation-free variant of the P_0 / u_0 solve.  The paper has no counterpart: this entry
+ * point exists for callers that are not allowed to allocate device memory at the moment they
+ * need a solve -- code running inside a memory-pool or allocator callback, a plugin whose host
+ * framework owns every device allocation, or a real-time loop in which cudaMalloc (which may
+ * synchronise the whole device and take an unbounded time) is forbidden.  ttc_lqr_solve cannot
+ * serve them because its scan path keeps one value matrix per instance plus a status word in a
+ * workspace obtained with cudaMalloc.
+ *
+ * It computes, with the symplectic-pair scan (method TTC_SCAN, TTC_OUT_FIRST_ONLY), exactly what
+ *     ttc_lqr_solve(h, A, B, Q, R, x0, H, NULL, P0, NULL, u0, info, TTC_OUT_FIRST_ONLY, stream)
+ * computes on a TTC_SCAN handle of the same shape: P0 [N][n][n], u0 [N][m], info [N] (each may be
+ * NULL; x0 may be NULL when u0 is).  No handle is needed.  The scratch (one n x n value matrix and
+ * one int32 per instance) lives in a fixed array of TTC_NOALLOC_SCRATCH_BYTES bytes that is part
+ * of the library image: every GPU on which the library is loaded holds those bytes until the
+ * process exits.  The call makes no cudaMalloc / cudaFree and calls no allocating library
+ * routine; the caller still provides every input and output buffer.
+ *
+ * Limits and rules:
+ *  - N * (4*n*n) rounded up to 256, plus 4*N, must not exceed TTC_NOALLOC_SCRATCH_BYTES; larger
+ *    problems are rejected with TTC_STATUS_INVALID_ARGUMENT and a message naming both numbers
+ *    (nothing is enqueued).  Split the batch, or use ttc_lqr_solve.
+ *  - The first call on a device looks up the device address of the scratch array (once per
+ *    device, with that device current).  Make that first call before starting any stream
+ *    capture.
+ *  - Every call on a device shares the one array.  Nothing in it has to start at zero (each call
+ *    writes every word it later reads) and it keeps the previous call's contents.  Two calls
+ *    whose kernels can overlap on the GPU (different streams, or different host threads without
+ *    ordering) race on it: order them on one stream or with events.
+ * Errors otherwise as for ttc_lqr_solve.
+ */
+#define TTC_NOALLOC_SCRATCH_BYTES (4u << 20)
+int ttc_lqr_solve_first_noalloc(int32_t n, int32_t m, const int64_t batch[3], int32_t device,
+                                const ttc_operand* A, const ttc_operand* B, const ttc_operand* Q,
+                                const ttc_operand* R, const ttc_operand* x0, int32_t H,
+                                float* P0, float* u0, int32_t* info, void* cuda_stream);
+
 /* Free the handle and its workspace (synchronises the handle's device).  NULL is OK. */
 int ttc_lqr_destroy(ttc_lqr_handle* h);
 

@@ -5,6 +5,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "common.cuh"
@@ -386,3 +387,108 @@ int ttc_lqr_solve_host(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operan
 }
 
 } // extern "C"
+
+// ---------------------------------------------------------------------------------------------
+// Allocation-free P_0 / u_0 solve for callers that must not allocate device memory (allocator
+// callbacks, plugins whose host owns all device memory, real-time loops).  Same kernels as the
+// TTC_SCAN first-only path of ttc_lqr_solve; the per-instance scratch (P_1 and a status word)
+// sits in a fixed array inside the library image instead of a cudaMalloc'd workspace.
+// ---------------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_noalloc_scratch[TTC_NOALLOC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_noalloc_mutex;
+void* g_noalloc_dev_ptr[kMaxDevices] = {};   // device address of g_noalloc_scratch, per device ordinal
+int g_noalloc_sm_count[kMaxDevices] = {};
+
+// In host code `g_noalloc_scratch` is only a handle for the runtime, not a device address: the
+// address each device gave the array is looked up once per device, with that device current.
+int noalloc_scratch_for_device(int device, void** ptr, int* sm_count)
+{
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (!g_noalloc_dev_ptr[device]) {
+        void* p = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
+        if (e != cudaSuccess || !p)
+            return fail(TTC_STATUS_CUDA_ERROR, "cudaGetSymbolAddress(scratch) on device %d: %s", device,
+                        cudaGetErrorString(e));
+        int major = 0, sms = 0;
+        TTC_CUDA(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device));
+        TTC_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
+        if (major != 10)
+            return fail(TTC_STATUS_CUDA_ERROR, "device %d is not an sm_100 device", device);
+        g_noalloc_sm_count[device] = sms;
+        g_noalloc_dev_ptr[device] = p;
+    }
+    *ptr = g_noalloc_dev_ptr[device];
+    *sm_count = g_noalloc_sm_count[device];
+    return TTC_OK;
+}
+} // namespace
+
+extern "C" int ttc_lqr_solve_first_noalloc(int32_t n, int32_t m, const int64_t batch[3], int32_t device,
+                                           const ttc_operand* A, const ttc_operand* B, const ttc_operand* Q,
+                                           const ttc_operand* R, const ttc_operand* x0, int32_t H, float* P0,
+                                           float* u0, int32_t* info, void* cuda_stream)
+{
+    if (n < 1 || n > 64 || m < 1 || m > 64)
+        return fail(TTC_STATUS_INVALID_ARGUMENT, "n=%d, m=%d outside [1, 64]", n, m);
+    if (!batch)
+        return fail(TTC_STATUS_INVALID_ARGUMENT, "null batch");
+    if (H < 1 || H > 65536)
+        return fail(TTC_STATUS_INVALID_ARGUMENT, "H=%d outside [1, 65536]", H);
+    if (device < 0 || device >= kMaxDevices)
+        return fail(TTC_STATUS_INVALID_ARGUMENT, "device %d outside [0, %d)", device, kMaxDevices);
+    long long N = 1;
+    for (int d = 0; d < 3; ++d) {
+        if (batch[d] < 1 || batch[d] > (1ll << 31))
+            return fail(TTC_STATUS_INVALID_ARGUMENT, "batch[%d]=%lld out of range", d, (long long)batch[d]);
+        N *= batch[d];
+        if (N > (1ll << 31))
+            return fail(TTC_STATUS_INVALID_ARGUMENT, "more than 2^31 instances");
+    }
+    const size_t p1_bytes = ((size_t)N * n * n * sizeof(float) + 255) & ~(size_t)255;
+    const size_t need = p1_bytes + (size_t)N * sizeof(int);
+    if (need > (size_t)TTC_NOALLOC_SCRATCH_BYTES)
+        return fail(TTC_STATUS_INVALID_ARGUMENT,
+                    "allocation-free solve: %lld instances of n=%d need %zu bytes of scratch but the built-in "
+                    "array holds %u; split the batch or use ttc_lqr_solve",
+                    N, n, need, (unsigned)TTC_NOALLOC_SCRATCH_BYTES);
+    int s;
+    if ((s = check_operand("A", A, false, false))) return s;
+    if ((s = check_operand("B", B, false, false))) return s;
+    if ((s = check_operand("Q", Q, true, false))) return s;
+    if ((s = check_operand("R", R, false, false))) return s;
+    if ((s = check_operand("x0", x0, true, u0 == nullptr))) return s;
+    if (!P0 && !u0 && !info)
+        return fail(TTC_STATUS_INVALID_ARGUMENT, "no output requested");
+    const void* outs[3] = {P0, u0, info};
+    for (int i = 0; i < 3; ++i)
+        if (outs[i] && (reinterpret_cast<uintptr_t>(outs[i]) & 15u))
+            return fail(TTC_STATUS_INVALID_ARGUMENT, "an output pointer is not 16-byte aligned");
+    int ndev = 0;
+    TTC_CUDA(cudaGetDeviceCount(&ndev));
+    if (device >= ndev)
+        return fail(TTC_STATUS_CUDA_ERROR, "device %d not present (%d devices)", device, ndev);
+    TTC_CUDA(cudaSetDevice(device));
+    void* scratch = nullptr;
+    int sm_count = 0;
+    if ((s = noalloc_scratch_for_device(device, &scratch, &sm_count))) return s;
+
+    SolveParams p;
+    p.n = n; p.m = m; p.H = H;
+    p.b0 = batch[0]; p.b1 = batch[1]; p.b2 = batch[2]; p.N = N;
+    p.A = to_dev(A); p.B = to_dev(B); p.Q = to_dev(Q); p.R = to_dev(R); p.x0 = to_dev(x0);
+    p.K = nullptr; p.P = P0; p.x = nullptr; p.u = u0; p.info = info;
+    p.Kws = nullptr;
+    p.first_only = 1;
+    float* p1 = static_cast<float*>(scratch);
+    int* flags = reinterpret_cast<int*>(static_cast<unsigned char*>(scratch) + p1_bytes);
+    int launches = 0;
+    cudaError_t e = launch_scan_path(p, p1, flags, /*pfull=*/0, sm_count, static_cast<cudaStream_t>(cuda_stream),
+                                     &launches);
+    if (e != cudaSuccess)
+        return fail(TTC_STATUS_CUDA_ERROR, "allocation-free solve launch: %s", cudaGetErrorString(e));
+    return TTC_OK;
+}

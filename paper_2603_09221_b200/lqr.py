@@ -24,8 +24,9 @@ KERNEL_NAMES = {0: "none", 1: "riccati_cta", 2: "riccati_warp", 3: "riccati_mma"
 
 EXPORTS = (
     "ttc_lqr_create", "ttc_lqr_solve", "ttc_lqr_solve_host", "ttc_lqr_destroy", "ttc_lqr_query",
-    "ttc_lqr_status_string", "ttc_lqr_last_error",
+    "ttc_lqr_status_string", "ttc_lqr_last_error", "ttc_lqr_solve_first_noalloc",
 )
+TTC_NOALLOC_SCRATCH_BYTES = 4 << 20
 
 
 class ttc_operand(ctypes.Structure):
@@ -77,6 +78,9 @@ def load_library():
     lib.ttc_lqr_status_string.argtypes = [ctypes.c_int]
     lib.ttc_lqr_last_error.restype = ctypes.c_char_p
     lib.ttc_lqr_last_error.argtypes = []
+    lib.ttc_lqr_solve_first_noalloc.restype = ctypes.c_int
+    lib.ttc_lqr_solve_first_noalloc.argtypes = [ctypes.c_int32, ctypes.c_int32, P(ctypes.c_int64), ctypes.c_int32,
+                                                opp, opp, opp, opp, opp, ctypes.c_int32] + [ctypes.c_void_p] * 4
     _lib = lib
     return lib
 
@@ -199,3 +203,24 @@ def alloc_outputs(n, m, H, N, device, first_only=False, want=("K", "P", "x", "u"
     if "info" in want:
         out["info"] = torch.empty((N,), dtype=torch.int32, **kw)
     return out
+
+
+def solve_first_noalloc(A, B, Q, R, x0, H, batch, P0=None, u0=None, info=None, device=0, stream=None):
+    """``ttc_lqr_solve_first_noalloc``: P_0 / u_0 by the scan method without any device allocation
+    by the library -- for callers that may not allocate (allocator callbacks, hosts that own all
+    device memory, real-time loops).  The scratch is a fixed ``TTC_NOALLOC_SCRATCH_BYTES`` array
+    inside the library; problems that need more are rejected with ``TtcError``.  Calls share that
+    array, so do not let two of them overlap on the GPU."""
+    lib = load_library()
+    batch = tuple(int(b) for b in batch)
+    batch = (1,) * (3 - len(batch)) + batch
+    n, m = B.shape[-2], B.shape[-1]
+    ops = [_operand(A, 2, batch), _operand(B, 2, batch), _operand(Q, 2, batch), _operand(R, 2, batch),
+           _operand(x0, 1, batch)]
+    refs = [ctypes.byref(o) if o is not None else None for o in ops]
+    if stream is None:
+        stream = torch.cuda.current_stream(device)
+    barr = (ctypes.c_int64 * 3)(*batch)
+    ptr = LqrSolver._ptr
+    _check(lib.ttc_lqr_solve_first_noalloc(n, m, barr, device, *refs, int(H), ptr(P0), ptr(u0), ptr(info),
+                                           ctypes.c_void_p(stream.cuda_stream)))
