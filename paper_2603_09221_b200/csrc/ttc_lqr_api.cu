@@ -10,6 +10,7 @@
 
 #include "common.cuh"
 #include "riccati_cta.cuh"
+#include "riccati_mma64.cuh"
 #include "scan_pair.cuh"
 
 using namespace ttc;
@@ -301,6 +302,27 @@ int ttc_lqr_solve(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B,
         if (!K && rollout_needs_all_K) {
             if ((s = ensure(h->ws_K, sizeof(float) * (size_t)h->N * H * m * n))) return s;
             p.Kws = static_cast<float*>(h->ws_K.ptr);
+        }
+        const bool bf16_in = (Q->dtype == TTC_BF16) || (x0 && x0->ptr && x0->dtype == TTC_BF16);
+        const bool want_tf32 = h->cfg.math == TTC_MATH_TF32 || (h->cfg.math == TTC_MATH_AUTO && bf16_in);
+        const bool head_shared = A->bstride[2] == 0 && B->bstride[2] == 0 && R->bstride[2] == 0;
+        if (want_tf32 && n == 64 && m == 64 && head_shared) {
+            // tensor-core kernel: persistent CTAs, work items handed out by an atomic counter
+            if ((s = ensure(h->ws_E, sizeof(int) * 4))) return s;
+            int* counter = static_cast<int*>(h->ws_E.ptr);
+            TTC_CUDA(cudaMemsetAsync(counter, 0, sizeof(int), st));
+            const size_t smem = mma64::smem_bytes();
+            TTC_CUDA(cudaFuncSetAttribute(mma64::riccati_mma64_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          (int)smem));
+            const long long chunks = p.b0 * p.b1 * ((p.b2 + mma64::CHUNK - 1) / mma64::CHUNK);
+            long long grid = h->sm_count;
+            if (grid > chunks) grid = chunks;
+            mma64::riccati_mma64_kernel<<<(unsigned)grid, mma64::THREADS, smem, st>>>(p, counter);
+            TTC_CUDA(cudaGetLastError());
+            h->last_launches = 1;
+            h->last_kernel = TTC_KERNEL_RICCATI_MMA;
+            h->total_launches += h->last_launches;
+            return TTC_OK;
         }
         const size_t smem = riccati_cta_smem_bytes(n, m);
         TTC_CUDA(cudaFuncSetAttribute(riccati_cta_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
