@@ -170,6 +170,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--cpu-sample", type=int, default=256, help="instances the oracle is timed on")
     ap.add_argument("--ref-instances", type=int, default=256)
+    ap.add_argument("--tokens", type=int, default=0, help="override the token count (small profiling captures)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -193,8 +194,11 @@ def main():
     dev = torch.device("cuda", local)
     peaks = measured_peaks()
 
-    c = workloads.CONFIGS[cid]
-    w = workloads.make_workload(cid, device=dev, seed=workloads.SEED0 + cid + 1000 * rank)
+    c = dict(workloads.CONFIGS[cid])
+    if args.tokens > 0:
+        c["batch"] = (c["batch"][0], c["batch"][1], args.tokens)
+        c["name"] += "_tokens%d" % args.tokens
+    w = workloads.make_workload(cid, device=dev, batch=c["batch"], seed=workloads.SEED0 + cid + 1000 * rank)
     n, m, H = c["n"], c["m"], c["H"]
     N = int(np.prod(c["batch"]))
     first = c["first_only"]
