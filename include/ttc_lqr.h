@@ -71,6 +71,8 @@ extern "C" {
 #define TTC_QUERY_WORKSPACE_BYTES  2  /* device bytes currently owned by the handle    */
 #define TTC_QUERY_LAST_KERNEL      3  /* id of the main kernel of the last solve       */
 #define TTC_QUERY_TOTAL_LAUNCHES   4  /* kernels launched since create                 */
+#define TTC_QUERY_DEVICE_ERROR     5  /* 0, or non-zero if a bounded wait inside the last
+                                         kernel ran out (synchronises the device)       */
 
 /* ids returned by TTC_QUERY_LAST_KERNEL */
 #define TTC_KERNEL_NONE           0
@@ -78,6 +80,7 @@ extern "C" {
 #define TTC_KERNEL_RICCATI_WARP   2  /* register-tiled FFMA, several instances per CTA */
 #define TTC_KERNEL_RICCATI_MMA    3  /* tensor-core contractions, n = m = 64           */
 #define TTC_KERNEL_SCAN           4  /* symplectic-pair scan + gain/rollout kernel     */
+#define TTC_KERNEL_RICCATI_UMMA   5  /* tcgen05 contractions (tensor memory), n = m = 64 */
 
 typedef struct ttc_lqr_handle ttc_lqr_handle; /* opaque; owned by the library */
 

@@ -1,0 +1,742 @@
+// Riccati-backward kernel for n = m = 64 on the 5th-generation tensor cores (tcgen05.mma,
+// kind::tf32, fp32 accumulators in tensor memory).
+//
+// One persistent CTA per SM, 256 threads = 2 warpgroups.  A warpgroup owns a PAIR of instances
+// (a, b) of one head at a time and walks their horizon together; the two warpgroups are
+// independent (own operands, own barriers, own half of tensor memory), so the tensor pipe works
+// for one pair while the other pair is in its factorisation.
+//
+// Per step (Prop. 3.1), with P symmetric and the per-head operand BA = [B'; A'] (128 x 64):
+//   (1)  W  = BA * [P_a P_b]          -> W_x = [V_x'; T_x'] = [(P_x B)'; (P_x A)']        SS, M128 N128
+//   (2x) F_x  = W_x * B  = [S_x - R ; Y_x']   DP_x = W_x * A = [ . ; A'P_x A]              TS (A operand
+//        read from tensor memory, no round trip through shared memory), N64 each
+//   S_x = R + (S_x - R) -> shared, fp32;  Linv_x = chol(S_x)^{-1}   2 warps per instance, blocked:
+//        32 x 32 diagonal blocks in registers (one row per lane), off-diagonal work as 3 x tf32
+//        (error-compensated) mma.sync products
+//   (4)  Z' = [Y_a'; Y_b'] * [Linv_a' Linv_b']   (diagonal blocks Z_a', Z_b')              SS, M128 N128
+//   (5x) DP_x -= Z_x' Z_x                                                                   SS, N64
+//   P_x <- Q_x + DP_x            (P_t = Q + A'P A - Y'S^{-1}Y)
+// Tensor-memory map of a warpgroup (256 columns): R0 = W_a then DP_b, R1 = W_b, R2 = F_a then F_b,
+// R3 = DP_a; Z' reuses R1|R2.
+//
+// Shared-memory operands use the canonical K-major layout without swizzle: 8 x 4 (rows x k) core
+// matrices of 128 contiguous bytes, chunk stride 128 B along k, 2048 B between 8-row groups.  A row
+// owner writes its row with conflict-free 16-byte stores.
+//
+// Every wait on an MMA-completion barrier is bounded; on a timeout the warpgroup records an error,
+// stops taking work and the kernel still releases tensor memory before it returns.
+#pragma once
+
+#include "common.cuh"
+
+namespace ttc {
+namespace umma64 {
+
+constexpr int N = 64;
+constexpr int WG_THREADS = 128;
+constexpr int NUM_WG = 2;
+constexpr int THREADS = NUM_WG * WG_THREADS;
+constexpr int CHUNK = 16;                       // tokens per work item (8 pairs)
+constexpr uint32_t SC = 128;                    // bytes between consecutive 4-wide k chunks
+constexpr uint32_t SR = 2048;                   // bytes between 8-row groups (16 chunks)
+constexpr uint32_t MAT_BYTES = 8 * SR;          // one 64 x 64 matrix
+constexpr uint32_t BUF_BYTES = 2 * MAT_BYTES;   // 128 rows
+constexpr int SPIN_LIMIT = 1 << 22;
+
+// per-warpgroup shared memory: BA | X0 | X1 (X0 and X1 adjacent: step (5a) starts its A operand
+// 64 rows before X1) followed by small scratch.
+constexpr uint32_t OFF_BA = 0;
+constexpr uint32_t OFF_X0 = BUF_BYTES;
+constexpr uint32_t OFF_X1 = 2 * BUF_BYTES;
+constexpr uint32_t OFF_MISC = 3 * BUF_BYTES;
+struct Misc {
+    unsigned long long mbar;     // MMA completion barrier
+    int chunk;                   // current work item
+    int dead;                    // set when a wait timed out
+    int flag[2];                 // first failed pivot per instance (0 = none)
+    float x0[2][N];
+    float y0[2][N];
+    float v[2][N];
+};
+constexpr uint32_t WG_BYTES = OFF_MISC + ((sizeof(Misc) + 127) / 128) * 128;
+constexpr uint32_t SMEM_BYTES = NUM_WG * WG_BYTES + 128;     // + slot for the tensor-memory base address
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+// byte offset of element (r, c) of a row-major matrix stored as 8 x 4 core matrices
+__device__ __forceinline__ uint32_t toff(int r, int c)
+{
+    return (uint32_t)(r >> 3) * SR + (uint32_t)(c >> 2) * SC + (uint32_t)(r & 7) * 16u + (uint32_t)(c & 3) * 4u;
+}
+// private layout of a 32 x 32 scratch inside the (rows 0..31, cols 32..63) block of a matrix: element (i, c)
+// sits in core matrix (i/8, 8 + i%8) at row (c/4) ^ (i%8); conflict-free for "lane = c" 4-byte accesses and
+// for "lane = i" 16-byte accesses.
+__device__ __forceinline__ uint32_t soff(int i, int c)
+{
+    return (uint32_t)(i >> 3) * SR + (uint32_t)(8 + (i & 7)) * SC + (uint32_t)(((c >> 2) ^ i) & 7) * 16u + (uint32_t)(c & 3) * 4u;
+}
+__device__ __forceinline__ float& elem(unsigned char* base, uint32_t off) { return *reinterpret_cast<float*>(base + off); }
+
+__device__ __forceinline__ uint32_t to_tf32(float x)
+{
+    uint32_t r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+    return r;
+}
+__device__ __forceinline__ float round_tf32(float x) { return __uint_as_float(to_tf32(x)); }
+
+// ---- tcgen05 wrappers ---------------------------------------------------------------------------------
+// shared-memory matrix descriptor: K-major, no swizzle; `saddr` = address of the first core matrix of
+// this k step (a k step of 8 tf32 values spans 2 chunks)
+__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr)
+{
+    return (uint64_t)((saddr >> 4) & 0x3FFFu) | ((uint64_t)(SC >> 4) << 16) | ((uint64_t)(SR >> 4) << 32) |
+           ((uint64_t)1 << 46);
+}
+// instruction descriptor: tf32 x tf32 -> f32, both operands K-major, M = 128
+__device__ __forceinline__ uint32_t instr_desc(int ncols, int negate_a)
+{
+    return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)negate_a << 13) | ((uint32_t)(ncols >> 3) << 17) |
+           ((uint32_t)(128 >> 4) << 24);
+}
+__device__ __forceinline__ void mma_ss(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}\n"
+                 :: "r"(d), "l"(a), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void mma_ts(uint32_t d, uint32_t a_tmem, uint64_t b, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, p;\n\t}\n"
+                 :: "r"(d), "r"(a_tmem), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
+}
+// D (128 x ncols) (+)= A (smem, 128 x 64) * B' (smem, ncols x 64), 8 k steps
+__device__ __forceinline__ void gemm_ss(uint32_t d, uint32_t a_smem, uint32_t b_smem, int ncols, int negate_a, bool accumulate)
+{
+    const uint32_t id = instr_desc(ncols, negate_a);
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+        mma_ss(d, smem_desc(a_smem + 2 * j * SC), smem_desc(b_smem + 2 * j * SC), id, (accumulate || j > 0) ? 1u : 0u);
+}
+// D (128 x ncols) = A (tensor memory, 128 lanes x 64 columns) * B' (smem, ncols x 64)
+__device__ __forceinline__ void gemm_ts(uint32_t d, uint32_t a_tmem, uint32_t b_smem, int ncols)
+{
+    const uint32_t id = instr_desc(ncols, 0);
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+        mma_ts(d, a_tmem + 8 * j, smem_desc(b_smem + 2 * j * SC), id, j > 0 ? 1u : 0u);
+}
+__device__ __forceinline__ void mma_commit(uint32_t mbar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(mbar) : "memory");
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t mbar, uint32_t parity)
+{
+    for (int it = 0; it < SPIN_LIMIT; ++it) {
+        uint32_t ok;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
+                     : "=r"(ok) : "r"(mbar), "r"(parity) : "memory");
+        if (ok)
+            return true;
+    }
+    return false;
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void async_proxy_fence() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// 32 lanes x 32 consecutive columns of tensor memory -> 32 registers per thread (lane = row)
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32])
+{
+    uint32_t r[32];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                 "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                   "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                   "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                 : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i)
+        v[i] = __uint_as_float(r[i]);
+}
+
+__device__ __forceinline__ void wg_barrier(int wg) { asm volatile("bar.sync %0, %1;" :: "r"(1 + wg), "r"(WG_THREADS) : "memory"); }
+__device__ __forceinline__ void pair_barrier(int wg, int x) { asm volatile("bar.sync %0, %1;" :: "r"(3 + 2 * wg + x), "r"(64) : "memory"); }
+
+// ---- warp-level 32 x 32 Cholesky, one row per lane -----------------------------------------------------------
+// s[c] = row `lane` of an SPD block.  On return s holds row `lane` of L (entries right of the diagonal are
+// meaningless) and rs_own = 1 / L[lane][lane].  The update of the trailing rows uses s_ij * s_cj / d_j, so
+// that the broadcast of column j does not wait for the reciprocal.  Returns 0 or 1 + the first bad pivot.
+__device__ __forceinline__ int warp_chol32(float (&s)[32], float& rs_own, int lane)
+{
+    int bad = 0;
+    rs_own = 1.f;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+        float d = __shfl_sync(0xffffffffu, s[j], j);
+        const float sj = s[j];
+        if (!(d > 0.f)) {
+            if (!bad)
+                bad = j + 1;
+            d = 1.f;
+        }
+        const float rinv = __frcp_rn(d);
+        const float f = sj * rinv;
+#pragma unroll
+        for (int c = j + 1; c < 32; ++c) {
+            const float lc = __shfl_sync(0xffffffffu, sj, c);
+            s[c] = fmaf(-f, lc, s[c]);
+        }
+        const float rs = rsqrtf(d);
+        s[j] = sj * rs;
+        if (lane == j)
+            rs_own = rs;
+    }
+    return bad;
+}
+
+// Lt(k, i) = L[i][k] in the private scratch layout of `scr`.  Lane c computes column c of L^{-1}:
+// x[i] = Linv[i][c] (0 for i < c).
+__device__ __forceinline__ void warp_trinv32(float (&x)[32], unsigned char* scr, float rs_own, int lane)
+{
+    float a[32];
+#pragma unroll
+    for (int i = 0; i < 32; ++i)
+        a[i] = 0.f;
+#pragma unroll
+    for (int k = 0; k < 32; ++k) {
+        const float rsk = __shfl_sync(0xffffffffu, rs_own, k);
+        const float xk = (k == lane) ? rsk : ((k > lane) ? -a[k] * rsk : 0.f);
+        x[k] = xk;
+#pragma unroll
+        for (int i4 = (k + 1) & ~3; i4 < 32; i4 += 4) {
+            const float4 l4 = *reinterpret_cast<const float4*>(scr + soff(k, i4));
+            if (i4 + 0 > k) a[i4 + 0] = fmaf(l4.x, xk, a[i4 + 0]);
+            if (i4 + 1 > k) a[i4 + 1] = fmaf(l4.y, xk, a[i4 + 1]);
+            if (i4 + 2 > k) a[i4 + 2] = fmaf(l4.z, xk, a[i4 + 2]);
+            if (i4 + 3 > k) a[i4 + 3] = fmaf(l4.w, xk, a[i4 + 3]);
+        }
+    }
+}
+
+// One warp: factor the 32 x 32 SPD diagonal block (d0, d0) of the matrix at `M` and overwrite it with the
+// inverse of its Cholesky factor (lower triangular, zeros above the diagonal).  Scratch: block (0, 1) of M.
+__device__ __forceinline__ int warp_factor_block(unsigned char* M, int d0, int lane)
+{
+    float s[32];
+#pragma unroll
+    for (int c = 0; c < 32; c += 4) {
+        const float4 v = *reinterpret_cast<const float4*>(M + toff(d0 + lane, d0 + c));
+        s[c] = v.x; s[c + 1] = v.y; s[c + 2] = v.z; s[c + 3] = v.w;
+    }
+    float rs_own;
+    const int bad = warp_chol32(s, rs_own, lane);
+#pragma unroll
+    for (int k = 0; k < 32; ++k)
+        elem(M, soff(k, lane)) = s[k];                  // Lt(k, i = lane) = L[i][k]
+    __syncwarp();
+    float x[32];
+    warp_trinv32(x, M, rs_own, lane);
+    __syncwarp();
+#pragma unroll
+    for (int i = 0; i < 32; ++i)
+        elem(M, soff(i, lane)) = x[i];                  // bounce: column owner -> row owner
+    __syncwarp();
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+        const float4 v = *reinterpret_cast<const float4*>(M + soff(lane, 4 * q));
+        *reinterpret_cast<float4*>(M + toff(d0 + lane, d0 + 4 * q)) = v;
+    }
+    __syncwarp();
+    return bad;
+}
+
+// ---- 3 x tf32 warp-level products on 16 x 32 tiles (fp32-grade accuracy) ---------------------------------------
+__device__ __forceinline__ void mma_16x8x8(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                           uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+                 "{%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void split_tf32(float x, uint32_t& hi, uint32_t& lo)
+{
+    hi = to_tf32(x);
+    lo = to_tf32(x - __uint_as_float(hi));
+}
+// acc[nt] (16 x 8 tiles, nt = 0..3) += sign * A(16 x 32) * B(32 x 32).  A(r, k) is read at M + toff(ar + r, ac + k).
+// B(k, n) is read at M + toff(br + n, bc + k) when BT (B given by its transpose, row n contiguous in k), else at
+// M + toff(br + k, bc + n).  K tiles outside [ktlo(nt), kthi(nt)] are skipped (triangular operands).
+template <bool NEG, bool BT, class KLo, class KHi>
+__device__ __forceinline__ void mma3x_16x32x32(float (&acc)[4][4], const unsigned char* M, int ar, int ac, int br, int bc,
+                                               int g, int t, KLo ktlo, KHi kthi)
+{
+#pragma unroll
+    for (int kt = 0; kt < 4; ++kt) {
+        float a[4];
+        a[0] = *reinterpret_cast<const float*>(M + toff(ar + g, ac + 8 * kt + t));
+        a[1] = *reinterpret_cast<const float*>(M + toff(ar + g + 8, ac + 8 * kt + t));
+        a[2] = *reinterpret_cast<const float*>(M + toff(ar + g, ac + 8 * kt + t + 4));
+        a[3] = *reinterpret_cast<const float*>(M + toff(ar + g + 8, ac + 8 * kt + t + 4));
+        uint32_t ah[4], al[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            split_tf32(NEG ? -a[e] : a[e], ah[e], al[e]);
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) {
+            if (kt < ktlo(nt) || kt > kthi(nt))
+                continue;
+            float b0, b1;
+            if (BT) {
+                b0 = *reinterpret_cast<const float*>(M + toff(br + 8 * nt + g, bc + 8 * kt + t));
+                b1 = *reinterpret_cast<const float*>(M + toff(br + 8 * nt + g, bc + 8 * kt + t + 4));
+            } else {
+                b0 = *reinterpret_cast<const float*>(M + toff(br + 8 * kt + t, bc + 8 * nt + g));
+                b1 = *reinterpret_cast<const float*>(M + toff(br + 8 * kt + t + 4, bc + 8 * nt + g));
+            }
+            uint32_t bh0, bl0, bh1, bl1;
+            split_tf32(b0, bh0, bl0);
+            split_tf32(b1, bh1, bl1);
+            mma_16x8x8(acc[nt], al[0], al[1], al[2], al[3], bh0, bh1);
+            mma_16x8x8(acc[nt], ah[0], ah[1], ah[2], ah[3], bl0, bl1);
+            mma_16x8x8(acc[nt], ah[0], ah[1], ah[2], ah[3], bh0, bh1);
+        }
+    }
+}
+__device__ __forceinline__ void zero4x4(float (&acc)[4][4])
+{
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            acc[nt][e] = 0.f;
+}
+// accumulator tiles <-> rows r0 + g, r0 + g + 8 ; columns c0 + 8 nt + 2t, +1
+template <bool ROUND>
+__device__ __forceinline__ void store_tiles(unsigned char* M, int r0, int c0, const float (&acc)[4][4], int g, int t)
+{
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt) {
+        const int c = c0 + 8 * nt + 2 * t;
+        float2 lo = make_float2(acc[nt][0], acc[nt][1]), hi = make_float2(acc[nt][2], acc[nt][3]);
+        if (ROUND) {
+            lo.x = round_tf32(lo.x); lo.y = round_tf32(lo.y); hi.x = round_tf32(hi.x); hi.y = round_tf32(hi.y);
+        }
+        *reinterpret_cast<float2*>(M + toff(r0 + g, c)) = lo;
+        *reinterpret_cast<float2*>(M + toff(r0 + g + 8, c)) = hi;
+    }
+}
+__device__ __forceinline__ void load_tiles(float (&acc)[4][4], const unsigned char* M, int r0, int c0, int g, int t)
+{
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt) {
+        const int c = c0 + 8 * nt + 2 * t;
+        const float2 lo = *reinterpret_cast<const float2*>(M + toff(r0 + g, c));
+        const float2 hi = *reinterpret_cast<const float2*>(M + toff(r0 + g + 8, c));
+        acc[nt][0] = lo.x; acc[nt][1] = lo.y; acc[nt][2] = hi.x; acc[nt][3] = hi.y;
+    }
+}
+
+// Two warps (pw = 0, 1; 64 threads) replace the SPD matrix S at `M` (fp32, core-matrix layout) by
+// Linv = chol(S)^{-1}: lower triangle fp32 values rounded to tf32, zeros above the diagonal.
+// 2 x 2 blocks of 32:  Linv11 = chol(S11)^{-1};  L21 = S21 Linv11';  S22 -= L21 L21';  W = L21 Linv11;
+// Linv22 = chol(S22)^{-1};  Linv21 = -Linv22 W.   A non-positive pivot is recorded in *flag as code0 + index.
+__device__ __forceinline__ void pair_factor_invert(unsigned char* M, int wg, int x, int pw, int lane, int* flag, int code0)
+{
+    const int g = lane >> 2, t = lane & 3;
+    const int r0 = 32 + 16 * pw;                       // the 16 rows of the lower half owned by this warp
+    if (pw == 0) {
+        const int bad = warp_factor_block(M, 0, lane);
+        if (bad && lane == 0 && *flag == 0)
+            *flag = code0 + bad;
+    }
+    pair_barrier(wg, x);
+    float acc[4][4];
+    // L21 = S21 Linv11'   (Linv11[n][k] = 0 for k > n)
+    zero4x4(acc);
+    mma3x_16x32x32<false, true>(acc, M, r0, 0, 0, 0, g, t, [](int) { return 0; }, [](int nt) { return nt; });
+    __syncwarp();
+    store_tiles<false>(M, r0, 0, acc, g, t);
+    pair_barrier(wg, x);
+    // S22 -= L21 L21'
+    load_tiles(acc, M, r0, 32, g, t);
+    mma3x_16x32x32<true, true>(acc, M, r0, 0, 32, 0, g, t, [](int) { return 0; }, [](int) { return 3; });
+    store_tiles<false>(M, r0, 32, acc, g, t);
+    pair_barrier(wg, x);
+    // W = L21 Linv11 over the own rows   (Linv11[k][n] = 0 for k < n)
+    zero4x4(acc);
+    mma3x_16x32x32<false, false>(acc, M, r0, 0, 0, 0, g, t, [](int nt) { return nt; }, [](int) { return 3; });
+    __syncwarp();
+    store_tiles<false>(M, r0, 0, acc, g, t);
+    if (pw == 1) {
+        const int bad = warp_factor_block(M, 32, lane);
+        if (bad && lane == 0 && *flag == 0)
+            *flag = code0 + 32 + bad;
+    }
+    pair_barrier(wg, x);
+    // Linv21 = -Linv22 W     (Linv22[r][k] = 0 for k > r)
+    zero4x4(acc);
+    {
+        const int kmax = (r0 - 32 + 15) >> 3;
+        mma3x_16x32x32<true, false>(acc, M, r0, 32, 32, 0, g, t, [](int) { return 0; }, [kmax](int) { return kmax; });
+    }
+    pair_barrier(wg, x);                               // every read of W is done
+    store_tiles<true>(M, r0, 0, acc, g, t);
+    // round the diagonal blocks to tf32 in place and clear block (0, 1) (scratch until now)
+    {
+        const int d0 = 32 * pw;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            float4 v = *reinterpret_cast<float4*>(M + toff(d0 + lane, d0 + 4 * q));
+            v.x = round_tf32(v.x); v.y = round_tf32(v.y); v.z = round_tf32(v.z); v.w = round_tf32(v.w);
+            *reinterpret_cast<float4*>(M + toff(d0 + lane, d0 + 4 * q)) = v;
+        }
+        if (pw == 0) {
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                *reinterpret_cast<float4*>(M + toff(lane, 32 + 4 * q)) = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+    }
+}
+
+// ---- global-memory helpers --------------------------------------------------------------------------------------
+// row j (64 values) of the Q matrix of one instance
+__device__ __forceinline__ void load_q_row(float (&q)[64], const OperandDev& Q, long long oq, int j)
+{
+    if (Q.dtype == TTC_BF16) {
+        const uint4* src = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(Q.ptr) + oq + (long long)j * N);
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            const uint4 v = __ldg(src + c);
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                q[8 * c + 2 * e] = __uint_as_float(w[e] << 16);
+                q[8 * c + 2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u);
+            }
+        }
+    } else {
+        const float4* src = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(Q.ptr) + oq + (long long)j * N);
+#pragma unroll
+        for (int c = 0; c < 16; ++c) {
+            const float4 v = __ldg(src + c);
+            q[4 * c] = v.x; q[4 * c + 1] = v.y; q[4 * c + 2] = v.z; q[4 * c + 3] = v.w;
+        }
+    }
+}
+// row `r` of a 128-row operand buffer <- 64 values rounded to tf32
+__device__ __forceinline__ void store_row_tf32(unsigned char* buf, int r, const float (&v)[64])
+{
+#pragma unroll
+    for (int c = 0; c < 16; ++c)
+        *reinterpret_cast<float4*>(buf + toff(r, 4 * c)) =
+            make_float4(round_tf32(v[4 * c]), round_tf32(v[4 * c + 1]), round_tf32(v[4 * c + 2]), round_tf32(v[4 * c + 3]));
+}
+__device__ __forceinline__ void store_row_global(float* dst, const float (&v)[64])
+{
+#pragma unroll
+    for (int c = 0; c < 16; ++c)
+        reinterpret_cast<float4*>(dst)[c] = make_float4(v[4 * c], v[4 * c + 1], v[4 * c + 2], v[4 * c + 3]);
+}
+
+__device__ __forceinline__ void wg_fail_instance(const SolveParams& p, long long inst, int code, int wt)
+{
+    const float qn = quiet_nan();
+    if (p.P) {
+        const long long cnt = (long long)(p.first_only ? 1 : p.H + 1) * N * N;
+        for (long long e = wt; e < cnt; e += WG_THREADS)
+            p.P[inst * cnt + e] = qn;
+    }
+    if (p.u && p.first_only && wt < N)
+        p.u[inst * (long long)N + wt] = qn;
+    if (p.info && wt == 0)
+        p.info[inst] = code;
+}
+
+// Supported requests: P (every P_t, or P_0 with first_only), u_0 (first_only), info.  K, x and the full u
+// are served by other kernels.
+__global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams p, int* chunk_counter, int* error_flag)
+{
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    const int tid = threadIdx.x;
+    const int wg = tid / WG_THREADS;
+    const int wt = tid % WG_THREADS;
+    const int warp = wt >> 5;                  // warp in warpgroup: owns tensor-memory lanes 32 warp .. 32 warp + 31
+    const int lane = wt & 31;
+    unsigned char* wsm = smem_raw + (size_t)wg * WG_BYTES;
+    unsigned char* BA = wsm + OFF_BA;          // rows 0..63: B' (row j = column j of B), rows 64..127: A'
+    unsigned char* X0 = wsm + OFF_X0;          // [P_a; P_b] -> [Y_a'; Y_b'] -> next [P_a; P_b]
+    unsigned char* X1 = wsm + OFF_X1;          // [S_a; S_b] -> [Linv_a; Linv_b] -> [Z_a'; Z_b']
+    Misc& misc = *reinterpret_cast<Misc*>(wsm + OFF_MISC);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_raw + (size_t)NUM_WG * WG_BYTES);
+    const uint32_t mbar = smem_u32(&misc.mbar);
+
+    if (wt == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(mbar) : "memory");
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        misc.dead = 0;
+    }
+    if (tid < 32) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(smem_u32(tmem_slot)), "r"(512) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tm = *tmem_slot + 256u * wg;
+    const uint32_t R0 = tm, R1 = tm + 64, R2 = tm + 128, R3 = tm + 192;
+    const uint32_t lane_sel = (uint32_t)(32 * warp) << 16;
+    uint32_t parity = 0;
+
+    const int H = p.H;
+    const long long chunks_per_head = (p.b2 + CHUNK - 1) / CHUNK;
+    const long long nchunks = p.b0 * p.b1 * chunks_per_head;
+    const bool want_u0 = (p.u != nullptr) && p.first_only;
+    long long offA_loaded = -1, offB_loaded = -1, offR_loaded = -1;
+    const float* Rg = nullptr;
+    bool dead = false;
+
+    // wait for the MMAs committed last; a timeout marks the warpgroup dead (checked after the next barrier)
+    auto wait_mma = [&]() {
+        if (!mbar_wait(mbar, parity)) {
+            misc.dead = 1;
+            atomicExch(error_flag, 1);
+        }
+        parity ^= 1u;
+        tc_fence_after();
+    };
+
+    while (!dead) {
+        if (wt == 0)
+            misc.chunk = atomicAdd(chunk_counter, 1);
+        wg_barrier(wg);
+        const long long chunk = misc.chunk;
+        if (chunk >= nchunks)
+            break;
+        const long long head = chunk / chunks_per_head;
+        const long long tok0 = (chunk % chunks_per_head) * CHUNK;
+        const long long inst0 = head * p.b2 + tok0;
+        const int ntok = (int)min((long long)CHUNK, p.b2 - tok0);
+        {
+            const long long oa = operand_offset(p.A, inst0, p.b1, p.b2);
+            const long long ob = operand_offset(p.B, inst0, p.b1, p.b2);
+            const long long orr = operand_offset(p.R, inst0, p.b1, p.b2);
+            if (oa != offA_loaded || ob != offB_loaded) {
+                const float* Ag = reinterpret_cast<const float*>(p.A.ptr) + oa;
+                const float* Bg = reinterpret_cast<const float*>(p.B.ptr) + ob;
+                for (int e = wt; e < N * N; e += WG_THREADS) {
+                    const int k = e >> 6, j = e & 63;
+                    elem(BA, toff(j, k)) = round_tf32(__ldg(Bg + e));
+                    elem(BA, toff(64 + j, k)) = round_tf32(__ldg(Ag + e));
+                }
+                offA_loaded = oa; offB_loaded = ob;
+            }
+            offR_loaded = orr;
+            Rg = reinterpret_cast<const float*>(p.R.ptr) + orr;
+        }
+
+        for (int tk = 0; tk < ntok && !dead; tk += 2) {
+            const long long inst_x[2] = {inst0 + tk, inst0 + min(tk + 1, ntok - 1)};
+            const bool valid_b = tk + 1 < ntok;
+            const long long oq_x[2] = {operand_offset(p.Q, inst_x[0], p.b1, p.b2), operand_offset(p.Q, inst_x[1], p.b1, p.b2)};
+            // ---- P_H = Q: warps 2, 3 own the rows of the value matrices
+            if (warp >= 2) {
+                const int j = wt - 64;
+#pragma unroll 1
+                for (int x = 0; x < 2; ++x) {
+                    float q[64];
+                    load_q_row(q, p.Q, oq_x[x], j);
+                    store_row_tf32(X0, 64 * x + j, q);
+                    if (p.P && !p.first_only && (x == 0 || valid_b))
+                        store_row_global(p.P + (inst_x[x] * (long long)(H + 1) + H) * N * N + (long long)j * N, q);
+                }
+            } else if (want_u0) {
+                const int x = warp, j0 = 2 * lane;             // warp x stages x_0 of instance x
+                const long long ox = operand_offset(p.x0, inst_x[x], p.b1, p.b2);
+                misc.x0[x][j0] = load_elem(p.x0, ox + j0);
+                misc.x0[x][j0 + 1] = load_elem(p.x0, ox + j0 + 1);
+            }
+            if (wt < 2)
+                misc.flag[wt] = 0;
+            async_proxy_fence();
+            wg_barrier(wg);
+
+            for (int ts = H - 1; ts >= 0 && !dead; --ts) {
+                // (1) W = BA [P_a P_b]' -> R0|R1 ; (2a) F_a -> R2, DP_a -> R3
+                if (wt == 0) {
+                    tc_fence_after();
+                    gemm_ss(R0, smem_u32(BA), smem_u32(X0), 128, 0, false);
+                    gemm_ts(R2, R0, smem_u32(BA), 64);
+                    gemm_ts(R3, R0, smem_u32(BA) + MAT_BYTES, 64);
+                    mma_commit(mbar);
+                }
+                // operands that do not depend on the MMA: R row (warps 0, 1)
+                float rrow[64];
+                if (warp < 2) {
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) {
+                        const float4 v = __ldg(reinterpret_cast<const float4*>(Rg + (long long)wt * N) + c);
+                        rrow[4 * c] = v.x; rrow[4 * c + 1] = v.y; rrow[4 * c + 2] = v.z; rrow[4 * c + 3] = v.w;
+                    }
+                }
+                wait_mma();
+                // (2b) back half first: DP_b -> R0 (W_a is dead), runs while F_a is read out
+                if (wt == 0)
+                    gemm_ts(R0, R1, smem_u32(BA) + MAT_BYTES, 64);
+#pragma unroll 1
+                for (int x = 0; x < 2; ++x) {
+                    if (x == 1) {
+                        wait_mma();
+                    }
+                    float f[64];
+                    {
+                        float h0[32], h1[32];
+                        tmem_ld32(R2 + lane_sel, h0);
+                        tmem_ld32(R2 + lane_sel + 32, h1);
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) {
+                            f[c] = h0[c];
+                            f[32 + c] = h1[c];
+                        }
+                    }
+                    if (warp < 2) {                    // S_x = R + B'P_x B, fp32 -> X1
+#pragma unroll
+                        for (int c = 0; c < 16; ++c)
+                            *reinterpret_cast<float4*>(X1 + x * MAT_BYTES + toff(wt, 4 * c)) =
+                                make_float4(f[4 * c] + rrow[4 * c], f[4 * c + 1] + rrow[4 * c + 1],
+                                            f[4 * c + 2] + rrow[4 * c + 2], f[4 * c + 3] + rrow[4 * c + 3]);
+                    } else {                           // Y_x' -> X0 (P is dead once (1) has completed)
+                        store_row_tf32(X0, 64 * x + (wt - 64), f);
+                    }
+                    tc_fence_before();
+                    wg_barrier(wg);
+                    dead = misc.dead != 0;
+                    if (x == 0 && wt == 0) {           // F_a has been read by every warp: (2b) front half -> R2
+                        tc_fence_after();
+                        gemm_ts(R2, R1, smem_u32(BA), 64);
+                        mma_commit(mbar);
+                    }
+                }
+                // ---- factorisation: warps 0, 1 -> instance a, warps 2, 3 -> instance b
+                {
+                    const int x = warp >> 1, pw = warp & 1;
+                    pair_factor_invert(X1 + x * MAT_BYTES, wg, x, pw, lane, &misc.flag[x], ts * N);
+                    if (ts == 0 && want_u0) {
+                        // u_0 = -Linv'(Linv (Y x_0)), fp32, by the 64 threads of the pair
+                        unsigned char* Lx = X1 + x * MAT_BYTES;
+                        const int i = 32 * pw + lane;
+                        pair_barrier(wg, x);
+                        float s = 0.f;
+#pragma unroll 8
+                        for (int j = 0; j < N; ++j)
+                            s = fmaf(elem(X0, toff(64 * x + j, i)), misc.x0[x][j], s);     // Y[i][j] = Y'[j][i]
+                        misc.y0[x][i] = s;
+                        pair_barrier(wg, x);
+                        s = 0.f;
+                        for (int k = 0; k <= i; ++k)
+                            s = fmaf(elem(Lx, toff(i, k)), misc.y0[x][k], s);
+                        misc.v[x][i] = s;
+                        pair_barrier(wg, x);
+                        s = 0.f;
+                        for (int k = i; k < N; ++k)
+                            s = fmaf(elem(Lx, toff(k, i)), misc.v[x][k], s);
+                        if (x == 0 || valid_b)
+                            p.u[inst_x[x] * (long long)N + i] = -s;
+                    }
+                }
+                async_proxy_fence();
+                wg_barrier(wg);
+                // (4) Z' = [Y_a'; Y_b'] [Linv_a' Linv_b'] -> R1|R2
+                if (wt == 0) {
+                    tc_fence_after();
+                    gemm_ss(R1, smem_u32(X0), smem_u32(X1), 128, 0, false);
+                    mma_commit(mbar);
+                }
+                wait_mma();
+                {
+                    // Z_a' = lanes 0..63 of columns 0..63, Z_b' = lanes 64..127 of columns 64..127
+                    const int x = warp >> 1;
+                    float z[64];
+                    float h0[32], h1[32];
+                    tmem_ld32(R1 + 64 * x + lane_sel, h0);
+                    tmem_ld32(R1 + 64 * x + lane_sel + 32, h1);
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) {
+                        z[c] = h0[c];
+                        z[32 + c] = h1[c];
+                    }
+                    store_row_tf32(X1, wt, z);         // row wt of [Z_a'; Z_b'] (Linv is dead)
+                }
+                tc_fence_before();
+                async_proxy_fence();
+                wg_barrier(wg);
+                dead = misc.dead != 0;
+                // (5a) DP_a (R3, lanes 64..127) -= Z_a' Z_a : A operand rows 64..127 = Z_a' (rows 0..63 = tail of X0, unused)
+                // (5b) DP_b (R0, lanes 64..127) -= Z_b' Z_b : A operand = [Z_a'; Z_b']
+                if (wt == 0) {
+                    tc_fence_after();
+                    gemm_ss(R3, smem_u32(X1) - MAT_BYTES, smem_u32(X1), 64, 1, true);
+                    gemm_ss(R0, smem_u32(X1), smem_u32(X1) + MAT_BYTES, 64, 1, true);
+                    mma_commit(mbar);
+                }
+                // P_t = Q + DP: warps 2, 3 own the rows (lanes 64..127)
+                float q[64];
+                if (warp >= 2)
+                    load_q_row(q, p.Q, oq_x[0], wt - 64);
+                wait_mma();
+                if (warp >= 2) {
+                    const int j = wt - 64;
+#pragma unroll 1
+                    for (int x = 0; x < 2; ++x) {
+                        if (x == 1)
+                            load_q_row(q, p.Q, oq_x[1], j);
+                        float h0[32], h1[32];
+                        const uint32_t src = (x == 0 ? R3 : R0) + lane_sel;
+                        tmem_ld32(src, h0);
+                        tmem_ld32(src + 32, h1);
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) {
+                            q[c] += h0[c];
+                            q[32 + c] += h1[c];
+                        }
+                        if (ts > 0)
+                            store_row_tf32(X0, 64 * x + j, q);
+                        if (p.P && (x == 0 || valid_b) && (!p.first_only || ts == 0))
+                            store_row_global(p.P + (inst_x[x] * (long long)(p.first_only ? 1 : H + 1) + (p.first_only ? 0 : ts)) * N * N +
+                                                 (long long)j * N, q);
+                    }
+                }
+                tc_fence_before();
+                async_proxy_fence();
+                wg_barrier(wg);
+                dead = dead || misc.dead != 0;
+            }
+            if (dead)
+                break;
+            // ---- status / failed instances
+#pragma unroll 1
+            for (int x = 0; x < (valid_b ? 2 : 1); ++x) {
+                const int fl = misc.flag[x];
+                if (fl)
+                    wg_fail_instance(p, inst_x[x], fl, wt);
+                else if (p.info && wt == 0)
+                    p.info[inst_x[x]] = 0;
+            }
+            wg_barrier(wg);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (tid < 32)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(*tmem_slot), "r"(512) : "memory");
+    (void)offR_loaded;
+}
+
+inline size_t smem_bytes() { return SMEM_BYTES; }
+
+} // namespace umma64
+} // namespace ttc

@@ -11,6 +11,7 @@
 #include "common.cuh"
 #include "riccati_cta.cuh"
 #include "riccati_mma64.cuh"
+#include "riccati_umma64.cuh"
 #include "scan_pair.cuh"
 
 using namespace ttc;
@@ -250,6 +251,18 @@ int ttc_lqr_query(const ttc_lqr_handle* h, int32_t key, int64_t* value)
     case TTC_QUERY_WORKSPACE_BYTES: *value = (int64_t)workspace_bytes(h); return TTC_OK;
     case TTC_QUERY_LAST_KERNEL: *value = h->last_kernel; return TTC_OK;
     case TTC_QUERY_TOTAL_LAUNCHES: *value = h->total_launches; return TTC_OK;
+    case TTC_QUERY_DEVICE_ERROR: {
+        // word 1 of the small workspace: set by a kernel whose bounded wait ran out
+        *value = 0;
+        if (h->ws_E.ptr && h->ws_E.bytes >= 2 * sizeof(int) && h->last_kernel == TTC_KERNEL_RICCATI_UMMA) {
+            int flag = 0;
+            if (cudaSetDevice(h->cfg.device) != cudaSuccess ||
+                cudaMemcpy(&flag, static_cast<int*>(h->ws_E.ptr) + 1, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess)
+                return fail(TTC_STATUS_CUDA_ERROR, "reading the device error word failed");
+            *value = flag;
+        }
+        return TTC_OK;
+    }
     default: return fail(TTC_STATUS_INVALID_ARGUMENT, "unknown query key %d", key);
     }
 }
@@ -306,6 +319,25 @@ int ttc_lqr_solve(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B,
         const bool bf16_in = (Q->dtype == TTC_BF16) || (x0 && x0->ptr && x0->dtype == TTC_BF16);
         const bool want_tf32 = h->cfg.math == TTC_MATH_TF32 || (h->cfg.math == TTC_MATH_AUTO && bf16_in);
         const bool head_shared = A->bstride[2] == 0 && B->bstride[2] == 0 && R->bstride[2] == 0;
+        const bool umma_outputs = !K && !x && (!u || p.first_only);
+        if (want_tf32 && n == 64 && m == 64 && head_shared && umma_outputs) {
+            // tcgen05 kernel (P_t / P_0, u_0): persistent CTAs, two independent warpgroups each
+            if ((s = ensure(h->ws_E, sizeof(int) * 4))) return s;
+            int* counter = static_cast<int*>(h->ws_E.ptr);
+            TTC_CUDA(cudaMemsetAsync(counter, 0, 2 * sizeof(int), st));
+            const size_t smem = umma64::smem_bytes();
+            TTC_CUDA(cudaFuncSetAttribute(umma64::riccati_umma64_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          (int)smem));
+            const long long chunks = p.b0 * p.b1 * ((p.b2 + umma64::CHUNK - 1) / umma64::CHUNK);
+            long long grid = h->sm_count;
+            if (2 * grid > chunks) grid = (chunks + 1) / 2;
+            umma64::riccati_umma64_kernel<<<(unsigned)grid, umma64::THREADS, smem, st>>>(p, counter, counter + 1);
+            TTC_CUDA(cudaGetLastError());
+            h->last_launches = 1;
+            h->last_kernel = TTC_KERNEL_RICCATI_UMMA;
+            h->total_launches += h->last_launches;
+            return TTC_OK;
+        }
         if (want_tf32 && n == 64 && m == 64 && head_shared) {
             // tensor-core kernel: persistent CTAs, work items handed out by an atomic counter
             if ((s = ensure(h->ws_E, sizeof(int) * 4))) return s;

@@ -61,6 +61,7 @@ def run_gpu(w, method=lqr.TTC_RICCATI, want=("K", "P", "x", "u", "info"), first_
     torch.cuda.synchronize(dev)
     out["kernel"] = solver.query(lqr.TTC_QUERY_LAST_KERNEL)
     out["launches"] = solver.query(lqr.TTC_QUERY_LAST_LAUNCHES)
+    assert solver.query(lqr.TTC_QUERY_DEVICE_ERROR) == 0, "a bounded wait inside the kernel ran out"
     if own:
         solver.close()
     return out
