@@ -10,14 +10,14 @@
 //   (1)  W  = BA * [P_a P_b]          -> W_x = [V_x'; T_x'] = [(P_x B)'; (P_x A)']        SS, M128 N128
 //   (2x) F_x  = W_x * B  = [S_x - R ; Y_x']   DP_x = W_x * A = [ . ; A'P_x A]              TS (A operand
 //        read from tensor memory, no round trip through shared memory), N64 each
-//   S_x = R + (S_x - R) -> shared, fp32;  Linv_x = chol(S_x)^{-1}   2 warps per instance, blocked:
-//        32 x 32 diagonal blocks in registers (one row per lane), off-diagonal work as 3 x tf32
-//        (error-compensated) mma.sync products
-//   (4)  Z' = [Y_a'; Y_b'] * [Linv_a' Linv_b']   (diagonal blocks Z_a', Z_b')              SS, M128 N128
+//   S_x = R + (S_x - R) and Y_x' -> shared, fp32.  Two warps per instance run a right-looking blocked
+//        Cholesky (8-wide panels) on the tall matrix [S_x; Y_x']: diagonal blocks in registers, panel rows by
+//        forward substitution, trailing updates as 3 x tf32 (error-compensated) mma.sync.  It leaves
+//        L (S_x = L L') and Z_x' = Y_x' L^{-T}: no explicit inverse, no extra contraction for Z.
 //   (5x) DP_x -= Z_x' Z_x                                                                   SS, N64
 //   P_x <- Q_x + DP_x            (P_t = Q + A'P A - Y'S^{-1}Y)
 // Tensor-memory map of a warpgroup (256 columns): R0 = W_a then DP_b, R1 = W_b, R2 = F_a then F_b,
-// R3 = DP_a; Z' reuses R1|R2.
+// R3 = DP_a.
 //
 // Shared-memory operands use the canonical K-major layout without swizzle: 8 x 4 (rows x k) core
 // matrices of 128 contiguous bytes, chunk stride 128 B along k, 2048 B between 8-row groups.  A row
@@ -43,8 +43,8 @@ constexpr uint32_t MAT_BYTES = 8 * SR;          // one 64 x 64 matrix
 constexpr uint32_t BUF_BYTES = 2 * MAT_BYTES;   // 128 rows
 constexpr int SPIN_LIMIT = 1 << 22;
 
-// per-warpgroup shared memory: BA | X0 | X1 (X0 and X1 adjacent: step (5a) starts its A operand
-// 64 rows before X1) followed by small scratch.
+// per-warpgroup shared memory: BA | X0 | X1 (BA and X0 adjacent: step (5a) starts its A operand
+// 64 rows before X0) followed by small scratch.
 constexpr uint32_t OFF_BA = 0;
 constexpr uint32_t OFF_X0 = BUF_BYTES;
 constexpr uint32_t OFF_X1 = 2 * BUF_BYTES;
@@ -54,9 +54,8 @@ struct Misc {
     int chunk;                   // current work item
     int dead;                    // set when a wait timed out
     int flag[2];                 // first failed pivot per instance (0 = none)
-    float x0[2][N];
-    float y0[2][N];
-    float v[2][N];
+    alignas(16) float x0[2][N];
+    alignas(16) float y0[2][N];
 };
 constexpr uint32_t WG_BYTES = OFF_MISC + ((sizeof(Misc) + 127) / 128) * 128;
 constexpr uint32_t SMEM_BYTES = NUM_WG * WG_BYTES + 128;     // + slot for the tensor-memory base address
@@ -68,20 +67,13 @@ __device__ __forceinline__ uint32_t toff(int r, int c)
 {
     return (uint32_t)(r >> 3) * SR + (uint32_t)(c >> 2) * SC + (uint32_t)(r & 7) * 16u + (uint32_t)(c & 3) * 4u;
 }
-// private layout of a 32 x 32 scratch inside the (rows 0..31, cols 32..63) block of a matrix: element (i, c)
-// sits in core matrix (i/8, 8 + i%8) at row (c/4) ^ (i%8); conflict-free for "lane = c" 4-byte accesses and
-// for "lane = i" 16-byte accesses.
-__device__ __forceinline__ uint32_t soff(int i, int c)
-{
-    return (uint32_t)(i >> 3) * SR + (uint32_t)(8 + (i & 7)) * SC + (uint32_t)(((c >> 2) ^ i) & 7) * 16u + (uint32_t)(c & 3) * 4u;
-}
 __device__ __forceinline__ float& elem(unsigned char* base, uint32_t off) { return *reinterpret_cast<float*>(base + off); }
 
+// fp32 -> tf32 (10 explicit mantissa bits), round to nearest with ties away from zero, on the integer
+// pipe (cvt.rna.tf32.f32 issues on the transcendental pipe at a fraction of the rate).
 __device__ __forceinline__ uint32_t to_tf32(float x)
 {
-    uint32_t r;
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
-    return r;
+    return (__float_as_uint(x) + 0x1000u) & 0xffffe000u;
 }
 __device__ __forceinline__ float round_tf32(float x) { return __uint_as_float(to_tf32(x)); }
 
@@ -166,95 +158,7 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32])
 __device__ __forceinline__ void wg_barrier(int wg) { asm volatile("bar.sync %0, %1;" :: "r"(1 + wg), "r"(WG_THREADS) : "memory"); }
 __device__ __forceinline__ void pair_barrier(int wg, int x) { asm volatile("bar.sync %0, %1;" :: "r"(3 + 2 * wg + x), "r"(64) : "memory"); }
 
-// ---- warp-level 32 x 32 Cholesky, one row per lane -----------------------------------------------------------
-// s[c] = row `lane` of an SPD block.  On return s holds row `lane` of L (entries right of the diagonal are
-// meaningless) and rs_own = 1 / L[lane][lane].  The update of the trailing rows uses s_ij * s_cj / d_j, so
-// that the broadcast of column j does not wait for the reciprocal.  Returns 0 or 1 + the first bad pivot.
-__device__ __forceinline__ int warp_chol32(float (&s)[32], float& rs_own, int lane)
-{
-    int bad = 0;
-    rs_own = 1.f;
-#pragma unroll
-    for (int j = 0; j < 32; ++j) {
-        float d = __shfl_sync(0xffffffffu, s[j], j);
-        const float sj = s[j];
-        if (!(d > 0.f)) {
-            if (!bad)
-                bad = j + 1;
-            d = 1.f;
-        }
-        const float rinv = __frcp_rn(d);
-        const float f = sj * rinv;
-#pragma unroll
-        for (int c = j + 1; c < 32; ++c) {
-            const float lc = __shfl_sync(0xffffffffu, sj, c);
-            s[c] = fmaf(-f, lc, s[c]);
-        }
-        const float rs = rsqrtf(d);
-        s[j] = sj * rs;
-        if (lane == j)
-            rs_own = rs;
-    }
-    return bad;
-}
-
-// Lt(k, i) = L[i][k] in the private scratch layout of `scr`.  Lane c computes column c of L^{-1}:
-// x[i] = Linv[i][c] (0 for i < c).
-__device__ __forceinline__ void warp_trinv32(float (&x)[32], unsigned char* scr, float rs_own, int lane)
-{
-    float a[32];
-#pragma unroll
-    for (int i = 0; i < 32; ++i)
-        a[i] = 0.f;
-#pragma unroll
-    for (int k = 0; k < 32; ++k) {
-        const float rsk = __shfl_sync(0xffffffffu, rs_own, k);
-        const float xk = (k == lane) ? rsk : ((k > lane) ? -a[k] * rsk : 0.f);
-        x[k] = xk;
-#pragma unroll
-        for (int i4 = (k + 1) & ~3; i4 < 32; i4 += 4) {
-            const float4 l4 = *reinterpret_cast<const float4*>(scr + soff(k, i4));
-            if (i4 + 0 > k) a[i4 + 0] = fmaf(l4.x, xk, a[i4 + 0]);
-            if (i4 + 1 > k) a[i4 + 1] = fmaf(l4.y, xk, a[i4 + 1]);
-            if (i4 + 2 > k) a[i4 + 2] = fmaf(l4.z, xk, a[i4 + 2]);
-            if (i4 + 3 > k) a[i4 + 3] = fmaf(l4.w, xk, a[i4 + 3]);
-        }
-    }
-}
-
-// One warp: factor the 32 x 32 SPD diagonal block (d0, d0) of the matrix at `M` and overwrite it with the
-// inverse of its Cholesky factor (lower triangular, zeros above the diagonal).  Scratch: block (0, 1) of M.
-__device__ __forceinline__ int warp_factor_block(unsigned char* M, int d0, int lane)
-{
-    float s[32];
-#pragma unroll
-    for (int c = 0; c < 32; c += 4) {
-        const float4 v = *reinterpret_cast<const float4*>(M + toff(d0 + lane, d0 + c));
-        s[c] = v.x; s[c + 1] = v.y; s[c + 2] = v.z; s[c + 3] = v.w;
-    }
-    float rs_own;
-    const int bad = warp_chol32(s, rs_own, lane);
-#pragma unroll
-    for (int k = 0; k < 32; ++k)
-        elem(M, soff(k, lane)) = s[k];                  // Lt(k, i = lane) = L[i][k]
-    __syncwarp();
-    float x[32];
-    warp_trinv32(x, M, rs_own, lane);
-    __syncwarp();
-#pragma unroll
-    for (int i = 0; i < 32; ++i)
-        elem(M, soff(i, lane)) = x[i];                  // bounce: column owner -> row owner
-    __syncwarp();
-#pragma unroll
-    for (int q = 0; q < 8; ++q) {
-        const float4 v = *reinterpret_cast<const float4*>(M + soff(lane, 4 * q));
-        *reinterpret_cast<float4*>(M + toff(d0 + lane, d0 + 4 * q)) = v;
-    }
-    __syncwarp();
-    return bad;
-}
-
-// ---- 3 x tf32 warp-level products on 16 x 32 tiles (fp32-grade accuracy) ---------------------------------------
+// ---- blocked Cholesky of S fused with the forward substitution Z' = Y' L^{-T} --------------------------------------
 __device__ __forceinline__ void mma_16x8x8(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                            uint32_t b0, uint32_t b1)
 {
@@ -263,143 +167,182 @@ __device__ __forceinline__ void mma_16x8x8(float (&d)[4], uint32_t a0, uint32_t 
                  : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
+// x = hi + lo with hi exactly representable in tf32 (truncation); the tensor core ignores the low 13 bits
+// of lo, an error of 2^-21 |x|.  hi*hi + hi*lo + lo*hi then has fp32-grade accuracy.
 __device__ __forceinline__ void split_tf32(float x, uint32_t& hi, uint32_t& lo)
 {
-    hi = to_tf32(x);
-    lo = to_tf32(x - __uint_as_float(hi));
-}
-// acc[nt] (16 x 8 tiles, nt = 0..3) += sign * A(16 x 32) * B(32 x 32).  A(r, k) is read at M + toff(ar + r, ac + k).
-// B(k, n) is read at M + toff(br + n, bc + k) when BT (B given by its transpose, row n contiguous in k), else at
-// M + toff(br + k, bc + n).  K tiles outside [ktlo(nt), kthi(nt)] are skipped (triangular operands).
-template <bool NEG, bool BT, class KLo, class KHi>
-__device__ __forceinline__ void mma3x_16x32x32(float (&acc)[4][4], const unsigned char* M, int ar, int ac, int br, int bc,
-                                               int g, int t, KLo ktlo, KHi kthi)
-{
-#pragma unroll
-    for (int kt = 0; kt < 4; ++kt) {
-        float a[4];
-        a[0] = *reinterpret_cast<const float*>(M + toff(ar + g, ac + 8 * kt + t));
-        a[1] = *reinterpret_cast<const float*>(M + toff(ar + g + 8, ac + 8 * kt + t));
-        a[2] = *reinterpret_cast<const float*>(M + toff(ar + g, ac + 8 * kt + t + 4));
-        a[3] = *reinterpret_cast<const float*>(M + toff(ar + g + 8, ac + 8 * kt + t + 4));
-        uint32_t ah[4], al[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e)
-            split_tf32(NEG ? -a[e] : a[e], ah[e], al[e]);
-#pragma unroll
-        for (int nt = 0; nt < 4; ++nt) {
-            if (kt < ktlo(nt) || kt > kthi(nt))
-                continue;
-            float b0, b1;
-            if (BT) {
-                b0 = *reinterpret_cast<const float*>(M + toff(br + 8 * nt + g, bc + 8 * kt + t));
-                b1 = *reinterpret_cast<const float*>(M + toff(br + 8 * nt + g, bc + 8 * kt + t + 4));
-            } else {
-                b0 = *reinterpret_cast<const float*>(M + toff(br + 8 * kt + t, bc + 8 * nt + g));
-                b1 = *reinterpret_cast<const float*>(M + toff(br + 8 * kt + t + 4, bc + 8 * nt + g));
-            }
-            uint32_t bh0, bl0, bh1, bl1;
-            split_tf32(b0, bh0, bl0);
-            split_tf32(b1, bh1, bl1);
-            mma_16x8x8(acc[nt], al[0], al[1], al[2], al[3], bh0, bh1);
-            mma_16x8x8(acc[nt], ah[0], ah[1], ah[2], ah[3], bl0, bl1);
-            mma_16x8x8(acc[nt], ah[0], ah[1], ah[2], ah[3], bh0, bh1);
-        }
-    }
-}
-__device__ __forceinline__ void zero4x4(float (&acc)[4][4])
-{
-#pragma unroll
-    for (int nt = 0; nt < 4; ++nt)
-#pragma unroll
-        for (int e = 0; e < 4; ++e)
-            acc[nt][e] = 0.f;
-}
-// accumulator tiles <-> rows r0 + g, r0 + g + 8 ; columns c0 + 8 nt + 2t, +1
-template <bool ROUND>
-__device__ __forceinline__ void store_tiles(unsigned char* M, int r0, int c0, const float (&acc)[4][4], int g, int t)
-{
-#pragma unroll
-    for (int nt = 0; nt < 4; ++nt) {
-        const int c = c0 + 8 * nt + 2 * t;
-        float2 lo = make_float2(acc[nt][0], acc[nt][1]), hi = make_float2(acc[nt][2], acc[nt][3]);
-        if (ROUND) {
-            lo.x = round_tf32(lo.x); lo.y = round_tf32(lo.y); hi.x = round_tf32(hi.x); hi.y = round_tf32(hi.y);
-        }
-        *reinterpret_cast<float2*>(M + toff(r0 + g, c)) = lo;
-        *reinterpret_cast<float2*>(M + toff(r0 + g + 8, c)) = hi;
-    }
-}
-__device__ __forceinline__ void load_tiles(float (&acc)[4][4], const unsigned char* M, int r0, int c0, int g, int t)
-{
-#pragma unroll
-    for (int nt = 0; nt < 4; ++nt) {
-        const int c = c0 + 8 * nt + 2 * t;
-        const float2 lo = *reinterpret_cast<const float2*>(M + toff(r0 + g, c));
-        const float2 hi = *reinterpret_cast<const float2*>(M + toff(r0 + g + 8, c));
-        acc[nt][0] = lo.x; acc[nt][1] = lo.y; acc[nt][2] = hi.x; acc[nt][3] = hi.y;
-    }
+    hi = __float_as_uint(x) & 0xffffe000u;
+    lo = __float_as_uint(x - __uint_as_float(hi));
 }
 
-// Two warps (pw = 0, 1; 64 threads) replace the SPD matrix S at `M` (fp32, core-matrix layout) by
-// Linv = chol(S)^{-1}: lower triangle fp32 values rounded to tf32, zeros above the diagonal.
-// 2 x 2 blocks of 32:  Linv11 = chol(S11)^{-1};  L21 = S21 Linv11';  S22 -= L21 L21';  W = L21 Linv11;
-// Linv22 = chol(S22)^{-1};  Linv21 = -Linv22 W.   A non-positive pivot is recorded in *flag as code0 + index.
-__device__ __forceinline__ void pair_factor_invert(unsigned char* M, int wg, int x, int pw, int lane, int* flag, int code0)
+// In-thread Cholesky of an 8 x 8 SPD block: l (lower triangle) is overwritten by L, rinv[i] = 1 / L[i][i].
+// Returns 0 or 1 + the index of the first non-positive pivot.
+__device__ __forceinline__ int chol8(float (&l)[8][8], float (&rinv)[8])
+{
+    int bad = 0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        float d = l[j][j];
+        if (!(d > 0.f)) {
+            if (!bad)
+                bad = j + 1;
+            d = 1.f;
+        }
+        float rs;
+        asm("rsqrt.approx.ftz.f32 %0, %1;" : "=f"(rs) : "f"(d));
+        rs = rs * fmaf(-0.5f * d * rs, rs, 1.5f);            // one Newton step: full fp32 accuracy
+        rinv[j] = rs;
+        l[j][j] = d * rs;
+#pragma unroll
+        for (int i = j + 1; i < 8; ++i)
+            l[i][j] *= rs;
+#pragma unroll
+        for (int i = j + 1; i < 8; ++i)
+#pragma unroll
+            for (int c = j + 1; c <= i; ++c)
+                l[i][c] = fmaf(-l[i][j], l[c][j], l[i][c]);
+    }
+    return bad;
+}
+// x (a row vector of 8) <- x L^{-T}  (forward substitution with the lower factor L)
+__device__ __forceinline__ void fsub8(float (&x)[8], const float (&l)[8][8], const float (&rinv)[8])
+{
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        float v = x[i];
+#pragma unroll
+        for (int j = 0; j < i; ++j)
+            v = fmaf(-l[i][j], x[j], v);
+        x[i] = v * rinv[i];
+    }
+}
+__device__ __forceinline__ void load_row8(float (&x)[8], const unsigned char* p)
+{
+    const float4 a = *reinterpret_cast<const float4*>(p);
+    const float4 b = *reinterpret_cast<const float4*>(p + SC);
+    x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
+}
+template <bool ROUND>
+__device__ __forceinline__ void store_row8(unsigned char* p, const float (&x)[8])
+{
+    float4 a = make_float4(x[0], x[1], x[2], x[3]), b = make_float4(x[4], x[5], x[6], x[7]);
+    if (ROUND) {
+        a.x = round_tf32(a.x); a.y = round_tf32(a.y); a.z = round_tf32(a.z); a.w = round_tf32(a.w);
+        b.x = round_tf32(b.x); b.y = round_tf32(b.y); b.z = round_tf32(b.z); b.w = round_tf32(b.w);
+    }
+    *reinterpret_cast<float4*>(p) = a;
+    *reinterpret_cast<float4*>(p + SC) = b;
+}
+
+// Two warps (pw = 0, 1; 64 threads) work on the tall matrix G = [S; Y'] (128 x 64, fp32): S (64 x 64 SPD,
+// lower triangle used) at `Sm`, Y' at `Ym`, both in the core-matrix layout.  Right-looking blocked Cholesky
+// with 8-wide panels, applied to all 128 rows: on return the lower triangle of Sm holds L (S = L L') and
+// Ym holds Z' = Y' L^{-T} rounded to tf32, so that Z'Z' ' = Y' S^{-1} Y.  Per panel k:
+//   every thread factors the 8 x 8 diagonal block in registers (redundantly: nothing to exchange),
+//   row owners replace G[r][panel] by G[r][panel] L_d^{-T}  (rows of S below the block, every row of Y'),
+//   the trailing columns get the rank-8 update G[r][c] -= G[r][panel] . S[c][panel] as 3 x tf32 mma.
+// Fragment addresses are a per-thread constant plus compile-time offsets.  A non-positive pivot is recorded
+// in *flag as code0 + index.
+__device__ __forceinline__ void pair_chol_solve(unsigned char* Sm, unsigned char* Ym, int wg, int x, int pw, int lane,
+                                                int* flag, int code0)
 {
     const int g = lane >> 2, t = lane & 3;
-    const int r0 = 32 + 16 * pw;                       // the 16 rows of the lower half owned by this warp
-    if (pw == 0) {
-        const int bad = warp_factor_block(M, 0, lane);
-        if (bad && lane == 0 && *flag == 0)
-            *flag = code0 + bad;
-    }
-    pair_barrier(wg, x);
-    float acc[4][4];
-    // L21 = S21 Linv11'   (Linv11[n][k] = 0 for k > n)
-    zero4x4(acc);
-    mma3x_16x32x32<false, true>(acc, M, r0, 0, 0, 0, g, t, [](int) { return 0; }, [](int nt) { return nt; });
-    __syncwarp();
-    store_tiles<false>(M, r0, 0, acc, g, t);
-    pair_barrier(wg, x);
-    // S22 -= L21 L21'
-    load_tiles(acc, M, r0, 32, g, t);
-    mma3x_16x32x32<true, true>(acc, M, r0, 0, 32, 0, g, t, [](int) { return 0; }, [](int) { return 3; });
-    store_tiles<false>(M, r0, 32, acc, g, t);
-    pair_barrier(wg, x);
-    // W = L21 Linv11 over the own rows   (Linv11[k][n] = 0 for k < n)
-    zero4x4(acc);
-    mma3x_16x32x32<false, false>(acc, M, r0, 0, 0, 0, g, t, [](int nt) { return nt; }, [](int) { return 3; });
-    __syncwarp();
-    store_tiles<false>(M, r0, 0, acc, g, t);
-    if (pw == 1) {
-        const int bad = warp_factor_block(M, 32, lane);
-        if (bad && lane == 0 && *flag == 0)
-            *flag = code0 + 32 + bad;
-    }
-    pair_barrier(wg, x);
-    // Linv21 = -Linv22 W     (Linv22[r][k] = 0 for k > r)
-    zero4x4(acc);
-    {
-        const int kmax = (r0 - 32 + 15) >> 3;
-        mma3x_16x32x32<true, false>(acc, M, r0, 32, 32, 0, g, t, [](int) { return 0; }, [kmax](int) { return kmax; });
-    }
-    pair_barrier(wg, x);                               // every read of W is done
-    store_tiles<true>(M, r0, 0, acc, g, t);
-    // round the diagonal blocks to tf32 in place and clear block (0, 1) (scratch until now)
-    {
-        const int d0 = 32 * pw;
+    const int tid2 = 32 * pw + lane;
+    const uint32_t frag_ab = (uint32_t)g * 16u + (uint32_t)t * 4u;                                     // (row g, col t) of a core matrix
+    const uint32_t frag_c = (uint32_t)g * 16u + (uint32_t)(t >> 1) * SC + (uint32_t)((2 * t) & 3) * 4u; // (row g, cols 2t, 2t+1) of a tile
+    const uint32_t own_row = (uint32_t)(tid2 >> 3) * SR + (uint32_t)(tid2 & 7) * 16u;                 // row tid2, column 0
+#pragma unroll 1
+    for (int k = 0; k < 8; ++k) {
+        const uint32_t kcol = 2u * k * SC;             // byte offset of columns 8k .. 8k+7 inside a row
+        unsigned char* dblk = Sm + (uint32_t)k * SR + kcol;
+        float l[8][8], rinv[8];
 #pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            float4 v = *reinterpret_cast<float4*>(M + toff(d0 + lane, d0 + 4 * q));
-            v.x = round_tf32(v.x); v.y = round_tf32(v.y); v.z = round_tf32(v.z); v.w = round_tf32(v.w);
-            *reinterpret_cast<float4*>(M + toff(d0 + lane, d0 + 4 * q)) = v;
-        }
-        if (pw == 0) {
+        for (int i = 0; i < 8; ++i)
+            load_row8(l[i], dblk + i * 16);
+        const bool has_s = tid2 + 8 * k + 8 < N;
+        unsigned char* py = Ym + own_row + kcol;
+        unsigned char* ps = Sm + own_row + (uint32_t)(k + 1) * SR + kcol;       // row tid2 + 8k + 8
+        float xy[8], xs[8];
+        load_row8(xy, py);
+        if (has_s)
+            load_row8(xs, ps);
+        const int bad = chol8(l, rinv);
+        if (bad && tid2 == 0 && *flag == 0)
+            *flag = code0 + 8 * k + bad;
+        fsub8(xy, l, rinv);
+        if (has_s)
+            fsub8(xs, l, rinv);
+        store_row8<true>(py, xy);
+        if (has_s)
+            store_row8<false>(ps, xs);
+        pair_barrier(wg, x);                           // panel written; every thread has read the diagonal block
+        if (tid2 < 8) {                                // keep L_d for the back substitution
 #pragma unroll
-            for (int q = 0; q < 8; ++q)
-                *reinterpret_cast<float4*>(M + toff(lane, 32 + 4 * q)) = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int i = 0; i < 8; ++i)
+                if (tid2 == i)
+                    store_row8<false>(dblk + i * 16, l[i]);
         }
+        if (k == 7)
+            break;
+        // ---- trailing update: B fragments = rows 8j + g of S, columns 8k + t, 8k + t + 4
+        uint32_t bh[7][2], bl[7][2];
+        {
+            const unsigned char* pb = Sm + frag_ab + kcol;
+#pragma unroll
+            for (int j = 1; j < 8; ++j)
+                if (j > k) {
+                    split_tf32(*reinterpret_cast<const float*>(pb + j * SR), bh[j - 1][0], bl[j - 1][0]);
+                    split_tf32(*reinterpret_cast<const float*>(pb + j * SR + SC), bh[j - 1][1], bl[j - 1][1]);
+                }
+        }
+#pragma unroll
+        for (int uu = 0; uu < 4; ++uu) {
+            const int u = 2 * uu + pw;                 // tiles 0..3: rows of S, 4..7: rows of Y'
+            const bool is_s = u < 4;
+            const int mt = u & 3;
+            if (is_s && 16 * mt + 15 < 8 * k + 8)
+                continue;
+            unsigned char* Mt = is_s ? Sm : Ym;
+            uint32_t ah[4], al[4];
+            {
+                const unsigned char* pa = Mt + frag_ab + kcol + 2 * mt * SR;
+                split_tf32(-*reinterpret_cast<const float*>(pa), ah[0], al[0]);
+                split_tf32(-*reinterpret_cast<const float*>(pa + SR), ah[1], al[1]);
+                split_tf32(-*reinterpret_cast<const float*>(pa + SC), ah[2], al[2]);
+                split_tf32(-*reinterpret_cast<const float*>(pa + SR + SC), ah[3], al[3]);
+            }
+            // all C tiles of this row tile first, then three independent mma passes, then the stores
+            unsigned char* pc = Mt + frag_c + 2 * mt * SR;
+            float acc[7][4];
+#pragma unroll
+            for (int j = 1; j < 8; ++j) {
+                if (j <= k || (is_s && j > 2 * mt + 1))
+                    continue;
+                const float2 lo = *reinterpret_cast<const float2*>(pc + 2 * j * SC);
+                const float2 hi = *reinterpret_cast<const float2*>(pc + 2 * j * SC + SR);
+                acc[j - 1][0] = lo.x; acc[j - 1][1] = lo.y; acc[j - 1][2] = hi.x; acc[j - 1][3] = hi.y;
+            }
+#pragma unroll
+            for (int j = 1; j < 8; ++j)
+                if (!(j <= k || (is_s && j > 2 * mt + 1)))
+                    mma_16x8x8(acc[j - 1], al[0], al[1], al[2], al[3], bh[j - 1][0], bh[j - 1][1]);
+#pragma unroll
+            for (int j = 1; j < 8; ++j)
+                if (!(j <= k || (is_s && j > 2 * mt + 1)))
+                    mma_16x8x8(acc[j - 1], ah[0], ah[1], ah[2], ah[3], bl[j - 1][0], bl[j - 1][1]);
+#pragma unroll
+            for (int j = 1; j < 8; ++j)
+                if (!(j <= k || (is_s && j > 2 * mt + 1)))
+                    mma_16x8x8(acc[j - 1], ah[0], ah[1], ah[2], ah[3], bh[j - 1][0], bh[j - 1][1]);
+#pragma unroll
+            for (int j = 1; j < 8; ++j) {
+                if (j <= k || (is_s && j > 2 * mt + 1))
+                    continue;
+                *reinterpret_cast<float2*>(pc + 2 * j * SC) = make_float2(acc[j - 1][0], acc[j - 1][1]);
+                *reinterpret_cast<float2*>(pc + 2 * j * SC + SR) = make_float2(acc[j - 1][2], acc[j - 1][3]);
+            }
+        }
+        pair_barrier(wg, x);
     }
 }
 
@@ -436,6 +379,12 @@ __device__ __forceinline__ void store_row_tf32(unsigned char* buf, int r, const 
         *reinterpret_cast<float4*>(buf + toff(r, 4 * c)) =
             make_float4(round_tf32(v[4 * c]), round_tf32(v[4 * c + 1]), round_tf32(v[4 * c + 2]), round_tf32(v[4 * c + 3]));
 }
+__device__ __forceinline__ void store_row_f32(unsigned char* buf, int r, const float (&v)[64])
+{
+#pragma unroll
+    for (int c = 0; c < 16; ++c)
+        *reinterpret_cast<float4*>(buf + toff(r, 4 * c)) = make_float4(v[4 * c], v[4 * c + 1], v[4 * c + 2], v[4 * c + 3]);
+}
 __device__ __forceinline__ void store_row_global(float* dst, const float (&v)[64])
 {
 #pragma unroll
@@ -469,8 +418,8 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
     const int lane = wt & 31;
     unsigned char* wsm = smem_raw + (size_t)wg * WG_BYTES;
     unsigned char* BA = wsm + OFF_BA;          // rows 0..63: B' (row j = column j of B), rows 64..127: A'
-    unsigned char* X0 = wsm + OFF_X0;          // [P_a; P_b] -> [Y_a'; Y_b'] -> next [P_a; P_b]
-    unsigned char* X1 = wsm + OFF_X1;          // [S_a; S_b] -> [Linv_a; Linv_b] -> [Z_a'; Z_b']
+    unsigned char* X0 = wsm + OFF_X0;          // [P_a; P_b] -> [Y_a'; Y_b'] -> [Z_a'; Z_b'] -> next [P_a; P_b]
+    unsigned char* X1 = wsm + OFF_X1;          // [S_a; S_b] -> [L_a; L_b]
     Misc& misc = *reinterpret_cast<Misc*>(wsm + OFF_MISC);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_raw + (size_t)NUM_WG * WG_BYTES);
     const uint32_t mbar = smem_u32(&misc.mbar);
@@ -609,8 +558,8 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
                             *reinterpret_cast<float4*>(X1 + x * MAT_BYTES + toff(wt, 4 * c)) =
                                 make_float4(f[4 * c] + rrow[4 * c], f[4 * c + 1] + rrow[4 * c + 1],
                                             f[4 * c + 2] + rrow[4 * c + 2], f[4 * c + 3] + rrow[4 * c + 3]);
-                    } else {                           // Y_x' -> X0 (P is dead once (1) has completed)
-                        store_row_tf32(X0, 64 * x + (wt - 64), f);
+                    } else {                           // Y_x' -> X0, fp32 (P is dead once (1) has completed)
+                        store_row_f32(X0, 64 * x + (wt - 64), f);
                     }
                     tc_fence_before();
                     wg_barrier(wg);
@@ -621,66 +570,63 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
                         mma_commit(mbar);
                     }
                 }
-                // ---- factorisation: warps 0, 1 -> instance a, warps 2, 3 -> instance b
+                // ---- S = L L' and Z' = Y' L^{-T}: warps 0, 1 -> instance a, warps 2, 3 -> instance b
                 {
                     const int x = warp >> 1, pw = warp & 1;
-                    pair_factor_invert(X1 + x * MAT_BYTES, wg, x, pw, lane, &misc.flag[x], ts * N);
+                    unsigned char* Sm = X1 + x * MAT_BYTES;
+                    unsigned char* Ym = X0 + x * MAT_BYTES;
+                    pair_chol_solve(Sm, Ym, wg, x, pw, lane, &misc.flag[x], ts * N);
                     if (ts == 0 && want_u0) {
-                        // u_0 = -Linv'(Linv (Y x_0)), fp32, by the 64 threads of the pair
-                        unsigned char* Lx = X1 + x * MAT_BYTES;
+                        // u_0 = K_0 x_0 = -L^{-T} (Z x_0), fp32, by the 64 threads of the pair
                         const int i = 32 * pw + lane;
                         pair_barrier(wg, x);
-                        float s = 0.f;
+                        float zi = 0.f;
 #pragma unroll 8
-                        for (int j = 0; j < N; ++j)
-                            s = fmaf(elem(X0, toff(64 * x + j, i)), misc.x0[x][j], s);     // Y[i][j] = Y'[j][i]
-                        misc.y0[x][i] = s;
-                        pair_barrier(wg, x);
-                        s = 0.f;
-                        for (int k = 0; k <= i; ++k)
-                            s = fmaf(elem(Lx, toff(i, k)), misc.y0[x][k], s);
-                        misc.v[x][i] = s;
-                        pair_barrier(wg, x);
-                        s = 0.f;
-                        for (int k = i; k < N; ++k)
-                            s = fmaf(elem(Lx, toff(k, i)), misc.v[x][k], s);
-                        if (x == 0 || valid_b)
-                            p.u[inst_x[x] * (long long)N + i] = -s;
-                    }
-                }
-                async_proxy_fence();
-                wg_barrier(wg);
-                // (4) Z' = [Y_a'; Y_b'] [Linv_a' Linv_b'] -> R1|R2
-                if (wt == 0) {
-                    tc_fence_after();
-                    gemm_ss(R1, smem_u32(X0), smem_u32(X1), 128, 0, false);
-                    mma_commit(mbar);
-                }
-                wait_mma();
-                {
-                    // Z_a' = lanes 0..63 of columns 0..63, Z_b' = lanes 64..127 of columns 64..127
-                    const int x = warp >> 1;
-                    float z[64];
-                    float h0[32], h1[32];
-                    tmem_ld32(R1 + 64 * x + lane_sel, h0);
-                    tmem_ld32(R1 + 64 * x + lane_sel + 32, h1);
+                        for (int c = 0; c < N; ++c)
+                            zi = fmaf(elem(Ym, toff(c, i)), misc.x0[x][c], zi);          // Z[i][c] = Z'[c][i]
+                        misc.y0[x][i] = zi;
+#pragma unroll 1
+                        for (int kb = 7; kb >= 0; --kb) {       // back substitution L' w = Z x_0 in 8-wide blocks
+                            pair_barrier(wg, x);
+                            const int c0 = 8 * kb;
+                            float l[8][8], w[8];
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) {
-                        z[c] = h0[c];
-                        z[32 + c] = h1[c];
+                            for (int r = 0; r < 8; ++r) {
+                                load_row8(l[r], Sm + toff(c0 + r, c0));
+                                w[r] = misc.y0[x][c0 + r];
+                            }
+#pragma unroll
+                            for (int r = 7; r >= 0; --r) {
+                                float v = w[r];
+#pragma unroll
+                                for (int j = r + 1; j < 8; ++j)
+                                    v = fmaf(-l[j][r], w[j], v);
+                                w[r] = v / l[r][r];
+                            }
+                            if (i < c0) {
+#pragma unroll
+                                for (int r = 0; r < 8; ++r)
+                                    zi = fmaf(-elem(Sm, toff(c0 + r, i)), w[r], zi);
+                            }
+                            pair_barrier(wg, x);
+                            if (i < c0)
+                                misc.y0[x][i] = zi;
+#pragma unroll
+                            for (int r = 0; r < 8; ++r)
+                                if (i == c0 + r && (x == 0 || valid_b))
+                                    p.u[inst_x[x] * (long long)N + i] = -w[r];
+                        }
                     }
-                    store_row_tf32(X1, wt, z);         // row wt of [Z_a'; Z_b'] (Linv is dead)
                 }
-                tc_fence_before();
                 async_proxy_fence();
                 wg_barrier(wg);
-                dead = misc.dead != 0;
-                // (5a) DP_a (R3, lanes 64..127) -= Z_a' Z_a : A operand rows 64..127 = Z_a' (rows 0..63 = tail of X0, unused)
+                dead = dead || misc.dead != 0;
+                // (5a) DP_a (R3, lanes 64..127) -= Z_a' Z_a : A operand rows 64..127 = Z_a' (rows 0..63 = the A' rows of BA, unused)
                 // (5b) DP_b (R0, lanes 64..127) -= Z_b' Z_b : A operand = [Z_a'; Z_b']
                 if (wt == 0) {
                     tc_fence_after();
-                    gemm_ss(R3, smem_u32(X1) - MAT_BYTES, smem_u32(X1), 64, 1, true);
-                    gemm_ss(R0, smem_u32(X1), smem_u32(X1) + MAT_BYTES, 64, 1, true);
+                    gemm_ss(R3, smem_u32(X0) - MAT_BYTES, smem_u32(X0), 64, 1, true);
+                    gemm_ss(R0, smem_u32(X0), smem_u32(X0) + MAT_BYTES, 64, 1, true);
                     mma_commit(mbar);
                 }
                 // P_t = Q + DP: warps 2, 3 own the rows (lanes 64..127)
