@@ -379,12 +379,6 @@ __device__ __forceinline__ void store_row_tf32(unsigned char* buf, int r, const 
         *reinterpret_cast<float4*>(buf + toff(r, 4 * c)) =
             make_float4(round_tf32(v[4 * c]), round_tf32(v[4 * c + 1]), round_tf32(v[4 * c + 2]), round_tf32(v[4 * c + 3]));
 }
-__device__ __forceinline__ void store_row_f32(unsigned char* buf, int r, const float (&v)[64])
-{
-#pragma unroll
-    for (int c = 0; c < 16; ++c)
-        *reinterpret_cast<float4*>(buf + toff(r, 4 * c)) = make_float4(v[4 * c], v[4 * c + 1], v[4 * c + 2], v[4 * c + 3]);
-}
 __device__ __forceinline__ void store_row_global(float* dst, const float (&v)[64])
 {
 #pragma unroll
@@ -523,15 +517,6 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
                     gemm_ts(R3, R0, smem_u32(BA) + MAT_BYTES, 64);
                     mma_commit(mbar);
                 }
-                // operands that do not depend on the MMA: R row (warps 0, 1)
-                float rrow[64];
-                if (warp < 2) {
-#pragma unroll
-                    for (int c = 0; c < 16; ++c) {
-                        const float4 v = __ldg(reinterpret_cast<const float4*>(Rg + (long long)wt * N) + c);
-                        rrow[4 * c] = v.x; rrow[4 * c + 1] = v.y; rrow[4 * c + 2] = v.z; rrow[4 * c + 3] = v.w;
-                    }
-                }
                 wait_mma();
                 // (2b) back half first: DP_b -> R0 (W_a is dead), runs while F_a is read out
                 if (wt == 0)
@@ -541,25 +526,24 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
                     if (x == 1) {
                         wait_mma();
                     }
-                    float f[64];
-                    {
-                        float h0[32], h1[32];
-                        tmem_ld32(R2 + lane_sel, h0);
-                        tmem_ld32(R2 + lane_sel + 32, h1);
 #pragma unroll
-                        for (int c = 0; c < 32; ++c) {
-                            f[c] = h0[c];
-                            f[32 + c] = h1[c];
+                    for (int half = 0; half < 2; ++half) {
+                        float h[32];
+                        tmem_ld32(R2 + lane_sel + 32 * half, h);
+                        if (warp < 2) {                // S_x = R + B'P_x B, fp32 -> X1
+                            const float4* rr = reinterpret_cast<const float4*>(Rg + (long long)wt * N + 32 * half);
+#pragma unroll
+                            for (int c = 0; c < 8; ++c) {
+                                const float4 r4 = __ldg(rr + c);
+                                *reinterpret_cast<float4*>(X1 + x * MAT_BYTES + toff(wt, 32 * half + 4 * c)) =
+                                    make_float4(h[4 * c] + r4.x, h[4 * c + 1] + r4.y, h[4 * c + 2] + r4.z, h[4 * c + 3] + r4.w);
+                            }
+                        } else {                       // Y_x' -> X0, fp32 (P is dead once (1) has completed)
+#pragma unroll
+                            for (int c = 0; c < 8; ++c)
+                                *reinterpret_cast<float4*>(X0 + toff(64 * x + (wt - 64), 32 * half + 4 * c)) =
+                                    make_float4(h[4 * c], h[4 * c + 1], h[4 * c + 2], h[4 * c + 3]);
                         }
-                    }
-                    if (warp < 2) {                    // S_x = R + B'P_x B, fp32 -> X1
-#pragma unroll
-                        for (int c = 0; c < 16; ++c)
-                            *reinterpret_cast<float4*>(X1 + x * MAT_BYTES + toff(wt, 4 * c)) =
-                                make_float4(f[4 * c] + rrow[4 * c], f[4 * c + 1] + rrow[4 * c + 1],
-                                            f[4 * c + 2] + rrow[4 * c + 2], f[4 * c + 3] + rrow[4 * c + 3]);
-                    } else {                           // Y_x' -> X0, fp32 (P is dead once (1) has completed)
-                        store_row_f32(X0, 64 * x + (wt - 64), f);
                     }
                     tc_fence_before();
                     wg_barrier(wg);
