@@ -322,10 +322,12 @@ __device__ __forceinline__ void pair_chol_solve(unsigned char* Sm, unsigned char
                 const float2 hi = *reinterpret_cast<const float2*>(pc + 2 * j * SC + SR);
                 acc[j - 1][0] = lo.x; acc[j - 1][1] = lo.y; acc[j - 1][2] = hi.x; acc[j - 1][3] = hi.y;
             }
+            if (is_s) {                                // rows of Y' in the panel are already tf32: their low part is zero
 #pragma unroll
-            for (int j = 1; j < 8; ++j)
-                if (!(j <= k || (is_s && j > 2 * mt + 1)))
-                    mma_16x8x8(acc[j - 1], al[0], al[1], al[2], al[3], bh[j - 1][0], bh[j - 1][1]);
+                for (int j = 1; j < 8; ++j)
+                    if (!(j <= k || j > 2 * mt + 1))
+                        mma_16x8x8(acc[j - 1], al[0], al[1], al[2], al[3], bh[j - 1][0], bh[j - 1][1]);
+            }
 #pragma unroll
             for (int j = 1; j < 8; ++j)
                 if (!(j <= k || (is_s && j > 2 * mt + 1)))
