@@ -1,0 +1,408 @@
+// Riccati-backward + rollout kernel for n = m = 16 or 32, fp32 FFMA throughout.
+//
+// N lanes of a warp own one instance (two instances per warp when N = 16); lane c holds COLUMN c of
+// every per-instance matrix in registers.  Because P, S, Q and R are symmetric, column c of them is
+// also row c, so no transposition is ever needed:
+//   V[:,c] = P B[:,c], T[:,c] = P A[:,c]      rows of P broadcast from the instance's scratch
+//   S[:,c] = R[:,c] + B' V[:,c]               rows of B broadcast from the per-head operands
+//   Y[:,c] = B' T[:,c],  Pn[:,c] = Q[:,c] + A' T[:,c]
+//   S = L L'                                  warp-level Cholesky, one row per lane (row c = column c)
+//   Z[:,c] = L^{-1} Y[:,c]                    in-lane forward substitution, columns of L broadcast
+//   Pn[:,c] -= Z' Z[:,c]                      rows of Z broadcast          (P_t = Q + A'P A - Y'S^{-1}Y)
+//   K[:,c] = -L^{-T} Z[:,c]                   in-lane back substitution (only when gains are needed)
+// (Prop. 3.1; Alg. 1 backward loop), then the forward loop of Alg. 1 with one output row per lane.
+// All cross-lane traffic goes through broadcast reads of shared memory rows (row stride N + 4 floats:
+// 16-byte vector accesses by row owners and 4-byte accesses by column owners are both conflict-free).
+//
+// CTAs of 4 warps take chunks of consecutive tokens of one (sequence, head) from an atomic counter
+// and keep that head's A, B, R in shared memory.
+#pragma once
+
+#include "common.cuh"
+
+namespace ttc {
+namespace rwarp {
+
+constexpr int WARPS = 4;
+constexpr int THREADS = 32 * WARPS;
+
+template <int N>
+struct Shape {
+    static constexpr int LD = N + 4;               // row stride in floats
+    static constexpr int IPW = 32 / N;             // instances per warp
+    static constexpr int SLOTS = WARPS * IPW;      // instances in flight per CTA = tokens per chunk
+    static constexpr int MAT = N * LD;
+};
+
+template <int N>
+struct Smem {
+    float A[Shape<N>::MAT], B[Shape<N>::MAT], R[Shape<N>::MAT];
+    struct Slot {
+        float buf0[Shape<N>::MAT];     // rows of P, then rows of Z
+        float L[Shape<N>::MAT];        // rows of L
+        float Lt[Shape<N>::MAT];       // rows of L' (columns of L); K_0 rows when only u_0 is wanted
+        float rinv[N];                 // 1 / L[i][i]
+        float x[N], u[N];
+    } slot[Shape<N>::SLOTS];
+    int chunk;
+};
+
+// Cholesky of an N x N SPD matrix spread over N lanes (lane i = row i = column i).  On return s holds
+// row `c` of L (entries right of the diagonal are meaningless), rs_own = 1 / L[c][c].  The trailing
+// update uses s_ij s_cj / d_j so that the broadcast of column j does not wait for the reciprocal.
+// Returns 0 or 1 + the index of the first non-positive pivot.
+template <int N>
+__device__ __forceinline__ int seg_chol(float (&s)[N], float& rs_own, int c)
+{
+    int bad = 0;
+    rs_own = 1.f;
+#pragma unroll
+    for (int j = 0; j < N; ++j) {
+        const float sj = s[j];
+        float d = __shfl_sync(0xffffffffu, sj, j, N);
+        if (!(d > 0.f)) {
+            if (!bad)
+                bad = j + 1;
+            d = 1.f;
+        }
+        const float rinv = __frcp_rn(d);
+        const float f = sj * rinv;
+#pragma unroll
+        for (int cc = j + 1; cc < N; ++cc) {
+            const float lc = __shfl_sync(0xffffffffu, sj, cc, N);
+            s[cc] = fmaf(-f, lc, s[cc]);
+        }
+        const float rs = rsqrtf(d);
+        s[j] = sj * rs;
+        if (c == j)
+            rs_own = rs;
+    }
+    return bad;
+}
+
+template <int N>
+__device__ __forceinline__ void load_row(float (&v)[N], const float* row)
+{
+#pragma unroll
+    for (int q = 0; q < N / 4; ++q) {
+        const float4 t = *reinterpret_cast<const float4*>(row + 4 * q);
+        v[4 * q] = t.x; v[4 * q + 1] = t.y; v[4 * q + 2] = t.z; v[4 * q + 3] = t.w;
+    }
+}
+template <int N>
+__device__ __forceinline__ void store_row(float* row, const float (&v)[N])
+{
+#pragma unroll
+    for (int q = 0; q < N / 4; ++q)
+        *reinterpret_cast<float4*>(row + 4 * q) = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+}
+// row c of the (symmetric) Q of one instance, fp32 or bf16 in global memory
+template <int N>
+__device__ __forceinline__ void load_q_row(float (&q)[N], const OperandDev& Q, long long off)
+{
+    if (Q.dtype == TTC_BF16) {
+        const uint4* src = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(Q.ptr) + off);
+#pragma unroll
+        for (int g = 0; g < N / 8; ++g) {
+            const uint4 v = __ldg(src + g);
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                q[8 * g + 2 * e] = __uint_as_float(w[e] << 16);
+                q[8 * g + 2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u);
+            }
+        }
+    } else {
+        const float4* src = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(Q.ptr) + off);
+#pragma unroll
+        for (int g = 0; g < N / 4; ++g) {
+            const float4 v = __ldg(src + g);
+            q[4 * g] = v.x; q[4 * g + 1] = v.y; q[4 * g + 2] = v.z; q[4 * g + 3] = v.w;
+        }
+    }
+}
+// acc[l] += w * row[l]
+template <int N>
+__device__ __forceinline__ void axpy_row(float (&acc)[N], float w, const float* row)
+{
+#pragma unroll
+    for (int q = 0; q < N / 4; ++q) {
+        const float4 t = *reinterpret_cast<const float4*>(row + 4 * q);
+        acc[4 * q] = fmaf(w, t.x, acc[4 * q]);
+        acc[4 * q + 1] = fmaf(w, t.y, acc[4 * q + 1]);
+        acc[4 * q + 2] = fmaf(w, t.z, acc[4 * q + 2]);
+        acc[4 * q + 3] = fmaf(w, t.w, acc[4 * q + 3]);
+    }
+}
+
+template <int N>
+__global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kernel(SolveParams p, int* chunk_counter)
+{
+    using S = Shape<N>;
+    constexpr int LD = S::LD;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    Smem<N>& sm = *reinterpret_cast<Smem<N>*>(smem_raw);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int sub = lane / N, c = lane % N;
+    typename Smem<N>::Slot& sl = sm.slot[warp * S::IPW + sub];
+    const int H = p.H;
+    const long long chunks_per_head = (p.b2 + S::SLOTS - 1) / S::SLOTS;
+    const long long nchunks = p.b0 * p.b1 * chunks_per_head;
+    const bool need_K_all = (p.K != nullptr) || (p.x != nullptr) || (p.u != nullptr && !p.first_only);
+    const bool want_u0 = (p.u != nullptr) && p.first_only && !need_K_all;
+    float* Kbase = p.K ? p.K : p.Kws;
+    long long offA = -1, offB = -1, offR = -1;
+
+    for (;;) {
+        __syncthreads();
+        if (tid == 0)
+            sm.chunk = atomicAdd(chunk_counter, 1);
+        __syncthreads();
+        const long long chunk = sm.chunk;
+        if (chunk >= nchunks)
+            break;
+        const long long head = chunk / chunks_per_head;
+        const long long tok0 = (chunk % chunks_per_head) * S::SLOTS;
+        const long long inst0 = head * p.b2 + tok0;
+        const int ntok = (int)min((long long)S::SLOTS, p.b2 - tok0);
+        {
+            const long long oa = operand_offset(p.A, inst0, p.b1, p.b2);
+            const long long ob = operand_offset(p.B, inst0, p.b1, p.b2);
+            const long long orr = operand_offset(p.R, inst0, p.b1, p.b2);
+            if (oa != offA || ob != offB || orr != offR) {
+                const float* Ag = reinterpret_cast<const float*>(p.A.ptr) + oa;
+                const float* Bg = reinterpret_cast<const float*>(p.B.ptr) + ob;
+                const float* Rg = reinterpret_cast<const float*>(p.R.ptr) + orr;
+                for (int e = tid; e < N * N; e += THREADS) {
+                    const int r = e / N, cc = e % N;
+                    sm.A[r * LD + cc] = __ldg(Ag + e);
+                    sm.B[r * LD + cc] = __ldg(Bg + e);
+                    sm.R[r * LD + cc] = __ldg(Rg + e);
+                }
+                offA = oa; offB = ob; offR = orr;
+            }
+        }
+        __syncthreads();
+        const int slot_idx = warp * S::IPW + sub;
+        const bool active = slot_idx < ntok;                  // idle segments shadow the chunk's first instance
+        const long long inst = inst0 + (active ? slot_idx : 0);
+        const long long oq = operand_offset(p.Q, inst, p.b1, p.b2) + (long long)c * N;
+
+        float* Pout = (p.P && active) ? p.P + inst * (long long)(p.first_only ? 1 : H + 1) * N * N : nullptr;
+        float* Kout = (Kbase && need_K_all) ? Kbase + inst * (long long)H * N * N : nullptr;
+        float pcol[N];
+        load_q_row<N>(pcol, p.Q, oq);                         // P_H = Q
+        if (Pout && !p.first_only) {
+#pragma unroll
+            for (int l = 0; l < N; ++l)
+                Pout[(long long)H * N * N + l * N + c] = pcol[l];
+        }
+        store_row<N>(sl.buf0 + c * LD, pcol);
+        if (p.x0.ptr)
+            sl.x[c] = load_elem(p.x0, operand_offset(p.x0, inst, p.b1, p.b2) + c);
+        __syncwarp();
+        int fail = 0;
+
+#pragma unroll 1
+        for (int ts = H - 1; ts >= 0; --ts) {
+            float vcol[N], tcol[N];
+#pragma unroll
+            for (int k = 0; k < N; ++k) {
+                vcol[k] = 0.f;
+                tcol[k] = 0.f;
+            }
+#pragma unroll 4
+            for (int i = 0; i < N; ++i) {                     // V[:,c] = P B[:,c], T[:,c] = P A[:,c]
+                const float bic = sm.B[i * LD + c], aic = sm.A[i * LD + c];
+                const float* prow = sl.buf0 + i * LD;
+#pragma unroll
+                for (int q = 0; q < N / 4; ++q) {
+                    const float4 t = *reinterpret_cast<const float4*>(prow + 4 * q);
+                    vcol[4 * q] = fmaf(t.x, bic, vcol[4 * q]);
+                    vcol[4 * q + 1] = fmaf(t.y, bic, vcol[4 * q + 1]);
+                    vcol[4 * q + 2] = fmaf(t.z, bic, vcol[4 * q + 2]);
+                    vcol[4 * q + 3] = fmaf(t.w, bic, vcol[4 * q + 3]);
+                    tcol[4 * q] = fmaf(t.x, aic, tcol[4 * q]);
+                    tcol[4 * q + 1] = fmaf(t.y, aic, tcol[4 * q + 1]);
+                    tcol[4 * q + 2] = fmaf(t.z, aic, tcol[4 * q + 2]);
+                    tcol[4 * q + 3] = fmaf(t.w, aic, tcol[4 * q + 3]);
+                }
+            }
+            // stage the two columns in the instance's scratch (own column only: no exchange) so that the next loop
+            // can run over k without indexing registers dynamically
+#pragma unroll
+            for (int k = 0; k < N; ++k) {
+                sl.L[k * LD + c] = vcol[k];
+                sl.Lt[k * LD + c] = tcol[k];
+            }
+            float s[N], y[N];
+            load_row<N>(s, sm.R + c * LD);                    // S[:,c] = R[:,c] + B' V[:,c]
+#pragma unroll
+            for (int l = 0; l < N; ++l)
+                y[l] = 0.f;
+            load_q_row<N>(pcol, p.Q, oq);                     // Pn[:,c] = Q[:,c] + A' T[:,c] ; Y[:,c] = B' T[:,c]
+#pragma unroll 4
+            for (int k = 0; k < N; ++k) {
+                const float vk = sl.L[k * LD + c], tk = sl.Lt[k * LD + c];
+                axpy_row<N>(s, vk, sm.B + k * LD);
+                axpy_row<N>(y, tk, sm.B + k * LD);
+                axpy_row<N>(pcol, tk, sm.A + k * LD);
+            }
+            float rs_own;
+            const int bad = seg_chol<N>(s, rs_own, c);
+            if (bad && !fail)
+                fail = ts * N + bad;
+            __syncwarp();                                     // every lane is done with the rows of P in buf0
+            store_row<N>(sl.L + c * LD, s);
+#pragma unroll
+            for (int k = 0; k < N; ++k)
+                sl.Lt[k * LD + c] = s[k];
+            sl.rinv[c] = rs_own;
+            __syncwarp();
+            float rinv[N];
+            load_row<N>(rinv, sl.rinv);
+#pragma unroll
+            for (int k = 0; k < N; ++k) {                     // Z[:,c] = L^{-1} Y[:,c]
+                const float zk = y[k] * rinv[k];
+                y[k] = zk;
+                const float* lt = sl.Lt + k * LD;
+#pragma unroll
+                for (int i4 = (k + 1) & ~3; i4 < N; i4 += 4) {
+                    const float4 l4 = *reinterpret_cast<const float4*>(lt + i4);
+                    if (i4 + 0 > k) y[i4 + 0] = fmaf(-l4.x, zk, y[i4 + 0]);
+                    if (i4 + 1 > k) y[i4 + 1] = fmaf(-l4.y, zk, y[i4 + 1]);
+                    if (i4 + 2 > k) y[i4 + 2] = fmaf(-l4.z, zk, y[i4 + 2]);
+                    if (i4 + 3 > k) y[i4 + 3] = fmaf(-l4.w, zk, y[i4 + 3]);
+                }
+            }
+#pragma unroll
+            for (int q = 0; q < N; ++q)
+                sl.buf0[q * LD + c] = y[q];                   // rows of Z
+            __syncwarp();
+#pragma unroll 4
+            for (int q = 0; q < N; ++q)                       // Pn[:,c] -= Z' Z[:,c]
+                axpy_row<N>(pcol, -sl.buf0[q * LD + c], sl.buf0 + q * LD);
+            const bool gains = need_K_all || (want_u0 && ts == 0);
+            if (gains) {                                      // K[:,c] = -L^{-T} Z[:,c]
+#pragma unroll
+                for (int k = N - 1; k >= 0; --k) {
+                    const float xk = y[k] * rinv[k];
+                    y[k] = xk;
+                    const float* lr = sl.L + k * LD;
+#pragma unroll
+                    for (int i4 = 0; i4 < k; i4 += 4) {
+                        const float4 l4 = *reinterpret_cast<const float4*>(lr + i4);
+                        if (i4 + 0 < k) y[i4 + 0] = fmaf(-l4.x, xk, y[i4 + 0]);
+                        if (i4 + 1 < k) y[i4 + 1] = fmaf(-l4.y, xk, y[i4 + 1]);
+                        if (i4 + 2 < k) y[i4 + 2] = fmaf(-l4.z, xk, y[i4 + 2]);
+                        if (i4 + 3 < k) y[i4 + 3] = fmaf(-l4.w, xk, y[i4 + 3]);
+                    }
+                }
+                if (need_K_all) {
+                    if (active) {
+                        float* kt = Kout + (long long)ts * N * N + c;
+#pragma unroll
+                        for (int l = 0; l < N; ++l)
+                            kt[l * N] = -y[l];
+                    }
+                } else {                                      // K_0 rows -> Lt (free after the forward substitution)
+#pragma unroll
+                    for (int l = 0; l < N; ++l)
+                        sl.Lt[l * LD + c] = -y[l];
+                }
+            }
+            if (Pout && (!p.first_only || ts == 0)) {
+                float* pt = Pout + (long long)(p.first_only ? 0 : ts) * N * N + c;
+#pragma unroll
+                for (int l = 0; l < N; ++l)
+                    pt[l * N] = pcol[l];
+            }
+            __syncwarp();                                     // rows of Z consumed
+            store_row<N>(sl.buf0 + c * LD, pcol);             // rows of P_t (row c = column c)
+            __syncwarp();
+        }
+
+        // A failure is known to every lane of the segment.  Control flow stays warp-uniform (the two
+        // segments of a warp may differ): a failed instance only loses its stores.
+        if (fail && active) {
+            const float qn = quiet_nan();
+            if (p.K)
+                for (long long e = c; e < (long long)H * N * N; e += N)
+                    p.K[inst * (long long)H * N * N + e] = qn;
+            if (p.P) {
+                const long long cnt = (long long)(p.first_only ? 1 : H + 1) * N * N;
+                for (long long e = c; e < cnt; e += N)
+                    p.P[inst * cnt + e] = qn;
+            }
+            if (p.x)
+                for (long long e = c; e < (long long)(H + 1) * N; e += N)
+                    p.x[inst * (long long)(H + 1) * N + e] = qn;
+            if (p.u) {
+                const long long cnt = p.first_only ? N : (long long)H * N;
+                for (long long e = c; e < cnt; e += N)
+                    p.u[inst * cnt + e] = qn;
+            }
+        }
+        if (p.info && active && c == 0)
+            p.info[inst] = fail;
+        const bool store_ok = active && !fail;
+
+        // ---- forward loop of Alg. 1: lane c computes u_t[c] and x_{t+1}[c]
+        if (want_u0) {
+            float kr[N], xv[N];
+            load_row<N>(kr, sl.Lt + c * LD);
+            load_row<N>(xv, sl.x);
+            float uc = 0.f;
+#pragma unroll
+            for (int j = 0; j < N; ++j)
+                uc = fmaf(kr[j], xv[j], uc);
+            if (store_ok)
+                p.u[inst * (long long)N + c] = uc;
+        } else if (p.x || p.u) {
+            float* xo = (p.x && store_ok) ? p.x + inst * (long long)(H + 1) * N : nullptr;
+            float* uo = (p.u && store_ok) ? p.u + inst * (long long)(p.first_only ? N : H * N) : nullptr;
+            float arow[N], brow[N];
+            load_row<N>(arow, sm.A + c * LD);
+            load_row<N>(brow, sm.B + c * LD);
+            if (xo)
+                xo[c] = sl.x[c];
+            __syncwarp();                                     // K_t written by the other lanes are visible
+#pragma unroll 1
+            for (int ts = 0; ts < H; ++ts) {
+                float xv[N];
+                load_row<N>(xv, sl.x);
+                const float4* kr = reinterpret_cast<const float4*>(Kout + (long long)ts * N * N + c * N);
+                float uc = 0.f;
+#pragma unroll
+                for (int q = 0; q < N / 4; ++q) {
+                    const float4 k4 = kr[q];
+                    uc = fmaf(k4.x, xv[4 * q], uc);
+                    uc = fmaf(k4.y, xv[4 * q + 1], uc);
+                    uc = fmaf(k4.z, xv[4 * q + 2], uc);
+                    uc = fmaf(k4.w, xv[4 * q + 3], uc);
+                }
+                sl.u[c] = uc;
+                if (uo && (!p.first_only || ts == 0))
+                    uo[(p.first_only ? 0 : ts * N) + c] = uc;
+                __syncwarp();
+                float uv[N];
+                load_row<N>(uv, sl.u);
+                float xc = 0.f;
+#pragma unroll
+                for (int j = 0; j < N; ++j)
+                    xc = fmaf(arow[j], xv[j], fmaf(brow[j], uv[j], xc));
+                __syncwarp();                                 // x_t consumed by every lane
+                sl.x[c] = xc;
+                if (xo)
+                    xo[(long long)(ts + 1) * N + c] = xc;
+                __syncwarp();
+            }
+        }
+    }
+}
+
+template <int N>
+inline size_t smem_bytes() { return sizeof(Smem<N>); }
+
+} // namespace rwarp
+} // namespace ttc

@@ -12,6 +12,7 @@
 #include "riccati_cta.cuh"
 #include "riccati_mma64.cuh"
 #include "riccati_umma64.cuh"
+#include "riccati_warp.cuh"
 #include "scan_pair.cuh"
 
 using namespace ttc;
@@ -353,6 +354,32 @@ int ttc_lqr_solve(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B,
             TTC_CUDA(cudaGetLastError());
             h->last_launches = 1;
             h->last_kernel = TTC_KERNEL_RICCATI_MMA;
+            h->total_launches += h->last_launches;
+            return TTC_OK;
+        }
+        if (head_shared && n == m && (n == 16 || n == 32)) {
+            // fp32 warp kernel: one instance per 16 / 32 lanes, chunks of tokens handed out by an atomic counter
+            if ((s = ensure(h->ws_E, sizeof(int) * 4))) return s;
+            int* counter = static_cast<int*>(h->ws_E.ptr);
+            TTC_CUDA(cudaMemsetAsync(counter, 0, sizeof(int), st));
+            if (n == 32) {
+                const size_t smem = rwarp::smem_bytes<32>();
+                TTC_CUDA(cudaFuncSetAttribute(rwarp::riccati_warp_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+                const long long chunks = p.b0 * p.b1 * ((p.b2 + rwarp::Shape<32>::SLOTS - 1) / rwarp::Shape<32>::SLOTS);
+                long long grid = (long long)h->sm_count * 3;
+                if (grid > chunks) grid = chunks;
+                rwarp::riccati_warp_kernel<32><<<(unsigned)grid, rwarp::THREADS, smem, st>>>(p, counter);
+            } else {
+                const size_t smem = rwarp::smem_bytes<16>();
+                TTC_CUDA(cudaFuncSetAttribute(rwarp::riccati_warp_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+                const long long chunks = p.b0 * p.b1 * ((p.b2 + rwarp::Shape<16>::SLOTS - 1) / rwarp::Shape<16>::SLOTS);
+                long long grid = (long long)h->sm_count * 4;
+                if (grid > chunks) grid = chunks;
+                rwarp::riccati_warp_kernel<16><<<(unsigned)grid, rwarp::THREADS, smem, st>>>(p, counter);
+            }
+            TTC_CUDA(cudaGetLastError());
+            h->last_launches = 1;
+            h->last_kernel = TTC_KERNEL_RICCATI_WARP;
             h->total_launches += h->last_launches;
             return TTC_OK;
         }
