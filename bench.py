@@ -285,7 +285,7 @@ def main():
     t_hbm = alg_bytes / (peaks["hbm_gbs"] * 1e9)
     fp32_peak = SM_COUNT * FP32_LANES_PER_SM * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12
     tf32_peak = peaks["bf16_tflops_sustained"] * TF32_TO_BF16_RATIO
-    if kname in ("riccati_mma", "riccati_umma"):
+    if kname == "riccati_umma":
         bound, peak, unit, ach = "tensor", tf32_peak, "TFLOP/s", alg_flops / (kernel_ms * 1e-3) / 1e12
         peak_note = "tf32 = measured sustained bf16 x 0.5 (nominal ratio), of %s" % peaks["source"]
     else:
@@ -321,7 +321,7 @@ def main():
 
     line = {"metric": "lqr_instances_per_sec", "value": value, "unit": "instances/s", "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "tf32" if kname in ("riccati_mma", "riccati_umma") else "f32",
+            "scaling": "weak", "vs_baseline": None, "dtype": "tf32" if kname == "riccati_umma" else "f32",
             "data": "synthetic",
             "config": {"workload": c["name"], "n": n, "m": m, "H": H, "instances": N, "batch": list(c["batch"]),
                        "q_x0_dtype": c["q_dtype"], "outputs": list(want), "method": args.method, "kernel": kname,

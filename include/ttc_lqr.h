@@ -61,7 +61,7 @@ extern "C" {
 /* ttc_lqr_config.math : arithmetic of the n x n contractions */
 #define TTC_MATH_AUTO  0  /* FP32 when every input is F32, TF32 when Q or x0 is BF16  */
 #define TTC_MATH_FP32  1  /* FFMA, fp32 throughout                                    */
-#define TTC_MATH_TF32  2  /* tensor cores, tf32 operands, fp32 accumulate (n = m = 64)*/
+#define TTC_MATH_TF32  2  /* tcgen05 tensor cores, tf32 operands, fp32 accumulate (n = m = 64) */
 
 /* ttc_lqr_solve flags */
 #define TTC_OUT_FIRST_ONLY  1u  /* P is [N][n][n] = P_0 and u is [N][m] = u_0          */
@@ -78,7 +78,7 @@ extern "C" {
 #define TTC_KERNEL_NONE           0
 #define TTC_KERNEL_RICCATI_CTA    1  /* generic: one CTA per instance, FFMA            */
 #define TTC_KERNEL_RICCATI_WARP   2  /* register-tiled FFMA, several instances per CTA */
-#define TTC_KERNEL_RICCATI_MMA    3  /* tensor-core contractions, n = m = 64           */
+#define TTC_KERNEL_RICCATI_MMA    3  /* retired id (mma.sync kernel); never returned   */
 #define TTC_KERNEL_SCAN           4  /* symplectic-pair scan + gain/rollout kernel     */
 #define TTC_KERNEL_RICCATI_UMMA   5  /* tcgen05 contractions (tensor memory), n = m = 64 */
 

@@ -348,6 +348,96 @@ __device__ __forceinline__ void pair_chol_solve(unsigned char* Sm, unsigned char
     }
 }
 
+// Gains (Eq. 4): K = -L^{-T} Z, i.e. row c of K' is -(row c of Z') L^{-1}.  Same two warps, same blocked scheme
+// run backwards: per 8-wide block kb = 7..0 every row owner solves x L_d = z for its row of Z' (in place in
+// `Ym`), then the columns left of the block get the update Z'[c][j] -= x[c][kb] . L[kb][j] as 3 x tf32 mma.
+// On return row c of Ym holds (Z' L^{-1})[c][:] = -K[:, c] (fp32).
+__device__ __forceinline__ void pair_gain_solve(const unsigned char* Sm, unsigned char* Ym, int wg, int x, int pw, int lane)
+{
+    const int g = lane >> 2, t = lane & 3;
+    const int tid2 = 32 * pw + lane;
+    const uint32_t frag_ab = (uint32_t)g * 16u + (uint32_t)t * 4u;
+    const uint32_t frag_c = (uint32_t)g * 16u + (uint32_t)(t >> 1) * SC + (uint32_t)((2 * t) & 3) * 4u;
+    const uint32_t frag_b = (uint32_t)t * 16u + (uint32_t)(g >> 2) * SC + (uint32_t)(g & 3) * 4u;   // (row t, col g) of a tile
+    const uint32_t own_row = (uint32_t)(tid2 >> 3) * SR + (uint32_t)(tid2 & 7) * 16u;
+#pragma unroll 1
+    for (int kb = 7; kb >= 0; --kb) {
+        const uint32_t kcol = 2u * kb * SC;
+        const unsigned char* dblk = Sm + (uint32_t)kb * SR + kcol;
+        float l[8][8], xr[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            load_row8(l[i], dblk + i * 16);
+        unsigned char* py = Ym + own_row + kcol;
+        load_row8(xr, py);
+#pragma unroll
+        for (int j = 7; j >= 0; --j) {                 // x L_d = z, L_d lower triangular
+            float v = xr[j];
+#pragma unroll
+            for (int i = j + 1; i < 8; ++i)
+                v = fmaf(-xr[i], l[i][j], v);
+            xr[j] = __fdividef(v, l[j][j]);
+        }
+        store_row8<false>(py, xr);
+        if (kb == 0)
+            break;
+        pair_barrier(wg, x);
+        // B fragments: rows 8kb + t, 8kb + t + 4 of L, columns 8j + g (j < kb)
+        uint32_t bh[7][2], bl[7][2];
+        {
+            const unsigned char* pb = Sm + (uint32_t)kb * SR + frag_b;
+#pragma unroll
+            for (int j = 0; j < 7; ++j)
+                if (j < kb) {
+                    split_tf32(*reinterpret_cast<const float*>(pb + 2 * j * SC), bh[j][0], bl[j][0]);
+                    split_tf32(*reinterpret_cast<const float*>(pb + 2 * j * SC + 64), bh[j][1], bl[j][1]);
+                }
+        }
+#pragma unroll
+        for (int uu = 0; uu < 2; ++uu) {
+            const int mt = 2 * uu + pw;
+            uint32_t ah[4], al[4];
+            {
+                const unsigned char* pa = Ym + frag_ab + kcol + 2 * mt * SR;
+                split_tf32(-*reinterpret_cast<const float*>(pa), ah[0], al[0]);
+                split_tf32(-*reinterpret_cast<const float*>(pa + SR), ah[1], al[1]);
+                split_tf32(-*reinterpret_cast<const float*>(pa + SC), ah[2], al[2]);
+                split_tf32(-*reinterpret_cast<const float*>(pa + SR + SC), ah[3], al[3]);
+            }
+            unsigned char* pc = Ym + frag_c + 2 * mt * SR;
+            float acc[7][4];
+#pragma unroll
+            for (int j = 0; j < 7; ++j) {
+                if (j >= kb)
+                    continue;
+                const float2 lo = *reinterpret_cast<const float2*>(pc + 2 * j * SC);
+                const float2 hi = *reinterpret_cast<const float2*>(pc + 2 * j * SC + SR);
+                acc[j][0] = lo.x; acc[j][1] = lo.y; acc[j][2] = hi.x; acc[j][3] = hi.y;
+            }
+#pragma unroll
+            for (int j = 0; j < 7; ++j)
+                if (j < kb)
+                    mma_16x8x8(acc[j], al[0], al[1], al[2], al[3], bh[j][0], bh[j][1]);
+#pragma unroll
+            for (int j = 0; j < 7; ++j)
+                if (j < kb)
+                    mma_16x8x8(acc[j], ah[0], ah[1], ah[2], ah[3], bl[j][0], bl[j][1]);
+#pragma unroll
+            for (int j = 0; j < 7; ++j)
+                if (j < kb)
+                    mma_16x8x8(acc[j], ah[0], ah[1], ah[2], ah[3], bh[j][0], bh[j][1]);
+#pragma unroll
+            for (int j = 0; j < 7; ++j) {
+                if (j >= kb)
+                    continue;
+                *reinterpret_cast<float2*>(pc + 2 * j * SC) = make_float2(acc[j][0], acc[j][1]);
+                *reinterpret_cast<float2*>(pc + 2 * j * SC + SR) = make_float2(acc[j][2], acc[j][3]);
+            }
+        }
+        pair_barrier(wg, x);
+    }
+}
+
 // ---- global-memory helpers --------------------------------------------------------------------------------------
 // row j (64 values) of the Q matrix of one instance
 __device__ __forceinline__ void load_q_row(float (&q)[64], const OperandDev& Q, long long oq, int j)
@@ -391,19 +481,31 @@ __device__ __forceinline__ void store_row_global(float* dst, const float (&v)[64
 __device__ __forceinline__ void wg_fail_instance(const SolveParams& p, long long inst, int code, int wt)
 {
     const float qn = quiet_nan();
+    const int H = p.H;
+    if (p.K)
+        for (long long e = wt; e < (long long)H * N * N; e += WG_THREADS)
+            p.K[inst * (long long)H * N * N + e] = qn;
     if (p.P) {
-        const long long cnt = (long long)(p.first_only ? 1 : p.H + 1) * N * N;
+        const long long cnt = (long long)(p.first_only ? 1 : H + 1) * N * N;
         for (long long e = wt; e < cnt; e += WG_THREADS)
             p.P[inst * cnt + e] = qn;
     }
-    if (p.u && p.first_only && wt < N)
-        p.u[inst * (long long)N + wt] = qn;
+    if (p.x)
+        for (long long e = wt; e < (long long)(H + 1) * N; e += WG_THREADS)
+            p.x[inst * (long long)(H + 1) * N + e] = qn;
+    if (p.u) {
+        const long long cnt = p.first_only ? N : (long long)H * N;
+        for (long long e = wt; e < cnt; e += WG_THREADS)
+            p.u[inst * cnt + e] = qn;
+    }
     if (p.info && wt == 0)
         p.info[inst] = code;
 }
 
-// Supported requests: P (every P_t, or P_0 with first_only), u_0 (first_only), info.  K, x and the full u
-// are served by other kernels.
+// Every output of the solve: K_t, P_t (or P_0), x_t, u_t (or u_0), info.  When the rollout needs gains that the
+// caller did not ask for they go to the workspace p.Kws.
+// GAINS = the request needs every K_t (K, x or the full u wanted); the other instantiation carries none of that code.
+template <bool GAINS>
 __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams p, int* chunk_counter, int* error_flag)
 {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
@@ -440,7 +542,10 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
     const int H = p.H;
     const long long chunks_per_head = (p.b2 + CHUNK - 1) / CHUNK;
     const long long nchunks = p.b0 * p.b1 * chunks_per_head;
-    const bool want_u0 = (p.u != nullptr) && p.first_only;
+    constexpr bool need_K_all = GAINS;
+    const bool want_u0 = (p.u != nullptr) && p.first_only && !need_K_all;
+    const bool rollout = (p.x != nullptr) || (p.u != nullptr && need_K_all);
+    float* Kbase = p.K ? p.K : p.Kws;
     long long offA_loaded = -1, offB_loaded = -1, offR_loaded = -1;
     const float* Rg = nullptr;
     bool dead = false;
@@ -499,7 +604,7 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
                     if (p.P && !p.first_only && (x == 0 || valid_b))
                         store_row_global(p.P + (inst_x[x] * (long long)(H + 1) + H) * N * N + (long long)j * N, q);
                 }
-            } else if (want_u0) {
+            } else if (p.x0.ptr) {
                 const int x = warp, j0 = 2 * lane;             // warp x stages x_0 of instance x
                 const long long ox = operand_offset(p.x0, inst_x[x], p.b1, p.b2);
                 misc.x0[x][j0] = load_elem(p.x0, ox + j0);
@@ -617,9 +722,31 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
                 }
                 // P_t = Q + DP: warps 2, 3 own the rows (lanes 64..127)
                 float q[64];
-                if (warp >= 2)
+                if (!need_K_all && warp >= 2)
                     load_q_row(q, p.Q, oq_x[0], wt - 64);
                 wait_mma();
+                if (need_K_all) {
+                    // (5) has consumed Z': turn it into the gains in place, K_t[i][c] = -(Z' L^{-1})[c][i]
+                    const int x = warp >> 1, pw = warp & 1;
+                    unsigned char* Ym = X0 + x * MAT_BYTES;
+                    pair_gain_solve(X1 + x * MAT_BYTES, Ym, wg, x, pw, lane);
+                    const int cidx = 32 * pw + lane;
+                    if (x == 0 || valid_b) {
+                        float* kt = Kbase + (inst_x[x] * (long long)H + ts) * N * N + cidx;
+                        const unsigned char* row = Ym + (uint32_t)(cidx >> 3) * SR + (uint32_t)(cidx & 7) * 16u;
+#pragma unroll
+                        for (int q4 = 0; q4 < 16; ++q4) {
+                            const float4 v = *reinterpret_cast<const float4*>(row + q4 * SC);
+                            kt[(4 * q4 + 0) * N] = -v.x;
+                            kt[(4 * q4 + 1) * N] = -v.y;
+                            kt[(4 * q4 + 2) * N] = -v.z;
+                            kt[(4 * q4 + 3) * N] = -v.w;
+                        }
+                    }
+                    wg_barrier(wg);                    // X0 is free for the next value matrices
+                    if (warp >= 2)
+                        load_q_row(q, p.Q, oq_x[0], wt - 64);
+                }
                 if (warp >= 2) {
                     const int j = wt - 64;
 #pragma unroll 1
@@ -649,6 +776,47 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
             }
             if (dead)
                 break;
+            if (rollout) {
+                // forward loop of Alg. 1 by the 64 threads of each instance: u_t = K_t x_t, x_{t+1} = A x_t + B u_t (fp32)
+                const int x = warp >> 1, i = 32 * (warp & 1) + lane;
+                const bool st = (x == 0 || valid_b) && misc.flag[x] == 0;
+                const long long inst = inst_x[x];
+                float* xo = (p.x && st) ? p.x + inst * (long long)(H + 1) * N : nullptr;
+                float* uo = (p.u && st) ? p.u + inst * (long long)(p.first_only ? 1 : H) * N : nullptr;
+                const float4* Ar = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(p.A.ptr) + offA_loaded + (long long)i * N);
+                const float4* Br = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(p.B.ptr) + offB_loaded + (long long)i * N);
+                if (xo)
+                    xo[i] = misc.x0[x][i];
+#pragma unroll 1
+                for (int ts = 0; ts < H; ++ts) {
+                    const float4* kr = reinterpret_cast<const float4*>(Kbase + (inst * (long long)H + ts) * N * N + (long long)i * N);
+                    float ui = 0.f;
+#pragma unroll
+                    for (int c4 = 0; c4 < 16; ++c4) {
+                        const float4 kv = kr[c4];
+                        const float4 xv = *reinterpret_cast<const float4*>(&misc.x0[x][4 * c4]);
+                        ui = fmaf(kv.x, xv.x, fmaf(kv.y, xv.y, fmaf(kv.z, xv.z, fmaf(kv.w, xv.w, ui))));
+                    }
+                    misc.y0[x][i] = ui;
+                    if (uo && (!p.first_only || ts == 0))
+                        uo[(p.first_only ? 0 : (long long)ts * N) + i] = ui;
+                    pair_barrier(wg, x);
+                    float xi = 0.f;
+#pragma unroll
+                    for (int c4 = 0; c4 < 16; ++c4) {
+                        const float4 av = __ldg(Ar + c4), bv = __ldg(Br + c4);
+                        const float4 xv = *reinterpret_cast<const float4*>(&misc.x0[x][4 * c4]);
+                        const float4 uv = *reinterpret_cast<const float4*>(&misc.y0[x][4 * c4]);
+                        xi = fmaf(av.x, xv.x, fmaf(av.y, xv.y, fmaf(av.z, xv.z, fmaf(av.w, xv.w, xi))));
+                        xi = fmaf(bv.x, uv.x, fmaf(bv.y, uv.y, fmaf(bv.z, uv.z, fmaf(bv.w, uv.w, xi))));
+                    }
+                    pair_barrier(wg, x);               // x_t and u_t consumed
+                    misc.x0[x][i] = xi;
+                    if (xo)
+                        xo[(long long)(ts + 1) * N + i] = xi;
+                    pair_barrier(wg, x);
+                }
+            }
             // ---- status / failed instances
 #pragma unroll 1
             for (int x = 0; x < (valid_b ? 2 : 1); ++x) {

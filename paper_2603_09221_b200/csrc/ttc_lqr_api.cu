@@ -10,7 +10,6 @@
 
 #include "common.cuh"
 #include "riccati_cta.cuh"
-#include "riccati_mma64.cuh"
 #include "riccati_umma64.cuh"
 #include "riccati_warp.cuh"
 #include "scan_pair.cuh"
@@ -320,40 +319,21 @@ int ttc_lqr_solve(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B,
         const bool bf16_in = (Q->dtype == TTC_BF16) || (x0 && x0->ptr && x0->dtype == TTC_BF16);
         const bool want_tf32 = h->cfg.math == TTC_MATH_TF32 || (h->cfg.math == TTC_MATH_AUTO && bf16_in);
         const bool head_shared = A->bstride[2] == 0 && B->bstride[2] == 0 && R->bstride[2] == 0;
-        const bool umma_outputs = !K && !x && (!u || p.first_only);
-        if (want_tf32 && n == 64 && m == 64 && head_shared && umma_outputs) {
-            // tcgen05 kernel (P_t / P_0, u_0): persistent CTAs, two independent warpgroups each
+        if (want_tf32 && n == 64 && m == 64 && head_shared) {
+            // tcgen05 kernel: persistent CTAs, two independent warpgroups each
             if ((s = ensure(h->ws_E, sizeof(int) * 4))) return s;
             int* counter = static_cast<int*>(h->ws_E.ptr);
             TTC_CUDA(cudaMemsetAsync(counter, 0, 2 * sizeof(int), st));
             const size_t smem = umma64::smem_bytes();
-            TTC_CUDA(cudaFuncSetAttribute(umma64::riccati_umma64_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          (int)smem));
+            auto kern = rollout_needs_all_K || K ? umma64::riccati_umma64_kernel<true> : umma64::riccati_umma64_kernel<false>;
+            TTC_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
             const long long chunks = p.b0 * p.b1 * ((p.b2 + umma64::CHUNK - 1) / umma64::CHUNK);
             long long grid = h->sm_count;
             if (2 * grid > chunks) grid = (chunks + 1) / 2;
-            umma64::riccati_umma64_kernel<<<(unsigned)grid, umma64::THREADS, smem, st>>>(p, counter, counter + 1);
+            kern<<<(unsigned)grid, umma64::THREADS, smem, st>>>(p, counter, counter + 1);
             TTC_CUDA(cudaGetLastError());
             h->last_launches = 1;
             h->last_kernel = TTC_KERNEL_RICCATI_UMMA;
-            h->total_launches += h->last_launches;
-            return TTC_OK;
-        }
-        if (want_tf32 && n == 64 && m == 64 && head_shared) {
-            // tensor-core kernel: persistent CTAs, work items handed out by an atomic counter
-            if ((s = ensure(h->ws_E, sizeof(int) * 4))) return s;
-            int* counter = static_cast<int*>(h->ws_E.ptr);
-            TTC_CUDA(cudaMemsetAsync(counter, 0, sizeof(int), st));
-            const size_t smem = mma64::smem_bytes();
-            TTC_CUDA(cudaFuncSetAttribute(mma64::riccati_mma64_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          (int)smem));
-            const long long chunks = p.b0 * p.b1 * ((p.b2 + mma64::CHUNK - 1) / mma64::CHUNK);
-            long long grid = h->sm_count;
-            if (grid > chunks) grid = chunks;
-            mma64::riccati_mma64_kernel<<<(unsigned)grid, mma64::THREADS, smem, st>>>(p, counter);
-            TTC_CUDA(cudaGetLastError());
-            h->last_launches = 1;
-            h->last_kernel = TTC_KERNEL_RICCATI_MMA;
             h->total_launches += h->last_launches;
             return TTC_OK;
         }

@@ -21,7 +21,7 @@ TTC_MATH_AUTO, TTC_MATH_FP32, TTC_MATH_TF32 = 0, 1, 2
 TTC_OUT_FIRST_ONLY = 1
 TTC_QUERY_LAST_LAUNCHES, TTC_QUERY_WORKSPACE_BYTES, TTC_QUERY_LAST_KERNEL, TTC_QUERY_TOTAL_LAUNCHES = 1, 2, 3, 4
 TTC_QUERY_DEVICE_ERROR = 5
-KERNEL_NAMES = {0: "none", 1: "riccati_cta", 2: "riccati_warp", 3: "riccati_mma", 4: "scan", 5: "riccati_umma"}
+KERNEL_NAMES = {0: "none", 1: "riccati_cta", 2: "riccati_warp", 4: "scan", 5: "riccati_umma"}
 
 EXPORTS = (
     "ttc_lqr_create", "ttc_lqr_solve", "ttc_lqr_solve_host", "ttc_lqr_destroy", "ttc_lqr_query",
