@@ -121,17 +121,46 @@ __device__ __forceinline__ void load_q_row(float (&q)[N], const OperandDev& Q, l
         }
     }
 }
-// acc[l] += w * row[l]
+// ---- packed fp32 pairs: fma.rn.f32x2 does two FMAs per issued instruction (the dense loops are issue-bound)
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float a, float b)
+{
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+    return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float& a, float& b)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+}
+__device__ __forceinline__ void fma2(f32x2& acc, f32x2 a, f32x2 b)
+{
+    asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(acc) : "l"(a), "l"(b));
+}
 template <int N>
-__device__ __forceinline__ void axpy_row(float (&acc)[N], float w, const float* row)
+__device__ __forceinline__ void pack_row(f32x2 (&v2)[N / 2], const float (&v)[N])
 {
 #pragma unroll
+    for (int i = 0; i < N / 2; ++i)
+        v2[i] = pack2(v[2 * i], v[2 * i + 1]);
+}
+template <int N>
+__device__ __forceinline__ void unpack_row(float (&v)[N], const f32x2 (&v2)[N / 2])
+{
+#pragma unroll
+    for (int i = 0; i < N / 2; ++i)
+        unpack2(v2[i], v[2 * i], v[2 * i + 1]);
+}
+// acc[l] += w * row[l], l = 0..N-1
+template <int N>
+__device__ __forceinline__ void axpy_row(f32x2 (&acc)[N / 2], float w, const float* row)
+{
+    const f32x2 ww = pack2(w, w);
+#pragma unroll
     for (int q = 0; q < N / 4; ++q) {
-        const float4 t = *reinterpret_cast<const float4*>(row + 4 * q);
-        acc[4 * q] = fmaf(w, t.x, acc[4 * q]);
-        acc[4 * q + 1] = fmaf(w, t.y, acc[4 * q + 1]);
-        acc[4 * q + 2] = fmaf(w, t.z, acc[4 * q + 2]);
-        acc[4 * q + 3] = fmaf(w, t.w, acc[4 * q + 3]);
+        const ulonglong2 t = *reinterpret_cast<const ulonglong2*>(row + 4 * q);
+        fma2(acc[2 * q], ww, t.x);
+        fma2(acc[2 * q + 1], ww, t.y);
     }
 }
 
@@ -205,49 +234,59 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
 
 #pragma unroll 1
         for (int ts = H - 1; ts >= 0; --ts) {
-            float vcol[N], tcol[N];
+            f32x2 vcol[N / 2], tcol[N / 2];
 #pragma unroll
-            for (int k = 0; k < N; ++k) {
-                vcol[k] = 0.f;
-                tcol[k] = 0.f;
+            for (int k = 0; k < N / 2; ++k) {
+                vcol[k] = 0ull;
+                tcol[k] = 0ull;
             }
 #pragma unroll 4
             for (int i = 0; i < N; ++i) {                     // V[:,c] = P B[:,c], T[:,c] = P A[:,c]
                 const float bic = sm.B[i * LD + c], aic = sm.A[i * LD + c];
+                const f32x2 b2 = pack2(bic, bic), a2 = pack2(aic, aic);
                 const float* prow = sl.buf0 + i * LD;
 #pragma unroll
                 for (int q = 0; q < N / 4; ++q) {
-                    const float4 t = *reinterpret_cast<const float4*>(prow + 4 * q);
-                    vcol[4 * q] = fmaf(t.x, bic, vcol[4 * q]);
-                    vcol[4 * q + 1] = fmaf(t.y, bic, vcol[4 * q + 1]);
-                    vcol[4 * q + 2] = fmaf(t.z, bic, vcol[4 * q + 2]);
-                    vcol[4 * q + 3] = fmaf(t.w, bic, vcol[4 * q + 3]);
-                    tcol[4 * q] = fmaf(t.x, aic, tcol[4 * q]);
-                    tcol[4 * q + 1] = fmaf(t.y, aic, tcol[4 * q + 1]);
-                    tcol[4 * q + 2] = fmaf(t.z, aic, tcol[4 * q + 2]);
-                    tcol[4 * q + 3] = fmaf(t.w, aic, tcol[4 * q + 3]);
+                    const ulonglong2 t = *reinterpret_cast<const ulonglong2*>(prow + 4 * q);
+                    fma2(vcol[2 * q], t.x, b2);
+                    fma2(vcol[2 * q + 1], t.y, b2);
+                    fma2(tcol[2 * q], t.x, a2);
+                    fma2(tcol[2 * q + 1], t.y, a2);
                 }
             }
             // stage the two columns in the instance's scratch (own column only: no exchange) so that the next loop
             // can run over k without indexing registers dynamically
 #pragma unroll
-            for (int k = 0; k < N; ++k) {
-                sl.L[k * LD + c] = vcol[k];
-                sl.Lt[k * LD + c] = tcol[k];
+            for (int k = 0; k < N / 2; ++k) {
+                float v0, v1, t0, t1;
+                unpack2(vcol[k], v0, v1);
+                unpack2(tcol[k], t0, t1);
+                sl.L[(2 * k) * LD + c] = v0;
+                sl.L[(2 * k + 1) * LD + c] = v1;
+                sl.Lt[(2 * k) * LD + c] = t0;
+                sl.Lt[(2 * k + 1) * LD + c] = t1;
             }
-            float s[N], y[N];
-            load_row<N>(s, sm.R + c * LD);                    // S[:,c] = R[:,c] + B' V[:,c]
+            f32x2 s2[N / 2], y2[N / 2], p2[N / 2];
+            {
+                float tmp[N];
+                load_row<N>(tmp, sm.R + c * LD);              // S[:,c] = R[:,c] + B' V[:,c]
+                pack_row<N>(s2, tmp);
+                load_q_row<N>(tmp, p.Q, oq);                  // Pn[:,c] = Q[:,c] + A' T[:,c] ; Y[:,c] = B' T[:,c]
+                pack_row<N>(p2, tmp);
+            }
 #pragma unroll
-            for (int l = 0; l < N; ++l)
-                y[l] = 0.f;
-            load_q_row<N>(pcol, p.Q, oq);                     // Pn[:,c] = Q[:,c] + A' T[:,c] ; Y[:,c] = B' T[:,c]
+            for (int l = 0; l < N / 2; ++l)
+                y2[l] = 0ull;
 #pragma unroll 4
             for (int k = 0; k < N; ++k) {
                 const float vk = sl.L[k * LD + c], tk = sl.Lt[k * LD + c];
-                axpy_row<N>(s, vk, sm.B + k * LD);
-                axpy_row<N>(y, tk, sm.B + k * LD);
-                axpy_row<N>(pcol, tk, sm.A + k * LD);
+                axpy_row<N>(s2, vk, sm.B + k * LD);
+                axpy_row<N>(y2, tk, sm.B + k * LD);
+                axpy_row<N>(p2, tk, sm.A + k * LD);
             }
+            float s[N], y[N];
+            unpack_row<N>(s, s2);
+            unpack_row<N>(y, y2);
             float rs_own;
             const int bad = seg_chol<N>(s, rs_own, c);
             if (bad && !fail)
@@ -281,7 +320,8 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
             __syncwarp();
 #pragma unroll 4
             for (int q = 0; q < N; ++q)                       // Pn[:,c] -= Z' Z[:,c]
-                axpy_row<N>(pcol, -sl.buf0[q * LD + c], sl.buf0 + q * LD);
+                axpy_row<N>(p2, -sl.buf0[q * LD + c], sl.buf0 + q * LD);
+            unpack_row<N>(pcol, p2);
             const bool gains = need_K_all || (want_u0 && ts == 0);
             if (gains) {                                      // K[:,c] = -L^{-T} Z[:,c]
 #pragma unroll
