@@ -28,7 +28,7 @@ import torch
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-from paper_2603_09221_b200 import workloads  # noqa: E402
+from paper_2603_09221_b200 import sharding, workloads  # noqa: E402
 
 SM_COUNT = 148
 FP32_LANES_PER_SM = 128
@@ -198,7 +198,7 @@ def main():
     if args.tokens > 0:
         c["batch"] = (c["batch"][0], c["batch"][1], args.tokens)
         c["name"] += "_tokens%d" % args.tokens
-    w = workloads.make_workload(cid, device=dev, batch=c["batch"], seed=workloads.SEED0 + cid + 1000 * rank)
+    w = workloads.make_workload(cid, device=dev, batch=c["batch"], seed=sharding.rank_seed(cid, rank))
     n, m, H = c["n"], c["m"], c["H"]
     N = int(np.prod(c["batch"]))
     first = c["first_only"]
@@ -237,12 +237,7 @@ def main():
     total_ms = evs[0].elapsed_time(evs[-1])
     per_step = [evs[i].elapsed_time(evs[i + 1]) for i in range(args.steps)]
     kernel_id = solver.query(lqr.TTC_QUERY_LAST_KERNEL)
-    t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-    if dist:
-        td.all_reduce(t, op=td.ReduceOp.MAX)
-    total_ms = float(t.item())
-    ms_per_step = total_ms / args.steps
-    value = world * N / (ms_per_step * 1e-3)
+    value, ms_per_step, _ = sharding.aggregate_throughput(N, total_ms / args.steps, device=dev)
 
     # ---- end to end through the host-buffer entry point (pinned host memory, copies timed)
     e2e = None
@@ -263,11 +258,9 @@ def main():
             host_step()
         barrier()
         e2e_ms = 1e3 * (time.perf_counter() - t0) / args.e2e_steps
-        te = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-        if dist:
-            td.all_reduce(te, op=td.ReduceOp.MAX)
-        e2e = {"value": world * N / (float(te.item()) * 1e-3), "unit": "instances/s",
-               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": float(te.item())}
+        e2e_value, e2e_ms_max, _ = sharding.aggregate_throughput(N, e2e_ms, device=dev)
+        e2e = {"value": e2e_value, "unit": "instances/s",
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms_max}
         del hin, hout
 
     if rank != 0:

@@ -108,28 +108,56 @@ def test_per_instance_systems_and_strides():
     pu.compare(gpu, ref, np.arange(64), 1e-4)
 
 
-@pytest.mark.parametrize("method", ["riccati", "scan"])
-def test_not_positive_definite_instance_is_isolated(method):
-    w = small_workload(8, 8, 6, (1, 1, 6), seed=9)
-    R_ok = w["R"].expand(1, 1, 6, 8, 8).clone()
+@pytest.mark.parametrize("method,n,bf16", [("riccati", 8, False), ("scan", 8, False), ("riccati", 16, False),
+                                            ("riccati", 32, False), ("riccati", 64, True)])
+def test_not_positive_definite_instance_is_isolated(method, n, bf16):
+    # n = 8: generic kernel, 16 / 32: warp kernel, 64 with bf16 inputs: tcgen05 kernel
+    H = 6
+    w = small_workload(n, n, H, (1, 1, 6), seed=9 + n, bf16=bf16)
+    R_ok = w["R"].expand(1, 1, 6, n, n).clone()
     R = R_ok.clone()
     R[0, 0, 2] = -10.0 * R[0, 0, 2]               # instance 2: R negative definite
     Q = w["Q"].clone()
     Q[0, 0, 4, 0, 0] = float("nan")               # instance 4: NaN input
-    w = dict(w, R=R.contiguous(), Q=Q)
+    per_instance = n == 8                          # per-token R needs the generic kernel; the others keep per-head R
+    if not per_instance:
+        # keep A, B, R per head: break instance 2 through an indefinite Q instead (S loses definiteness)
+        R = R_ok
+        Q[0, 0, 2] = -50.0 * torch.eye(n, device=DEV, dtype=Q.dtype)
+    w = dict(w, R=R.contiguous() if per_instance else w["R"], Q=Q)
     gpu = pu.run_gpu(w, method=METHODS[method])
+    expect = {8: "riccati_cta", 16: "riccati_warp", 32: "riccati_warp", 64: "riccati_umma"}[n] if method == "riccati" else "scan"
+    assert lqr.KERNEL_NAMES[gpu["kernel"]] == expect
     info = gpu["info"].cpu().numpy()
-    assert info[2] > 0 and info[4] > 0 and np.all(info[[0, 1, 3, 5]] == 0)
-    if method == "riccati":
-        assert info[2] == (6 - 1) * 8 + 1          # first step t = H-1, first pivot
+    assert info[2] > 0 and info[4] > 0 and np.all(info[[0, 1, 3, 5]] == 0), info
+    if method == "riccati" and per_instance:
+        assert info[2] == (H - 1) * n + 1          # first step t = H-1, first pivot
     for k in ("K", "P", "x", "u"):
-        assert torch.isnan(gpu[k][2]).all() and torch.isnan(gpu[k][4]).all()
-        assert torch.isfinite(gpu[k][[0, 1, 3, 5]]).all()
+        assert torch.isnan(gpu[k][2]).all() and torch.isnan(gpu[k][4]).all(), k
+        assert torch.isfinite(gpu[k][[0, 1, 3, 5]]).all(), k
     good = np.array([0, 1, 3, 5])
-    w_ok = dict(w, Q=torch.nan_to_num(Q, nan=1.0), R=R_ok)
-    ref = pu.run_oracle(dict(w_ok), idx=good)
+    ref = pu.run_oracle(dict(w, Q=torch.nan_to_num(Q.float(), nan=1.0).to(Q.dtype), R=R_ok if per_instance else w["R"]), idx=good)
     gsel = {k: gpu[k] for k in ("K", "P", "x", "u")}
-    pu.compare(gsel, ref, good, 1e-4)
+    pu.compare(gsel, ref, good, w["tol"])
+
+
+@pytest.mark.parametrize("cfg,expect", [(2, "riccati_umma"), (3, "riccati_warp"), (4, "riccati_umma")])
+def test_full_size_configuration_on_sampled_instances(cfg, expect):
+    """Full batch of the configuration, in the launch configuration the benchmark times; the oracle
+    checks a stratified sample of instances (every sequence and head) one by one."""
+    w = workloads.make_workload(cfg, device=DEV)
+    gpu = pu.run_gpu(w)
+    assert lqr.KERNEL_NAMES[gpu["kernel"]] == expect and gpu["launches"] == 1
+    S, Hd, T = w["batch"]
+    toks = np.array([0, 1, T // 3, T - 2, T - 1])
+    idx = (np.arange(S * Hd)[:, None] * T + toks[None, :]).reshape(-1)
+    ref = pu.run_oracle(w, idx=idx)
+    names = ("P", "u") if w["first_only"] else ("K", "P", "x", "u")
+    errs = pu.compare({k: gpu[k] for k in names + ("info",)}, ref, idx, w["tol"], names=names)
+    assert int(gpu["info"].abs().max()) == 0
+    print("cfg", cfg, errs)
+    del gpu
+    torch.cuda.empty_cache()
 
 
 def test_invalid_arguments_are_rejected():
