@@ -19,6 +19,7 @@ struct OperandDev {
 struct SolveParams {
     int n, m, H;
     long long b0, b1, b2, N;   // batch dims and their product
+    long long t0, tcount;      // token window [t0, t0 + tcount) of the last batch dimension solved by this launch
     OperandDev A, B, Q, R, x0;
     float* K;      // [N][H][m][n] or null
     float* P;      // [N][H+1][n][n] ([N][n][n] when first_only) or null
@@ -37,6 +38,12 @@ __device__ __forceinline__ long long operand_offset(const OperandDev& o, long lo
     long long i1 = r % b1;
     long long i0 = r / b1;
     return i0 * o.s0 + i1 * o.s1 + i2 * o.s2;
+}
+
+// w-th instance of the launch's token window (w in [0, b0 * b1 * tcount)) -> instance index
+__device__ __forceinline__ long long window_instance(const SolveParams& p, long long w)
+{
+    return (w / p.tcount) * p.b2 + p.t0 + w % p.tcount;
 }
 
 __device__ __forceinline__ float load_elem(const OperandDev& o, long long idx)

@@ -213,7 +213,8 @@ __global__ void __launch_bounds__(256) riccati_cta_kernel(SolveParams p)
     float* su = sxn + n;
     float* scol = su + m;
 
-    for (long long inst = blockIdx.x; inst < p.N; inst += gridDim.x) {
+    for (long long widx = blockIdx.x; widx < p.b0 * p.b1 * p.tcount; widx += gridDim.x) {
+        const long long inst = window_instance(p, widx);
         __syncthreads();
         load_to_smem(sA, p.A, operand_offset(p.A, inst, p.b1, p.b2), n * n);
         load_to_smem(sB, p.B, operand_offset(p.B, inst, p.b1, p.b2), n * m);

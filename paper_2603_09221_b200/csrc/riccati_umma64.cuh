@@ -540,7 +540,7 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
     uint32_t parity = 0;
 
     const int H = p.H;
-    const long long chunks_per_head = (p.b2 + CHUNK - 1) / CHUNK;
+    const long long chunks_per_head = (p.tcount + CHUNK - 1) / CHUNK;
     const long long nchunks = p.b0 * p.b1 * chunks_per_head;
     constexpr bool need_K_all = GAINS;
     const bool want_u0 = (p.u != nullptr) && p.first_only && !need_K_all;
@@ -568,9 +568,9 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
         if (chunk >= nchunks)
             break;
         const long long head = chunk / chunks_per_head;
-        const long long tok0 = (chunk % chunks_per_head) * CHUNK;
+        const long long tok0 = p.t0 + (chunk % chunks_per_head) * CHUNK;
         const long long inst0 = head * p.b2 + tok0;
-        const int ntok = (int)min((long long)CHUNK, p.b2 - tok0);
+        const int ntok = (int)min((long long)CHUNK, p.t0 + p.tcount - tok0);
         {
             const long long oa = operand_offset(p.A, inst0, p.b1, p.b2);
             const long long ob = operand_offset(p.B, inst0, p.b1, p.b2);

@@ -175,7 +175,7 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
     const int sub = lane / N, c = lane % N;
     typename Smem<N>::Slot& sl = sm.slot[warp * S::IPW + sub];
     const int H = p.H;
-    const long long chunks_per_head = (p.b2 + S::SLOTS - 1) / S::SLOTS;
+    const long long chunks_per_head = (p.tcount + S::SLOTS - 1) / S::SLOTS;
     const long long nchunks = p.b0 * p.b1 * chunks_per_head;
     const bool need_K_all = (p.K != nullptr) || (p.x != nullptr) || (p.u != nullptr && !p.first_only);
     const bool want_u0 = (p.u != nullptr) && p.first_only && !need_K_all;
@@ -191,9 +191,9 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
         if (chunk >= nchunks)
             break;
         const long long head = chunk / chunks_per_head;
-        const long long tok0 = (chunk % chunks_per_head) * S::SLOTS;
+        const long long tok0 = p.t0 + (chunk % chunks_per_head) * S::SLOTS;
         const long long inst0 = head * p.b2 + tok0;
-        const int ntok = (int)min((long long)S::SLOTS, p.b2 - tok0);
+        const int ntok = (int)min((long long)S::SLOTS, p.t0 + p.tcount - tok0);
         {
             const long long oa = operand_offset(p.A, inst0, p.b1, p.b2);
             const long long ob = operand_offset(p.B, inst0, p.b1, p.b2);

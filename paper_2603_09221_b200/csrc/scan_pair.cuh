@@ -188,7 +188,8 @@ __global__ void __launch_bounds__(256) scan_pair_kernel(SolveParams p, float* Pb
     float* W = T1 + d * d;
     float* scol = W + 3 * d * d;
 
-    for (long long inst = blockIdx.x; inst < p.N; inst += gridDim.x) {
+    for (long long widx = blockIdx.x; widx < p.b0 * p.b1 * p.tcount; widx += gridDim.x) {
+        const long long inst = window_instance(p, widx);
         __syncthreads();
         int fail = 0;
         // ---- step element: Ae = A, Je = Q, Ce = B R^{-1} B'
@@ -311,7 +312,8 @@ __global__ void __launch_bounds__(256) gain_rollout_kernel(SolveParams p, const 
     float* scol = su + m;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
 
-    for (long long inst = blockIdx.x; inst < p.N; inst += gridDim.x) {
+    for (long long widx = blockIdx.x; widx < p.b0 * p.b1 * p.tcount; widx += gridDim.x) {
+        const long long inst = window_instance(p, widx);
         __syncthreads();
         int fail = fail_flag ? fail_flag[inst] : 0;
         if (fail) {
@@ -427,8 +429,9 @@ inline cudaError_t launch_scan_path(const SolveParams& p, float* Pbuf, int* fail
     if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o1, scan_pair_kernel, 256, sm1))) return e;
     if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o2, gain_rollout_kernel, 256, sm2))) return e;
     long long g1 = (long long)sm_count * (o1 < 1 ? 1 : o1), g2 = (long long)sm_count * (o2 < 1 ? 1 : o2);
-    if (g1 > p.N) g1 = p.N;
-    if (g2 > p.N) g2 = p.N;
+    const long long nwin = p.b0 * p.b1 * p.tcount;
+    if (g1 > nwin) g1 = nwin;
+    if (g2 > nwin) g2 = nwin;
     scan_pair_kernel<<<(unsigned)g1, 256, sm1, st>>>(p, Pbuf, fail_flag, pfull);
     if ((e = cudaGetLastError())) return e;
     gain_rollout_kernel<<<(unsigned)g2, 256, sm2, st>>>(p, Pbuf, fail_flag, pfull);

@@ -36,6 +36,8 @@ int fail(int status, const char* fmt, ...)
             return fail(TTC_STATUS_CUDA_ERROR, "%s: %s", #call, cudaGetErrorString(e_)); \
     } while (0)
 
+constexpr int kMaxSlices = 8;    // token slices of the pipelined host-buffer entry point
+
 struct DevBuf {
     void* ptr = nullptr;
     size_t bytes = 0;
@@ -49,7 +51,10 @@ struct ttc_lqr_handle {
     int sm_count;
     DevBuf ws_K, ws_P, ws_E;       // scratch used by kernels
     DevBuf st_in[5], st_out[5];    // device staging of ttc_lqr_solve_host
-    cudaStream_t host_stream;
+    cudaStream_t host_stream;      // compute stream of ttc_lqr_solve_host
+    cudaStream_t in_stream, out_stream;   // its copy streams (host -> device, device -> host)
+    cudaEvent_t ev_in[kMaxSlices], ev_done[kMaxSlices];
+    bool host_pipeline_ready;
     long long last_launches, total_launches;
     int last_kernel;
 };
@@ -216,6 +221,8 @@ int ttc_lqr_create(const ttc_lqr_config* cfg, ttc_lqr_handle** out)
     h->N = N;
     h->sm_count = prop.multiProcessorCount;
     h->host_stream = nullptr;
+    h->in_stream = h->out_stream = nullptr;
+    h->host_pipeline_ready = false;
     h->last_launches = h->total_launches = 0;
     h->last_kernel = TTC_KERNEL_NONE;
     *out = h;
@@ -235,6 +242,14 @@ int ttc_lqr_destroy(ttc_lqr_handle* h)
     for (int i = 0; i < 5; ++i) {
         release(h->st_in[i]);
         release(h->st_out[i]);
+    }
+    if (h->host_pipeline_ready) {
+        for (int i = 0; i < kMaxSlices; ++i) {
+            cudaEventDestroy(h->ev_in[i]);
+            cudaEventDestroy(h->ev_done[i]);
+        }
+        cudaStreamDestroy(h->in_stream);
+        cudaStreamDestroy(h->out_stream);
     }
     if (h->host_stream)
         cudaStreamDestroy(h->host_stream);
@@ -267,25 +282,28 @@ int ttc_lqr_query(const ttc_lqr_handle* h, int32_t key, int64_t* value)
     }
 }
 
-int ttc_lqr_solve(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, const ttc_operand* Q,
-                  const ttc_operand* R, const ttc_operand* x0, int32_t H, float* K, float* P, float* x,
-                  float* u, int32_t* info, uint32_t flags, void* cuda_stream)
+} // extern "C"
+
+namespace {
+
+// Enqueue the solve of the token window [t0, t0 + tcount) of the last batch dimension (all of it for
+// ttc_lqr_solve; one slice at a time for the pipelined host-buffer entry point).  Arguments validated.
+int solve_window(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, const ttc_operand* Q,
+                 const ttc_operand* R, const ttc_operand* x0, int32_t H, float* K, float* P, float* x,
+                 float* u, int32_t* info, uint32_t flags, cudaStream_t st, long long t0, long long tcount)
 {
-    int s = validate_common(h, A, B, Q, R, x0, H, K, P, x, u, info, flags);
-    if (s)
-        return s;
-    TTC_CUDA(cudaSetDevice(h->cfg.device));
-    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    int s;
     const int n = h->cfg.n, m = h->cfg.m;
 
     SolveParams p;
     p.n = n; p.m = m; p.H = H;
     p.b0 = h->cfg.batch[0]; p.b1 = h->cfg.batch[1]; p.b2 = h->cfg.batch[2]; p.N = h->N;
+    p.t0 = t0; p.tcount = tcount;
+    const long long nwin = p.b0 * p.b1 * tcount;          // instances of this launch
     p.A = to_dev(A); p.B = to_dev(B); p.Q = to_dev(Q); p.R = to_dev(R); p.x0 = to_dev(x0);
     p.K = K; p.P = P; p.x = x; p.u = u; p.info = info;
     p.Kws = nullptr;
     p.first_only = (flags & TTC_OUT_FIRST_ONLY) ? 1 : 0;
-    h->last_launches = 0;
 
     const int method = pick_method(h);
     // The rollout reads every K_t in forward order after the backward pass produced them in
@@ -309,8 +327,10 @@ int ttc_lqr_solve(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B,
         cudaError_t e = launch_scan_path(p, Pbuf, static_cast<int*>(h->ws_E.ptr), pfull, h->sm_count, st, &launches);
         if (e != cudaSuccess)
             return fail(TTC_STATUS_CUDA_ERROR, "scan path launch: %s", cudaGetErrorString(e));
-        h->last_launches = launches;
+        h->last_launches += launches;
+        h->total_launches += launches;
         h->last_kernel = TTC_KERNEL_SCAN;
+        return TTC_OK;
     } else {
         if (!K && rollout_needs_all_K) {
             if ((s = ensure(h->ws_K, sizeof(float) * (size_t)h->N * H * m * n))) return s;
@@ -327,14 +347,14 @@ int ttc_lqr_solve(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B,
             const size_t smem = umma64::smem_bytes();
             auto kern = rollout_needs_all_K || K ? umma64::riccati_umma64_kernel<true> : umma64::riccati_umma64_kernel<false>;
             TTC_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            const long long chunks = p.b0 * p.b1 * ((p.b2 + umma64::CHUNK - 1) / umma64::CHUNK);
+            const long long chunks = p.b0 * p.b1 * ((tcount + umma64::CHUNK - 1) / umma64::CHUNK);
             long long grid = h->sm_count;
             if (2 * grid > chunks) grid = (chunks + 1) / 2;
             kern<<<(unsigned)grid, umma64::THREADS, smem, st>>>(p, counter, counter + 1);
             TTC_CUDA(cudaGetLastError());
-            h->last_launches = 1;
+            h->last_launches += 1;
+            h->total_launches += 1;
             h->last_kernel = TTC_KERNEL_RICCATI_UMMA;
-            h->total_launches += h->last_launches;
             return TTC_OK;
         }
         if (head_shared && n == m && (n == 16 || n == 32)) {
@@ -345,22 +365,22 @@ int ttc_lqr_solve(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B,
             if (n == 32) {
                 const size_t smem = rwarp::smem_bytes<32>();
                 TTC_CUDA(cudaFuncSetAttribute(rwarp::riccati_warp_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-                const long long chunks = p.b0 * p.b1 * ((p.b2 + rwarp::Shape<32>::SLOTS - 1) / rwarp::Shape<32>::SLOTS);
+                const long long chunks = p.b0 * p.b1 * ((tcount + rwarp::Shape<32>::SLOTS - 1) / rwarp::Shape<32>::SLOTS);
                 long long grid = (long long)h->sm_count * 3;
                 if (grid > chunks) grid = chunks;
                 rwarp::riccati_warp_kernel<32><<<(unsigned)grid, rwarp::THREADS, smem, st>>>(p, counter);
             } else {
                 const size_t smem = rwarp::smem_bytes<16>();
                 TTC_CUDA(cudaFuncSetAttribute(rwarp::riccati_warp_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-                const long long chunks = p.b0 * p.b1 * ((p.b2 + rwarp::Shape<16>::SLOTS - 1) / rwarp::Shape<16>::SLOTS);
+                const long long chunks = p.b0 * p.b1 * ((tcount + rwarp::Shape<16>::SLOTS - 1) / rwarp::Shape<16>::SLOTS);
                 long long grid = (long long)h->sm_count * 4;
                 if (grid > chunks) grid = chunks;
                 rwarp::riccati_warp_kernel<16><<<(unsigned)grid, rwarp::THREADS, smem, st>>>(p, counter);
             }
             TTC_CUDA(cudaGetLastError());
-            h->last_launches = 1;
+            h->last_launches += 1;
+            h->total_launches += 1;
             h->last_kernel = TTC_KERNEL_RICCATI_WARP;
-            h->total_launches += h->last_launches;
             return TTC_OK;
         }
         const size_t smem = riccati_cta_smem_bytes(n, m);
@@ -369,14 +389,32 @@ int ttc_lqr_solve(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B,
         TTC_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, riccati_cta_kernel, 256, smem));
         if (per_sm < 1) per_sm = 1;
         long long grid = (long long)h->sm_count * per_sm;
-        if (grid > h->N) grid = h->N;
+        if (grid > nwin) grid = nwin;
         riccati_cta_kernel<<<(unsigned)grid, 256, smem, st>>>(p);
         TTC_CUDA(cudaGetLastError());
-        h->last_launches = 1;
+        h->last_launches += 1;
+        h->total_launches += 1;
         h->last_kernel = TTC_KERNEL_RICCATI_CTA;
     }
-    h->total_launches += h->last_launches;
     return TTC_OK;
+}
+
+
+} // namespace
+
+extern "C" {
+
+int ttc_lqr_solve(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, const ttc_operand* Q,
+                  const ttc_operand* R, const ttc_operand* x0, int32_t H, float* K, float* P, float* x,
+                  float* u, int32_t* info, uint32_t flags, void* cuda_stream)
+{
+    int s = validate_common(h, A, B, Q, R, x0, H, K, P, x, u, info, flags);
+    if (s)
+        return s;
+    TTC_CUDA(cudaSetDevice(h->cfg.device));
+    h->last_launches = 0;
+    return solve_window(h, A, B, Q, R, x0, H, K, P, x, u, info, flags, static_cast<cudaStream_t>(cuda_stream), 0,
+                        h->cfg.batch[2]);
 }
 
 int ttc_lqr_solve_host(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, const ttc_operand* Q,
@@ -388,16 +426,27 @@ int ttc_lqr_solve_host(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operan
     // alignment of host pointers is irrelevant; validate the rest through a relaxed copy
     if (H < 1 || H > h->cfg.max_horizon)
         return fail(TTC_STATUS_INVALID_ARGUMENT, "H=%d outside [1, max_horizon=%d]", H, h->cfg.max_horizon);
+    if (flags & ~TTC_OUT_FIRST_ONLY)
+        return fail(TTC_STATUS_INVALID_ARGUMENT, "unknown flag bits 0x%x", flags);
     TTC_CUDA(cudaSetDevice(h->cfg.device));
-    if (!h->host_stream)
+    if (!h->host_pipeline_ready) {
         TTC_CUDA(cudaStreamCreateWithFlags(&h->host_stream, cudaStreamNonBlocking));
+        TTC_CUDA(cudaStreamCreateWithFlags(&h->in_stream, cudaStreamNonBlocking));
+        TTC_CUDA(cudaStreamCreateWithFlags(&h->out_stream, cudaStreamNonBlocking));
+        for (int i = 0; i < kMaxSlices; ++i) {
+            TTC_CUDA(cudaEventCreateWithFlags(&h->ev_in[i], cudaEventDisableTiming));
+            TTC_CUDA(cudaEventCreateWithFlags(&h->ev_done[i], cudaEventDisableTiming));
+        }
+        h->host_pipeline_ready = true;
+    }
     const int n = h->cfg.n, m = h->cfg.m;
-    const long long N = h->N;
+    const long long N = h->N, b0 = h->cfg.batch[0], b1 = h->cfg.batch[1], b2 = h->cfg.batch[2];
     const bool first = (flags & TTC_OUT_FIRST_ONLY) != 0;
     const ttc_operand* in[5] = {A, B, Q, R, x0};
     const char* names[5] = {"A", "B", "Q", "R", "x0"};
     const size_t elems[5] = {(size_t)n * n, (size_t)n * m, (size_t)n * n, (size_t)m * m, (size_t)n};
     ttc_operand dev[5];
+    size_t in_bytes[5] = {0, 0, 0, 0, 0};
     for (int i = 0; i < 5; ++i) {
         dev[i].ptr = nullptr; dev[i].dtype = TTC_F32; dev[i].reserved = 0;
         dev[i].bstride[0] = dev[i].bstride[1] = dev[i].bstride[2] = 0;
@@ -406,7 +455,7 @@ int ttc_lqr_solve_host(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operan
                 continue;
             return fail(TTC_STATUS_INVALID_ARGUMENT, "operand %s is null", names[i]);
         }
-        if (in[i]->dtype != TTC_F32 && in[i]->dtype != TTC_BF16)
+        if (in[i]->dtype != TTC_F32 && !(in[i]->dtype == TTC_BF16 && (i == 2 || i == 4)))
             return fail(TTC_STATUS_INVALID_ARGUMENT, "operand %s: dtype %d not supported", names[i], in[i]->dtype);
         size_t extent = elems[i];
         for (int d = 0; d < 3; ++d) {
@@ -414,35 +463,91 @@ int ttc_lqr_solve_host(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operan
                 return fail(TTC_STATUS_INVALID_ARGUMENT, "operand %s: negative stride", names[i]);
             extent += (size_t)(h->cfg.batch[d] - 1) * (size_t)in[i]->bstride[d];
         }
-        const size_t bytes = extent * (in[i]->dtype == TTC_BF16 ? 2 : 4);
-        int s = ensure(h->st_in[i], bytes);
+        in_bytes[i] = extent * (in[i]->dtype == TTC_BF16 ? 2 : 4);
+        int s = ensure(h->st_in[i], in_bytes[i]);
         if (s) return s;
-        TTC_CUDA(cudaMemcpyAsync(h->st_in[i].ptr, in[i]->ptr, bytes, cudaMemcpyHostToDevice, h->host_stream));
         dev[i] = *in[i];
         dev[i].ptr = h->st_in[i].ptr;
     }
     void* host_out[5] = {K, P, x, u, info};
-    const size_t out_bytes[5] = {
-        sizeof(float) * (size_t)N * H * m * n,
-        sizeof(float) * (size_t)N * (first ? 1 : H + 1) * n * n,
-        sizeof(float) * (size_t)N * (H + 1) * n,
-        sizeof(float) * (size_t)N * (first ? 1 : H) * m,
-        sizeof(int32_t) * (size_t)N};
+    const size_t per_out[5] = {                        // bytes per instance
+        sizeof(float) * (size_t)H * m * n, sizeof(float) * (size_t)(first ? 1 : H + 1) * n * n,
+        sizeof(float) * (size_t)(H + 1) * n, sizeof(float) * (size_t)(first ? 1 : H) * m, sizeof(int32_t)};
     void* dev_out[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
-    for (int i = 0; i < 5; ++i)
+    size_t total_bytes = 0;
+    for (int i = 0; i < 5; ++i) {
+        total_bytes += in_bytes[i];
         if (host_out[i]) {
-            int s = ensure(h->st_out[i], out_bytes[i]);
+            int s = ensure(h->st_out[i], per_out[i] * (size_t)N);
             if (s) return s;
             dev_out[i] = h->st_out[i].ptr;
+            total_bytes += per_out[i] * (size_t)N;
         }
-    int s = ttc_lqr_solve(h, &dev[0], &dev[1], &dev[2], &dev[3], dev[4].ptr ? &dev[4] : nullptr, H,
-                          (float*)dev_out[0], (float*)dev_out[1], (float*)dev_out[2], (float*)dev_out[3],
-                          (int32_t*)dev_out[4], flags, h->host_stream);
-    if (s)
-        return s;
-    for (int i = 0; i < 5; ++i)
-        if (host_out[i])
-            TTC_CUDA(cudaMemcpyAsync(host_out[i], dev_out[i], out_bytes[i], cudaMemcpyDeviceToHost, h->host_stream));
+    }
+
+    // ---- slices of the token dimension: copy in, solve and copy out overlap across slices
+    int nslice = 1;
+    if (total_bytes >= ((size_t)64 << 20) && b2 >= 256) {
+        nslice = (int)(b2 / 128 < kMaxSlices ? b2 / 128 : kMaxSlices);
+        for (int i = 0; i < 5 && nslice > 1; ++i) {    // per-token operands must have separable rows
+            if (!dev[i].ptr || in[i]->bstride[2] == 0)
+                continue;
+            const long long s1 = in[i]->bstride[1], s2 = in[i]->bstride[2];
+            if (s2 < (long long)elems[i] || (b1 > 1 && s1 != 0 && s1 < (b2 - 1) * s2 + (long long)elems[i]))
+                nslice = 1;
+        }
+    }
+    long long tslice = (b2 + nslice - 1) / nslice;
+    tslice = (tslice + 15) / 16 * 16;
+    nslice = (int)((b2 + tslice - 1) / tslice);
+
+    h->last_launches = 0;
+    for (int i = 0; i < 5; ++i)                        // operands shared along the token dimension: whole, once
+        if (dev[i].ptr && (nslice == 1 || in[i]->bstride[2] == 0))
+            TTC_CUDA(cudaMemcpyAsync(h->st_in[i].ptr, in[i]->ptr, in_bytes[i], cudaMemcpyHostToDevice, h->in_stream));
+    for (int c = 0; c < nslice; ++c) {
+        const long long t0 = c * tslice, tc = (b2 - t0 < tslice) ? b2 - t0 : tslice;
+        if (nslice > 1)
+            for (int i = 0; i < 5; ++i) {
+                if (!dev[i].ptr || in[i]->bstride[2] == 0)
+                    continue;
+                const size_t es = in[i]->dtype == TTC_BF16 ? 2 : 4;
+                const long long s0 = in[i]->bstride[0], s1 = in[i]->bstride[1], s2 = in[i]->bstride[2];
+                const size_t width = ((size_t)(tc - 1) * s2 + elems[i]) * es;
+                const size_t rows = (s1 == 0) ? 1 : (size_t)b1;
+                const size_t pitch = rows > 1 ? (size_t)s1 * es : width;
+                for (long long i0 = 0; i0 < (s0 == 0 ? 1 : b0); ++i0) {
+                    const size_t off = ((size_t)i0 * s0 + (size_t)t0 * s2) * es;
+                    TTC_CUDA(cudaMemcpy2DAsync(static_cast<char*>(h->st_in[i].ptr) + off, pitch,
+                                               static_cast<const char*>(in[i]->ptr) + off, pitch, width, rows,
+                                               cudaMemcpyHostToDevice, h->in_stream));
+                }
+            }
+        TTC_CUDA(cudaEventRecord(h->ev_in[c], h->in_stream));
+        TTC_CUDA(cudaStreamWaitEvent(h->host_stream, h->ev_in[c], 0));
+        int s = solve_window(h, &dev[0], &dev[1], &dev[2], &dev[3], dev[4].ptr ? &dev[4] : nullptr, H,
+                             (float*)dev_out[0], (float*)dev_out[1], (float*)dev_out[2], (float*)dev_out[3],
+                             (int32_t*)dev_out[4], flags, h->host_stream, t0, tc);
+        if (s) {
+            cudaDeviceSynchronize();
+            return s;
+        }
+        TTC_CUDA(cudaEventRecord(h->ev_done[c], h->host_stream));
+        TTC_CUDA(cudaStreamWaitEvent(h->out_stream, h->ev_done[c], 0));
+        for (int i = 0; i < 5; ++i) {
+            if (!host_out[i])
+                continue;
+            if (nslice == 1) {
+                TTC_CUDA(cudaMemcpyAsync(host_out[i], dev_out[i], per_out[i] * (size_t)N, cudaMemcpyDeviceToHost, h->out_stream));
+            } else {                                   // rows = (sequence, head), one run of tc instances per row
+                const size_t off = (size_t)t0 * per_out[i], pitch = (size_t)b2 * per_out[i];
+                TTC_CUDA(cudaMemcpy2DAsync(static_cast<char*>(host_out[i]) + off, pitch,
+                                           static_cast<const char*>(dev_out[i]) + off, pitch, (size_t)tc * per_out[i],
+                                           (size_t)(b0 * b1), cudaMemcpyDeviceToHost, h->out_stream));
+            }
+        }
+    }
+    TTC_CUDA(cudaStreamSynchronize(h->out_stream));
     TTC_CUDA(cudaStreamSynchronize(h->host_stream));
     return TTC_OK;
 }
@@ -540,6 +645,7 @@ extern "C" int ttc_lqr_solve_first_noalloc(int32_t n, int32_t m, const int64_t b
     SolveParams p;
     p.n = n; p.m = m; p.H = H;
     p.b0 = batch[0]; p.b1 = batch[1]; p.b2 = batch[2]; p.N = N;
+    p.t0 = 0; p.tcount = batch[2];
     p.A = to_dev(A); p.B = to_dev(B); p.Q = to_dev(Q); p.R = to_dev(R); p.x0 = to_dev(x0);
     p.K = nullptr; p.P = P0; p.x = nullptr; p.u = u0; p.info = info;
     p.Kws = nullptr;

@@ -195,3 +195,25 @@ def test_host_buffer_entry_point_matches_device_entry_point():
     s.close()
     for k in ("K", "P", "x", "u", "info"):
         assert torch.equal(out[k], gpu[k].cpu()), k
+
+
+@pytest.mark.parametrize("n,H,batch,bf16", [(16, 6, (2, 2, 2000), False), (64, 4, (1, 2, 512), True)])
+def test_host_buffer_entry_point_pipelined_slices(n, H, batch, bf16):
+    """Large enough for the host-buffer entry point to cut the token dimension into slices whose copies and
+    solves overlap (ragged last slice at 2000 tokens): results must equal the device entry point's bit for bit."""
+    w = small_workload(n, n, H, batch, seed=31 + n, bf16=bf16)
+    N = int(np.prod(batch))
+    gpu = pu.run_gpu(w)
+    s = lqr.LqrSolver(n, n, H, batch)
+    host = {k: w[k].cpu().pin_memory() for k in ("A", "B", "Q", "R", "x0")}
+    out = lqr.alloc_outputs(n, n, H, N, "cpu", pin=True)
+    for v in out.values():
+        v.fill_(7)
+    s.solve_host(host["A"], host["B"], host["Q"], host["R"], host["x0"], H, **out)
+    assert s.query(lqr.TTC_QUERY_LAST_LAUNCHES) > 1, "expected more than one slice"
+    s.solve_host(host["A"], host["B"], host["Q"], host["R"], host["x0"], H, **out)      # staging buffers reused
+    s.close()
+    for k in ("K", "P", "x", "u", "info"):
+        assert torch.equal(out[k], gpu[k].cpu()), k
+    ref = pu.run_oracle(w, idx=np.arange(0, N, max(1, N // 64)))
+    pu.compare({k: out[k] for k in ("K", "P", "x", "u")}, ref, np.arange(0, N, max(1, N // 64)), w["tol"])
