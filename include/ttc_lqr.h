@@ -145,10 +145,13 @@ int ttc_lqr_solve(ttc_lqr_handle* h,
 
 /*
  * Same computation with HOST buffers (same problem statement as ttc_lqr_solve): operand
- * pointers and all outputs are host memory (pinned memory makes the copies faster but is
- * not required).  The call copies the inputs to device staging buffers owned by the handle,
- * runs ttc_lqr_solve on an internal stream, copies the requested outputs back and returns
- * after everything has completed (synchronous).  Strides have the same meaning.
+ * pointers and all outputs are host memory (pinned memory lets the copies run asynchronously;
+ * pageable memory works but serialises them).  The call copies the inputs to device staging
+ * buffers owned by the handle, solves on internal streams, copies the requested outputs back
+ * and returns after everything has completed (synchronous).  Large problems are cut into up to
+ * 8 slices of the last batch dimension so that the copy-in of one slice, the solve of the
+ * previous one and the copy-out of the one before overlap; results are identical to
+ * ttc_lqr_solve.  Strides have the same meaning.
  */
 int ttc_lqr_solve_host(ttc_lqr_handle* h,
                        const ttc_operand* A, const ttc_operand* B, const ttc_operand* Q,
