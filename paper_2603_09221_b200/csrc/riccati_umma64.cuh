@@ -67,6 +67,15 @@ __device__ __forceinline__ uint32_t toff(int r, int c)
 {
     return (uint32_t)(r >> 3) * SR + (uint32_t)(c >> 2) * SC + (uint32_t)(r & 7) * 16u + (uint32_t)(c & 3) * 4u;
 }
+// Private variant of the layout for matrices that are read and updated by the factorisation (S, and the columns
+// of Y' that are still being updated): in odd k-chunks the 8 rows of a core matrix are rotated by 4.  The 8-byte
+// accumulator-tile accesses of the mma updates (row g, columns 2t, 2t+1: two lanes 128 B apart) then hit
+// different banks; row owners (16 bytes) and fragment loads (4 bytes) stay conflict-free.
+__device__ __forceinline__ uint32_t toff_rot(int r, int c)
+{
+    return (uint32_t)(r >> 3) * SR + (uint32_t)(c >> 2) * SC + (uint32_t)(((r & 7) + (((c >> 2) & 1) << 2)) & 7) * 16u +
+           (uint32_t)(c & 3) * 4u;
+}
 __device__ __forceinline__ float& elem(unsigned char* base, uint32_t off) { return *reinterpret_cast<float*>(base + off); }
 
 // fp32 -> tf32 (10 explicit mantissa bits), round to nearest with ties away from zero, on the integer
@@ -216,22 +225,25 @@ __device__ __forceinline__ void fsub8(float (&x)[8], const float (&l)[8][8], con
         x[i] = v * rinv[i];
     }
 }
-__device__ __forceinline__ void load_row8(float (&x)[8], const unsigned char* p)
+// 8 consecutive columns (an even chunk and the odd chunk after it) of one row.  `grp` points at the even chunk
+// of the row's 8-row group, `slot` = row & 7.  ROT: rotated layout (odd chunk at slot + 4), else canonical.
+template <bool ROT>
+__device__ __forceinline__ void load_row8(float (&x)[8], const unsigned char* grp, int slot)
 {
-    const float4 a = *reinterpret_cast<const float4*>(p);
-    const float4 b = *reinterpret_cast<const float4*>(p + SC);
+    const float4 a = *reinterpret_cast<const float4*>(grp + slot * 16);
+    const float4 b = *reinterpret_cast<const float4*>(grp + SC + (ROT ? ((slot + 4) & 7) : slot) * 16);
     x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
 }
-template <bool ROUND>
-__device__ __forceinline__ void store_row8(unsigned char* p, const float (&x)[8])
+template <bool ROT, bool ROUND>
+__device__ __forceinline__ void store_row8(unsigned char* grp, int slot, const float (&x)[8])
 {
     float4 a = make_float4(x[0], x[1], x[2], x[3]), b = make_float4(x[4], x[5], x[6], x[7]);
     if (ROUND) {
         a.x = round_tf32(a.x); a.y = round_tf32(a.y); a.z = round_tf32(a.z); a.w = round_tf32(a.w);
         b.x = round_tf32(b.x); b.y = round_tf32(b.y); b.z = round_tf32(b.z); b.w = round_tf32(b.w);
     }
-    *reinterpret_cast<float4*>(p) = a;
-    *reinterpret_cast<float4*>(p + SC) = b;
+    *reinterpret_cast<float4*>(grp + slot * 16) = a;
+    *reinterpret_cast<float4*>(grp + SC + (ROT ? ((slot + 4) & 7) : slot) * 16) = b;
 }
 
 // Two warps (pw = 0, 1; 64 threads) work on the tall matrix G = [S; Y'] (128 x 64, fp32): S (64 x 64 SPD,
@@ -248,9 +260,13 @@ __device__ __forceinline__ void pair_chol_solve(unsigned char* Sm, unsigned char
 {
     const int g = lane >> 2, t = lane & 3;
     const int tid2 = 32 * pw + lane;
-    const uint32_t frag_ab = (uint32_t)g * 16u + (uint32_t)t * 4u;                                     // (row g, col t) of a core matrix
-    const uint32_t frag_c = (uint32_t)g * 16u + (uint32_t)(t >> 1) * SC + (uint32_t)((2 * t) & 3) * 4u; // (row g, cols 2t, 2t+1) of a tile
-    const uint32_t own_row = (uint32_t)(tid2 >> 3) * SR + (uint32_t)(tid2 & 7) * 16u;                 // row tid2, column 0
+    // fragment offsets inside an (8-row group, even chunk): S and the pending columns of Y' are in the rotated layout
+    const uint32_t frag_ab = (uint32_t)g * 16u + (uint32_t)t * 4u;                        // (row g, col t), even chunk
+    const uint32_t frag_ab1 = SC + (uint32_t)((g + 4) & 7) * 16u + (uint32_t)t * 4u;      // (row g, col t + 4), rotated odd chunk
+    const uint32_t frag_ab1c = SC + (uint32_t)g * 16u + (uint32_t)t * 4u;                 // the same, canonical
+    const uint32_t frag_c = (uint32_t)((g + 4 * (t >> 1)) & 7) * 16u + (uint32_t)(t >> 1) * SC + (uint32_t)((2 * t) & 3) * 4u; // (row g, cols 2t, 2t+1), rotated
+    const uint32_t own_grp = (uint32_t)(tid2 >> 3) * SR;                                  // 8-row group of row tid2
+    const int own_slot = tid2 & 7;
 #pragma unroll 1
     for (int k = 0; k < 8; ++k) {
         const uint32_t kcol = 2u * k * SC;             // byte offset of columns 8k .. 8k+7 inside a row
@@ -258,41 +274,41 @@ __device__ __forceinline__ void pair_chol_solve(unsigned char* Sm, unsigned char
         float l[8][8], rinv[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i)
-            load_row8(l[i], dblk + i * 16);
+            load_row8<true>(l[i], dblk, i);
         const bool has_s = tid2 + 8 * k + 8 < N;
-        unsigned char* py = Ym + own_row + kcol;
-        unsigned char* ps = Sm + own_row + (uint32_t)(k + 1) * SR + kcol;       // row tid2 + 8k + 8
+        unsigned char* py = Ym + own_grp + kcol;
+        unsigned char* ps = Sm + own_grp + (uint32_t)(k + 1) * SR + kcol;       // row tid2 + 8k + 8
         float xy[8], xs[8];
-        load_row8(xy, py);
+        load_row8<true>(xy, py, own_slot);
         if (has_s)
-            load_row8(xs, ps);
+            load_row8<true>(xs, ps, own_slot);
         const int bad = chol8(l, rinv);
         if (bad && tid2 == 0 && *flag == 0)
             *flag = code0 + 8 * k + bad;
         fsub8(xy, l, rinv);
         if (has_s)
             fsub8(xs, l, rinv);
-        store_row8<true>(py, xy);
+        store_row8<false, true>(py, own_slot, xy);    // final columns of Z': canonical layout, tf32
         if (has_s)
-            store_row8<false>(ps, xs);
+            store_row8<true, false>(ps, own_slot, xs);
         pair_barrier(wg, x);                           // panel written; every thread has read the diagonal block
         if (tid2 < 8) {                                // keep L_d for the back substitution
 #pragma unroll
             for (int i = 0; i < 8; ++i)
                 if (tid2 == i)
-                    store_row8<false>(dblk + i * 16, l[i]);
+                    store_row8<true, false>(dblk, i, l[i]);
         }
         if (k == 7)
             break;
         // ---- trailing update: B fragments = rows 8j + g of S, columns 8k + t, 8k + t + 4
         uint32_t bh[7][2], bl[7][2];
         {
-            const unsigned char* pb = Sm + frag_ab + kcol;
+            const unsigned char* pb = Sm + kcol;
 #pragma unroll
             for (int j = 1; j < 8; ++j)
                 if (j > k) {
-                    split_tf32(*reinterpret_cast<const float*>(pb + j * SR), bh[j - 1][0], bl[j - 1][0]);
-                    split_tf32(*reinterpret_cast<const float*>(pb + j * SR + SC), bh[j - 1][1], bl[j - 1][1]);
+                    split_tf32(*reinterpret_cast<const float*>(pb + j * SR + frag_ab), bh[j - 1][0], bl[j - 1][0]);
+                    split_tf32(*reinterpret_cast<const float*>(pb + j * SR + frag_ab1), bh[j - 1][1], bl[j - 1][1]);
                 }
         }
 #pragma unroll
@@ -305,11 +321,12 @@ __device__ __forceinline__ void pair_chol_solve(unsigned char* Sm, unsigned char
             unsigned char* Mt = is_s ? Sm : Ym;
             uint32_t ah[4], al[4];
             {
-                const unsigned char* pa = Mt + frag_ab + kcol + 2 * mt * SR;
-                split_tf32(-*reinterpret_cast<const float*>(pa), ah[0], al[0]);
-                split_tf32(-*reinterpret_cast<const float*>(pa + SR), ah[1], al[1]);
-                split_tf32(-*reinterpret_cast<const float*>(pa + SC), ah[2], al[2]);
-                split_tf32(-*reinterpret_cast<const float*>(pa + SR + SC), ah[3], al[3]);
+                const unsigned char* pa = Mt + kcol + 2 * mt * SR;
+                const uint32_t odd = is_s ? frag_ab1 : frag_ab1c;              // the panel of Y' has just been stored canonically
+                split_tf32(-*reinterpret_cast<const float*>(pa + frag_ab), ah[0], al[0]);
+                split_tf32(-*reinterpret_cast<const float*>(pa + SR + frag_ab), ah[1], al[1]);
+                split_tf32(-*reinterpret_cast<const float*>(pa + odd), ah[2], al[2]);
+                split_tf32(-*reinterpret_cast<const float*>(pa + SR + odd), ah[3], al[3]);
             }
             // all C tiles of this row tile first, then three independent mma passes, then the stores
             unsigned char* pc = Mt + frag_c + 2 * mt * SR;
@@ -358,8 +375,11 @@ __device__ __forceinline__ void pair_gain_solve(const unsigned char* Sm, unsigne
     const int tid2 = 32 * pw + lane;
     const uint32_t frag_ab = (uint32_t)g * 16u + (uint32_t)t * 4u;
     const uint32_t frag_c = (uint32_t)g * 16u + (uint32_t)(t >> 1) * SC + (uint32_t)((2 * t) & 3) * 4u;
-    const uint32_t frag_b = (uint32_t)t * 16u + (uint32_t)(g >> 2) * SC + (uint32_t)(g & 3) * 4u;   // (row t, col g) of a tile
-    const uint32_t own_row = (uint32_t)(tid2 >> 3) * SR + (uint32_t)(tid2 & 7) * 16u;
+    // (row t, col g) and (row t + 4, col g) of a tile of L (rotated layout: the chunk parity is g >> 2)
+    const uint32_t frag_b = (uint32_t)((t + 4 * (g >> 2)) & 7) * 16u + (uint32_t)(g >> 2) * SC + (uint32_t)(g & 3) * 4u;
+    const uint32_t frag_b4 = (uint32_t)((t + 4 + 4 * (g >> 2)) & 7) * 16u + (uint32_t)(g >> 2) * SC + (uint32_t)(g & 3) * 4u;
+    const uint32_t own_grp = (uint32_t)(tid2 >> 3) * SR;
+    const int own_slot = tid2 & 7;
 #pragma unroll 1
     for (int kb = 7; kb >= 0; --kb) {
         const uint32_t kcol = 2u * kb * SC;
@@ -367,9 +387,9 @@ __device__ __forceinline__ void pair_gain_solve(const unsigned char* Sm, unsigne
         float l[8][8], xr[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i)
-            load_row8(l[i], dblk + i * 16);
-        unsigned char* py = Ym + own_row + kcol;
-        load_row8(xr, py);
+            load_row8<true>(l[i], dblk, i);
+        unsigned char* py = Ym + own_grp + kcol;
+        load_row8<false>(xr, py, own_slot);
 #pragma unroll
         for (int j = 7; j >= 0; --j) {                 // x L_d = z, L_d lower triangular
             float v = xr[j];
@@ -378,19 +398,19 @@ __device__ __forceinline__ void pair_gain_solve(const unsigned char* Sm, unsigne
                 v = fmaf(-xr[i], l[i][j], v);
             xr[j] = __fdividef(v, l[j][j]);
         }
-        store_row8<false>(py, xr);
+        store_row8<false, false>(py, own_slot, xr);
         if (kb == 0)
             break;
         pair_barrier(wg, x);
         // B fragments: rows 8kb + t, 8kb + t + 4 of L, columns 8j + g (j < kb)
         uint32_t bh[7][2], bl[7][2];
         {
-            const unsigned char* pb = Sm + (uint32_t)kb * SR + frag_b;
+            const unsigned char* pb = Sm + (uint32_t)kb * SR;
 #pragma unroll
             for (int j = 0; j < 7; ++j)
                 if (j < kb) {
-                    split_tf32(*reinterpret_cast<const float*>(pb + 2 * j * SC), bh[j][0], bl[j][0]);
-                    split_tf32(*reinterpret_cast<const float*>(pb + 2 * j * SC + 64), bh[j][1], bl[j][1]);
+                    split_tf32(*reinterpret_cast<const float*>(pb + 2 * j * SC + frag_b), bh[j][0], bl[j][0]);
+                    split_tf32(*reinterpret_cast<const float*>(pb + 2 * j * SC + frag_b4), bh[j][1], bl[j][1]);
                 }
         }
 #pragma unroll
@@ -642,13 +662,13 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
 #pragma unroll
                             for (int c = 0; c < 8; ++c) {
                                 const float4 r4 = __ldg(rr + c);
-                                *reinterpret_cast<float4*>(X1 + x * MAT_BYTES + toff(wt, 32 * half + 4 * c)) =
+                                *reinterpret_cast<float4*>(X1 + x * MAT_BYTES + toff_rot(wt, 32 * half + 4 * c)) =
                                     make_float4(h[4 * c] + r4.x, h[4 * c + 1] + r4.y, h[4 * c + 2] + r4.z, h[4 * c + 3] + r4.w);
                             }
                         } else {                       // Y_x' -> X0, fp32 (P is dead once (1) has completed)
 #pragma unroll
                             for (int c = 0; c < 8; ++c)
-                                *reinterpret_cast<float4*>(X0 + toff(64 * x + (wt - 64), 32 * half + 4 * c)) =
+                                *reinterpret_cast<float4*>(X0 + toff_rot(64 * x + (wt - 64), 32 * half + 4 * c)) =
                                     make_float4(h[4 * c], h[4 * c + 1], h[4 * c + 2], h[4 * c + 3]);
                         }
                     }
@@ -683,7 +703,7 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
                             float l[8][8], w[8];
 #pragma unroll
                             for (int r = 0; r < 8; ++r) {
-                                load_row8(l[r], Sm + toff(c0 + r, c0));
+                                load_row8<true>(l[r], Sm + toff(c0, c0), r);
                                 w[r] = misc.y0[x][c0 + r];
                             }
 #pragma unroll
@@ -697,7 +717,7 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
                             if (i < c0) {
 #pragma unroll
                                 for (int r = 0; r < 8; ++r)
-                                    zi = fmaf(-elem(Sm, toff(c0 + r, i)), w[r], zi);
+                                    zi = fmaf(-elem(Sm, toff_rot(c0 + r, i)), w[r], zi);
                             }
                             pair_barrier(wg, x);
                             if (i < c0)
