@@ -185,6 +185,8 @@ __device__ __forceinline__ void split_tf32(float x, uint32_t& hi, uint32_t& lo)
 }
 
 // In-thread Cholesky of an 8 x 8 SPD block: l (lower triangle) is overwritten by L, rinv[i] = 1 / L[i][i].
+// The trailing update uses l_ij l_cj / d_j with the hardware reciprocal, so that the chain from one pivot to
+// the next is reciprocal -> multiply -> fma; the scaling by 1 / sqrt(d_j) is off that chain.
 // Returns 0 or 1 + the index of the first non-positive pivot.
 __device__ __forceinline__ int chol8(float (&l)[8][8], float (&rinv)[8])
 {
@@ -197,19 +199,21 @@ __device__ __forceinline__ int chol8(float (&l)[8][8], float (&rinv)[8])
                 bad = j + 1;
             d = 1.f;
         }
-        float rs;
+        float rd, rs;
+        asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(rd) : "f"(d));
         asm("rsqrt.approx.ftz.f32 %0, %1;" : "=f"(rs) : "f"(d));
-        rs = rs * fmaf(-0.5f * d * rs, rs, 1.5f);            // one Newton step: full fp32 accuracy
+#pragma unroll
+        for (int i = j + 1; i < 8; ++i) {
+            const float f = l[i][j] * rd;
+#pragma unroll
+            for (int c = j + 1; c <= i; ++c)
+                l[i][c] = fmaf(-f, l[c][j], l[i][c]);
+        }
         rinv[j] = rs;
         l[j][j] = d * rs;
 #pragma unroll
         for (int i = j + 1; i < 8; ++i)
             l[i][j] *= rs;
-#pragma unroll
-        for (int i = j + 1; i < 8; ++i)
-#pragma unroll
-            for (int c = j + 1; c <= i; ++c)
-                l[i][c] = fmaf(-l[i][j], l[c][j], l[i][c]);
     }
     return bad;
 }
