@@ -280,9 +280,18 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
 #pragma unroll 4
             for (int k = 0; k < N; ++k) {
                 const float vk = sl.L[k * LD + c], tk = sl.Lt[k * LD + c];
-                axpy_row<N>(s2, vk, sm.B + k * LD);
-                axpy_row<N>(y2, tk, sm.B + k * LD);
-                axpy_row<N>(p2, tk, sm.A + k * LD);
+                const f32x2 vv = pack2(vk, vk), tt = pack2(tk, tk);
+#pragma unroll
+                for (int q = 0; q < N / 4; ++q) {             // each row of B and A is read once
+                    const ulonglong2 b4 = *reinterpret_cast<const ulonglong2*>(sm.B + k * LD + 4 * q);
+                    const ulonglong2 a4 = *reinterpret_cast<const ulonglong2*>(sm.A + k * LD + 4 * q);
+                    fma2(s2[2 * q], vv, b4.x);
+                    fma2(s2[2 * q + 1], vv, b4.y);
+                    fma2(y2[2 * q], tt, b4.x);
+                    fma2(y2[2 * q + 1], tt, b4.y);
+                    fma2(p2[2 * q], tt, a4.x);
+                    fma2(p2[2 * q + 1], tt, a4.y);
+                }
             }
             float s[N], y[N];
             unpack_row<N>(s, s2);
