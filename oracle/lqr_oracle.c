@@ -24,9 +24,19 @@
  * t >= 1 and P_0 = P_0(paper) + Q.  S^{-1} is applied through a Cholesky
  * factorisation (S is positive definite when R is and P is semi-definite).
  *
+ * Time-varying problems (Definition A.1 with A_t, B_t, Q_t, R_t and a terminal weight Q_f,
+ * Prop. A.1 / Alg. 1 with time indices kept): lqr_oracle_solve_tv takes, per operand, the element
+ * stride between consecutive time indices (0 = the same matrix at every t):
+ *   P_H = Q_f ;  S = R_t + B_t' P_{t+1} B_t ;  Y = B_t' P_{t+1} A_t ;  K_t = -S^{-1} Y ;
+ *   P_t = Q_t + A_t' P_{t+1} A_t + Y' K_t ;  u_t = K_t x_t ;  x_{t+1} = A_t x_t + B_t u_t,
+ * with cost sum_{t<H} (x_t'Q_t x_t + u_t'R_t u_t) + x_H'Q_f x_H.  The paper's h_t = A_t h_{t-1} + B_t u_t
+ * (t = 1..T) maps to x_t = h_t, A_t(here) = A_{t+1}(paper), likewise B and R, Q_t(here) = Q_t(paper),
+ * Q_f = Q_T.  The time-invariant entry points are this function with all strides 0 and Q_f = Q.
+ *
  * All matrices are row-major and contiguous.  Parity status: pinned (brute-force
  * KKT solve, closed forms, invariants, DARE limit, symplectic cross-identity --
- * see tests/test_oracle_*.py).
+ * see tests/test_oracle_*.py; the time-varying function by a brute-force KKT solve with
+ * time-varying blocks, tail consistency and the cost identity -- tests/test_oracle_tv_pins.py).
  */
 #include <math.h>
 #include <stdint.h>
@@ -112,9 +122,9 @@ static void chol_solve(int m, int n, const double *L, double *Y)
  * S = R + B'P_{t+1}B at time index t was not positive; outputs are then
  * unspecified.  Returns -1 on bad sizes / allocation failure.
  */
-int lqr_oracle_solve(int n, int m, int H, const double *A, const double *B, const double *Q,
-                     const double *R, const double *x0, double *K, double *P, double *x,
-                     double *u, int first_only)
+int lqr_oracle_solve_tv(int n, int m, int H, const double *A0, int64_t sA, const double *B0, int64_t sB,
+                        const double *Q0, int64_t sQ, const double *R0, int64_t sR, const double *Qf,
+                        const double *x0, double *K, double *P, double *x, double *u, int first_only)
 {
     if (n < 1 || m < 1 || H < 1)
         return -1;
@@ -135,11 +145,12 @@ int lqr_oracle_solve(int n, int m, int H, const double *A, const double *B, cons
     double *xt = S + mm, *xn = xt + n, *ut = xn + n;
     int info = 0;
 
-    memcpy(Pall + nn * (size_t)H, Q, sizeof(double) * nn);          /* P_H = Q */
+    memcpy(Pall + nn * (size_t)H, Qf, sizeof(double) * nn);         /* P_H = Q_f */
     for (int t = H - 1; t >= 0 && info == 0; --t) {
         const double *Pn = Pall + nn * (size_t)(t + 1);
         double *Pt = Pall + nn * (size_t)t;
         double *Kt = Kall + nm * (size_t)t;
+        const double *A = A0 + sA * t, *B = B0 + sB * t, *Q = Q0 + sQ * t, *R = R0 + sR * t;
         mm_nn(n, m, n, Pn, B, PB);
         mm_tn(m, m, n, B, PB, S);                                   /* B'(P B)  */
         for (size_t i = 0; i < mm; ++i)
@@ -178,6 +189,7 @@ int lqr_oracle_solve(int n, int m, int H, const double *A, const double *B, cons
             memcpy(x, xt, sizeof(double) * (size_t)n);
         for (int t = 0; t < H; ++t) {
             const double *Kt = Kall + nm * (size_t)t;
+            const double *A = A0 + sA * t, *B = B0 + sB * t;
             for (int i = 0; i < m; ++i) {
                 double s = 0.0;
                 for (int j = 0; j < n; ++j)
@@ -205,6 +217,14 @@ int lqr_oracle_solve(int n, int m, int H, const double *A, const double *B, cons
     return info;
 }
 
+/* Time-invariant problem: every stride 0, terminal weight Q (Prop. 3.1 with P_T = Q). */
+int lqr_oracle_solve(int n, int m, int H, const double *A, const double *B, const double *Q,
+                     const double *R, const double *x0, double *K, double *P, double *x,
+                     double *u, int first_only)
+{
+    return lqr_oracle_solve_tv(n, m, H, A, 0, B, 0, Q, 0, R, 0, Q, x0, K, P, x, u, first_only);
+}
+
 /*
  * N independent instances.  off*[i] is the element offset of instance i's
  * operand inside the corresponding base array (this is how operands shared by a
@@ -212,14 +232,15 @@ int lqr_oracle_solve(int n, int m, int H, const double *A, const double *B, cons
  * Instances are distributed over `nthreads` OpenMP threads.  Returns the number
  * of threads actually used.
  */
-int lqr_oracle_solve_batch(int64_t N, int n, int m, int H,
-                           const double *A, const int64_t *offA,
-                           const double *B, const int64_t *offB,
-                           const double *Q, const int64_t *offQ,
-                           const double *R, const int64_t *offR,
-                           const double *x0, const int64_t *offx,
-                           double *K, double *P, double *x, double *u, int32_t *info,
-                           int first_only, int nthreads)
+int lqr_oracle_solve_batch_tv(int64_t N, int n, int m, int H,
+                              const double *A, const int64_t *offA, int64_t sA,
+                              const double *B, const int64_t *offB, int64_t sB,
+                              const double *Q, const int64_t *offQ, int64_t sQ,
+                              const double *R, const int64_t *offR, int64_t sR,
+                              const double *Qf, const int64_t *offQf,
+                              const double *x0, const int64_t *offx,
+                              double *K, double *P, double *x, double *u, int32_t *info,
+                              int first_only, int nthreads)
 {
     size_t nn = (size_t)n * n, nm = (size_t)n * m;
     size_t sP = first_only ? nn : nn * (size_t)(H + 1);
@@ -234,8 +255,8 @@ int lqr_oracle_solve_batch(int64_t N, int n, int m, int H,
         used = omp_get_num_threads();
 #pragma omp for schedule(dynamic, 1)
         for (int64_t i = 0; i < N; ++i) {
-            int r = lqr_oracle_solve(n, m, H, A + offA[i], B + offB[i], Q + offQ[i], R + offR[i],
-                                     x0 + offx[i], K ? K + (size_t)i * nm * H : NULL,
+            int r = lqr_oracle_solve_tv(n, m, H, A + offA[i], sA, B + offB[i], sB, Q + offQ[i], sQ, R + offR[i], sR,
+                                     Qf + offQf[i], x0 + offx[i], K ? K + (size_t)i * nm * H : NULL,
                                      P ? P + (size_t)i * sP : NULL,
                                      x ? x + (size_t)i * n * (H + 1) : NULL,
                                      u ? u + (size_t)i * su : NULL, first_only);
@@ -246,8 +267,8 @@ int lqr_oracle_solve_batch(int64_t N, int n, int m, int H,
 #else
     (void)nthreads;
     for (int64_t i = 0; i < N; ++i) {
-        int r = lqr_oracle_solve(n, m, H, A + offA[i], B + offB[i], Q + offQ[i], R + offR[i],
-                                 x0 + offx[i], K ? K + (size_t)i * nm * H : NULL,
+        int r = lqr_oracle_solve_tv(n, m, H, A + offA[i], sA, B + offB[i], sB, Q + offQ[i], sQ, R + offR[i], sR,
+                                 Qf + offQf[i], x0 + offx[i], K ? K + (size_t)i * nm * H : NULL,
                                  P ? P + (size_t)i * sP : NULL,
                                  x ? x + (size_t)i * n * (H + 1) : NULL,
                                  u ? u + (size_t)i * su : NULL, first_only);
@@ -256,4 +277,18 @@ int lqr_oracle_solve_batch(int64_t N, int n, int m, int H,
     }
 #endif
     return used;
+}
+
+/* Time-invariant batch: strides 0, Q_f = Q. */
+int lqr_oracle_solve_batch(int64_t N, int n, int m, int H,
+                           const double *A, const int64_t *offA,
+                           const double *B, const int64_t *offB,
+                           const double *Q, const int64_t *offQ,
+                           const double *R, const int64_t *offR,
+                           const double *x0, const int64_t *offx,
+                           double *K, double *P, double *x, double *u, int32_t *info,
+                           int first_only, int nthreads)
+{
+    return lqr_oracle_solve_batch_tv(N, n, m, H, A, offA, 0, B, offB, 0, Q, offQ, 0, R, offR, 0, Q, offQ,
+                                     x0, offx, K, P, x, u, info, first_only, nthreads);
 }

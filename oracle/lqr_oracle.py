@@ -49,6 +49,16 @@ def _load():
             + [dp] * 4
             + [ctypes.POINTER(ctypes.c_int32), ctypes.c_int, ctypes.c_int]
         )
+        lib.lqr_oracle_solve_tv.restype = ctypes.c_int
+        lib.lqr_oracle_solve_tv.argtypes = [ctypes.c_int] * 3 + [dp, ctypes.c_int64] * 4 + [dp] * 6 + [ctypes.c_int]
+        lib.lqr_oracle_solve_batch_tv.restype = ctypes.c_int
+        lib.lqr_oracle_solve_batch_tv.argtypes = (
+            [ctypes.c_int64, ctypes.c_int, ctypes.c_int, ctypes.c_int]
+            + [dp, ip, ctypes.c_int64] * 4
+            + [dp, ip] * 2
+            + [dp] * 4
+            + [ctypes.POINTER(ctypes.c_int32), ctypes.c_int, ctypes.c_int]
+        )
         _lib = lib
     return _lib
 
@@ -134,6 +144,64 @@ def solve_batch(A, B, Q, R, x0, H, batch=None, first_only=False, nthreads=0,
     for k, v in (("K", K), ("P", P), ("x", x), ("u", u)):
         if v is not None:
             out[k] = v
+    out["info"] = info
+    out["threads"] = used
+    return out
+
+
+def solve_tv(A, B, Q, R, Qf, x0, H, first_only=False):
+    """One time-varying instance (Definition A.1 / Prop. A.1 with A_t, B_t, Q_t, R_t, terminal weight Qf).
+
+    ``A`` is ``[H,n,n]`` or ``[n,n]`` (the same at every t); likewise ``B [H,n,m]``, ``Q [H,n,n]``,
+    ``R [H,m,m]``.  Index t of each is the matrix of step t: ``x_{t+1} = A_t x_t + B_t u_t``, stage cost
+    ``x_t'Q_t x_t + u_t'R_t u_t``, terminal cost ``x_H'Qf x_H``.  Returns ``(K, P, x, u, info)``.
+    """
+    A, B, Q, R, Qf, x0 = map(_f64, (A, B, Q, R, Qf, x0))
+    n, m = B.shape[-2:]
+    strides = []
+    for a, tail in ((A, (n, n)), (B, (n, m)), (Q, (n, n)), (R, (m, m))):
+        assert a.shape in (tail, (H,) + tail), (a.shape, tail)
+        strides.append(0 if a.ndim == 2 else tail[0] * tail[1])
+    assert Qf.shape == (n, n) and x0.shape == (n,)
+    K = np.empty((H, m, n))
+    P = np.empty((n, n) if first_only else (H + 1, n, n))
+    x = np.empty((H + 1, n))
+    u = np.empty((m,) if first_only else (H, m))
+    info = _load().lqr_oracle_solve_tv(
+        n, m, H, _dptr(A), strides[0], _dptr(B), strides[1], _dptr(Q), strides[2], _dptr(R), strides[3],
+        _dptr(Qf), _dptr(x0), _dptr(K), _dptr(P), _dptr(x), _dptr(u), int(first_only))
+    return K, P, x, u, info
+
+
+def solve_batch_tv(A, B, Q, R, Qf, x0, H, batch, tv=("A", "B", "Q", "R"), first_only=False, nthreads=0,
+                   want=("K", "P", "x", "u")):
+    """Many time-varying instances.  Operands named in ``tv`` carry a time axis of length ``H`` right after
+    their (broadcastable) batch dimensions, e.g. ``A [..batch.., H, n, n]``; the others are ``[..batch.., n, n]``.
+    Returns the same dict as :func:`solve_batch`."""
+    n, m = np.asarray(B).shape[-2:]
+    batch = tuple(int(b) for b in batch)
+    N = int(np.prod(batch))
+    ops, offs, strides = {}, {}, {}
+    for name, arr, tail in (("A", A, (n, n)), ("B", B, (n, m)), ("Q", Q, (n, n)), ("R", R, (m, m))):
+        full_tail = ((H,) + tail) if name in tv else tail
+        ops[name], offs[name] = _offsets(arr, batch, full_tail)
+        strides[name] = tail[0] * tail[1] if name in tv else 0
+    Qf_, oQf = _offsets(Qf, batch, (n, n))
+    x_, ox = _offsets(x0, batch, (n,))
+    K = np.empty((N, H, m, n)) if "K" in want else None
+    P = (np.empty((N, n, n) if first_only else (N, H + 1, n, n))) if "P" in want else None
+    x = np.empty((N, H + 1, n)) if "x" in want else None
+    u = (np.empty((N, m) if first_only else (N, H, m))) if "u" in want else None
+    info = np.zeros(N, dtype=np.int32)
+    ip = ctypes.POINTER(ctypes.c_int64)
+    args = []
+    for name in ("A", "B", "Q", "R"):
+        args += [_dptr(ops[name]), offs[name].ctypes.data_as(ip), strides[name]]
+    used = _load().lqr_oracle_solve_batch_tv(
+        N, n, m, H, *args, _dptr(Qf_), oQf.ctypes.data_as(ip), _dptr(x_), ox.ctypes.data_as(ip),
+        _dptr(K), _dptr(P), _dptr(x), _dptr(u),
+        info.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)), int(first_only), int(nthreads))
+    out = {k: v for k, v in (("K", K), ("P", P), ("x", x), ("u", u)) if v is not None}
     out["info"] = info
     out["threads"] = used
     return out
