@@ -144,6 +144,26 @@ int ttc_lqr_solve(ttc_lqr_handle* h,
                   uint32_t flags, void* cuda_stream);
 
 /*
+ * Time-varying problem (Definition A.1 / Prop. A.1 with A_t, B_t, Q_t, R_t and a terminal weight Q_f;
+ * Alg. 1 with the time indices kept):
+ *     minimise   sum_{t=0}^{H-1} ( x_t' Q_t x_t + u_t' R_t u_t ) + x_H' Q_f x_H ,   x_{t+1} = A_t x_t + B_t u_t
+ *     P_H = Q_f ;  K_t = -(R_t + B_t' P_{t+1} B_t)^{-1} B_t' P_{t+1} A_t ;  P_t = Q_t + A_t' P_{t+1} A_t + (B_t' P_{t+1} A_t)' K_t .
+ * With the paper's h_t = A_t h_{t-1} + B_t u_t (t = 1..T): x_t = h_t, A_t(here) = A_{t+1}(paper), likewise B and R,
+ * Q_t(here) = Q_t(paper), Q_f = Q_T.
+ * tstride[0..3] are the element strides between consecutive time indices of A, B, Q, R (0 = the same matrix
+ * at every t); the matrix of step t of instance i starts at the operand's batch offset + t * tstride.
+ * Qf [n][n] (F32 or BF16, batch strides like any operand) is the terminal weight; it may be NULL only when
+ * tstride[2] == 0, and then Q_f = Q.  Everything else (outputs, info, flags, stream, errors) as ttc_lqr_solve.
+ * Served by the fp32 kernels (n = m = 16 / 32 warp kernel, generic kernel otherwise); TTC_SCAN handles
+ * time-invariant problems only and returns TTC_STATUS_UNSUPPORTED here.
+ */
+int ttc_lqr_solve_tv(ttc_lqr_handle* h,
+                     const ttc_operand* A, const ttc_operand* B, const ttc_operand* Q, const ttc_operand* R,
+                     const int64_t tstride[4], const ttc_operand* Qf, const ttc_operand* x0, int32_t H,
+                     float* K, float* P, float* x, float* u, int32_t* info,
+                     uint32_t flags, void* cuda_stream);
+
+/*
  * Same computation with HOST buffers (same problem statement as ttc_lqr_solve): operand
  * pointers and all outputs are host memory (pinned memory lets the copies run asynchronously;
  * pageable memory works but serialises them).  The call copies the inputs to device staging

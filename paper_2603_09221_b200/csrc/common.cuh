@@ -14,6 +14,7 @@ struct OperandDev {
     const void* ptr;
     int dtype;            // TTC_F32 | TTC_BF16
     long long s0, s1, s2; // element strides of the three batch dimensions (0 = shared)
+    long long st;         // element stride between consecutive time indices (0 = the same matrix at every t)
 };
 
 struct SolveParams {
@@ -21,6 +22,7 @@ struct SolveParams {
     long long b0, b1, b2, N;   // batch dims and their product
     long long t0, tcount;      // token window [t0, t0 + tcount) of the last batch dimension solved by this launch
     OperandDev A, B, Q, R, x0;
+    OperandDev Qf;             // terminal weight P_H (ptr null: P_H = Q)
     float* K;      // [N][H][m][n] or null
     float* P;      // [N][H+1][n][n] ([N][n][n] when first_only) or null
     float* x;      // [N][H+1][n] or null

@@ -126,8 +126,8 @@ __device__ __forceinline__ float warp_dot(const float* row, const float* v, int 
 
 // Forward rollout of Alg. 1 for one instance by one CTA.  Kt_src: gains [H][m][n] in global
 // memory (or, when only u_0 is wanted, the K_0 left in shared memory: pass Ksm and H_roll = 1).
-__device__ __forceinline__ void cta_rollout(const SolveParams& p, long long inst, const float* sA,
-                                            const float* sB, const float* Kglob, const float* Ksm,
+__device__ __forceinline__ void cta_rollout(const SolveParams& p, long long inst, float* sA,
+                                            float* sB, const float* Kglob, const float* Ksm,
                                             float* sx, float* sxn, float* su, int steps)
 {
     const int n = p.n, m = p.m, H = p.H;
@@ -139,6 +139,13 @@ __device__ __forceinline__ void cta_rollout(const SolveParams& p, long long inst
             xo[e] = sx[e];
     for (int t = 0; t < steps; ++t) {
         const float* Kt = Ksm ? Ksm : Kglob + (long long)t * m * n;
+        if (p.A.st || p.B.st) {                      // time-varying dynamics: A_t, B_t of this step
+            if (p.A.st)
+                load_to_smem(sA, p.A, operand_offset(p.A, inst, p.b1, p.b2) + t * p.A.st, n * n);
+            if (p.B.st)
+                load_to_smem(sB, p.B, operand_offset(p.B, inst, p.b1, p.b2) + t * p.B.st, n * m);
+            __syncthreads();
+        }
         for (int i = warp; i < m; i += nw) {
             const float s = warp_dot(Kt + i * n, sx, n);
             if (lane == 0)
@@ -221,10 +228,10 @@ __global__ void __launch_bounds__(256) riccati_cta_kernel(SolveParams p)
         load_to_smem(sR, p.R, operand_offset(p.R, inst, p.b1, p.b2), m * m);
         {
             const long long oq = operand_offset(p.Q, inst, p.b1, p.b2);
+            const long long of = p.Qf.ptr ? operand_offset(p.Qf, inst, p.b1, p.b2) : 0;
             for (int e = threadIdx.x; e < n * n; e += blockDim.x) {
-                const float q = load_elem(p.Q, oq + e);
-                sQ[e] = q;
-                sP[e] = q;
+                sQ[e] = load_elem(p.Q, oq + e);
+                sP[e] = p.Qf.ptr ? load_elem(p.Qf, of + e) : sQ[e];       // P_H = Q_f
             }
         }
         if (p.x0.ptr)
@@ -236,10 +243,17 @@ __global__ void __launch_bounds__(256) riccati_cta_kernel(SolveParams p)
         float* Pout = p.P ? p.P + inst * (long long)(p.first_only ? 1 : H + 1) * n * n : nullptr;
         if (Pout && !p.first_only)
             for (int e = threadIdx.x; e < n * n; e += blockDim.x)
-                Pout[(long long)H * n * n + e] = sQ[e];      // P_H = Q
+                Pout[(long long)H * n * n + e] = sP[e];      // P_H
 
         int fail = 0;
         for (int t = H - 1; t >= 0; --t) {
+            if (p.A.st || p.B.st || p.Q.st || p.R.st) {                      // time-varying operands of step t
+                if (p.A.st) load_to_smem(sA, p.A, operand_offset(p.A, inst, p.b1, p.b2) + t * p.A.st, n * n);
+                if (p.B.st) load_to_smem(sB, p.B, operand_offset(p.B, inst, p.b1, p.b2) + t * p.B.st, n * m);
+                if (p.R.st) load_to_smem(sR, p.R, operand_offset(p.R, inst, p.b1, p.b2) + t * p.R.st, m * m);
+                if (p.Q.st) load_to_smem(sQ, p.Q, operand_offset(p.Q, inst, p.b1, p.b2) + t * p.Q.st, n * n);
+                __syncthreads();
+            }
             smem_gemm<false>(n, m, n, sP, n, sB, m, sV, m, nullptr, 0);      // V = P B
             smem_gemm<false>(n, n, n, sP, n, sA, n, sT, n, nullptr, 0);      // T = P A
             __syncthreads();

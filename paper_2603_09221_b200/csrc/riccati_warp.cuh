@@ -164,7 +164,25 @@ __device__ __forceinline__ void axpy_row(f32x2 (&acc)[N / 2], float w, const flo
     }
 }
 
+// Per-head operands of time index t -> shared memory (all threads of the CTA; the caller synchronises).
 template <int N>
+__device__ __forceinline__ void load_head_operands(Smem<N>& sm, const SolveParams& p, long long oa, long long ob, long long orr,
+                                                   int t, bool la, bool lb, bool lr)
+{
+    constexpr int LD = Shape<N>::LD;
+    const float* Ag = reinterpret_cast<const float*>(p.A.ptr) + oa + t * p.A.st;
+    const float* Bg = reinterpret_cast<const float*>(p.B.ptr) + ob + t * p.B.st;
+    const float* Rg = reinterpret_cast<const float*>(p.R.ptr) + orr + t * p.R.st;
+    for (int e = threadIdx.x; e < N * N; e += THREADS) {
+        const int r = e / N, cc = e % N;
+        if (la) sm.A[r * LD + cc] = __ldg(Ag + e);
+        if (lb) sm.B[r * LD + cc] = __ldg(Bg + e);
+        if (lr) sm.R[r * LD + cc] = __ldg(Rg + e);
+    }
+}
+
+// TV = time-varying request (time strides or a terminal weight): the other instantiation carries none of that code.
+template <int N, bool TV>
 __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kernel(SolveParams p, int* chunk_counter)
 {
     using S = Shape<N>;
@@ -194,22 +212,13 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
         const long long tok0 = p.t0 + (chunk % chunks_per_head) * S::SLOTS;
         const long long inst0 = head * p.b2 + tok0;
         const int ntok = (int)min((long long)S::SLOTS, p.t0 + p.tcount - tok0);
-        {
-            const long long oa = operand_offset(p.A, inst0, p.b1, p.b2);
-            const long long ob = operand_offset(p.B, inst0, p.b1, p.b2);
-            const long long orr = operand_offset(p.R, inst0, p.b1, p.b2);
-            if (oa != offA || ob != offB || orr != offR) {
-                const float* Ag = reinterpret_cast<const float*>(p.A.ptr) + oa;
-                const float* Bg = reinterpret_cast<const float*>(p.B.ptr) + ob;
-                const float* Rg = reinterpret_cast<const float*>(p.R.ptr) + orr;
-                for (int e = tid; e < N * N; e += THREADS) {
-                    const int r = e / N, cc = e % N;
-                    sm.A[r * LD + cc] = __ldg(Ag + e);
-                    sm.B[r * LD + cc] = __ldg(Bg + e);
-                    sm.R[r * LD + cc] = __ldg(Rg + e);
-                }
-                offA = oa; offB = ob; offR = orr;
-            }
+        const long long oa = operand_offset(p.A, inst0, p.b1, p.b2);
+        const long long ob = operand_offset(p.B, inst0, p.b1, p.b2);
+        const long long orr = operand_offset(p.R, inst0, p.b1, p.b2);
+        const bool tv_head = TV && (p.A.st | p.B.st | p.R.st) != 0;      // per-head operands change with the time index
+        if (tv_head || oa != offA || ob != offB || orr != offR) {
+            load_head_operands<N>(sm, p, oa, ob, orr, TV ? H - 1 : 0, true, true, true);
+            offA = oa; offB = ob; offR = orr;
         }
         __syncthreads();
         const int slot_idx = warp * S::IPW + sub;
@@ -220,7 +229,10 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
         float* Pout = (p.P && active) ? p.P + inst * (long long)(p.first_only ? 1 : H + 1) * N * N : nullptr;
         float* Kout = (Kbase && need_K_all) ? Kbase + inst * (long long)H * N * N : nullptr;
         float pcol[N];
-        load_q_row<N>(pcol, p.Q, oq);                         // P_H = Q
+        if (TV && p.Qf.ptr)
+            load_q_row<N>(pcol, p.Qf, operand_offset(p.Qf, inst, p.b1, p.b2) + (long long)c * N);   // P_H = Q_f
+        else
+            load_q_row<N>(pcol, p.Q, oq);                     // P_H = Q
         if (Pout && !p.first_only) {
 #pragma unroll
             for (int l = 0; l < N; ++l)
@@ -234,6 +246,11 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
 
 #pragma unroll 1
         for (int ts = H - 1; ts >= 0; --ts) {
+            if (tv_head && ts != H - 1) {                     // A_t, B_t, R_t of this step (the whole CTA is in step)
+                __syncthreads();
+                load_head_operands<N>(sm, p, oa, ob, orr, ts, p.A.st != 0, p.B.st != 0, p.R.st != 0);
+                __syncthreads();
+            }
             f32x2 vcol[N / 2], tcol[N / 2];
 #pragma unroll
             for (int k = 0; k < N / 2; ++k) {
@@ -271,7 +288,7 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
                 float tmp[N];
                 load_row<N>(tmp, sm.R + c * LD);              // S[:,c] = R[:,c] + B' V[:,c]
                 pack_row<N>(s2, tmp);
-                load_q_row<N>(tmp, p.Q, oq);                  // Pn[:,c] = Q[:,c] + A' T[:,c] ; Y[:,c] = B' T[:,c]
+                load_q_row<N>(tmp, p.Q, TV ? oq + ts * p.Q.st : oq);    // Pn[:,c] = Q_t[:,c] + A' T[:,c] ; Y[:,c] = B' T[:,c]
                 pack_row<N>(p2, tmp);
             }
 #pragma unroll
@@ -411,13 +428,24 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
             float* xo = (p.x && store_ok) ? p.x + inst * (long long)(H + 1) * N : nullptr;
             float* uo = (p.u && store_ok) ? p.u + inst * (long long)(p.first_only ? N : H * N) : nullptr;
             float arow[N], brow[N];
-            load_row<N>(arow, sm.A + c * LD);
-            load_row<N>(brow, sm.B + c * LD);
+            if (!tv_head) {
+                load_row<N>(arow, sm.A + c * LD);
+                load_row<N>(brow, sm.B + c * LD);
+            }
             if (xo)
                 xo[c] = sl.x[c];
             __syncwarp();                                     // K_t written by the other lanes are visible
 #pragma unroll 1
             for (int ts = 0; ts < H; ++ts) {
+                if (tv_head) {                                // A_t, B_t of this step (after the backward pass they hold t = 0)
+                    if (ts > 0) {
+                        __syncthreads();
+                        load_head_operands<N>(sm, p, oa, ob, orr, ts, p.A.st != 0, p.B.st != 0, false);
+                        __syncthreads();
+                    }
+                    load_row<N>(arow, sm.A + c * LD);
+                    load_row<N>(brow, sm.B + c * LD);
+                }
                 float xv[N];
                 load_row<N>(xv, sl.x);
                 const float4* kr = reinterpret_cast<const float4*>(Kout + (long long)ts * N * N + c * N);

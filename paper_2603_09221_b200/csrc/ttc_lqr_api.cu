@@ -121,6 +121,7 @@ OperandDev to_dev(const ttc_operand* o)
         d.ptr = nullptr;
         d.dtype = TTC_F32;
         d.s0 = d.s1 = d.s2 = 0;
+        d.st = 0;
         return d;
     }
     d.ptr = o->ptr;
@@ -128,6 +129,7 @@ OperandDev to_dev(const ttc_operand* o)
     d.s0 = o->bstride[0];
     d.s1 = o->bstride[1];
     d.s2 = o->bstride[2];
+    d.st = 0;
     return d;
 }
 
@@ -290,7 +292,8 @@ namespace {
 // ttc_lqr_solve; one slice at a time for the pipelined host-buffer entry point).  Arguments validated.
 int solve_window(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, const ttc_operand* Q,
                  const ttc_operand* R, const ttc_operand* x0, int32_t H, float* K, float* P, float* x,
-                 float* u, int32_t* info, uint32_t flags, cudaStream_t st, long long t0, long long tcount)
+                 float* u, int32_t* info, uint32_t flags, cudaStream_t st, long long t0, long long tcount,
+                 const int64_t* tstride = nullptr, const ttc_operand* Qf = nullptr)
 {
     int s;
     const int n = h->cfg.n, m = h->cfg.m;
@@ -301,11 +304,18 @@ int solve_window(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, 
     p.t0 = t0; p.tcount = tcount;
     const long long nwin = p.b0 * p.b1 * tcount;          // instances of this launch
     p.A = to_dev(A); p.B = to_dev(B); p.Q = to_dev(Q); p.R = to_dev(R); p.x0 = to_dev(x0);
+    p.Qf = to_dev(Qf);
+    if (tstride) {
+        p.A.st = tstride[0]; p.B.st = tstride[1]; p.Q.st = tstride[2]; p.R.st = tstride[3];
+    }
+    const bool time_varying = p.Qf.ptr != nullptr || (p.A.st | p.B.st | p.Q.st | p.R.st) != 0;
     p.K = K; p.P = P; p.x = x; p.u = u; p.info = info;
     p.Kws = nullptr;
     p.first_only = (flags & TTC_OUT_FIRST_ONLY) ? 1 : 0;
 
     const int method = pick_method(h);
+    if (method == TTC_SCAN && time_varying)
+        return fail(TTC_STATUS_UNSUPPORTED, "the scan method handles time-invariant problems only");
     // The rollout reads every K_t in forward order after the backward pass produced them in
     // reverse order; when the caller does not want K they live in the workspace.
     const bool rollout_needs_all_K = (x != nullptr) || (u != nullptr && !p.first_only);
@@ -339,7 +349,7 @@ int solve_window(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, 
         const bool bf16_in = (Q->dtype == TTC_BF16) || (x0 && x0->ptr && x0->dtype == TTC_BF16);
         const bool want_tf32 = h->cfg.math == TTC_MATH_TF32 || (h->cfg.math == TTC_MATH_AUTO && bf16_in);
         const bool head_shared = A->bstride[2] == 0 && B->bstride[2] == 0 && R->bstride[2] == 0;
-        if (want_tf32 && n == 64 && m == 64 && head_shared) {
+        if (want_tf32 && n == 64 && m == 64 && head_shared && !time_varying) {
             // tcgen05 kernel: persistent CTAs, two independent warpgroups each
             if ((s = ensure(h->ws_E, sizeof(int) * 4))) return s;
             int* counter = static_cast<int*>(h->ws_E.ptr);
@@ -362,21 +372,23 @@ int solve_window(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, 
             if ((s = ensure(h->ws_E, sizeof(int) * 4))) return s;
             int* counter = static_cast<int*>(h->ws_E.ptr);
             TTC_CUDA(cudaMemsetAsync(counter, 0, sizeof(int), st));
+            void (*kern)(SolveParams, int*);
+            size_t smem;
+            long long chunks, grid;
             if (n == 32) {
-                const size_t smem = rwarp::smem_bytes<32>();
-                TTC_CUDA(cudaFuncSetAttribute(rwarp::riccati_warp_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-                const long long chunks = p.b0 * p.b1 * ((tcount + rwarp::Shape<32>::SLOTS - 1) / rwarp::Shape<32>::SLOTS);
-                long long grid = (long long)h->sm_count * 3;
-                if (grid > chunks) grid = chunks;
-                rwarp::riccati_warp_kernel<32><<<(unsigned)grid, rwarp::THREADS, smem, st>>>(p, counter);
+                kern = time_varying ? rwarp::riccati_warp_kernel<32, true> : rwarp::riccati_warp_kernel<32, false>;
+                smem = rwarp::smem_bytes<32>();
+                chunks = p.b0 * p.b1 * ((tcount + rwarp::Shape<32>::SLOTS - 1) / rwarp::Shape<32>::SLOTS);
+                grid = (long long)h->sm_count * 3;
             } else {
-                const size_t smem = rwarp::smem_bytes<16>();
-                TTC_CUDA(cudaFuncSetAttribute(rwarp::riccati_warp_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-                const long long chunks = p.b0 * p.b1 * ((tcount + rwarp::Shape<16>::SLOTS - 1) / rwarp::Shape<16>::SLOTS);
-                long long grid = (long long)h->sm_count * 4;
-                if (grid > chunks) grid = chunks;
-                rwarp::riccati_warp_kernel<16><<<(unsigned)grid, rwarp::THREADS, smem, st>>>(p, counter);
+                kern = time_varying ? rwarp::riccati_warp_kernel<16, true> : rwarp::riccati_warp_kernel<16, false>;
+                smem = rwarp::smem_bytes<16>();
+                chunks = p.b0 * p.b1 * ((tcount + rwarp::Shape<16>::SLOTS - 1) / rwarp::Shape<16>::SLOTS);
+                grid = (long long)h->sm_count * 4;
             }
+            TTC_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            if (grid > chunks) grid = chunks;
+            kern<<<(unsigned)grid, rwarp::THREADS, smem, st>>>(p, counter);
             TTC_CUDA(cudaGetLastError());
             h->last_launches += 1;
             h->total_launches += 1;
@@ -415,6 +427,27 @@ int ttc_lqr_solve(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B,
     h->last_launches = 0;
     return solve_window(h, A, B, Q, R, x0, H, K, P, x, u, info, flags, static_cast<cudaStream_t>(cuda_stream), 0,
                         h->cfg.batch[2]);
+}
+
+int ttc_lqr_solve_tv(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, const ttc_operand* Q,
+                     const ttc_operand* R, const int64_t tstride[4], const ttc_operand* Qf, const ttc_operand* x0,
+                     int32_t H, float* K, float* P, float* x, float* u, int32_t* info, uint32_t flags,
+                     void* cuda_stream)
+{
+    int s = validate_common(h, A, B, Q, R, x0, H, K, P, x, u, info, flags);
+    if (s)
+        return s;
+    if (!tstride)
+        return fail(TTC_STATUS_INVALID_ARGUMENT, "null tstride");
+    for (int i = 0; i < 4; ++i)
+        if (tstride[i] < 0)
+            return fail(TTC_STATUS_INVALID_ARGUMENT, "negative time stride");
+    if ((s = check_operand("Qf", Qf, true, tstride[2] == 0)))
+        return s;
+    TTC_CUDA(cudaSetDevice(h->cfg.device));
+    h->last_launches = 0;
+    return solve_window(h, A, B, Q, R, x0, H, K, P, x, u, info, flags, static_cast<cudaStream_t>(cuda_stream), 0,
+                        h->cfg.batch[2], tstride, (Qf && Qf->ptr) ? Qf : nullptr);
 }
 
 int ttc_lqr_solve_host(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, const ttc_operand* Q,
@@ -647,6 +680,7 @@ extern "C" int ttc_lqr_solve_first_noalloc(int32_t n, int32_t m, const int64_t b
     p.b0 = batch[0]; p.b1 = batch[1]; p.b2 = batch[2]; p.N = N;
     p.t0 = 0; p.tcount = batch[2];
     p.A = to_dev(A); p.B = to_dev(B); p.Q = to_dev(Q); p.R = to_dev(R); p.x0 = to_dev(x0);
+    p.Qf = to_dev(nullptr);
     p.K = nullptr; p.P = P0; p.x = nullptr; p.u = u0; p.info = info;
     p.Kws = nullptr;
     p.first_only = 1;

@@ -25,7 +25,7 @@ KERNEL_NAMES = {0: "none", 1: "riccati_cta", 2: "riccati_warp", 4: "scan", 5: "r
 
 EXPORTS = (
     "ttc_lqr_create", "ttc_lqr_solve", "ttc_lqr_solve_host", "ttc_lqr_destroy", "ttc_lqr_query",
-    "ttc_lqr_status_string", "ttc_lqr_last_error", "ttc_lqr_solve_first_noalloc",
+    "ttc_lqr_status_string", "ttc_lqr_last_error", "ttc_lqr_solve_first_noalloc", "ttc_lqr_solve_tv",
 )
 TTC_NOALLOC_SCRATCH_BYTES = 4 << 20
 
@@ -67,6 +67,9 @@ def load_library():
     opp = P(ttc_operand)
     lib.ttc_lqr_solve.restype = ctypes.c_int
     lib.ttc_lqr_solve.argtypes = [ctypes.c_void_p, opp, opp, opp, opp, opp, ctypes.c_int32] + \
+        [ctypes.c_void_p] * 5 + [ctypes.c_uint32, ctypes.c_void_p]
+    lib.ttc_lqr_solve_tv.restype = ctypes.c_int
+    lib.ttc_lqr_solve_tv.argtypes = [ctypes.c_void_p, opp, opp, opp, opp, P(ctypes.c_int64), opp, opp, ctypes.c_int32] + \
         [ctypes.c_void_p] * 5 + [ctypes.c_uint32, ctypes.c_void_p]
     lib.ttc_lqr_solve_host.restype = ctypes.c_int
     lib.ttc_lqr_solve_host.argtypes = [ctypes.c_void_p, opp, opp, opp, opp, opp, ctypes.c_int32] + \
@@ -178,6 +181,31 @@ class LqrSolver:
         _check(load_library().ttc_lqr_solve(
             self._h, *refs, int(H), self._ptr(K), self._ptr(P), self._ptr(x), self._ptr(u), self._ptr(info),
             int(flags), ctypes.c_void_p(stream.cuda_stream)))
+
+    def solve_tv(self, A, B, Q, R, Qf, x0, H, tv=("A", "B", "Q", "R"), K=None, P=None, x=None, u=None, info=None,
+                 flags=0, stream=None):
+        """Enqueue ``ttc_lqr_solve_tv``.  Operands named in ``tv`` carry a time axis of length >= H right after
+        their batch dimensions (``A [..batch.., H, n, n]``); the others are as for :meth:`solve`.  ``Qf`` is the
+        terminal weight (may be None when Q is not time-varying)."""
+        ops, tstride = [], (ctypes.c_int64 * 4)()
+        for i, (name, t, tail) in enumerate((("A", A, 2), ("B", B, 2), ("Q", Q, 2), ("R", R, 2))):
+            if name in tv:
+                if t.shape[-3] < H:
+                    raise ValueError("operand %s has %d time steps, H = %d" % (name, t.shape[-3], H))
+                ops.append(_operand(t[..., 0, :, :], 2, self.batch))
+                tstride[i] = t.stride(-3)
+            else:
+                ops.append(_operand(t, 2, self.batch))
+                tstride[i] = 0
+        oqf = _operand(Qf, 2, self.batch)
+        ox = _operand(x0, 1, self.batch)
+        ref = lambda o: ctypes.byref(o) if o is not None else None
+        if stream is None:
+            stream = torch.cuda.current_stream(self.device)
+        _check(load_library().ttc_lqr_solve_tv(
+            self._h, ref(ops[0]), ref(ops[1]), ref(ops[2]), ref(ops[3]), tstride, ref(oqf), ref(ox), int(H),
+            self._ptr(K), self._ptr(P), self._ptr(x), self._ptr(u), self._ptr(info), int(flags),
+            ctypes.c_void_p(stream.cuda_stream)))
 
     def solve_host(self, A, B, Q, R, x0, H, K=None, P=None, x=None, u=None, info=None, flags=0):
         """``ttc_lqr_solve_host``: all tensors live in host memory; returns when the results are there."""
