@@ -54,6 +54,8 @@ def algorithmic_counts(c):
     flops = (3 * n**3 + 5 * n * n * m + 3 * n * m * m + m**3 / 3.0 + 2 * n * n + 4 * n * m) * H
     esz = 2 if c["q_dtype"] == "bf16" else 4
     bytes_in = (n * n + n) * esz
+    if c.get("tv"):                  # per-token Q_t for every step plus the terminal weight; head operands are shared
+        bytes_in = ((H + 1) * n * n + n) * esz
     if c["first_only"]:
         bytes_out = 4 * (n * n + m)
     else:
@@ -116,30 +118,36 @@ def oracle_sample(w, count):
 def time_oracle(w, idx, first_only):
     from tests import parity_util as pu
     t0 = time.perf_counter()
-    ref = pu.run_oracle(w, idx=idx, first_only=first_only)
+    ref = (pu.run_oracle_tv if w.get("tv") else pu.run_oracle)(w, idx=idx, first_only=first_only)
     dt = time.perf_counter() - t0
     return ref, dt
 
 
-def run_reference(args, cid):
+def run_reference(args, cid, tv_key=None):
     """--impl reference: the float64 oracle on the host cores, bounded sample per step."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    c = workloads.CONFIGS[cid]
+    c = workloads.TV_CONFIGS[tv_key] if tv_key else workloads.CONFIGS[cid]
     S, Hd, T = c["batch"]
     tok = max(1, min(T, args.ref_instances // (S * Hd)))
-    w = workloads.make_workload(cid, device="cpu", batch=(S, Hd, tok))
     n_inst = S * Hd * tok
     from oracle import lqr_oracle as orc
-    from paper_2603_09221_b200.workloads import to_float64_numpy
-    d = to_float64_numpy(w)
     want = ("P", "u") if c["first_only"] else ("K", "P", "x", "u")
+    if tv_key:
+        w = workloads.make_tv_workload(tv_key, device="cpu", batch=(S, Hd, tok))
+        d = {k: w[k].to(torch.float64).numpy() for k in ("A", "B", "Q", "R", "Qf", "x0")}
+        solve = lambda: orc.solve_batch_tv(d["A"], d["B"], d["Q"], d["R"], d["Qf"], d["x0"], c["H"], (S, Hd, tok),
+                                           tv=c["tv"], first_only=c["first_only"], want=want)
+    else:
+        from paper_2603_09221_b200.workloads import to_float64_numpy
+        d = to_float64_numpy(workloads.make_workload(cid, device="cpu", batch=(S, Hd, tok)))
+        solve = lambda: orc.solve_batch(d["A"], d["B"], d["Q"], d["R"], d["x0"], c["H"], batch=(S, Hd, tok),
+                                        first_only=c["first_only"], want=want)
     times, threads = [], 0
     for it in range(args.warmup + args.steps):
         t0 = time.perf_counter()
-        out = orc.solve_batch(d["A"], d["B"], d["Q"], d["R"], d["x0"], c["H"], batch=(S, Hd, tok),
-                              first_only=c["first_only"], want=want)
+        out = solve()
         dt = time.perf_counter() - t0
         threads = out["threads"]
         if it >= args.warmup:
@@ -174,9 +182,10 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
-    cid = int(args.workload.replace("cfg", ""))
+    tv_key = args.workload if args.workload in workloads.TV_CONFIGS else None
+    cid = None if tv_key else int(args.workload.replace("cfg", ""))
     if args.impl == "reference":
-        run_reference(args, cid)
+        run_reference(args, cid, tv_key)
         return
     args.warmup = max(args.warmup, 3)
 
@@ -194,11 +203,15 @@ def main():
     dev = torch.device("cuda", local)
     peaks = measured_peaks()
 
-    c = dict(workloads.CONFIGS[cid])
+    c = dict(workloads.TV_CONFIGS[tv_key] if tv_key else workloads.CONFIGS[cid])
     if args.tokens > 0:
         c["batch"] = (c["batch"][0], c["batch"][1], args.tokens)
         c["name"] += "_tokens%d" % args.tokens
-    w = workloads.make_workload(cid, device=dev, batch=c["batch"], seed=sharding.rank_seed(cid, rank))
+    if tv_key:
+        w = workloads.make_tv_workload(tv_key, device=dev, batch=c["batch"], seed=sharding.rank_seed(100, rank))
+        args.no_e2e = True           # the host-buffer entry point covers the time-invariant solve only
+    else:
+        w = workloads.make_workload(cid, device=dev, batch=c["batch"], seed=sharding.rank_seed(cid, rank))
     n, m, H = c["n"], c["m"], c["H"]
     N = int(np.prod(c["batch"]))
     first = c["first_only"]
@@ -210,6 +223,10 @@ def main():
     flags = lqr.TTC_OUT_FIRST_ONLY if first else 0
 
     def step():
+        if tv_key:
+            solver.solve_tv(w["A"], w["B"], w["Q"], w["R"], w["Qf"], w["x0"], H, tv=c["tv"], K=out.get("K"),
+                            P=out.get("P"), x=out.get("x"), u=out.get("u"), info=out.get("info"), flags=flags)
+            return
         solver.solve(w["A"], w["B"], w["Q"], w["R"], w["x0"], H, K=out.get("K"), P=out.get("P"), x=out.get("x"),
                      u=out.get("u"), info=out.get("info"), flags=flags)
 
@@ -317,7 +334,7 @@ def main():
             "scaling": "weak", "vs_baseline": None, "dtype": "tf32" if kname == "riccati_umma" else "f32",
             "data": "synthetic",
             "config": {"workload": c["name"], "n": n, "m": m, "H": H, "instances": N, "batch": list(c["batch"]),
-                       "q_x0_dtype": c["q_dtype"], "outputs": list(want), "method": args.method, "kernel": kname,
+                       "q_x0_dtype": c["q_dtype"], "time_varying": list(c.get("tv", ())), "outputs": list(want), "method": args.method, "kernel": kname,
                        "l2": "inputs+outputs per step exceed L2 (%.2f GB)" % (alg_bytes / 1e9)
                        if alg_bytes > 126e6 else "workload fits L2: latency-bound case"},
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches),

@@ -36,6 +36,51 @@ CONFIGS = {
 }
 
 
+# Time-varying workload shaped like the paper's TTC layer: state dimension 16, 16 heads, horizon 32.  Dynamics and
+# control cost belong to the head and change with the time index, state cost / terminal weight / initial state
+# belong to the token.  Stand-in for the layer's learned parameters (near-identity A_t, diagonal-dominant R_t,
+# rank-16 Q_t): A_t = I + 0.1 G_t / sqrt(n), B_t ~ N(0, 1/n), R_t = diag(U[0.5, 1.5]) + 0.05 M_t M_t'/m,
+# Q_t = L_t L_t'/n + 0.05 I, Q_f likewise, x0 ~ N(0, I).
+TV_CONFIGS = {
+    "tv16": dict(name="tv16_ttc_layer_d16_T32", batch=(4, 16, 1024), n=16, m=16, H=32, q_dtype="f32",
+                 first_only=True, tol=1e-4, tv=("A", "B", "Q", "R")),
+}
+
+
+def make_tv_workload(key="tv16", device="cpu", batch=None, seed=None, chunk=4096):
+    """Inputs of a time-varying configuration: ``A, B, R [1,Hd,1,H,...]`` (float32, per head and time index),
+    ``Q [S,Hd,T,H,n,n]``, ``Qf [S,Hd,T,n,n]``, ``x0 [S,Hd,T,n]`` plus the configuration fields."""
+    c = dict(TV_CONFIGS[key])
+    if batch is not None:
+        c["batch"] = tuple(int(b) for b in batch)
+    S, Hd, T = c["batch"]
+    n, m, H = c["n"], c["m"], c["H"]
+    seed = SEED0 + 100 if seed is None else seed
+    gen = torch.Generator(device=device)
+    gen.manual_seed(seed)
+    rn = lambda *shape: torch.randn(shape, generator=gen, device=device)
+    eye_n, eye_m = torch.eye(n, device=device), torch.eye(m, device=device)
+    A = eye_n + 0.1 * rn(1, Hd, 1, H, n, n) / n ** 0.5
+    B = rn(1, Hd, 1, H, n, m) / n ** 0.5
+    M = rn(1, Hd, 1, H, m, m)
+    R = torch.diag_embed(0.5 + torch.rand((1, Hd, 1, H, m), generator=gen, device=device)) + 0.05 * M @ M.transpose(-1, -2) / m
+    R = 0.5 * (R + R.transpose(-1, -2))
+    N = S * Hd * T
+    Q = torch.empty((N, H, n, n), dtype=torch.float32, device=device)
+    for s0 in range(0, N, chunk):
+        cnt = min(chunk, N - s0)
+        L = rn(cnt, H, n, n)
+        q = L @ L.transpose(-1, -2) / n + 0.05 * eye_n
+        Q[s0:s0 + cnt] = 0.5 * (q + q.transpose(-1, -2))
+    Lf = rn(N, n, n)
+    Qf = Lf @ Lf.transpose(-1, -2) / n + 0.05 * eye_n
+    Qf = 0.5 * (Qf + Qf.transpose(-1, -2))
+    x0 = rn(N, n)
+    c.update(A=A.contiguous(), B=B.contiguous(), R=R.contiguous(), Q=Q.reshape(S, Hd, T, H, n, n),
+             Qf=Qf.reshape(S, Hd, T, n, n), x0=x0.reshape(S, Hd, T, n), seed=seed)
+    return c
+
+
 def _system(rng, n, m, rho):
     G = rng.standard_normal((n, n))
     A = G * (rho / np.max(np.abs(np.linalg.eigvals(G))))

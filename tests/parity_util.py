@@ -90,6 +90,28 @@ def run_oracle(w, idx=None, first_only=None, H=None, nthreads=0):
     return orc.solve_batch(A, B, Q, R, x0, H, batch=(len(idx),), first_only=first_only, nthreads=nthreads)
 
 
+def run_oracle_tv(w, idx=None, first_only=None, H=None, nthreads=0):
+    """The time-varying oracle on the instances ``idx`` of a workload whose operands named in ``w["tv"]`` carry a
+    time axis after the batch dimensions."""
+    S, Hd, T = w["batch"]
+    n, m = w["n"], w["m"]
+    N = S * Hd * T
+    H = w["H"] if H is None else H
+    first_only = w["first_only"] if first_only is None else first_only
+    idx_t = torch.as_tensor(np.arange(N) if idx is None else idx, device=w["Q"].device, dtype=torch.long)
+
+    def sel(name, tail):
+        t = w[name]
+        if name in w["tv"]:
+            t = t[..., :H, :, :]
+            tail = (H,) + tuple(tail)
+        full = t.expand((S, Hd, T) + tuple(tail)).reshape((N,) + tuple(tail))
+        return full[idx_t].to(torch.float64).cpu().numpy()
+
+    return orc.solve_batch_tv(sel("A", (n, n)), sel("B", (n, m)), sel("Q", (n, n)), sel("R", (m, m)), sel("Qf", (n, n)),
+                              sel("x0", (n,)), H, (len(idx_t),), tv=w["tv"], first_only=first_only, nthreads=nthreads)
+
+
 def compare(gpu, ref, idx, tol, names=("K", "P", "x", "u")):
     """Returns {name: err}; asserts every requested output is within tol and info == 0."""
     n_dims = {"K": 2, "P": 2, "x": 1, "u": 1}

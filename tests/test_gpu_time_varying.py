@@ -105,3 +105,34 @@ def test_scan_method_rejects_time_varying_requests():
         s.solve_tv(w["A"], w["B"], w["Q"], w["R"], w["Qf"], w["x0"], 4, P=out["P"])
     assert "UNSUPPORTED" in str(ei.value)
     s.close()
+
+
+def test_ttc_layer_shaped_workload_full_size_on_sampled_instances():
+    """The time-varying benchmark configuration (d = 16, 16 heads, horizon 32) at full size, in the launch
+    configuration the benchmark times; the oracle solves a stratified sample of instances one by one."""
+    from paper_2603_09221_b200 import workloads
+    w = workloads.make_tv_workload("tv16", device=DEV)
+    n, m, H, batch = w["n"], w["m"], w["H"], w["batch"]
+    N = int(np.prod(batch))
+    s = lqr.LqrSolver(n, m, H, batch)
+    out = lqr.alloc_outputs(n, m, H, N, DEV, first_only=True, want=("P", "u", "info"))
+    out["P"].fill_(123456.0)
+    out["u"].fill_(123456.0)
+    out["info"].fill_(-7)
+    s.solve_tv(w["A"], w["B"], w["Q"], w["R"], w["Qf"], w["x0"], H, tv=w["tv"], P=out["P"], u=out["u"],
+               info=out["info"], flags=lqr.TTC_OUT_FIRST_ONLY)
+    torch.cuda.synchronize()
+    assert lqr.KERNEL_NAMES[s.query(lqr.TTC_QUERY_LAST_KERNEL)] == "riccati_warp"
+    assert s.query(lqr.TTC_QUERY_DEVICE_ERROR) == 0
+    s.close()
+    assert int(out["info"].abs().max()) == 0
+    assert not torch.any(out["P"] == 123456.0) and not torch.any(out["u"] == 123456.0)
+    S, Hd, T = batch
+    toks = np.array([0, 1, T // 2, T - 2, T - 1])
+    idx = (np.arange(S * Hd)[:, None] * T + toks[None, :]).reshape(-1)
+    ref = pu.run_oracle_tv(w, idx=idx, first_only=True)
+    errs = pu.compare(out, ref, idx, w["tol"], names=("P", "u"))
+    print("tv16 sampled parity:", errs)
+    # symmetry of P_0 holds at any size
+    P = out["P"][:: 97]
+    assert float((P - P.transpose(-1, -2)).abs().max() / P.abs().max()) < 1e-5
