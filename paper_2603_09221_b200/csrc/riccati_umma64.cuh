@@ -8,16 +8,19 @@
 //
 // Per step (Prop. 3.1), with P symmetric and the per-head operand BA = [B'; A'] (128 x 64):
 //   (1)  W  = BA * [P_a P_b]          -> W_x = [V_x'; T_x'] = [(P_x B)'; (P_x A)']        SS, M128 N128
-//   (2x) F_x  = W_x * B  = [S_x - R ; Y_x']   DP_x = W_x * A = [ . ; A'P_x A]              TS (A operand
-//        read from tensor memory, no round trip through shared memory), N64 each
-//   S_x = R + (S_x - R) and Y_x' -> shared, fp32.  Two warps per instance run a right-looking blocked
-//        Cholesky (8-wide panels) on the tall matrix [S_x; Y_x']: diagonal blocks in registers, panel rows by
-//        forward substitution, trailing updates as 3 x tf32 (error-compensated) mma.sync.  It leaves
-//        L (S_x = L L') and Z_x' = Y_x' L^{-T}: no explicit inverse, no extra contraction for Z.
+//   (2x) F_x  = W_x * B  = [S_x - R ; Y_x']                                               TS (A operand read from
+//        tensor memory, no round trip through shared memory), N64
+//   (3x) right-looking blocked Cholesky (8-wide panels) of the tall matrix G_x = [S_x; Y_x'] IN TENSOR MEMORY:
+//        thread r owns row r (lane r).  Per panel: load the row's 8 panel columns (tcgen05.ld), add R, publish the
+//        8 x 8 diagonal block, every thread factors it in registers and forward-substitutes its own row, writes
+//        the row of the panel as tf32 hi + lo parts to a 128 x 8 operand buffer, and ONE rank-8 tcgen05.mma
+//        (3 passes: hi*hi + lo*hi + hi*lo, error-compensated) applies the trailing update to all 128 rows.
+//        Both instances of the pair go through every panel together, so their dependency chains overlap.
+//        It leaves L (S_x = L L') and Z_x' = Y_x' L^{-T} (rows 64..127): no explicit inverse.
+//   (4x) DP_x = W_x * A = [ . ; A'P_x A]   (into the columns that held F_x)                TS, N64
 //   (5x) DP_x -= Z_x' Z_x                                                                   SS, N64
 //   P_x <- Q_x + DP_x            (P_t = Q + A'P A - Y'S^{-1}Y)
-// Tensor-memory map of a warpgroup (256 columns): R0 = W_a then DP_b, R1 = W_b, R2 = F_a then F_b,
-// R3 = DP_a.
+// Tensor-memory map of a warpgroup (256 columns): R0 = W_a, R1 = W_b, R2 = F_a then DP_a, R3 = F_b then DP_b.
 //
 // Shared-memory operands use the canonical K-major layout without swizzle: 8 x 4 (rows x k) core
 // matrices of 128 contiguous bytes, chunk stride 128 B along k, 2048 B between 8-row groups.  A row
@@ -48,17 +51,22 @@ constexpr int SPIN_LIMIT = 1 << 22;
 constexpr uint32_t OFF_BA = 0;
 constexpr uint32_t OFF_X0 = BUF_BYTES;
 constexpr uint32_t OFF_X1 = 2 * BUF_BYTES;
-constexpr uint32_t OFF_MISC = 3 * BUF_BYTES;
+constexpr uint32_t OFF_PAN = 3 * BUF_BYTES;     // panel operands: per instance 128 x 8 hi parts, 128 x 8 lo parts
+constexpr uint32_t PSR = 256;                   // bytes between 8-row groups of a panel buffer (2 chunks)
+constexpr uint32_t PAN_BYTES = 16 * PSR;        // one 128 x 8 buffer
+constexpr uint32_t OFF_MISC = OFF_PAN + 4 * PAN_BYTES;
 struct Misc {
     unsigned long long mbar;     // MMA completion barrier
     int chunk;                   // current work item
     int dead;                    // set when a wait timed out
     int flag[2];                 // first failed pivot per instance (0 = none)
     alignas(16) float x0[2][N];
-    alignas(16) float y0[2][N];
+    alignas(16) float y0[2][N];  // Y x_0 / u_t of the rollout; during the factorisation: the 8 x 8 diagonal blocks
+    alignas(16) float ld[2][36]; // current diagonal factors: strict lower triangle (28) + reciprocal pivots (8)
 };
 constexpr uint32_t WG_BYTES = OFF_MISC + ((sizeof(Misc) + 127) / 128) * 128;
 constexpr uint32_t SMEM_BYTES = NUM_WG * WG_BYTES + 128;     // + slot for the tensor-memory base address
+static_assert(SMEM_BYTES <= 227 * 1024, "shared memory of one CTA");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -92,6 +100,12 @@ __device__ __forceinline__ float round_tf32(float x) { return __uint_as_float(to
 __device__ __forceinline__ uint64_t smem_desc(uint32_t saddr)
 {
     return (uint64_t)((saddr >> 4) & 0x3FFFu) | ((uint64_t)(SC >> 4) << 16) | ((uint64_t)(SR >> 4) << 32) |
+           ((uint64_t)1 << 46);
+}
+// the same for a 128 x 8 panel buffer (8-row groups 256 B apart)
+__device__ __forceinline__ uint64_t panel_desc(uint32_t saddr)
+{
+    return (uint64_t)((saddr >> 4) & 0x3FFFu) | ((uint64_t)(SC >> 4) << 16) | ((uint64_t)(PSR >> 4) << 32) |
            ((uint64_t)1 << 46);
 }
 // instruction descriptor: tf32 x tf32 -> f32, both operands K-major, M = 128
@@ -163,6 +177,15 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32])
     for (int i = 0; i < 32; ++i)
         v[i] = __uint_as_float(r[i]);
 }
+
+// 32 lanes x 8 consecutive columns; the caller waits with tmem_wait_ld() before it reads v
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&r)[8])
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 __device__ __forceinline__ void wg_barrier(int wg) { asm volatile("bar.sync %0, %1;" :: "r"(1 + wg), "r"(WG_THREADS) : "memory"); }
 __device__ __forceinline__ void pair_barrier(int wg, int x) { asm volatile("bar.sync %0, %1;" :: "r"(3 + 2 * wg + x), "r"(64) : "memory"); }
@@ -248,125 +271,6 @@ __device__ __forceinline__ void store_row8(unsigned char* grp, int slot, const f
     }
     *reinterpret_cast<float4*>(grp + slot * 16) = a;
     *reinterpret_cast<float4*>(grp + SC + (ROT ? ((slot + 4) & 7) : slot) * 16) = b;
-}
-
-// Two warps (pw = 0, 1; 64 threads) work on the tall matrix G = [S; Y'] (128 x 64, fp32): S (64 x 64 SPD,
-// lower triangle used) at `Sm`, Y' at `Ym`, both in the core-matrix layout.  Right-looking blocked Cholesky
-// with 8-wide panels, applied to all 128 rows: on return the lower triangle of Sm holds L (S = L L') and
-// Ym holds Z' = Y' L^{-T} rounded to tf32, so that Z'Z' ' = Y' S^{-1} Y.  Per panel k:
-//   every thread factors the 8 x 8 diagonal block in registers (redundantly: nothing to exchange),
-//   row owners replace G[r][panel] by G[r][panel] L_d^{-T}  (rows of S below the block, every row of Y'),
-//   the trailing columns get the rank-8 update G[r][c] -= G[r][panel] . S[c][panel] as 3 x tf32 mma.
-// Fragment addresses are a per-thread constant plus compile-time offsets.  A non-positive pivot is recorded
-// in *flag as code0 + index.
-__device__ __forceinline__ void pair_chol_solve(unsigned char* Sm, unsigned char* Ym, int wg, int x, int pw, int lane,
-                                                int* flag, int code0)
-{
-    const int g = lane >> 2, t = lane & 3;
-    const int tid2 = 32 * pw + lane;
-    // fragment offsets inside an (8-row group, even chunk): S and the pending columns of Y' are in the rotated layout
-    const uint32_t frag_ab = (uint32_t)g * 16u + (uint32_t)t * 4u;                        // (row g, col t), even chunk
-    const uint32_t frag_ab1 = SC + (uint32_t)((g + 4) & 7) * 16u + (uint32_t)t * 4u;      // (row g, col t + 4), rotated odd chunk
-    const uint32_t frag_ab1c = SC + (uint32_t)g * 16u + (uint32_t)t * 4u;                 // the same, canonical
-    const uint32_t frag_c = (uint32_t)((g + 4 * (t >> 1)) & 7) * 16u + (uint32_t)(t >> 1) * SC + (uint32_t)((2 * t) & 3) * 4u; // (row g, cols 2t, 2t+1), rotated
-    const uint32_t own_grp = (uint32_t)(tid2 >> 3) * SR;                                  // 8-row group of row tid2
-    const int own_slot = tid2 & 7;
-#pragma unroll 1
-    for (int k = 0; k < 8; ++k) {
-        const uint32_t kcol = 2u * k * SC;             // byte offset of columns 8k .. 8k+7 inside a row
-        unsigned char* dblk = Sm + (uint32_t)k * SR + kcol;
-        float l[8][8], rinv[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i)
-            load_row8<true>(l[i], dblk, i);
-        const bool has_s = tid2 + 8 * k + 8 < N;
-        unsigned char* py = Ym + own_grp + kcol;
-        unsigned char* ps = Sm + own_grp + (uint32_t)(k + 1) * SR + kcol;       // row tid2 + 8k + 8
-        float xy[8], xs[8];
-        load_row8<true>(xy, py, own_slot);
-        if (has_s)
-            load_row8<true>(xs, ps, own_slot);
-        const int bad = chol8(l, rinv);
-        if (bad && tid2 == 0 && *flag == 0)
-            *flag = code0 + 8 * k + bad;
-        fsub8(xy, l, rinv);
-        if (has_s)
-            fsub8(xs, l, rinv);
-        store_row8<false, true>(py, own_slot, xy);    // final columns of Z': canonical layout, tf32
-        if (has_s)
-            store_row8<true, false>(ps, own_slot, xs);
-        pair_barrier(wg, x);                           // panel written; every thread has read the diagonal block
-        if (tid2 < 8) {                                // keep L_d for the back substitution
-#pragma unroll
-            for (int i = 0; i < 8; ++i)
-                if (tid2 == i)
-                    store_row8<true, false>(dblk, i, l[i]);
-        }
-        if (k == 7)
-            break;
-        // ---- trailing update: B fragments = rows 8j + g of S, columns 8k + t, 8k + t + 4
-        uint32_t bh[7][2], bl[7][2];
-        {
-            const unsigned char* pb = Sm + kcol;
-#pragma unroll
-            for (int j = 1; j < 8; ++j)
-                if (j > k) {
-                    split_tf32(*reinterpret_cast<const float*>(pb + j * SR + frag_ab), bh[j - 1][0], bl[j - 1][0]);
-                    split_tf32(*reinterpret_cast<const float*>(pb + j * SR + frag_ab1), bh[j - 1][1], bl[j - 1][1]);
-                }
-        }
-#pragma unroll
-        for (int uu = 0; uu < 4; ++uu) {
-            const int u = 2 * uu + pw;                 // tiles 0..3: rows of S, 4..7: rows of Y'
-            const bool is_s = u < 4;
-            const int mt = u & 3;
-            if (is_s && 16 * mt + 15 < 8 * k + 8)
-                continue;
-            unsigned char* Mt = is_s ? Sm : Ym;
-            uint32_t ah[4], al[4];
-            {
-                const unsigned char* pa = Mt + kcol + 2 * mt * SR;
-                const uint32_t odd = is_s ? frag_ab1 : frag_ab1c;              // the panel of Y' has just been stored canonically
-                split_tf32(-*reinterpret_cast<const float*>(pa + frag_ab), ah[0], al[0]);
-                split_tf32(-*reinterpret_cast<const float*>(pa + SR + frag_ab), ah[1], al[1]);
-                split_tf32(-*reinterpret_cast<const float*>(pa + odd), ah[2], al[2]);
-                split_tf32(-*reinterpret_cast<const float*>(pa + SR + odd), ah[3], al[3]);
-            }
-            // all C tiles of this row tile first, then three independent mma passes, then the stores
-            unsigned char* pc = Mt + frag_c + 2 * mt * SR;
-            float acc[7][4];
-#pragma unroll
-            for (int j = 1; j < 8; ++j) {
-                if (j <= k || (is_s && j > 2 * mt + 1))
-                    continue;
-                const float2 lo = *reinterpret_cast<const float2*>(pc + 2 * j * SC);
-                const float2 hi = *reinterpret_cast<const float2*>(pc + 2 * j * SC + SR);
-                acc[j - 1][0] = lo.x; acc[j - 1][1] = lo.y; acc[j - 1][2] = hi.x; acc[j - 1][3] = hi.y;
-            }
-            if (is_s) {                                // rows of Y' in the panel are already tf32: their low part is zero
-#pragma unroll
-                for (int j = 1; j < 8; ++j)
-                    if (!(j <= k || j > 2 * mt + 1))
-                        mma_16x8x8(acc[j - 1], al[0], al[1], al[2], al[3], bh[j - 1][0], bh[j - 1][1]);
-            }
-#pragma unroll
-            for (int j = 1; j < 8; ++j)
-                if (!(j <= k || (is_s && j > 2 * mt + 1)))
-                    mma_16x8x8(acc[j - 1], ah[0], ah[1], ah[2], ah[3], bl[j - 1][0], bl[j - 1][1]);
-#pragma unroll
-            for (int j = 1; j < 8; ++j)
-                if (!(j <= k || (is_s && j > 2 * mt + 1)))
-                    mma_16x8x8(acc[j - 1], ah[0], ah[1], ah[2], ah[3], bh[j - 1][0], bh[j - 1][1]);
-#pragma unroll
-            for (int j = 1; j < 8; ++j) {
-                if (j <= k || (is_s && j > 2 * mt + 1))
-                    continue;
-                *reinterpret_cast<float2*>(pc + 2 * j * SC) = make_float2(acc[j - 1][0], acc[j - 1][1]);
-                *reinterpret_cast<float2*>(pc + 2 * j * SC + SR) = make_float2(acc[j - 1][2], acc[j - 1][3]);
-            }
-        }
-        pair_barrier(wg, x);
-    }
 }
 
 // Gains (Eq. 4): K = -L^{-T} Z, i.e. row c of K' is -(row c of Z') L^{-1}.  Same two warps, same blocked scheme
@@ -540,8 +444,9 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
     const int lane = wt & 31;
     unsigned char* wsm = smem_raw + (size_t)wg * WG_BYTES;
     unsigned char* BA = wsm + OFF_BA;          // rows 0..63: B' (row j = column j of B), rows 64..127: A'
-    unsigned char* X0 = wsm + OFF_X0;          // [P_a; P_b] -> [Y_a'; Y_b'] -> [Z_a'; Z_b'] -> next [P_a; P_b]
-    unsigned char* X1 = wsm + OFF_X1;          // [S_a; S_b] -> [L_a; L_b]
+    unsigned char* X0 = wsm + OFF_X0;          // [P_a; P_b] -> [Z_a'; Z_b'] -> next [P_a; P_b]
+    unsigned char* X1 = wsm + OFF_X1;          // [L_a; L_b], fp32 (kept only when the gains or u_0 need it)
+    unsigned char* PAN = wsm + OFF_PAN;        // panel operands: hi_a | lo_a | hi_b | lo_b
     Misc& misc = *reinterpret_cast<Misc*>(wsm + OFF_MISC);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_raw + (size_t)NUM_WG * WG_BYTES);
     const uint32_t mbar = smem_u32(&misc.mbar);
@@ -640,57 +545,168 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
             wg_barrier(wg);
 
             for (int ts = H - 1; ts >= 0 && !dead; --ts) {
-                // (1) W = BA [P_a P_b]' -> R0|R1 ; (2a) F_a -> R2, DP_a -> R3
+                // (1) W = BA [P_a P_b]' -> R0|R1 ; (2) F_a -> R2, F_b -> R3
                 if (wt == 0) {
                     tc_fence_after();
                     gemm_ss(R0, smem_u32(BA), smem_u32(X0), 128, 0, false);
                     gemm_ts(R2, R0, smem_u32(BA), 64);
-                    gemm_ts(R3, R0, smem_u32(BA) + MAT_BYTES, 64);
+                    gemm_ts(R3, R1, smem_u32(BA), 64);
                     mma_commit(mbar);
                 }
                 wait_mma();
-                // (2b) back half first: DP_b -> R0 (W_a is dead), runs while F_a is read out
-                if (wt == 0)
-                    gemm_ts(R0, R1, smem_u32(BA) + MAT_BYTES, 64);
+                // (3) [S_x; Y_x'] = [L; Z'] L' panel by panel, thread wt owns row wt of both instances
+                const bool keep_l = need_K_all || (ts == 0 && want_u0);
+                float* diag = &misc.y0[0][0];                  // [2][8][8]
 #pragma unroll 1
-                for (int x = 0; x < 2; ++x) {
-                    if (x == 1) {
-                        wait_mma();
+                for (int pnl = 0; pnl < 8; ++pnl) {
+                    const int col = 8 * pnl;
+                    uint32_t raw[2][8];
+                    tmem_ld8(R2 + lane_sel + col, raw[0]);
+                    tmem_ld8(R3 + lane_sel + col, raw[1]);
+                    float4 r0 = make_float4(0.f, 0.f, 0.f, 0.f), r1 = r0;
+                    if (warp < 2) {
+                        r0 = __ldg(reinterpret_cast<const float4*>(Rg + (long long)wt * N + col));
+                        r1 = __ldg(reinterpret_cast<const float4*>(Rg + (long long)wt * N + col + 4));
                     }
+                    tmem_wait_ld();
+                    float v[2][8];
 #pragma unroll
-                    for (int half = 0; half < 2; ++half) {
-                        float h[32];
-                        tmem_ld32(R2 + lane_sel + 32 * half, h);
-                        if (warp < 2) {                // S_x = R + B'P_x B, fp32 -> X1
-                            const float4* rr = reinterpret_cast<const float4*>(Rg + (long long)wt * N + 32 * half);
+                    for (int x = 0; x < 2; ++x) {
+                        v[x][0] = __uint_as_float(raw[x][0]) + r0.x; v[x][1] = __uint_as_float(raw[x][1]) + r0.y;
+                        v[x][2] = __uint_as_float(raw[x][2]) + r0.z; v[x][3] = __uint_as_float(raw[x][3]) + r0.w;
+                        v[x][4] = __uint_as_float(raw[x][4]) + r1.x; v[x][5] = __uint_as_float(raw[x][5]) + r1.y;
+                        v[x][6] = __uint_as_float(raw[x][6]) + r1.z; v[x][7] = __uint_as_float(raw[x][7]) + r1.w;
+                    }
+                    if (warp == (pnl >> 2)) {
+                        // the 8 rows of the diagonal blocks belong to this warp: gather the blocks, factor them
+                        // (lanes 0..15 the block of instance a, lanes 16..31 that of b; redundantly within each
+                        // half) and publish L_d and the reciprocal pivots
+                        if ((unsigned)(wt - col) < 8u) {
 #pragma unroll
-                            for (int c = 0; c < 8; ++c) {
-                                const float4 r4 = __ldg(rr + c);
-                                *reinterpret_cast<float4*>(X1 + x * MAT_BYTES + toff_rot(wt, 32 * half + 4 * c)) =
-                                    make_float4(h[4 * c] + r4.x, h[4 * c + 1] + r4.y, h[4 * c + 2] + r4.z, h[4 * c + 3] + r4.w);
+                            for (int x = 0; x < 2; ++x) {
+                                float4* dst = reinterpret_cast<float4*>(diag + 64 * x + 8 * (wt - col));
+                                dst[0] = make_float4(v[x][0], v[x][1], v[x][2], v[x][3]);
+                                dst[1] = make_float4(v[x][4], v[x][5], v[x][6], v[x][7]);
                             }
-                        } else {                       // Y_x' -> X0, fp32 (P is dead once (1) has completed)
-#pragma unroll
-                            for (int c = 0; c < 8; ++c)
-                                *reinterpret_cast<float4*>(X0 + toff_rot(64 * x + (wt - 64), 32 * half + 4 * c)) =
-                                    make_float4(h[4 * c], h[4 * c + 1], h[4 * c + 2], h[4 * c + 3]);
                         }
+                        __syncwarp();
+                        const int hx = lane >> 4, hl = lane & 15;
+                        float l[8][8], rinv[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const float4 a4 = *reinterpret_cast<const float4*>(diag + 64 * hx + 8 * i);
+                            const float4 b4 = *reinterpret_cast<const float4*>(diag + 64 * hx + 8 * i + 4);
+                            l[i][0] = a4.x; l[i][1] = a4.y; l[i][2] = a4.z; l[i][3] = a4.w;
+                            l[i][4] = b4.x; l[i][5] = b4.y; l[i][6] = b4.z; l[i][7] = b4.w;
+                        }
+                        const int bad = chol8(l, rinv);
+                        if (hl == 0) {
+                            // strict lower triangle row by row (28 values), then the 8 reciprocal pivots
+                            float4* dst = reinterpret_cast<float4*>(&misc.ld[hx][0]);
+                            dst[0] = make_float4(l[1][0], l[2][0], l[2][1], l[3][0]);
+                            dst[1] = make_float4(l[3][1], l[3][2], l[4][0], l[4][1]);
+                            dst[2] = make_float4(l[4][2], l[4][3], l[5][0], l[5][1]);
+                            dst[3] = make_float4(l[5][2], l[5][3], l[5][4], l[6][0]);
+                            dst[4] = make_float4(l[6][1], l[6][2], l[6][3], l[6][4]);
+                            dst[5] = make_float4(l[6][5], l[7][0], l[7][1], l[7][2]);
+                            dst[6] = make_float4(l[7][3], l[7][4], l[7][5], l[7][6]);
+                            dst[7] = make_float4(rinv[0], rinv[1], rinv[2], rinv[3]);
+                            dst[8] = make_float4(rinv[4], rinv[5], rinv[6], rinv[7]);
+                        }
+                        if (hl == 0 && bad && misc.flag[hx] == 0)
+                            misc.flag[hx] = ts * N + col + bad;
                     }
                     tc_fence_before();
                     wg_barrier(wg);
-                    dead = misc.dead != 0;
-                    if (x == 0 && wt == 0) {           // F_a has been read by every warp: (2b) front half -> R2
+                    if (misc.dead != 0) {
+                        dead = true;
+                        break;
+                    }
+#pragma unroll
+                    for (int x = 0; x < 2; ++x) {
+                        float l[8][8], rinv[8];
+                        {
+                            const float4* src = reinterpret_cast<const float4*>(&misc.ld[x][0]);
+                            const float4 c0 = src[0], c1 = src[1], c2 = src[2], c3 = src[3], c4 = src[4], c5 = src[5],
+                                         c6 = src[6], c7 = src[7], c8 = src[8];
+                            l[1][0] = c0.x; l[2][0] = c0.y; l[2][1] = c0.z; l[3][0] = c0.w;
+                            l[3][1] = c1.x; l[3][2] = c1.y; l[4][0] = c1.z; l[4][1] = c1.w;
+                            l[4][2] = c2.x; l[4][3] = c2.y; l[5][0] = c2.z; l[5][1] = c2.w;
+                            l[5][2] = c3.x; l[5][3] = c3.y; l[5][4] = c3.z; l[6][0] = c3.w;
+                            l[6][1] = c4.x; l[6][2] = c4.y; l[6][3] = c4.z; l[6][4] = c4.w;
+                            l[6][5] = c5.x; l[7][0] = c5.y; l[7][1] = c5.z; l[7][2] = c5.w;
+                            l[7][3] = c6.x; l[7][4] = c6.y; l[7][5] = c6.z; l[7][6] = c6.w;
+                            rinv[0] = c7.x; rinv[1] = c7.y; rinv[2] = c7.z; rinv[3] = c7.w;
+                            rinv[4] = c8.x; rinv[5] = c8.y; rinv[6] = c8.z; rinv[7] = c8.w;
+                        }
+                        fsub8(v[x], l, rinv);
+                        if (warp < 2) {                        // L is lower triangular: row wt ends at column wt
+#pragma unroll
+                            for (int j = 0; j < 8; ++j)
+                                if (col + j > wt)
+                                    v[x][j] = 0.f;
+                        }
+                        float hi[8], lo[8];
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            hi[j] = round_tf32(v[x][j]);
+                            lo[j] = v[x][j] - hi[j];
+                        }
+                        unsigned char* ph = PAN + (uint32_t)x * 2u * PAN_BYTES + (uint32_t)(wt >> 3) * PSR + (uint32_t)(wt & 7) * 16u;
+                        *reinterpret_cast<float4*>(ph) = make_float4(hi[0], hi[1], hi[2], hi[3]);
+                        *reinterpret_cast<float4*>(ph + SC) = make_float4(hi[4], hi[5], hi[6], hi[7]);
+                        *reinterpret_cast<float4*>(ph + PAN_BYTES) = make_float4(lo[0], lo[1], lo[2], lo[3]);
+                        *reinterpret_cast<float4*>(ph + PAN_BYTES + SC) = make_float4(lo[4], lo[5], lo[6], lo[7]);
+                        if (warp >= 2) {                       // row wt - 64 of Z_x', tf32: operand of (5x)
+                            unsigned char* pz = X0 + (uint32_t)x * MAT_BYTES + (uint32_t)((wt - 64) >> 3) * SR + 2u * pnl * SC +
+                                                (uint32_t)(wt & 7) * 16u;
+                            *reinterpret_cast<float4*>(pz) = make_float4(hi[0], hi[1], hi[2], hi[3]);
+                            *reinterpret_cast<float4*>(pz + SC) = make_float4(hi[4], hi[5], hi[6], hi[7]);
+                        } else if (keep_l) {                   // row wt of L, fp32: gains / u_0
+                            store_row8<true, false>(X1 + (uint32_t)x * MAT_BYTES + (uint32_t)(wt >> 3) * SR + 2u * pnl * SC, wt & 7, v[x]);
+                        }
+                    }
+                    if (pnl == 7)
+                        break;
+                    async_proxy_fence();
+                    wg_barrier(wg);
+                    if (wt == 0) {                             // G_x -= panel * panel[0:64]'  (hi*hi + lo*hi + hi*lo)
                         tc_fence_after();
-                        gemm_ts(R2, R1, smem_u32(BA), 64);
+                        const uint32_t idn = instr_desc(64, 1);
+#pragma unroll
+                        for (int x = 0; x < 2; ++x) {
+                            const uint32_t d = x ? R3 : R2;
+                            const uint64_t dh = panel_desc(smem_u32(PAN) + (uint32_t)x * 2u * PAN_BYTES);
+                            const uint64_t dl = panel_desc(smem_u32(PAN) + (uint32_t)x * 2u * PAN_BYTES + PAN_BYTES);
+                            mma_ss(d, dh, dh, idn, 1u);
+                            mma_ss(d, dl, dh, idn, 1u);
+                            mma_ss(d, dh, dl, idn, 1u);
+                        }
                         mma_commit(mbar);
                     }
+                    wait_mma();
                 }
-                // ---- S = L L' and Z' = Y' L^{-T}: warps 0, 1 -> instance a, warps 2, 3 -> instance b
+                async_proxy_fence();
+                tc_fence_before();
+                wg_barrier(wg);
+                dead = dead || misc.dead != 0;
+                // (4x) DP_x = W_x A into the columns of F_x (lanes 64..127 = A'P_x A), then
+                // (5a) DP_a -= Z_a' Z_a : A operand rows 64..127 = Z_a' (rows 0..63 = the A' rows of BA, unused)
+                // (5b) DP_b -= Z_b' Z_b : A operand = [Z_a'; Z_b']
+                if (wt == 0 && !dead) {
+                    tc_fence_after();
+                    gemm_ts(R2, R0, smem_u32(BA) + MAT_BYTES, 64);
+                    gemm_ss(R2, smem_u32(X0) - MAT_BYTES, smem_u32(X0), 64, 1, true);
+                    gemm_ts(R3, R1, smem_u32(BA) + MAT_BYTES, 64);
+                    gemm_ss(R3, smem_u32(X0), smem_u32(X0) + MAT_BYTES, 64, 1, true);
+                    mma_commit(mbar);
+                }
+                if (dead)
+                    break;
                 {
                     const int x = warp >> 1, pw = warp & 1;
                     unsigned char* Sm = X1 + x * MAT_BYTES;
                     unsigned char* Ym = X0 + x * MAT_BYTES;
-                    pair_chol_solve(Sm, Ym, wg, x, pw, lane, &misc.flag[x], ts * N);
                     if (ts == 0 && want_u0) {
                         // u_0 = K_0 x_0 = -L^{-T} (Z x_0), fp32, by the 64 threads of the pair
                         const int i = 32 * pw + lane;
@@ -733,17 +749,6 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
                         }
                     }
                 }
-                async_proxy_fence();
-                wg_barrier(wg);
-                dead = dead || misc.dead != 0;
-                // (5a) DP_a (R3, lanes 64..127) -= Z_a' Z_a : A operand rows 64..127 = Z_a' (rows 0..63 = the A' rows of BA, unused)
-                // (5b) DP_b (R0, lanes 64..127) -= Z_b' Z_b : A operand = [Z_a'; Z_b']
-                if (wt == 0) {
-                    tc_fence_after();
-                    gemm_ss(R3, smem_u32(X0) - MAT_BYTES, smem_u32(X0), 64, 1, true);
-                    gemm_ss(R0, smem_u32(X0), smem_u32(X0) + MAT_BYTES, 64, 1, true);
-                    mma_commit(mbar);
-                }
                 // P_t = Q + DP: warps 2, 3 own the rows (lanes 64..127)
                 float q[64];
                 if (!need_K_all && warp >= 2)
@@ -778,7 +783,7 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
                         if (x == 1)
                             load_q_row(q, p.Q, oq_x[1], j);
                         float h0[32], h1[32];
-                        const uint32_t src = (x == 0 ? R3 : R0) + lane_sel;
+                        const uint32_t src = (x == 0 ? R2 : R3) + lane_sel;
                         tmem_ld32(src, h0);
                         tmem_ld32(src + 32, h1);
 #pragma unroll
