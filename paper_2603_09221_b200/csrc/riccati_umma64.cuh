@@ -208,8 +208,7 @@ __device__ __forceinline__ void split_tf32(float x, uint32_t& hi, uint32_t& lo)
 }
 
 // In-thread Cholesky of an 8 x 8 SPD block: l (lower triangle) is overwritten by L, rinv[i] = 1 / L[i][i].
-// The trailing update uses l_ij l_cj / d_j with the hardware reciprocal, so that the chain from one pivot to
-// the next is reciprocal -> multiply -> fma; the scaling by 1 / sqrt(d_j) is off that chain.
+// Right-looking; the chain from one pivot to the next is rsqrt -> multiply -> fma.
 // Returns 0 or 1 + the index of the first non-positive pivot.
 __device__ __forceinline__ int chol8(float (&l)[8][8], float (&rinv)[8])
 {
@@ -222,21 +221,18 @@ __device__ __forceinline__ int chol8(float (&l)[8][8], float (&rinv)[8])
                 bad = j + 1;
             d = 1.f;
         }
-        float rd, rs;
-        asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(rd) : "f"(d));
+        float rs;
         asm("rsqrt.approx.ftz.f32 %0, %1;" : "=f"(rs) : "f"(d));
-#pragma unroll
-        for (int i = j + 1; i < 8; ++i) {
-            const float f = l[i][j] * rd;
-#pragma unroll
-            for (int c = j + 1; c <= i; ++c)
-                l[i][c] = fmaf(-f, l[c][j], l[i][c]);
-        }
         rinv[j] = rs;
-        l[j][j] = d * rs;
 #pragma unroll
         for (int i = j + 1; i < 8; ++i)
             l[i][j] *= rs;
+#pragma unroll
+        for (int i = j + 1; i < 8; ++i)
+#pragma unroll
+            for (int c = j + 1; c <= i; ++c)
+                l[i][c] = fmaf(-l[i][j], l[c][j], l[i][c]);
+        l[j][j] = d * rs;
     }
     return bad;
 }
@@ -456,6 +452,11 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         misc.dead = 0;
     }
+    // rows 64..127 (Z') of the two low-part panel buffers stay zero: Z' is kept as tf32
+#pragma unroll
+    for (int x = 0; x < 2; ++x)
+        *reinterpret_cast<float4*>(PAN + (uint32_t)x * 2u * PAN_BYTES + PAN_BYTES + 8u * PSR + (uint32_t)wt * 16u) = make_float4(0.f, 0.f, 0.f, 0.f);
+    async_proxy_fence();
     if (tid < 32) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(smem_u32(tmem_slot)), "r"(512) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -467,6 +468,9 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
     const uint32_t R0 = tm, R1 = tm + 64, R2 = tm + 128, R3 = tm + 192;
     const uint32_t lane_sel = (uint32_t)(32 * warp) << 16;
     uint32_t parity = 0;
+    // one thread of warp 3 issues every MMA of the warpgroup (tensor-pipe order = its program order); the issue of
+    // a batch blocks that thread for about as long as the batch runs, and warps 0 and 1 factor the diagonal blocks
+    const bool issuer = wt == 96;
 
     const int H = p.H;
     const long long chunks_per_head = (p.tcount + CHUNK - 1) / CHUNK;
@@ -546,7 +550,7 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
 
             for (int ts = H - 1; ts >= 0 && !dead; --ts) {
                 // (1) W = BA [P_a P_b]' -> R0|R1 ; (2) F_a -> R2, F_b -> R3
-                if (wt == 0) {
+                if (issuer) {
                     tc_fence_after();
                     gemm_ss(R0, smem_u32(BA), smem_u32(X0), 128, 0, false);
                     gemm_ts(R2, R0, smem_u32(BA), 64);
@@ -557,19 +561,18 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
                 // (3) [S_x; Y_x'] = [L; Z'] L' panel by panel, thread wt owns row wt of both instances
                 const bool keep_l = need_K_all || (ts == 0 && want_u0);
                 float* diag = &misc.y0[0][0];                  // [2][8][8]
-#pragma unroll 1
-                for (int pnl = 0; pnl < 8; ++pnl) {
-                    const int col = 8 * pnl;
+                float v[2][8];                                 // this row's columns of the current panel
+                // columns c0 .. c0 + 7 of row wt (+ R for the rows of S)
+                auto load_cols = [&](int c0) {
                     uint32_t raw[2][8];
-                    tmem_ld8(R2 + lane_sel + col, raw[0]);
-                    tmem_ld8(R3 + lane_sel + col, raw[1]);
+                    tmem_ld8(R2 + lane_sel + c0, raw[0]);
+                    tmem_ld8(R3 + lane_sel + c0, raw[1]);
                     float4 r0 = make_float4(0.f, 0.f, 0.f, 0.f), r1 = r0;
                     if (warp < 2) {
-                        r0 = __ldg(reinterpret_cast<const float4*>(Rg + (long long)wt * N + col));
-                        r1 = __ldg(reinterpret_cast<const float4*>(Rg + (long long)wt * N + col + 4));
+                        r0 = __ldg(reinterpret_cast<const float4*>(Rg + (long long)wt * N + c0));
+                        r1 = __ldg(reinterpret_cast<const float4*>(Rg + (long long)wt * N + c0 + 4));
                     }
                     tmem_wait_ld();
-                    float v[2][8];
 #pragma unroll
                     for (int x = 0; x < 2; ++x) {
                         v[x][0] = __uint_as_float(raw[x][0]) + r0.x; v[x][1] = __uint_as_float(raw[x][1]) + r0.y;
@@ -577,6 +580,11 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
                         v[x][4] = __uint_as_float(raw[x][4]) + r1.x; v[x][5] = __uint_as_float(raw[x][5]) + r1.y;
                         v[x][6] = __uint_as_float(raw[x][6]) + r1.z; v[x][7] = __uint_as_float(raw[x][7]) + r1.w;
                     }
+                };
+                load_cols(0);
+#pragma unroll 1
+                for (int pnl = 0; pnl < 8; ++pnl) {
+                    const int col = 8 * pnl;
                     if (warp == (pnl >> 2)) {
                         // the 8 rows of the diagonal blocks belong to this warp: gather the blocks, factor them
                         // (lanes 0..15 the block of instance a, lanes 16..31 that of b; redundantly within each
@@ -622,6 +630,12 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
                         dead = true;
                         break;
                     }
+                    if (pnl == 7 && issuer) {
+                        // every row has read its last columns of F: (4x) DP_x = W_x A into the columns of F_x
+                        tc_fence_after();
+                        gemm_ts(R2, R0, smem_u32(BA) + MAT_BYTES, 64);
+                        gemm_ts(R3, R1, smem_u32(BA) + MAT_BYTES, 64);
+                    }
 #pragma unroll
                     for (int x = 0; x < 2; ++x) {
                         float l[8][8], rinv[8];
@@ -640,37 +654,38 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
                             rinv[4] = c8.x; rinv[5] = c8.y; rinv[6] = c8.z; rinv[7] = c8.w;
                         }
                         fsub8(v[x], l, rinv);
-                        if (warp < 2) {                        // L is lower triangular: row wt ends at column wt
+                        unsigned char* ph = PAN + (uint32_t)x * 2u * PAN_BYTES + (uint32_t)(wt >> 3) * PSR + (uint32_t)(wt & 7) * 16u;
+                        float hi[8];
+                        if (warp < 2) {                        // row wt of L: lower triangular, ends at column wt
+                            float lo[8];
 #pragma unroll
-                            for (int j = 0; j < 8; ++j)
+                            for (int j = 0; j < 8; ++j) {
                                 if (col + j > wt)
                                     v[x][j] = 0.f;
-                        }
-                        float hi[8], lo[8];
+                                hi[j] = round_tf32(v[x][j]);
+                                lo[j] = v[x][j] - hi[j];
+                            }
+                            *reinterpret_cast<float4*>(ph + PAN_BYTES) = make_float4(lo[0], lo[1], lo[2], lo[3]);
+                            *reinterpret_cast<float4*>(ph + PAN_BYTES + SC) = make_float4(lo[4], lo[5], lo[6], lo[7]);
+                            if (keep_l)                        // fp32 copy for the gains / u_0
+                                store_row8<true, false>(X1 + (uint32_t)x * MAT_BYTES + (uint32_t)(wt >> 3) * SR + 2u * pnl * SC, wt & 7, v[x]);
+                        } else {                               // row wt - 64 of Z_x': kept as tf32 (operand of (5x)), low part zero
 #pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            hi[j] = round_tf32(v[x][j]);
-                            lo[j] = v[x][j] - hi[j];
-                        }
-                        unsigned char* ph = PAN + (uint32_t)x * 2u * PAN_BYTES + (uint32_t)(wt >> 3) * PSR + (uint32_t)(wt & 7) * 16u;
-                        *reinterpret_cast<float4*>(ph) = make_float4(hi[0], hi[1], hi[2], hi[3]);
-                        *reinterpret_cast<float4*>(ph + SC) = make_float4(hi[4], hi[5], hi[6], hi[7]);
-                        *reinterpret_cast<float4*>(ph + PAN_BYTES) = make_float4(lo[0], lo[1], lo[2], lo[3]);
-                        *reinterpret_cast<float4*>(ph + PAN_BYTES + SC) = make_float4(lo[4], lo[5], lo[6], lo[7]);
-                        if (warp >= 2) {                       // row wt - 64 of Z_x', tf32: operand of (5x)
+                            for (int j = 0; j < 8; ++j)
+                                hi[j] = round_tf32(v[x][j]);
                             unsigned char* pz = X0 + (uint32_t)x * MAT_BYTES + (uint32_t)((wt - 64) >> 3) * SR + 2u * pnl * SC +
                                                 (uint32_t)(wt & 7) * 16u;
                             *reinterpret_cast<float4*>(pz) = make_float4(hi[0], hi[1], hi[2], hi[3]);
                             *reinterpret_cast<float4*>(pz + SC) = make_float4(hi[4], hi[5], hi[6], hi[7]);
-                        } else if (keep_l) {                   // row wt of L, fp32: gains / u_0
-                            store_row8<true, false>(X1 + (uint32_t)x * MAT_BYTES + (uint32_t)(wt >> 3) * SR + 2u * pnl * SC, wt & 7, v[x]);
                         }
+                        *reinterpret_cast<float4*>(ph) = make_float4(hi[0], hi[1], hi[2], hi[3]);
+                        *reinterpret_cast<float4*>(ph + SC) = make_float4(hi[4], hi[5], hi[6], hi[7]);
                     }
                     if (pnl == 7)
                         break;
                     async_proxy_fence();
                     wg_barrier(wg);
-                    if (wt == 0) {                             // G_x -= panel * panel[0:64]'  (hi*hi + lo*hi + hi*lo)
+                    if (issuer) {                              // G_x -= panel * panel[0:64]'  (hi*hi + lo*hi + hi*lo)
                         tc_fence_after();
                         const uint32_t idn = instr_desc(64, 1);
 #pragma unroll
@@ -685,19 +700,18 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
                         mma_commit(mbar);
                     }
                     wait_mma();
+                    load_cols(col + 8);
                 }
                 async_proxy_fence();
                 tc_fence_before();
                 wg_barrier(wg);
                 dead = dead || misc.dead != 0;
-                // (4x) DP_x = W_x A into the columns of F_x (lanes 64..127 = A'P_x A), then
+                // (4x) was issued at the last panel (lanes 64..127 of R2 / R3 = A'P_x A); then
                 // (5a) DP_a -= Z_a' Z_a : A operand rows 64..127 = Z_a' (rows 0..63 = the A' rows of BA, unused)
                 // (5b) DP_b -= Z_b' Z_b : A operand = [Z_a'; Z_b']
-                if (wt == 0 && !dead) {
+                if (issuer && !dead) {
                     tc_fence_after();
-                    gemm_ts(R2, R0, smem_u32(BA) + MAT_BYTES, 64);
                     gemm_ss(R2, smem_u32(X0) - MAT_BYTES, smem_u32(X0), 64, 1, true);
-                    gemm_ts(R3, R1, smem_u32(BA) + MAT_BYTES, 64);
                     gemm_ss(R3, smem_u32(X0), smem_u32(X0) + MAT_BYTES, 64, 1, true);
                     mma_commit(mbar);
                 }
