@@ -81,6 +81,7 @@ extern "C" {
 #define TTC_KERNEL_RICCATI_MMA    3  /* retired id (mma.sync kernel); never returned   */
 #define TTC_KERNEL_SCAN           4  /* symplectic-pair scan + gain/rollout kernel     */
 #define TTC_KERNEL_RICCATI_UMMA   5  /* tcgen05 contractions (tensor memory), n = m = 64 */
+#define TTC_KERNEL_LAYER          6  /* contextualised layer: parameters synthesised in-kernel */
 
 typedef struct ttc_lqr_handle ttc_lqr_handle; /* opaque; owned by the library */
 
@@ -162,6 +163,49 @@ int ttc_lqr_solve_tv(ttc_lqr_handle* h,
                      const int64_t tstride[4], const ttc_operand* Qf, const ttc_operand* x0, int32_t H,
                      float* K, float* P, float* x, float* u, int32_t* info,
                      uint32_t flags, void* cuda_stream);
+
+/*
+ * One Test-Time Control layer evaluation per instance with CONTEXTUALISED parameters
+ * (Contextualization and Parameterization paragraphs of the TTC-Net section): the LQR parameters
+ * of the planning horizon t = 1..T are synthesised inside the kernel from per-instance
+ * coefficient vectors and shared basis matrices and are never written to memory:
+ *     A_t = I + diag(exp(-t s_gamma_a) .* s_a)                        (diagonal)
+ *     B_t = (sum_i s_b[i] B_basis[i]) diag(exp(-t s_gamma_b))
+ *     Q_t = diag(exp(-t s_gamma_q)) (sum_i s_q[i] Q_basis[i]) diag(exp(-t s_gamma_q)),  Q_0 = 0,
+ *     Q_T = sum_i s_qf[i] Q_basis[i]                                  (terminal override)
+ *     R_t = diag(1 / r_inv)                                           (the layer is handed diag(R^-1))
+ * for the problem of the LQR section / Definition A.1 without affine terms,
+ *     h_t = A_t h_{t-1} + B_t u_t,  cost = sum_{t=1..T} h_t'Q_t h_t + u_t'R_t u_t,
+ * solved by the backward recursion of Prop. A.1 / Alg. 1.  Outputs: u1 = u_1* (the layer output,
+ * [N][n]) and P0 (the value matrix at t = 0, [N][n][n]: the optimal cost is h0'P0 h0), info [N]
+ * (0, or s*n + j + 1 for the first non-positive pivot j of R + B'PB at step s = t - 1; that
+ * instance's outputs are quiet NaN).  Each output may be NULL.
+ *
+ * The handle must have n == m in {16, 32} (else TTC_STATUS_UNSUPPORTED); N is the product of its
+ * batch dimensions and instance i of every array is row i.  All pointers are DEVICE memory,
+ * float32, dense row-major, 16-byte aligned, owned by the caller and read-only for the call:
+ * s_a, s_gamma_a, s_gamma_b, s_gamma_q, r_inv, h0 are [N][n]; s_b, s_q, s_qf are [N][r];
+ * B_basis, Q_basis are [r][n][n] (Q_basis[i] symmetric positive semi-definite), 1 <= r <= 64.
+ * s_gamma_* >= 0 and r_inv > 0 are the caller's responsibility (softplus outputs in the paper).
+ * 1 <= T <= max_horizon of the handle.  Asynchronous on cuda_stream like ttc_lqr_solve.
+ */
+typedef struct ttc_layer_inputs {
+    const float* s_a;
+    const float* s_gamma_a;
+    const float* s_gamma_b;
+    const float* s_gamma_q;
+    const float* s_b;
+    const float* s_q;
+    const float* s_qf;
+    const float* r_inv;
+    const float* h0;
+    const float* B_basis;
+    const float* Q_basis;
+    int32_t r;
+} ttc_layer_inputs;
+
+int ttc_lqr_solve_layer(ttc_lqr_handle* h, const ttc_layer_inputs* in, int32_t T,
+                        float* u1, float* P0, int32_t* info, void* cuda_stream);
 
 /*
  * Same computation with HOST buffers (same problem statement as ttc_lqr_solve): operand

@@ -1,0 +1,280 @@
+// One Test-Time Control layer evaluation per (token, head): the LQR parameters are synthesised
+// inside the kernel from the coefficient vectors (Contextualization / Parameterization paragraphs of
+// the TTC-Net section) and the backward Riccati recursion (Prop. A.1 / Alg. 1) runs on them; nothing
+// time-dependent is ever written to HBM.  Paper indices t = 1..T:
+//     A_t = I + diag(exp(-t g_A) a)                 (diagonal)
+//     B_t = Bbar diag(exp(-t g_B)),                 Bbar = sum_i s_B[i] B^(i)
+//     Q_t = diag(exp(-t g_Q)) Qbar diag(exp(-t g_Q)),  Qbar = sum_i s_Q[i] Q^(i),  Q_0 = 0,
+//     Q_T = sum_i s_Qf[i] Q^(i)                     (terminal override)
+//     R_t = diag(1 / r_inv)
+// and the layer output is the first optimal control u_1* = K_1 h_0.
+//
+// Same mapping as the dense fp32 warp kernel: N lanes own one instance, lane c holds COLUMN c of every
+// symmetric matrix (= row c), cross-lane traffic goes through broadcast reads of the instance's rows in
+// shared memory.  Step s = t - 1 (s = T-1 .. 0), P = P_{s+1}, with a = diag(A_t), g = exp(-t g_B), q = exp(-s g_Q):
+//     V[:,c] = g_c (P Bbar[:,c])                     one dense contraction (rows of P broadcast)
+//     T[:,c] = a_c P[:,c]                            A_t diagonal: no contraction
+//     S[:,c] = e_c / r_inv_c + g .* (Bbar' V[:,c])   one pass over the rows of Bbar yields S and Y
+//     Y[:,c] = g .* (Bbar' T[:,c])
+//     Pn[:,c] = q_c (q .* Qbar[:,c]) [s >= 1] + a .* T[:,c]
+//     S = L L',  Z[:,c] = L^{-1} Y[:,c],  Pn[:,c] -= Z' Z[:,c]        (P_s = Q_s + A'PA - Y'S^{-1}Y)
+// and at s = 0 the gain column K[:,c] = -L^{-T} Z[:,c] for u_1* = K h_0.
+#pragma once
+
+#include "riccati_warp.cuh"
+
+namespace ttc {
+namespace layer {
+
+struct LayerParams {
+    long long N;                 // instances
+    int T, r;
+    const float *s_a, *s_ga, *s_gb, *s_gq;   // [N][n]
+    const float *s_b, *s_q, *s_qf;           // [N][r]
+    const float *r_inv, *h0;                 // [N][n]
+    const float *B_basis, *Q_basis;          // [r][n][n]
+    float* u1;                   // [N][n] or null
+    float* P0;                   // [N][n][n] or null
+    int* info;                   // [N] or null
+};
+
+using rwarp::Shape;
+using rwarp::THREADS;
+using rwarp::WARPS;
+
+template <int N>
+struct Smem {
+    struct Slot {
+        float buf0[Shape<N>::MAT];     // rows of P, then rows of Z
+        float L[Shape<N>::MAT];        // staged V, then rows of L
+        float Lt[Shape<N>::MAT];       // staged T, then rows of L'; K_1 rows at the last step
+        float Bb[Shape<N>::MAT];       // rows of Bbar
+        float rinv[N];                 // 1 / L[i][i]
+        float x[N];                    // h_0
+        float at[N], gb[N], gq[N];     // diag(A_t), exp(-t g_B), exp(-s g_Q) of the current step
+    } slot[Shape<N>::SLOTS];
+    int chunk;
+};
+
+template <int N>
+__global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) ttc_layer_kernel(LayerParams p, int* chunk_counter)
+{
+    using S = Shape<N>;
+    using namespace rwarp;
+    constexpr int LD = S::LD;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    Smem<N>& sm = *reinterpret_cast<Smem<N>*>(smem_raw);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int sub = lane / N, c = lane % N;
+    typename Smem<N>::Slot& sl = sm.slot[warp * S::IPW + sub];
+    const int T = p.T, r = p.r;
+    const long long nchunks = (p.N + S::SLOTS - 1) / S::SLOTS;
+
+    for (;;) {
+        __syncthreads();
+        if (tid == 0)
+            sm.chunk = atomicAdd(chunk_counter, 1);
+        __syncthreads();
+        const long long chunk = sm.chunk;
+        if (chunk >= nchunks)
+            break;
+        const long long inst_raw = chunk * S::SLOTS + warp * S::IPW + sub;
+        const bool active = inst_raw < p.N;                   // idle segments shadow the chunk's first instance
+        const long long inst = active ? inst_raw : chunk * S::SLOTS;
+
+        // ---- synthesis of Bbar (rows -> shared), Qbar[:,c] (registers) and P_T = Q_T[:,c]
+        float qcol[N], pcol[N];
+        {
+            float bcol[N];
+#pragma unroll
+            for (int l = 0; l < N; ++l) {
+                bcol[l] = 0.f;
+                qcol[l] = 0.f;
+                pcol[l] = 0.f;
+            }
+            const float* sb = p.s_b + inst * r;
+            const float* sq = p.s_q + inst * r;
+            const float* sf = p.s_qf + inst * r;
+#pragma unroll 1
+            for (int i = 0; i < r; ++i) {
+                const float wb = __ldg(sb + i), wq = __ldg(sq + i), wf = __ldg(sf + i);
+                const float* Bi = p.B_basis + (long long)i * N * N + c;
+                const float* Qi = p.Q_basis + (long long)i * N * N + c;
+#pragma unroll
+                for (int l = 0; l < N; ++l) {
+                    const float qv = __ldg(Qi + l * N);
+                    bcol[l] = fmaf(wb, __ldg(Bi + l * N), bcol[l]);
+                    qcol[l] = fmaf(wq, qv, qcol[l]);
+                    pcol[l] = fmaf(wf, qv, pcol[l]);
+                }
+            }
+#pragma unroll
+            for (int l = 0; l < N; ++l)
+                sl.Bb[l * LD + c] = bcol[l];
+        }
+        const float a_c = __ldg(p.s_a + inst * N + c), ga_c = __ldg(p.s_ga + inst * N + c);
+        const float gb_c = __ldg(p.s_gb + inst * N + c), gq_c = __ldg(p.s_gq + inst * N + c);
+        const float r_c = 1.f / __ldg(p.r_inv + inst * N + c);
+        sl.x[c] = __ldg(p.h0 + inst * N + c);
+        store_row<N>(sl.buf0 + c * LD, pcol);                 // rows of P_T (row c = column c)
+        int fail = 0;
+
+#pragma unroll 1
+        for (int s = T - 1; s >= 0; --s) {
+            const float tt = (float)(s + 1);
+            const float at_c = fmaf(__expf(-tt * ga_c), a_c, 1.f);
+            const float g_c = __expf(-tt * gb_c);
+            const float q_c = (s >= 1) ? __expf(-(float)s * gq_c) : 0.f;     // Q_0 = 0
+            sl.at[c] = at_c;
+            sl.gb[c] = g_c;
+            sl.gq[c] = q_c;
+            __syncwarp();                                     // rows of P and the step's diagonals are in place
+            f32x2 vcol[N / 2];
+#pragma unroll
+            for (int k = 0; k < N / 2; ++k)
+                vcol[k] = 0ull;
+#pragma unroll 4
+            for (int i = 0; i < N; ++i) {                     // P Bbar[:,c]
+                const float bic = sl.Bb[i * LD + c];
+                axpy_row<N>(vcol, bic, sl.buf0 + i * LD);
+            }
+            // stage V[:,c] = g_c (P Bbar[:,c]) and T[:,c] = a_c P[:,c] (own column only) so that the next loop can
+            // run over k without indexing registers dynamically
+#pragma unroll
+            for (int k = 0; k < N / 2; ++k) {
+                float v0, v1;
+                unpack2(vcol[k], v0, v1);
+                sl.L[(2 * k) * LD + c] = g_c * v0;
+                sl.L[(2 * k + 1) * LD + c] = g_c * v1;
+                sl.Lt[(2 * k) * LD + c] = at_c * pcol[2 * k];
+                sl.Lt[(2 * k + 1) * LD + c] = at_c * pcol[2 * k + 1];
+            }
+            f32x2 s2[N / 2], y2[N / 2];
+#pragma unroll
+            for (int l = 0; l < N / 2; ++l) {
+                s2[l] = 0ull;
+                y2[l] = 0ull;
+            }
+#pragma unroll 4
+            for (int k = 0; k < N; ++k) {                     // Bbar' V[:,c] and Bbar' T[:,c]: each row of Bbar read once
+                const float vk = sl.L[k * LD + c], tk = sl.Lt[k * LD + c];
+                const f32x2 vv = pack2(vk, vk), t2 = pack2(tk, tk);
+#pragma unroll
+                for (int q = 0; q < N / 4; ++q) {
+                    const ulonglong2 b4 = *reinterpret_cast<const ulonglong2*>(sl.Bb + k * LD + 4 * q);
+                    fma2(s2[2 * q], vv, b4.x);
+                    fma2(s2[2 * q + 1], vv, b4.y);
+                    fma2(y2[2 * q], t2, b4.x);
+                    fma2(y2[2 * q + 1], t2, b4.y);
+                }
+            }
+            float sv[N], y[N], pn[N];
+            unpack_row<N>(sv, s2);
+            unpack_row<N>(y, y2);
+            {
+                float gv[N], av[N], qv[N];
+                load_row<N>(gv, sl.gb);
+                load_row<N>(av, sl.at);
+                load_row<N>(qv, sl.gq);
+#pragma unroll
+                for (int l = 0; l < N; ++l) {
+                    sv[l] *= gv[l];
+                    y[l] *= gv[l];
+                    // Pn[l][c] = q_l Qbar[l][c] q_c + a_l a_c P[l][c]
+                    pn[l] = fmaf(q_c * qv[l], qcol[l], av[l] * at_c * pcol[l]);
+                    if (l == c)
+                        sv[l] += r_c;
+                }
+            }
+            float rs_own;
+            const int bad = seg_chol<N>(sv, rs_own, c);
+            if (bad && !fail)
+                fail = s * N + bad;
+            __syncwarp();                                     // every lane is done with the rows of P in buf0 and the staged columns
+            store_row<N>(sl.L + c * LD, sv);
+#pragma unroll
+            for (int k = 0; k < N; ++k)
+                sl.Lt[k * LD + c] = sv[k];
+            sl.rinv[c] = rs_own;
+            __syncwarp();
+            float rinv[N];
+            load_row<N>(rinv, sl.rinv);
+#pragma unroll
+            for (int k = 0; k < N; ++k) {                     // Z[:,c] = L^{-1} Y[:,c]
+                const float zk = y[k] * rinv[k];
+                y[k] = zk;
+                const float* lt = sl.Lt + k * LD;
+#pragma unroll
+                for (int i4 = (k + 1) & ~3; i4 < N; i4 += 4) {
+                    const float4 l4 = *reinterpret_cast<const float4*>(lt + i4);
+                    if (i4 + 0 > k) y[i4 + 0] = fmaf(-l4.x, zk, y[i4 + 0]);
+                    if (i4 + 1 > k) y[i4 + 1] = fmaf(-l4.y, zk, y[i4 + 1]);
+                    if (i4 + 2 > k) y[i4 + 2] = fmaf(-l4.z, zk, y[i4 + 2]);
+                    if (i4 + 3 > k) y[i4 + 3] = fmaf(-l4.w, zk, y[i4 + 3]);
+                }
+            }
+#pragma unroll
+            for (int q = 0; q < N; ++q)
+                sl.buf0[q * LD + c] = y[q];                   // rows of Z
+            __syncwarp();
+            {
+                f32x2 p2[N / 2];
+                pack_row<N>(p2, pn);
+#pragma unroll 4
+                for (int q = 0; q < N; ++q)                   // Pn[:,c] -= Z' Z[:,c]
+                    axpy_row<N>(p2, -sl.buf0[q * LD + c], sl.buf0 + q * LD);
+                unpack_row<N>(pcol, p2);
+            }
+            if (s == 0 && p.u1) {                             // K[:,c] = -L^{-T} Z[:,c]; rows of K -> Lt
+#pragma unroll
+                for (int k = N - 1; k >= 0; --k) {
+                    const float xk = y[k] * rinv[k];
+                    y[k] = xk;
+                    const float* lr = sl.L + k * LD;
+#pragma unroll
+                    for (int i4 = 0; i4 < k; i4 += 4) {
+                        const float4 l4 = *reinterpret_cast<const float4*>(lr + i4);
+                        if (i4 + 0 < k) y[i4 + 0] = fmaf(-l4.x, xk, y[i4 + 0]);
+                        if (i4 + 1 < k) y[i4 + 1] = fmaf(-l4.y, xk, y[i4 + 1]);
+                        if (i4 + 2 < k) y[i4 + 2] = fmaf(-l4.z, xk, y[i4 + 2]);
+                        if (i4 + 3 < k) y[i4 + 3] = fmaf(-l4.w, xk, y[i4 + 3]);
+                    }
+                }
+#pragma unroll
+                for (int l = 0; l < N; ++l)
+                    sl.Lt[l * LD + c] = -y[l];
+            }
+            __syncwarp();                                     // rows of Z consumed
+            store_row<N>(sl.buf0 + c * LD, pcol);             // rows of P_s (row c = column c)
+        }
+        __syncwarp();
+
+        const bool store_ok = active && !fail;
+        if (p.P0 && active) {
+            float* pt = p.P0 + inst * (long long)N * N + c;
+            const float qn = quiet_nan();
+#pragma unroll
+            for (int l = 0; l < N; ++l)
+                pt[l * N] = fail ? qn : pcol[l];
+        }
+        if (p.u1) {                                           // u_1* = K_1 h_0: lane c takes row c of K_1
+            float kr[N], xv[N];
+            load_row<N>(kr, sl.Lt + c * LD);
+            load_row<N>(xv, sl.x);
+            float uc = 0.f;
+#pragma unroll
+            for (int j = 0; j < N; ++j)
+                uc = fmaf(kr[j], xv[j], uc);
+            if (active)
+                p.u1[inst * (long long)N + c] = store_ok ? uc : quiet_nan();
+        }
+        if (p.info && active && c == 0)
+            p.info[inst] = fail;
+    }
+}
+
+template <int N>
+inline size_t smem_bytes() { return sizeof(Smem<N>); }
+
+} // namespace layer
+} // namespace ttc

@@ -12,6 +12,7 @@
 #include "riccati_cta.cuh"
 #include "riccati_umma64.cuh"
 #include "riccati_warp.cuh"
+#include "ttc_layer.cuh"
 #include "scan_pair.cuh"
 
 using namespace ttc;
@@ -448,6 +449,68 @@ int ttc_lqr_solve_tv(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand*
     h->last_launches = 0;
     return solve_window(h, A, B, Q, R, x0, H, K, P, x, u, info, flags, static_cast<cudaStream_t>(cuda_stream), 0,
                         h->cfg.batch[2], tstride, (Qf && Qf->ptr) ? Qf : nullptr);
+}
+
+int ttc_lqr_solve_layer(ttc_lqr_handle* h, const ttc_layer_inputs* in, int32_t T, float* u1, float* P0,
+                        int32_t* info, void* cuda_stream)
+{
+    if (!h || !in)
+        return fail(TTC_STATUS_INVALID_ARGUMENT, "null handle or inputs");
+    const int n = h->cfg.n;
+    if (n != h->cfg.m || (n != 16 && n != 32))
+        return fail(TTC_STATUS_UNSUPPORTED, "layer solve needs n == m in {16, 32} (got n=%d, m=%d)", n, h->cfg.m);
+    if (T < 1 || T > h->cfg.max_horizon)
+        return fail(TTC_STATUS_INVALID_ARGUMENT, "T=%d outside [1, max_horizon=%d]", T, h->cfg.max_horizon);
+    if (in->r < 1 || in->r > 64)
+        return fail(TTC_STATUS_INVALID_ARGUMENT, "r=%d outside [1, 64]", in->r);
+    const void* ptrs[11] = {in->s_a, in->s_gamma_a, in->s_gamma_b, in->s_gamma_q, in->s_b, in->s_q, in->s_qf,
+                            in->r_inv, in->h0, in->B_basis, in->Q_basis};
+    for (int i = 0; i < 11; ++i) {
+        if (!ptrs[i])
+            return fail(TTC_STATUS_INVALID_ARGUMENT, "layer input %d is null", i);
+        if (reinterpret_cast<uintptr_t>(ptrs[i]) & 15u)
+            return fail(TTC_STATUS_INVALID_ARGUMENT, "layer input %d is not 16-byte aligned", i);
+    }
+    if ((reinterpret_cast<uintptr_t>(u1) | reinterpret_cast<uintptr_t>(P0)) & 15u)
+        return fail(TTC_STATUS_INVALID_ARGUMENT, "outputs must be 16-byte aligned");
+    TTC_CUDA(cudaSetDevice(h->cfg.device));
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    h->last_launches = 0;
+    int s;
+    if ((s = ensure(h->ws_E, sizeof(int) * 4))) return s;
+    int* counter = static_cast<int*>(h->ws_E.ptr);
+    TTC_CUDA(cudaMemsetAsync(counter, 0, sizeof(int), st));
+    layer::LayerParams p;
+    p.N = h->N;
+    p.T = T;
+    p.r = in->r;
+    p.s_a = in->s_a; p.s_ga = in->s_gamma_a; p.s_gb = in->s_gamma_b; p.s_gq = in->s_gamma_q;
+    p.s_b = in->s_b; p.s_q = in->s_q; p.s_qf = in->s_qf;
+    p.r_inv = in->r_inv; p.h0 = in->h0;
+    p.B_basis = in->B_basis; p.Q_basis = in->Q_basis;
+    p.u1 = u1; p.P0 = P0; p.info = info;
+    void (*kern)(layer::LayerParams, int*);
+    size_t smem;
+    long long chunks, grid;
+    if (n == 32) {
+        kern = layer::ttc_layer_kernel<32>;
+        smem = layer::smem_bytes<32>();
+        chunks = (p.N + rwarp::Shape<32>::SLOTS - 1) / rwarp::Shape<32>::SLOTS;
+        grid = (long long)h->sm_count * 3;
+    } else {
+        kern = layer::ttc_layer_kernel<16>;
+        smem = layer::smem_bytes<16>();
+        chunks = (p.N + rwarp::Shape<16>::SLOTS - 1) / rwarp::Shape<16>::SLOTS;
+        grid = (long long)h->sm_count * 4;
+    }
+    TTC_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    if (grid > chunks) grid = chunks;
+    kern<<<(unsigned)grid, rwarp::THREADS, smem, st>>>(p, counter);
+    TTC_CUDA(cudaGetLastError());
+    h->last_launches = 1;
+    h->total_launches += 1;
+    h->last_kernel = TTC_KERNEL_LAYER;
+    return TTC_OK;
 }
 
 int ttc_lqr_solve_host(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, const ttc_operand* Q,

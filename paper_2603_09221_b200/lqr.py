@@ -21,11 +21,12 @@ TTC_MATH_AUTO, TTC_MATH_FP32, TTC_MATH_TF32 = 0, 1, 2
 TTC_OUT_FIRST_ONLY = 1
 TTC_QUERY_LAST_LAUNCHES, TTC_QUERY_WORKSPACE_BYTES, TTC_QUERY_LAST_KERNEL, TTC_QUERY_TOTAL_LAUNCHES = 1, 2, 3, 4
 TTC_QUERY_DEVICE_ERROR = 5
-KERNEL_NAMES = {0: "none", 1: "riccati_cta", 2: "riccati_warp", 4: "scan", 5: "riccati_umma"}
+KERNEL_NAMES = {6: "ttc_layer", 0: "none", 1: "riccati_cta", 2: "riccati_warp", 4: "scan", 5: "riccati_umma"}
 
 EXPORTS = (
     "ttc_lqr_create", "ttc_lqr_solve", "ttc_lqr_solve_host", "ttc_lqr_destroy", "ttc_lqr_query",
     "ttc_lqr_status_string", "ttc_lqr_last_error", "ttc_lqr_solve_first_noalloc", "ttc_lqr_solve_tv",
+    "ttc_lqr_solve_layer",
 )
 TTC_NOALLOC_SCRATCH_BYTES = 4 << 20
 
@@ -33,6 +34,11 @@ TTC_NOALLOC_SCRATCH_BYTES = 4 << 20
 class ttc_operand(ctypes.Structure):
     _fields_ = [("ptr", ctypes.c_void_p), ("dtype", ctypes.c_int32), ("reserved", ctypes.c_int32),
                 ("bstride", ctypes.c_int64 * 3)]
+
+
+class ttc_layer_inputs(ctypes.Structure):
+    _fields_ = [(k, ctypes.c_void_p) for k in ("s_a", "s_gamma_a", "s_gamma_b", "s_gamma_q", "s_b", "s_q", "s_qf",
+                                               "r_inv", "h0", "B_basis", "Q_basis")] + [("r", ctypes.c_int32)]
 
 
 class ttc_lqr_config(ctypes.Structure):
@@ -71,6 +77,9 @@ def load_library():
     lib.ttc_lqr_solve_tv.restype = ctypes.c_int
     lib.ttc_lqr_solve_tv.argtypes = [ctypes.c_void_p, opp, opp, opp, opp, P(ctypes.c_int64), opp, opp, ctypes.c_int32] + \
         [ctypes.c_void_p] * 5 + [ctypes.c_uint32, ctypes.c_void_p]
+    lib.ttc_lqr_solve_layer.restype = ctypes.c_int
+    lib.ttc_lqr_solve_layer.argtypes = [ctypes.c_void_p, P(ttc_layer_inputs), ctypes.c_int32, ctypes.c_void_p,
+                                        ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
     lib.ttc_lqr_solve_host.restype = ctypes.c_int
     lib.ttc_lqr_solve_host.argtypes = [ctypes.c_void_p, opp, opp, opp, opp, opp, ctypes.c_int32] + \
         [ctypes.c_void_p] * 5 + [ctypes.c_uint32]
@@ -205,6 +214,30 @@ class LqrSolver:
         _check(load_library().ttc_lqr_solve_tv(
             self._h, ref(ops[0]), ref(ops[1]), ref(ops[2]), ref(ops[3]), tstride, ref(oqf), ref(ox), int(H),
             self._ptr(K), self._ptr(P), self._ptr(x), self._ptr(u), self._ptr(info), int(flags),
+            ctypes.c_void_p(stream.cuda_stream)))
+
+    def solve_layer(self, s_a, s_gamma_a, s_gamma_b, s_gamma_q, s_b, s_q, s_qf, r_inv, h0, B_basis, Q_basis, T,
+                    u1=None, P0=None, info=None, stream=None):
+        """Enqueue ``ttc_lqr_solve_layer``: contextualised TTC-layer evaluation.  Per-instance tensors are
+        ``[N, n]`` (``s_b, s_q, s_qf``: ``[N, r]``), the bases ``[r, n, n]``; all float32, contiguous, on the
+        solver's device.  ``u1 [N, n]``, ``P0 [N, n, n]``, ``info [N]`` (int32) are written if given."""
+        r = int(B_basis.shape[0])
+        n = self.n
+        N = self.N
+        per_n = dict(s_a=s_a, s_gamma_a=s_gamma_a, s_gamma_b=s_gamma_b, s_gamma_q=s_gamma_q, r_inv=r_inv, h0=h0)
+        per_r = dict(s_b=s_b, s_q=s_q, s_qf=s_qf)
+        inp = ttc_layer_inputs()
+        for name, t in list(per_n.items()) + list(per_r.items()) + [("B_basis", B_basis), ("Q_basis", Q_basis)]:
+            want = (N, n) if name in per_n else (N, r) if name in per_r else (r, n, n)
+            on_dev = t.device.type == "cuda" and (t.device.index or 0) == self.device
+            if tuple(t.shape) != want or t.dtype != torch.float32 or not t.is_contiguous() or not on_dev:
+                raise ValueError("%s must be a contiguous float32 tensor of shape %s on cuda:%d" % (name, want, self.device))
+            setattr(inp, name, t.data_ptr())
+        inp.r = r
+        if stream is None:
+            stream = torch.cuda.current_stream(self.device)
+        _check(load_library().ttc_lqr_solve_layer(
+            self._h, ctypes.byref(inp), int(T), self._ptr(u1), self._ptr(P0), self._ptr(info),
             ctypes.c_void_p(stream.cuda_stream)))
 
     def solve_host(self, A, B, Q, R, x0, H, K=None, P=None, x=None, u=None, info=None, flags=0):

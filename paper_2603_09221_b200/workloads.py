@@ -142,3 +142,38 @@ def make_workload(cfg_id, device="cpu", batch=None, seed=None, chunk=8192):
 def to_float64_numpy(w):
     """Widen a workload's tensors exactly to float64 numpy arrays (what the oracle reads)."""
     return {k: w[k].detach().to("cpu").to(torch.float64).numpy() for k in ("A", "B", "Q", "R", "x0")}
+
+
+# Contextualised TTC-layer workload (Contextualization paragraph): state dimension d = 16 per head, 16 heads,
+# r = 16 basis matrices shared by all heads, planning horizon T = 32; one instance per (sequence, head, token).
+# The coefficient layers' outputs are drawn directly (trained weights are not available): s_A ~ 0.3 N(0,1),
+# s_Gamma* = softplus(N(0,1) - 2) (decay rates mostly in (0.05, 0.5)), s_B ~ N(0, 1/r), s_Q, s_Qf = softplus(N(0,1)) / r,
+# r_inv = softplus(N(0,1)) + 0.5, h0 ~ N(0, I); B^(i) ~ N(0, 1/d), Q^(i) = Qc Qc' / sqrt(d) with Qc ~ N(0, 1).
+LAYER_CONFIGS = {
+    "layer16": dict(name="layer16_ctx_d16_r16_T32", batch=(4, 16, 1024), n=16, r=16, T=32, tol=1e-4),
+    "layer32": dict(name="layer32_ctx_d32_r16_T32", batch=(2, 8, 1024), n=32, r=16, T=32, tol=1e-4),
+}
+
+
+def make_layer_workload(key="layer16", device="cpu", batch=None, seed=None):
+    """Inputs of ``ttc_lqr_solve_layer`` for a contextualised-layer configuration (float32 tensors, instance-major)."""
+    c = dict(LAYER_CONFIGS[key])
+    if batch is not None:
+        c["batch"] = tuple(int(b) for b in batch)
+    N = c["batch"][0] * c["batch"][1] * c["batch"][2]
+    n, r = c["n"], c["r"]
+    seed = SEED0 + 200 if seed is None else seed
+    gen = torch.Generator(device=device)
+    gen.manual_seed(seed)
+    rn = lambda *shape: torch.randn(shape, generator=gen, device=device)
+    sp = torch.nn.functional.softplus
+    Qc = rn(r, n, n)
+    c.update(
+        s_a=(0.3 * rn(N, n)).contiguous(), s_gamma_a=sp(rn(N, n) - 2.0), s_gamma_b=sp(rn(N, n) - 2.0),
+        s_gamma_q=sp(rn(N, n) - 2.0), s_b=rn(N, r) / r ** 0.5, s_q=sp(rn(N, r)) / r, s_qf=sp(rn(N, r)) / r,
+        r_inv=sp(rn(N, n)) + 0.5, h0=rn(N, n), B_basis=rn(r, n, n) / n ** 0.5,
+        Q_basis=(Qc @ Qc.transpose(-1, -2) / n ** 0.5).contiguous(), seed=seed, N=N)
+    return c
+
+
+LAYER_KEYS = ("s_a", "s_gamma_a", "s_gamma_b", "s_gamma_q", "s_b", "s_q", "s_qf", "r_inv", "h0", "B_basis", "Q_basis")
