@@ -166,6 +166,178 @@ def run_reference(args, cid, tv_key=None):
     print(json.dumps(line))
 
 
+def layer_counts(c):
+    """Per-instance algorithmic flops and HBM bytes of the contextualised layer solve: per step P Bbar (2 n^3),
+    Bbar'V (n^3, S symmetric), Bbar'T (2 n^3), Cholesky (n^3 / 3), L^{-1}Y (n^3), Z'Z (n^3, symmetric); per
+    instance the synthesis of Bbar, Qbar, Q_T (6 r n^2).  Bytes: coefficient vectors in, u_1* and P_0 out."""
+    n, r, T = c["n"], c["r"], c["T"]
+    flops = (7.0 + 1.0 / 3.0) * n**3 * T + 6.0 * r * n * n
+    return flops, 4 * (6 * n + 3 * r), 4 * (n + n * n)
+
+
+def layer_oracle(w, idx, T):
+    from oracle import ttc_layer as lay
+    sel = lambda k: w[k][torch.as_tensor(idx, device=w[k].device)].to(torch.float64).cpu().numpy()
+    f64 = lambda k: w[k].to(torch.float64).cpu().numpy()
+    t0 = time.perf_counter()
+    ref = lay.solve_batch(sel("s_a"), sel("s_gamma_a"), sel("s_gamma_b"), sel("s_gamma_q"), sel("s_b"), sel("s_q"),
+                          sel("s_qf"), sel("r_inv"), sel("h0"), f64("B_basis"), f64("Q_basis"), T)
+    return ref, time.perf_counter() - t0
+
+
+def run_layer(args):
+    """--workload layer16 / layer32: one step = one ttc_lqr_solve_layer over the whole workload."""
+    key = args.workload
+    c = dict(workloads.LAYER_CONFIGS[key])
+    rank = int(os.environ.get("RANK", "0"))
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        S, Hd, Tk = c["batch"]
+        tok = max(1, min(Tk, args.ref_instances // (S * Hd)))
+        w = workloads.make_layer_workload(key, device="cpu", batch=(S, Hd, tok))
+        idx = np.arange(w["N"])
+        times, threads = [], 0
+        for it in range(args.warmup + args.steps):
+            ref, dt = layer_oracle(w, idx, c["T"])
+            threads = int(ref["threads"])
+            if it >= args.warmup:
+                times.append(dt)
+        ms = 1e3 * sum(times) / len(times)
+        val = w["N"] / (ms * 1e-3)
+        print(json.dumps({"impl": "reference", "metric": "lqr_instances_per_sec", "value": val, "unit": "instances/s",
+                          "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
+                          "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+                          "data": "synthetic",
+                          "config": {"workload": c["name"], "n": c["n"], "r": c["r"], "T": c["T"],
+                                     "instances_per_step": w["N"], "note": "bounded sample of the workload per step"},
+                          "cpu_baseline": {"value": val, "unit": "instances/s", "cores": threads, "kind": "oracle",
+                                           "sample": "%d instances per step (parameter synthesis in numpy + C recursion)" % w["N"]},
+                          "e2e": {"value": val, "unit": "instances/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                          "gpu_launches": 0}))
+        return
+    args.warmup = max(args.warmup, 3)
+    from paper_2603_09221_b200 import lqr
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the solver has no CPU path")
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = world > 1
+    if dist:
+        import torch.distributed as td
+        td.init_process_group("nccl", device_id=torch.device("cuda", local))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    peaks = measured_peaks()
+    if args.tokens > 0:
+        c["batch"] = (c["batch"][0], c["batch"][1], args.tokens)
+        c["name"] += "_tokens%d" % args.tokens
+    w = workloads.make_layer_workload(key, device=dev, batch=c["batch"], seed=sharding.rank_seed(200, rank))
+    n, r, T, N = c["n"], c["r"], c["T"], w["N"]
+    solver = lqr.LqrSolver(n, n, T, c["batch"], device=local)
+    u1 = torch.empty((N, n), device=dev)
+    P0 = torch.empty((N, n, n), device=dev)
+    info = torch.empty((N,), dtype=torch.int32, device=dev)
+    ins = [w[k] for k in workloads.LAYER_KEYS]
+
+    def step():
+        solver.solve_layer(*ins, T, u1=u1, P0=P0, info=info)
+
+    def barrier():
+        if dist:
+            td.barrier()
+        torch.cuda.synchronize(dev)
+
+    # the working set (a few MB) fits L2: flush it between timed steps by writing a buffer larger than L2
+    flush = torch.empty(192 * 1024 * 1024, dtype=torch.uint8, device=dev)
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    launches0 = solver.query(lqr.TTC_QUERY_TOTAL_LAUNCHES)
+    e0 = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    e1 = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    barrier()
+    for i in range(args.steps):
+        flush.fill_(i & 255)
+        e0[i].record()
+        step()
+        e1[i].record()
+    barrier()
+    launches = solver.query(lqr.TTC_QUERY_TOTAL_LAUNCHES) - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    per_step = [e0[i].elapsed_time(e1[i]) for i in range(args.steps)]
+    value, ms_per_step, _ = sharding.aggregate_throughput(N, sum(per_step) / len(per_step), device=dev)
+
+    e2e = None
+    if not args.no_e2e:
+        # end to end: coefficient vectors from pinned host memory, u_1* and P_0 back to pinned host memory
+        hin = [t.cpu().pin_memory() for t in ins]
+        din = [torch.empty_like(t) for t in ins]
+        hu, hP = torch.empty((N, n)).pin_memory(), torch.empty((N, n, n)).pin_memory()
+        h2d = sum(t.numel() * t.element_size() for t in hin)
+        d2h = hu.numel() * 4 + hP.numel() * 4
+
+        def host_step():
+            for d, h_ in zip(din, hin):
+                d.copy_(h_, non_blocking=True)
+            solver.solve_layer(*din, T, u1=u1, P0=P0, info=info)
+            hu.copy_(u1, non_blocking=True)
+            hP.copy_(P0, non_blocking=True)
+            torch.cuda.synchronize(dev)
+
+        host_step()
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(args.e2e_steps):
+            host_step()
+        barrier()
+        e2e_ms = 1e3 * (time.perf_counter() - t0) / args.e2e_steps
+        e2e_value, e2e_ms_max, _ = sharding.aggregate_throughput(N, e2e_ms, device=dev)
+        e2e = {"value": e2e_value, "unit": "instances/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+               "ms_per_step": e2e_ms_max,
+               "note": "the layer entry point takes device pointers; copies from/to pinned host memory are issued around it"}
+    if rank != 0:
+        if dist:
+            td.destroy_process_group()
+        return
+    flops_i, bin_i, bout_i = layer_counts(c)
+    kernel_ms = statistics.median(per_step)
+    fp32_peak = SM_COUNT * FP32_LANES_PER_SM * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12
+    ach = N * flops_i / (kernel_ms * 1e-3) / 1e12
+    roofline = {"bound": "alu", "achieved": ach, "peak": fp32_peak, "unit": "TFLOP/s", "frac": ach / fp32_peak,
+                "traffic": None, "kernel": "ttc_layer", "kernel_ms": kernel_ms,
+                "peak_note": "148 SMs x 128 FP32 lanes x 2 x %.0f MHz (derived)" % peaks["sm_max_mhz"],
+                "algorithmic_flops_per_launch": N * flops_i, "algorithmic_bytes_per_launch": N * (bin_i + bout_i),
+                "hbm_frac": (N * (bin_i + bout_i) / (kernel_ms * 1e-3) / 1e9) / peaks["hbm_gbs"]}
+    cpu = None
+    if not args.no_cpu_baseline and world == 1:
+        idx = np.unique(np.linspace(0, N - 1, args.cpu_sample).astype(np.int64))
+        ref, dt = layer_oracle(w, idx, T)
+        from tests import parity_util as pu
+        sel = torch.as_tensor(idx)
+        errs = {"P0": pu.block_rel_err(P0.cpu()[sel].numpy(), ref["P0"], 2),
+                "u1": pu.block_rel_err(u1.cpu()[sel].numpy(), ref["u1"], 1)}
+        assert all(v <= c["tol"] for v in errs.values()), errs
+        assert int(info.abs().max()) == 0
+        cpu = {"value": len(idx) / dt, "unit": "instances/s", "cores": int(ref["threads"]), "kind": "oracle",
+               "sample": "%d instances spread over the workload (parameter synthesis in numpy + C recursion)" % len(idx),
+               "seconds": dt, "parity_max_rel_err": errs, "speedup_gpu_over_cpu": value / (len(idx) / dt)}
+    print(json.dumps({"metric": "lqr_instances_per_sec", "value": value, "unit": "instances/s", "n_gpus": world,
+                      "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+                      "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                      "config": {"workload": c["name"], "n": n, "r": r, "T": T, "instances": N, "batch": list(c["batch"]),
+                                 "outputs": ["u1", "P0", "info"], "kernel": "ttc_layer",
+                                 "l2": "working set fits L2: a 192 MB buffer is written between timed steps"},
+                      "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches),
+                      "launches_per_step": launches / args.steps, "clocks": clocks}))
+    solver.close()
+    if dist:
+        td.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -182,6 +354,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
+    if args.workload in workloads.LAYER_CONFIGS:
+        run_layer(args)
+        return
     tv_key = args.workload if args.workload in workloads.TV_CONFIGS else None
     cid = None if tv_key else int(args.workload.replace("cfg", ""))
     if args.impl == "reference":
