@@ -19,6 +19,8 @@
 //     Pn[:,c] = q_c (q .* Qbar[:,c]) [s >= 1] + a .* T[:,c]
 //     S = L L',  Z[:,c] = L^{-1} Y[:,c],  Pn[:,c] -= Z' Z[:,c]        (P_s = Q_s + A'PA - Y'S^{-1}Y)
 // and at s = 0 the gain column K[:,c] = -L^{-T} Z[:,c] for u_1* = K h_0.
+// ttc_layer_kernel<N> is this one-column-per-lane form (used for N = 32); ttc_layer_kernel_c2<N> holds two columns
+// per lane (used for N = 16), which halves the row reads per FMA.
 #pragma once
 
 #include "riccati_warp.cuh"
@@ -272,6 +274,317 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) ttc_layer_kernel(L
             p.info[inst] = fail;
     }
 }
+
+// ---- two columns per lane ---------------------------------------------------------------------------------------
+// Same computation with N / 2 lanes per instance: lane j holds columns 2j and 2j + 1 of every matrix, so that one
+// broadcast read of a matrix row feeds the packed FMAs of two columns (the one-column kernel is bound by the
+// shared-memory pipe).  Four instances per warp when N = 16.
+template <int N>
+struct Shape2 {
+    static constexpr int LD = N + 4;
+    static constexpr int G = N / 2;                 // lanes per instance
+    static constexpr int IPW = 32 / G;
+    static constexpr int SLOTS = WARPS * IPW;
+    static constexpr int MAT = N * LD;
+};
+template <int N>
+struct Smem2 {
+    struct Slot {
+        float buf0[Shape2<N>::MAT], L[Shape2<N>::MAT], Lt[Shape2<N>::MAT], Bb[Shape2<N>::MAT];
+        float rinv[N], x[N], at[N], gb[N], gq[N];
+    } slot[Shape2<N>::SLOTS];
+    int chunk;
+};
+
+// Cholesky of an N x N SPD matrix spread over N / 2 lanes: lane j holds rows 2j (s0) and 2j + 1 (s1) (= columns, by
+// symmetry).  On return s0, s1 hold the rows of L (entries right of the diagonal are meaningless), rs0 / rs1 the
+// reciprocals of their diagonal entries.  Returns 0 or 1 + the index of the first non-positive pivot.
+template <int N>
+__device__ __forceinline__ int seg_chol2(float (&s0)[N], float (&s1)[N], float& rs0, float& rs1, int j)
+{
+    constexpr int G = N / 2;
+    int bad = 0;
+    rs0 = rs1 = 1.f;
+#pragma unroll
+    for (int p = 0; p < N; ++p) {
+        const float a0 = s0[p], a1 = s1[p];
+        float d = __shfl_sync(0xffffffffu, (p & 1) ? a1 : a0, p >> 1, G);
+        if (!(d > 0.f)) {
+            if (!bad)
+                bad = p + 1;
+            d = 1.f;
+        }
+        const float rinv = __frcp_rn(d);
+        const float f0 = a0 * rinv, f1 = a1 * rinv;
+#pragma unroll
+        for (int cc = p + 1; cc < N; ++cc) {
+            const float lc = __shfl_sync(0xffffffffu, (cc & 1) ? a1 : a0, cc >> 1, G);
+            s0[cc] = fmaf(-f0, lc, s0[cc]);
+            s1[cc] = fmaf(-f1, lc, s1[cc]);
+        }
+        const float rs = rsqrtf(d);
+        s0[p] = a0 * rs;
+        s1[p] = a1 * rs;
+        if (2 * j == p)
+            rs0 = rs;
+        if (2 * j + 1 == p)
+            rs1 = rs;
+    }
+    return bad;
+}
+
+// acc0[l] += w0 * row[l], acc1[l] += w1 * row[l]: one pass over the row for two columns
+template <int N>
+__device__ __forceinline__ void axpy_row2(rwarp::f32x2 (&acc0)[N / 2], rwarp::f32x2 (&acc1)[N / 2], float w0, float w1, const float* row)
+{
+    const rwarp::f32x2 ww0 = rwarp::pack2(w0, w0), ww1 = rwarp::pack2(w1, w1);
+#pragma unroll
+    for (int q = 0; q < N / 4; ++q) {
+        const ulonglong2 t = *reinterpret_cast<const ulonglong2*>(row + 4 * q);
+        rwarp::fma2(acc0[2 * q], ww0, t.x);
+        rwarp::fma2(acc0[2 * q + 1], ww0, t.y);
+        rwarp::fma2(acc1[2 * q], ww1, t.x);
+        rwarp::fma2(acc1[2 * q + 1], ww1, t.y);
+    }
+}
+
+template <int N>
+__global__ void __launch_bounds__(THREADS, 2) ttc_layer_kernel_c2(LayerParams p, int* chunk_counter)
+{
+    using S = Shape2<N>;
+    using namespace rwarp;
+    constexpr int LD = S::LD, G = S::G;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    Smem2<N>& sm = *reinterpret_cast<Smem2<N>*>(smem_raw);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int sub = lane / G, j = lane % G;
+    const int c0 = 2 * j, c1 = 2 * j + 1;
+    typename Smem2<N>::Slot& sl = sm.slot[warp * S::IPW + sub];
+    const int T = p.T, r = p.r;
+    const long long nchunks = (p.N + S::SLOTS - 1) / S::SLOTS;
+
+    for (;;) {
+        __syncthreads();
+        if (tid == 0)
+            sm.chunk = atomicAdd(chunk_counter, 1);
+        __syncthreads();
+        const long long chunk = sm.chunk;
+        if (chunk >= nchunks)
+            break;
+        const long long inst_raw = chunk * S::SLOTS + warp * S::IPW + sub;
+        const bool active = inst_raw < p.N;                   // idle segments shadow the chunk's first instance
+        const long long inst = active ? inst_raw : chunk * S::SLOTS;
+
+        // ---- synthesis of Bbar (rows -> shared), Qbar[:, c0..c1] (registers) and P_T = Q_T[:, c0..c1]
+        float q0[N], q1[N], p0[N], p1[N];
+        {
+            float b0[N], b1[N];
+#pragma unroll
+            for (int l = 0; l < N; ++l)
+                b0[l] = b1[l] = q0[l] = q1[l] = p0[l] = p1[l] = 0.f;
+            const float* sb = p.s_b + inst * r;
+            const float* sq = p.s_q + inst * r;
+            const float* sf = p.s_qf + inst * r;
+#pragma unroll 1
+            for (int i = 0; i < r; ++i) {
+                const float wb = __ldg(sb + i), wq = __ldg(sq + i), wf = __ldg(sf + i);
+                const float2* Bi = reinterpret_cast<const float2*>(p.B_basis + (long long)i * N * N + c0);
+                const float2* Qi = reinterpret_cast<const float2*>(p.Q_basis + (long long)i * N * N + c0);
+#pragma unroll
+                for (int l = 0; l < N; ++l) {
+                    const float2 bv = __ldg(Bi + l * (N / 2)), qv = __ldg(Qi + l * (N / 2));
+                    b0[l] = fmaf(wb, bv.x, b0[l]);
+                    b1[l] = fmaf(wb, bv.y, b1[l]);
+                    q0[l] = fmaf(wq, qv.x, q0[l]);
+                    q1[l] = fmaf(wq, qv.y, q1[l]);
+                    p0[l] = fmaf(wf, qv.x, p0[l]);
+                    p1[l] = fmaf(wf, qv.y, p1[l]);
+                }
+            }
+#pragma unroll
+            for (int l = 0; l < N; ++l)
+                *reinterpret_cast<float2*>(sl.Bb + l * LD + c0) = make_float2(b0[l], b1[l]);
+        }
+        const float2 a_c = __ldg(reinterpret_cast<const float2*>(p.s_a + inst * N + c0));
+        const float2 ga_c = __ldg(reinterpret_cast<const float2*>(p.s_ga + inst * N + c0));
+        const float2 gb_c = __ldg(reinterpret_cast<const float2*>(p.s_gb + inst * N + c0));
+        const float2 gq_c = __ldg(reinterpret_cast<const float2*>(p.s_gq + inst * N + c0));
+        const float2 ri_c = __ldg(reinterpret_cast<const float2*>(p.r_inv + inst * N + c0));
+        const float r_0 = 1.f / ri_c.x, r_1 = 1.f / ri_c.y;
+        *reinterpret_cast<float2*>(sl.x + c0) = __ldg(reinterpret_cast<const float2*>(p.h0 + inst * N + c0));
+        store_row<N>(sl.buf0 + c0 * LD, p0);                  // rows of P_T (row c = column c)
+        store_row<N>(sl.buf0 + c1 * LD, p1);
+        int fail = 0;
+
+#pragma unroll 1
+        for (int s = T - 1; s >= 0; --s) {
+            const float tt = (float)(s + 1);
+            const float at0 = fmaf(__expf(-tt * ga_c.x), a_c.x, 1.f), at1 = fmaf(__expf(-tt * ga_c.y), a_c.y, 1.f);
+            const float g0 = __expf(-tt * gb_c.x), g1 = __expf(-tt * gb_c.y);
+            const float qq0 = (s >= 1) ? __expf(-(float)s * gq_c.x) : 0.f;       // Q_0 = 0
+            const float qq1 = (s >= 1) ? __expf(-(float)s * gq_c.y) : 0.f;
+            *reinterpret_cast<float2*>(sl.at + c0) = make_float2(at0, at1);
+            *reinterpret_cast<float2*>(sl.gb + c0) = make_float2(g0, g1);
+            *reinterpret_cast<float2*>(sl.gq + c0) = make_float2(qq0, qq1);
+            __syncwarp();                                     // rows of P and the step's diagonals are in place
+            float v0[N], v1[N];
+            {
+                f32x2 a0[N / 2], a1[N / 2];
+#pragma unroll
+                for (int k = 0; k < N / 2; ++k)
+                    a0[k] = a1[k] = 0ull;
+#pragma unroll 4
+                for (int i = 0; i < N; ++i) {                 // P Bbar[:, c0..c1]
+                    const float2 b = *reinterpret_cast<const float2*>(sl.Bb + i * LD + c0);
+                    axpy_row2<N>(a0, a1, b.x, b.y, sl.buf0 + i * LD);
+                }
+                unpack_row<N>(v0, a0);
+                unpack_row<N>(v1, a1);
+            }
+            f32x2 s20[N / 2], s21[N / 2], y20[N / 2], y21[N / 2];
+#pragma unroll
+            for (int l = 0; l < N / 2; ++l)
+                s20[l] = s21[l] = y20[l] = y21[l] = 0ull;
+            // fully unrolled: V[k][c] = g_c v[k] and T[k][c] = a_c P[k][c] come straight from registers
+#pragma unroll
+            for (int k = 0; k < N; ++k) {                     // Bbar' V and Bbar' T for both columns: each row of Bbar read once
+                const f32x2 w0 = pack2(g0 * v0[k], g0 * v0[k]), w1 = pack2(g1 * v1[k], g1 * v1[k]);
+                const f32x2 u0 = pack2(at0 * p0[k], at0 * p0[k]), u1 = pack2(at1 * p1[k], at1 * p1[k]);
+#pragma unroll
+                for (int q = 0; q < N / 4; ++q) {
+                    const ulonglong2 b4 = *reinterpret_cast<const ulonglong2*>(sl.Bb + k * LD + 4 * q);
+                    fma2(s20[2 * q], w0, b4.x);
+                    fma2(s20[2 * q + 1], w0, b4.y);
+                    fma2(s21[2 * q], w1, b4.x);
+                    fma2(s21[2 * q + 1], w1, b4.y);
+                    fma2(y20[2 * q], u0, b4.x);
+                    fma2(y20[2 * q + 1], u0, b4.y);
+                    fma2(y21[2 * q], u1, b4.x);
+                    fma2(y21[2 * q + 1], u1, b4.y);
+                }
+            }
+            float s0[N], s1[N], y0[N], y1[N], pn0[N], pn1[N];
+            unpack_row<N>(s0, s20);
+            unpack_row<N>(s1, s21);
+            unpack_row<N>(y0, y20);
+            unpack_row<N>(y1, y21);
+            {
+                float gv[N], av[N], qv[N];
+                load_row<N>(gv, sl.gb);
+                load_row<N>(av, sl.at);
+                load_row<N>(qv, sl.gq);
+#pragma unroll
+                for (int l = 0; l < N; ++l) {
+                    s0[l] *= gv[l];
+                    s1[l] *= gv[l];
+                    y0[l] *= gv[l];
+                    y1[l] *= gv[l];
+                    pn0[l] = fmaf(qq0 * qv[l], q0[l], av[l] * at0 * p0[l]);
+                    pn1[l] = fmaf(qq1 * qv[l], q1[l], av[l] * at1 * p1[l]);
+                    if (l == c0)
+                        s0[l] += r_0;
+                    if (l == c1)
+                        s1[l] += r_1;
+                }
+            }
+            float rs0, rs1;
+            const int bad = seg_chol2<N>(s0, s1, rs0, rs1, j);
+            if (bad && !fail)
+                fail = s * N + bad;
+            __syncwarp();                                     // every lane is done with the rows of P in buf0
+            store_row<N>(sl.L + c0 * LD, s0);
+            store_row<N>(sl.L + c1 * LD, s1);
+#pragma unroll
+            for (int k = 0; k < N; ++k)
+                *reinterpret_cast<float2*>(sl.Lt + k * LD + c0) = make_float2(s0[k], s1[k]);
+            *reinterpret_cast<float2*>(sl.rinv + c0) = make_float2(rs0, rs1);
+            __syncwarp();
+            float rinv[N];
+            load_row<N>(rinv, sl.rinv);
+#pragma unroll
+            for (int k = 0; k < N; ++k) {                     // Z[:, c] = L^{-1} Y[:, c] for both columns
+                const float z0 = y0[k] * rinv[k], z1 = y1[k] * rinv[k];
+                y0[k] = z0;
+                y1[k] = z1;
+                const float* lt = sl.Lt + k * LD;
+#pragma unroll
+                for (int i4 = (k + 1) & ~3; i4 < N; i4 += 4) {
+                    const float4 l4 = *reinterpret_cast<const float4*>(lt + i4);
+                    if (i4 + 0 > k) { y0[i4 + 0] = fmaf(-l4.x, z0, y0[i4 + 0]); y1[i4 + 0] = fmaf(-l4.x, z1, y1[i4 + 0]); }
+                    if (i4 + 1 > k) { y0[i4 + 1] = fmaf(-l4.y, z0, y0[i4 + 1]); y1[i4 + 1] = fmaf(-l4.y, z1, y1[i4 + 1]); }
+                    if (i4 + 2 > k) { y0[i4 + 2] = fmaf(-l4.z, z0, y0[i4 + 2]); y1[i4 + 2] = fmaf(-l4.z, z1, y1[i4 + 2]); }
+                    if (i4 + 3 > k) { y0[i4 + 3] = fmaf(-l4.w, z0, y0[i4 + 3]); y1[i4 + 3] = fmaf(-l4.w, z1, y1[i4 + 3]); }
+                }
+            }
+#pragma unroll
+            for (int q = 0; q < N; ++q)
+                *reinterpret_cast<float2*>(sl.buf0 + q * LD + c0) = make_float2(y0[q], y1[q]);     // rows of Z
+            __syncwarp();
+            {
+                f32x2 p20[N / 2], p21[N / 2];
+                pack_row<N>(p20, pn0);
+                pack_row<N>(p21, pn1);
+#pragma unroll
+                for (int q = 0; q < N; ++q)                   // Pn[:, c] -= Z' Z[:, c]
+                    axpy_row2<N>(p20, p21, -y0[q], -y1[q], sl.buf0 + q * LD);
+                unpack_row<N>(p0, p20);
+                unpack_row<N>(p1, p21);
+            }
+            if (s == 0 && p.u1) {                             // K[:, c] = -L^{-T} Z[:, c]; rows of K -> Lt
+#pragma unroll
+                for (int k = N - 1; k >= 0; --k) {
+                    const float x0 = y0[k] * rinv[k], x1 = y1[k] * rinv[k];
+                    y0[k] = x0;
+                    y1[k] = x1;
+                    const float* lr = sl.L + k * LD;
+#pragma unroll
+                    for (int i4 = 0; i4 < k; i4 += 4) {
+                        const float4 l4 = *reinterpret_cast<const float4*>(lr + i4);
+                        if (i4 + 0 < k) { y0[i4 + 0] = fmaf(-l4.x, x0, y0[i4 + 0]); y1[i4 + 0] = fmaf(-l4.x, x1, y1[i4 + 0]); }
+                        if (i4 + 1 < k) { y0[i4 + 1] = fmaf(-l4.y, x0, y0[i4 + 1]); y1[i4 + 1] = fmaf(-l4.y, x1, y1[i4 + 1]); }
+                        if (i4 + 2 < k) { y0[i4 + 2] = fmaf(-l4.z, x0, y0[i4 + 2]); y1[i4 + 2] = fmaf(-l4.z, x1, y1[i4 + 2]); }
+                        if (i4 + 3 < k) { y0[i4 + 3] = fmaf(-l4.w, x0, y0[i4 + 3]); y1[i4 + 3] = fmaf(-l4.w, x1, y1[i4 + 3]); }
+                    }
+                }
+#pragma unroll
+                for (int l = 0; l < N; ++l)
+                    *reinterpret_cast<float2*>(sl.Lt + l * LD + c0) = make_float2(-y0[l], -y1[l]);
+            }
+            __syncwarp();                                     // rows of Z consumed
+            store_row<N>(sl.buf0 + c0 * LD, p0);              // rows of P_s (row c = column c)
+            store_row<N>(sl.buf0 + c1 * LD, p1);
+        }
+        __syncwarp();
+
+        const bool store_ok = active && !fail;
+        const float qn = quiet_nan();
+        if (p.P0 && active) {
+            float* pt = p.P0 + inst * (long long)N * N + c0;
+#pragma unroll
+            for (int l = 0; l < N; ++l)
+                *reinterpret_cast<float2*>(pt + l * N) = fail ? make_float2(qn, qn) : make_float2(p0[l], p1[l]);
+        }
+        if (p.u1) {                                           // u_1* = K_1 h_0: lane j takes rows c0, c1 of K_1
+            float k0[N], k1[N], xv[N];
+            load_row<N>(k0, sl.Lt + c0 * LD);
+            load_row<N>(k1, sl.Lt + c1 * LD);
+            load_row<N>(xv, sl.x);
+            float u0 = 0.f, u1v = 0.f;
+#pragma unroll
+            for (int l = 0; l < N; ++l) {
+                u0 = fmaf(k0[l], xv[l], u0);
+                u1v = fmaf(k1[l], xv[l], u1v);
+            }
+            if (active)
+                *reinterpret_cast<float2*>(p.u1 + inst * (long long)N + c0) = store_ok ? make_float2(u0, u1v) : make_float2(qn, qn);
+        }
+        if (p.info && active && j == 0)
+            p.info[inst] = fail;
+    }
+}
+
+template <int N>
+inline size_t smem_bytes_c2() { return sizeof(Smem2<N>); }
 
 template <int N>
 inline size_t smem_bytes() { return sizeof(Smem<N>); }

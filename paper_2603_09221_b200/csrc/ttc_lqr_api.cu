@@ -498,10 +498,10 @@ int ttc_lqr_solve_layer(ttc_lqr_handle* h, const ttc_layer_inputs* in, int32_t T
         chunks = (p.N + rwarp::Shape<32>::SLOTS - 1) / rwarp::Shape<32>::SLOTS;
         grid = (long long)h->sm_count * 3;
     } else {
-        kern = layer::ttc_layer_kernel<16>;
-        smem = layer::smem_bytes<16>();
-        chunks = (p.N + rwarp::Shape<16>::SLOTS - 1) / rwarp::Shape<16>::SLOTS;
-        grid = (long long)h->sm_count * 4;
+        kern = layer::ttc_layer_kernel_c2<16>;
+        smem = layer::smem_bytes_c2<16>();
+        chunks = (p.N + layer::Shape2<16>::SLOTS - 1) / layer::Shape2<16>::SLOTS;
+        grid = (long long)h->sm_count * 2;
     }
     TTC_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     if (grid > chunks) grid = chunks;
