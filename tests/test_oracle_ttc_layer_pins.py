@@ -159,3 +159,26 @@ def test_batch_matches_single():
         one = lay.solve(**c, B_basis=Bb, Q_basis=Qb, T=T)
         np.testing.assert_array_equal(out["u1"][i], one["u1"])
         np.testing.assert_array_equal(out["P0"][i], one["P0"])
+
+
+def test_first_control_matches_the_symplectic_iteration_theorem():
+    """Thm 3.3: u_1* = -R_1^{-1} B_1' A_1^{-T} Y1^{-1} Y2 h_0 with [Y1 Y2] = [I Q_T] Sigma_T ... Sigma_1, evaluated by
+    the oracle's restatement of Alg. 3 (a different algorithm from the backward recursion the layer oracle uses).
+    Short horizons only: the product is a shooting method and loses accuracy as T grows (printed, not asserted)."""
+    from oracle import symplectic as sym
+    rng = np.random.default_rng(21)
+    d, r = 6, 4
+    worst = {}
+    for T in (1, 3, 6, 24):
+        errs = []
+        for _ in range(8):
+            c, Bb, Qb = draw(rng, d, r)
+            A, B, Q, R = lay.synthesize(*(c[k] for k in ("s_a", "s_ga", "s_gb", "s_gq", "s_b", "s_q", "s_qf", "r_inv")), Bb, Qb, T)
+            Y1, Y2, lam0, u1 = sym.reverse_symplectic(A[1:], B[1:], Q, R[1:], c["h0"])
+            P0 = np.linalg.solve(Y1, Y2)
+            out = lay.solve(**c, B_basis=Bb, Q_basis=Qb, T=T)
+            errs.append(max(np.abs(u1 - out["u1"]).max() / np.abs(out["u1"]).max(),
+                            np.abs(P0 - out["P0"]).max() / np.abs(out["P0"]).max()))
+        worst[T] = max(errs)
+    print("symplectic iteration vs backward recursion, max relative difference by horizon:", worst)
+    assert worst[1] < 1e-10 and worst[3] < 1e-9 and worst[6] < 1e-7
