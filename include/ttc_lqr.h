@@ -208,6 +208,17 @@ int ttc_lqr_solve_layer(ttc_lqr_handle* h, const ttc_layer_inputs* in, int32_t T
                         float* u1, float* P0, int32_t* info, void* cuda_stream);
 
 /*
+ * ttc_lqr_solve_layer with HOST buffers: every pointer of `in` and u1 / P0 / info are host memory
+ * (pinned memory lets the copies run at full speed; pageable memory works).  The call copies the
+ * inputs to a device staging buffer owned by the handle, runs the same kernel on an internal
+ * stream, copies the requested outputs back and returns after everything has completed
+ * (synchronous).  No alignment requirement on host pointers.  Results are identical to
+ * ttc_lqr_solve_layer.
+ */
+int ttc_lqr_solve_layer_host(ttc_lqr_handle* h, const ttc_layer_inputs* in, int32_t T,
+                             float* u1, float* P0, int32_t* info);
+
+/*
  * Same computation with HOST buffers (same problem statement as ttc_lqr_solve): operand
  * pointers and all outputs are host memory (pinned memory lets the copies run asynchronously;
  * pageable memory works but serialises them).  The call copies the inputs to device staging

@@ -52,6 +52,7 @@ struct ttc_lqr_handle {
     int sm_count;
     DevBuf ws_K, ws_P, ws_E;       // scratch used by kernels
     DevBuf st_in[5], st_out[5];    // device staging of ttc_lqr_solve_host
+    DevBuf st_layer;               // device staging of ttc_lqr_solve_layer_host
     cudaStream_t host_stream;      // compute stream of ttc_lqr_solve_host
     cudaStream_t in_stream, out_stream;   // its copy streams (host -> device, device -> host)
     cudaEvent_t ev_in[kMaxSlices], ev_done[kMaxSlices];
@@ -92,7 +93,7 @@ void release(DevBuf& b)
 
 size_t workspace_bytes(const ttc_lqr_handle* h)
 {
-    size_t s = h->ws_K.bytes + h->ws_P.bytes + h->ws_E.bytes;
+    size_t s = h->ws_K.bytes + h->ws_P.bytes + h->ws_E.bytes + h->st_layer.bytes;
     for (int i = 0; i < 5; ++i)
         s += h->st_in[i].bytes + h->st_out[i].bytes;
     return s;
@@ -246,6 +247,7 @@ int ttc_lqr_destroy(ttc_lqr_handle* h)
         release(h->st_in[i]);
         release(h->st_out[i]);
     }
+    release(h->st_layer);
     if (h->host_pipeline_ready) {
         for (int i = 0; i < kMaxSlices; ++i) {
             cudaEventDestroy(h->ev_in[i]);
@@ -430,6 +432,22 @@ int ttc_lqr_solve(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B,
                         h->cfg.batch[2]);
 }
 
+// streams and events of the host-buffer entry points (created on first use)
+static int ensure_host_pipeline(ttc_lqr_handle* h)
+{
+    if (h->host_pipeline_ready)
+        return TTC_OK;
+    TTC_CUDA(cudaStreamCreateWithFlags(&h->host_stream, cudaStreamNonBlocking));
+    TTC_CUDA(cudaStreamCreateWithFlags(&h->in_stream, cudaStreamNonBlocking));
+    TTC_CUDA(cudaStreamCreateWithFlags(&h->out_stream, cudaStreamNonBlocking));
+    for (int i = 0; i < kMaxSlices; ++i) {
+        TTC_CUDA(cudaEventCreateWithFlags(&h->ev_in[i], cudaEventDisableTiming));
+        TTC_CUDA(cudaEventCreateWithFlags(&h->ev_done[i], cudaEventDisableTiming));
+    }
+    h->host_pipeline_ready = true;
+    return TTC_OK;
+}
+
 int ttc_lqr_solve_tv(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, const ttc_operand* Q,
                      const ttc_operand* R, const int64_t tstride[4], const ttc_operand* Qf, const ttc_operand* x0,
                      int32_t H, float* K, float* P, float* x, float* u, int32_t* info, uint32_t flags,
@@ -451,8 +469,8 @@ int ttc_lqr_solve_tv(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand*
                         h->cfg.batch[2], tstride, (Qf && Qf->ptr) ? Qf : nullptr);
 }
 
-int ttc_lqr_solve_layer(ttc_lqr_handle* h, const ttc_layer_inputs* in, int32_t T, float* u1, float* P0,
-                        int32_t* info, void* cuda_stream)
+static int check_layer_call(ttc_lqr_handle* h, const ttc_layer_inputs* in, int32_t T, bool device_pointers,
+                            const float* u1, const float* P0)
 {
     if (!h || !in)
         return fail(TTC_STATUS_INVALID_ARGUMENT, "null handle or inputs");
@@ -468,14 +486,19 @@ int ttc_lqr_solve_layer(ttc_lqr_handle* h, const ttc_layer_inputs* in, int32_t T
     for (int i = 0; i < 11; ++i) {
         if (!ptrs[i])
             return fail(TTC_STATUS_INVALID_ARGUMENT, "layer input %d is null", i);
-        if (reinterpret_cast<uintptr_t>(ptrs[i]) & 15u)
+        if (device_pointers && (reinterpret_cast<uintptr_t>(ptrs[i]) & 15u))
             return fail(TTC_STATUS_INVALID_ARGUMENT, "layer input %d is not 16-byte aligned", i);
     }
-    if ((reinterpret_cast<uintptr_t>(u1) | reinterpret_cast<uintptr_t>(P0)) & 15u)
+    if (device_pointers && ((reinterpret_cast<uintptr_t>(u1) | reinterpret_cast<uintptr_t>(P0)) & 15u))
         return fail(TTC_STATUS_INVALID_ARGUMENT, "outputs must be 16-byte aligned");
-    TTC_CUDA(cudaSetDevice(h->cfg.device));
-    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    h->last_launches = 0;
+    return TTC_OK;
+}
+
+// all pointers are device memory here
+static int launch_layer(ttc_lqr_handle* h, const ttc_layer_inputs* in, int32_t T, float* u1, float* P0, int32_t* info,
+                        cudaStream_t st)
+{
+    const int n = h->cfg.n;
     int s;
     if ((s = ensure(h->ws_E, sizeof(int) * 4))) return s;
     int* counter = static_cast<int*>(h->ws_E.ptr);
@@ -507,9 +530,72 @@ int ttc_lqr_solve_layer(ttc_lqr_handle* h, const ttc_layer_inputs* in, int32_t T
     if (grid > chunks) grid = chunks;
     kern<<<(unsigned)grid, rwarp::THREADS, smem, st>>>(p, counter);
     TTC_CUDA(cudaGetLastError());
-    h->last_launches = 1;
+    h->last_launches += 1;
     h->total_launches += 1;
     h->last_kernel = TTC_KERNEL_LAYER;
+    return TTC_OK;
+}
+
+int ttc_lqr_solve_layer(ttc_lqr_handle* h, const ttc_layer_inputs* in, int32_t T, float* u1, float* P0,
+                        int32_t* info, void* cuda_stream)
+{
+    int s = check_layer_call(h, in, T, true, u1, P0);
+    if (s)
+        return s;
+    TTC_CUDA(cudaSetDevice(h->cfg.device));
+    h->last_launches = 0;
+    return launch_layer(h, in, T, u1, P0, info, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int ttc_lqr_solve_layer_host(ttc_lqr_handle* h, const ttc_layer_inputs* in, int32_t T, float* u1, float* P0,
+                             int32_t* info)
+{
+    int s = check_layer_call(h, in, T, false, nullptr, nullptr);
+    if (s)
+        return s;
+    TTC_CUDA(cudaSetDevice(h->cfg.device));
+    if ((s = ensure_host_pipeline(h)))
+        return s;
+    h->last_launches = 0;
+    const size_t N = (size_t)h->N, n = (size_t)h->cfg.n, r = (size_t)in->r;
+    const void* src[11] = {in->s_a, in->s_gamma_a, in->s_gamma_b, in->s_gamma_q, in->s_b, in->s_q, in->s_qf,
+                           in->r_inv, in->h0, in->B_basis, in->Q_basis};
+    const size_t in_bytes[11] = {4 * N * n, 4 * N * n, 4 * N * n, 4 * N * n, 4 * N * r, 4 * N * r, 4 * N * r,
+                                 4 * N * n, 4 * N * n, 4 * r * n * n, 4 * r * n * n};
+    void* host_out[3] = {u1, P0, info};
+    const size_t out_bytes[3] = {4 * N * n, 4 * N * n * n, 4 * N};
+    auto pad = [](size_t b) { return (b + 255) & ~(size_t)255; };
+    size_t total = 0;
+    for (int i = 0; i < 11; ++i) total += pad(in_bytes[i]);
+    for (int i = 0; i < 3; ++i) total += host_out[i] ? pad(out_bytes[i]) : 0;
+    if ((s = ensure(h->st_layer, total)))
+        return s;
+    cudaStream_t st = h->host_stream;
+    unsigned char* base = static_cast<unsigned char*>(h->st_layer.ptr);
+    const float* dptr[11];
+    size_t off = 0;
+    for (int i = 0; i < 11; ++i) {
+        dptr[i] = reinterpret_cast<const float*>(base + off);
+        TTC_CUDA(cudaMemcpyAsync(base + off, src[i], in_bytes[i], cudaMemcpyHostToDevice, st));
+        off += pad(in_bytes[i]);
+    }
+    void* dev_out[3] = {nullptr, nullptr, nullptr};
+    for (int i = 0; i < 3; ++i)
+        if (host_out[i]) {
+            dev_out[i] = base + off;
+            off += pad(out_bytes[i]);
+        }
+    ttc_layer_inputs din = *in;
+    din.s_a = dptr[0]; din.s_gamma_a = dptr[1]; din.s_gamma_b = dptr[2]; din.s_gamma_q = dptr[3];
+    din.s_b = dptr[4]; din.s_q = dptr[5]; din.s_qf = dptr[6]; din.r_inv = dptr[7]; din.h0 = dptr[8];
+    din.B_basis = dptr[9]; din.Q_basis = dptr[10];
+    if ((s = launch_layer(h, &din, T, static_cast<float*>(dev_out[0]), static_cast<float*>(dev_out[1]),
+                          static_cast<int32_t*>(dev_out[2]), st)))
+        return s;
+    for (int i = 0; i < 3; ++i)
+        if (host_out[i])
+            TTC_CUDA(cudaMemcpyAsync(host_out[i], dev_out[i], out_bytes[i], cudaMemcpyDeviceToHost, st));
+    TTC_CUDA(cudaStreamSynchronize(st));
     return TTC_OK;
 }
 
@@ -525,16 +611,7 @@ int ttc_lqr_solve_host(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operan
     if (flags & ~TTC_OUT_FIRST_ONLY)
         return fail(TTC_STATUS_INVALID_ARGUMENT, "unknown flag bits 0x%x", flags);
     TTC_CUDA(cudaSetDevice(h->cfg.device));
-    if (!h->host_pipeline_ready) {
-        TTC_CUDA(cudaStreamCreateWithFlags(&h->host_stream, cudaStreamNonBlocking));
-        TTC_CUDA(cudaStreamCreateWithFlags(&h->in_stream, cudaStreamNonBlocking));
-        TTC_CUDA(cudaStreamCreateWithFlags(&h->out_stream, cudaStreamNonBlocking));
-        for (int i = 0; i < kMaxSlices; ++i) {
-            TTC_CUDA(cudaEventCreateWithFlags(&h->ev_in[i], cudaEventDisableTiming));
-            TTC_CUDA(cudaEventCreateWithFlags(&h->ev_done[i], cudaEventDisableTiming));
-        }
-        h->host_pipeline_ready = true;
-    }
+    { int sp = ensure_host_pipeline(h); if (sp) return sp; }
     const int n = h->cfg.n, m = h->cfg.m;
     const long long N = h->N, b0 = h->cfg.batch[0], b1 = h->cfg.batch[1], b2 = h->cfg.batch[2];
     const bool first = (flags & TTC_OUT_FIRST_ONLY) != 0;

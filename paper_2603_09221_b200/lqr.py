@@ -26,7 +26,7 @@ KERNEL_NAMES = {6: "ttc_layer", 0: "none", 1: "riccati_cta", 2: "riccati_warp", 
 EXPORTS = (
     "ttc_lqr_create", "ttc_lqr_solve", "ttc_lqr_solve_host", "ttc_lqr_destroy", "ttc_lqr_query",
     "ttc_lqr_status_string", "ttc_lqr_last_error", "ttc_lqr_solve_first_noalloc", "ttc_lqr_solve_tv",
-    "ttc_lqr_solve_layer",
+    "ttc_lqr_solve_layer", "ttc_lqr_solve_layer_host",
 )
 TTC_NOALLOC_SCRATCH_BYTES = 4 << 20
 
@@ -80,6 +80,9 @@ def load_library():
     lib.ttc_lqr_solve_layer.restype = ctypes.c_int
     lib.ttc_lqr_solve_layer.argtypes = [ctypes.c_void_p, P(ttc_layer_inputs), ctypes.c_int32, ctypes.c_void_p,
                                         ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+    lib.ttc_lqr_solve_layer_host.restype = ctypes.c_int
+    lib.ttc_lqr_solve_layer_host.argtypes = [ctypes.c_void_p, P(ttc_layer_inputs), ctypes.c_int32, ctypes.c_void_p,
+                                             ctypes.c_void_p, ctypes.c_void_p]
     lib.ttc_lqr_solve_host.restype = ctypes.c_int
     lib.ttc_lqr_solve_host.argtypes = [ctypes.c_void_p, opp, opp, opp, opp, opp, ctypes.c_int32] + \
         [ctypes.c_void_p] * 5 + [ctypes.c_uint32]
@@ -216,29 +219,44 @@ class LqrSolver:
             self._ptr(K), self._ptr(P), self._ptr(x), self._ptr(u), self._ptr(info), int(flags),
             ctypes.c_void_p(stream.cuda_stream)))
 
-    def solve_layer(self, s_a, s_gamma_a, s_gamma_b, s_gamma_q, s_b, s_q, s_qf, r_inv, h0, B_basis, Q_basis, T,
-                    u1=None, P0=None, info=None, stream=None):
-        """Enqueue ``ttc_lqr_solve_layer``: contextualised TTC-layer evaluation.  Per-instance tensors are
-        ``[N, n]`` (``s_b, s_q, s_qf``: ``[N, r]``), the bases ``[r, n, n]``; all float32, contiguous, on the
-        solver's device.  ``u1 [N, n]``, ``P0 [N, n, n]``, ``info [N]`` (int32) are written if given."""
+    def _layer_inputs(self, tensors, host):
+        s_a, s_gamma_a, s_gamma_b, s_gamma_q, s_b, s_q, s_qf, r_inv, h0, B_basis, Q_basis = tensors
         r = int(B_basis.shape[0])
-        n = self.n
-        N = self.N
+        n, N = self.n, self.N
         per_n = dict(s_a=s_a, s_gamma_a=s_gamma_a, s_gamma_b=s_gamma_b, s_gamma_q=s_gamma_q, r_inv=r_inv, h0=h0)
         per_r = dict(s_b=s_b, s_q=s_q, s_qf=s_qf)
         inp = ttc_layer_inputs()
         for name, t in list(per_n.items()) + list(per_r.items()) + [("B_basis", B_basis), ("Q_basis", Q_basis)]:
             want = (N, n) if name in per_n else (N, r) if name in per_r else (r, n, n)
-            on_dev = t.device.type == "cuda" and (t.device.index or 0) == self.device
-            if tuple(t.shape) != want or t.dtype != torch.float32 or not t.is_contiguous() or not on_dev:
-                raise ValueError("%s must be a contiguous float32 tensor of shape %s on cuda:%d" % (name, want, self.device))
+            if host:
+                placed = t.device.type == "cpu"
+            else:
+                placed = t.device.type == "cuda" and (t.device.index or 0) == self.device
+            if tuple(t.shape) != want or t.dtype != torch.float32 or not t.is_contiguous() or not placed:
+                raise ValueError("%s must be a contiguous float32 tensor of shape %s on %s" %
+                                 (name, want, "the host" if host else "cuda:%d" % self.device))
             setattr(inp, name, t.data_ptr())
         inp.r = r
+        return inp
+
+    def solve_layer(self, s_a, s_gamma_a, s_gamma_b, s_gamma_q, s_b, s_q, s_qf, r_inv, h0, B_basis, Q_basis, T,
+                    u1=None, P0=None, info=None, stream=None):
+        """Enqueue ``ttc_lqr_solve_layer``: contextualised TTC-layer evaluation.  Per-instance tensors are
+        ``[N, n]`` (``s_b, s_q, s_qf``: ``[N, r]``), the bases ``[r, n, n]``; all float32, contiguous, on the
+        solver's device.  ``u1 [N, n]``, ``P0 [N, n, n]``, ``info [N]`` (int32) are written if given."""
+        inp = self._layer_inputs((s_a, s_gamma_a, s_gamma_b, s_gamma_q, s_b, s_q, s_qf, r_inv, h0, B_basis, Q_basis), False)
         if stream is None:
             stream = torch.cuda.current_stream(self.device)
         _check(load_library().ttc_lqr_solve_layer(
             self._h, ctypes.byref(inp), int(T), self._ptr(u1), self._ptr(P0), self._ptr(info),
             ctypes.c_void_p(stream.cuda_stream)))
+
+    def solve_layer_host(self, s_a, s_gamma_a, s_gamma_b, s_gamma_q, s_b, s_q, s_qf, r_inv, h0, B_basis, Q_basis, T,
+                         u1=None, P0=None, info=None):
+        """``ttc_lqr_solve_layer_host``: all tensors live in host memory; returns when the results are there."""
+        inp = self._layer_inputs((s_a, s_gamma_a, s_gamma_b, s_gamma_q, s_b, s_q, s_qf, r_inv, h0, B_basis, Q_basis), True)
+        _check(load_library().ttc_lqr_solve_layer_host(
+            self._h, ctypes.byref(inp), int(T), self._ptr(u1), self._ptr(P0), self._ptr(info)))
 
     def solve_host(self, A, B, Q, R, x0, H, K=None, P=None, x=None, u=None, info=None, flags=0):
         """``ttc_lqr_solve_host``: all tensors live in host memory; returns when the results are there."""

@@ -119,3 +119,22 @@ def test_layer_rejects_unsupported_shapes():
     with pytest.raises(Exception):
         s.solve_layer(*(w[k] for k in workloads.LAYER_KEYS), 2)
     s.close()
+
+
+def test_host_buffer_entry_point_matches_device_entry_point():
+    w = workloads.make_layer_workload("layer16", device=DEV, batch=(2, 3, 37), seed=12)
+    T, n, N = 11, w["n"], w["N"]
+    u_d, P_d, info_d = run_gpu(w, T)
+    s = lqr.LqrSolver(n, n, T, w["batch"])
+    hin = [w[k].cpu() for k in workloads.LAYER_KEYS]
+    u_h = torch.full((N, n), 7.0).pin_memory()
+    P_h = torch.full((N, n, n), 7.0).pin_memory()
+    info_h = torch.full((N,), -3, dtype=torch.int32).pin_memory()
+    s.solve_layer_host(*hin, T, u1=u_h, P0=P_h, info=info_h)
+    assert s.query(lqr.TTC_QUERY_LAST_LAUNCHES) == 1
+    assert torch.equal(u_h, u_d.cpu()) and torch.equal(P_h, P_d.cpu()) and torch.equal(info_h, info_d.cpu())
+    # outputs are optional, pageable memory works, and the call can be repeated
+    u2 = torch.empty((N, n))
+    s.solve_layer_host(*hin, T, u1=u2)
+    assert torch.equal(u2, u_d.cpu())
+    s.close()
