@@ -11,6 +11,7 @@
 #include "common.cuh"
 #include "riccati_cta.cuh"
 #include "riccati_umma64.cuh"
+#include "riccati_umma64q.cuh"
 #include "riccati_warp.cuh"
 #include "ttc_layer.cuh"
 #include "scan_pair.cuh"
@@ -353,17 +354,17 @@ int solve_window(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, 
         const bool want_tf32 = h->cfg.math == TTC_MATH_TF32 || (h->cfg.math == TTC_MATH_AUTO && bf16_in);
         const bool head_shared = A->bstride[2] == 0 && B->bstride[2] == 0 && R->bstride[2] == 0;
         if (want_tf32 && n == 64 && m == 64 && head_shared && !time_varying) {
-            // tcgen05 kernel: persistent CTAs, two independent warpgroups each
+            // tcgen05 kernel: persistent CTAs, four independent warpgroups each
             if ((s = ensure(h->ws_E, sizeof(int) * 4))) return s;
             int* counter = static_cast<int*>(h->ws_E.ptr);
             TTC_CUDA(cudaMemsetAsync(counter, 0, 2 * sizeof(int), st));
-            const size_t smem = umma64::smem_bytes();
-            auto kern = rollout_needs_all_K || K ? umma64::riccati_umma64_kernel<true> : umma64::riccati_umma64_kernel<false>;
+            const size_t smem = umma64::smem4_bytes();
+            auto kern = rollout_needs_all_K || K ? umma64::riccati_umma64q_kernel<true> : umma64::riccati_umma64q_kernel<false>;
             TTC_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            const long long chunks = p.b0 * p.b1 * ((tcount + umma64::CHUNK - 1) / umma64::CHUNK);
+            const long long chunks = p.b0 * p.b1 * ((tcount + umma64::CHUNK4 - 1) / umma64::CHUNK4);
             long long grid = h->sm_count;
-            if (2 * grid > chunks) grid = (chunks + 1) / 2;
-            kern<<<(unsigned)grid, umma64::THREADS, smem, st>>>(p, counter, counter + 1);
+            if (grid > chunks) grid = chunks;
+            kern<<<(unsigned)grid, umma64::THREADS4, smem, st>>>(p, counter, counter + 1);
             TTC_CUDA(cudaGetLastError());
             h->last_launches += 1;
             h->total_launches += 1;
