@@ -1,33 +1,37 @@
 // Riccati-backward kernel for n = m = 64 on the 5th-generation tensor cores (tcgen05.mma,
 // kind::tf32, fp32 accumulators in tensor memory).
 //
-// One persistent CTA per SM, 256 threads = 2 warpgroups.  A warpgroup owns a PAIR of instances
-// (a, b) of one head at a time and walks their horizon together; the two warpgroups are
-// independent (own operands, own barriers, own half of tensor memory), so the tensor pipe works
-// for one pair while the other pair is in its factorisation.
+// One persistent CTA per SM, 512 threads = 4 warpgroups.  A warpgroup (128 threads = the 128 lanes of tensor
+// memory) walks ONE instance through the horizon; the four warpgroups are independent (own operands, own barriers,
+// own quarter of tensor memory) and share the per-head operand BA = [B'; A'] (128 x 64).  The step is one long
+// dependency chain (64 pivots in 8 panels); four chains per SM keep the tensor pipe, the shared-memory pipe and
+// the issue slots busier than fewer, longer ones (a thread has 128 registers).
 //
-// Per step (Prop. 3.1), with P symmetric and the per-head operand BA = [B'; A'] (128 x 64):
-//   (1)  W  = BA * [P_a P_b]          -> W_x = [V_x'; T_x'] = [(P_x B)'; (P_x A)']        SS, M128 N128
-//   (2x) F_x  = W_x * B  = [S_x - R ; Y_x']                                               TS (A operand read from
-//        tensor memory, no round trip through shared memory), N64
-//   (3x) right-looking blocked Cholesky (8-wide panels) of the tall matrix G_x = [S_x; Y_x'] IN TENSOR MEMORY:
-//        thread r owns row r (lane r).  Per panel: load the row's 8 panel columns (tcgen05.ld), add R, publish the
-//        8 x 8 diagonal block, every thread factors it in registers and forward-substitutes its own row, writes
-//        the row of the panel as tf32 hi + lo parts to a 128 x 8 operand buffer, and ONE rank-8 tcgen05.mma
-//        (3 passes: hi*hi + lo*hi + hi*lo, error-compensated) applies the trailing update to all 128 rows.
-//        Both instances of the pair go through every panel together, so their dependency chains overlap.
-//        It leaves L (S_x = L L') and Z_x' = Y_x' L^{-T} (rows 64..127): no explicit inverse.
-//   (4x) DP_x = W_x * A = [ . ; A'P_x A]   (into the columns that held F_x)                TS, N64
-//   (5x) DP_x -= Z_x' Z_x                                                                   SS, N64
-//   P_x <- Q_x + DP_x            (P_t = Q + A'P A - Y'S^{-1}Y)
-// Tensor-memory map of a warpgroup (256 columns): R0 = W_a, R1 = W_b, R2 = F_a then DP_a, R3 = F_b then DP_b.
+// Per step (Prop. 3.1), with P symmetric:
+//   (1)  W  = BA * P                  -> W = [V'; T'] = [(P B)'; (P A)']                    SS, M128 N64
+//   (2)  F  = W * B  = [S - R ; Y']                                                        TS (A operand read from
+//        tensor memory, no round trip through shared memory), N64.  The issuing thread waits for (1) first: an MMA
+//        that reads its A operand from tensor memory is not ordered after the MMAs that wrote it.
+//   (3)  right-looking blocked Cholesky (8-wide panels) of the tall matrix G = [S; Y'] IN TENSOR MEMORY:
+//        thread r owns row r (lane r).  Per panel: load the row's 8 panel columns (tcgen05.ld), add R, the warp that
+//        owns the 8 diagonal rows factors the 8 x 8 block in registers and publishes it, every thread
+//        forward-substitutes its own row, writes it as tf32 hi + lo parts to a 128 x 8 operand buffer, and ONE
+//        rank-8 tcgen05.mma (3 passes: hi*hi + lo*hi + hi*lo, error-compensated) applies the trailing update to all
+//        128 rows.  It leaves L (S = L L') and Z' = Y' L^{-T} (rows 64..127): no explicit inverse.
+//   (4)  DP = W * A = [ . ; A'P A]   (into the columns that held F)                         TS, N64
+//   (5)  DP -= Z' Z                                                                         SS, N64
+//   P <- Q + DP                  (P_t = Q + A'P A - Y'S^{-1}Y)
+// Tensor memory of a warpgroup (128 columns): R_W = W, R_F = F then DP.
+// Shared memory of a warpgroup: X1 (L in fp32, only when the gains or u_0 need it) | X0 (P, then Z') | panel hi |
+// panel lo | scratch.  X1 directly precedes X0: step (5) starts its A operand 64 rows before Z' so that Z' lands on
+// lanes 64..127 (what the first 64 rows multiply goes to lanes that are never read).
 //
 // Shared-memory operands use the canonical K-major layout without swizzle: 8 x 4 (rows x k) core
-// matrices of 128 contiguous bytes, chunk stride 128 B along k, 2048 B between 8-row groups.  A row
-// owner writes its row with conflict-free 16-byte stores.
+// matrices of 128 contiguous bytes, chunk stride 128 B along k, 2048 B between 8-row groups (256 B in the panel
+// buffers).  A row owner writes its row with conflict-free 16-byte stores.
 //
 // Every wait on an MMA-completion barrier is bounded; on a timeout the warpgroup records an error,
-// stops taking work and the kernel still releases tensor memory before it returns.
+// the CTA stops taking work and the kernel still releases tensor memory before it returns.
 #pragma once
 
 #include "common.cuh"
@@ -37,36 +41,14 @@ namespace umma64 {
 
 constexpr int N = 64;
 constexpr int WG_THREADS = 128;
-constexpr int NUM_WG = 2;
-constexpr int THREADS = NUM_WG * WG_THREADS;
-constexpr int CHUNK = 16;                       // tokens per work item (8 pairs)
 constexpr uint32_t SC = 128;                    // bytes between consecutive 4-wide k chunks
 constexpr uint32_t SR = 2048;                   // bytes between 8-row groups (16 chunks)
 constexpr uint32_t MAT_BYTES = 8 * SR;          // one 64 x 64 matrix
 constexpr uint32_t BUF_BYTES = 2 * MAT_BYTES;   // 128 rows
 constexpr int SPIN_LIMIT = 1 << 22;
 
-// per-warpgroup shared memory: BA | X0 | X1 (BA and X0 adjacent: step (5a) starts its A operand
-// 64 rows before X0) followed by small scratch.
-constexpr uint32_t OFF_BA = 0;
-constexpr uint32_t OFF_X0 = BUF_BYTES;
-constexpr uint32_t OFF_X1 = 2 * BUF_BYTES;
-constexpr uint32_t OFF_PAN = 3 * BUF_BYTES;     // panel operands: per instance 128 x 8 hi parts, 128 x 8 lo parts
 constexpr uint32_t PSR = 256;                   // bytes between 8-row groups of a panel buffer (2 chunks)
 constexpr uint32_t PAN_BYTES = 16 * PSR;        // one 128 x 8 buffer
-constexpr uint32_t OFF_MISC = OFF_PAN + 4 * PAN_BYTES;
-struct Misc {
-    unsigned long long mbar;     // MMA completion barrier
-    int chunk;                   // current work item
-    int dead;                    // set when a wait timed out
-    int flag[2];                 // first failed pivot per instance (0 = none)
-    alignas(16) float x0[2][N];
-    alignas(16) float y0[2][N];  // Y x_0 / u_t of the rollout; during the factorisation: the 8 x 8 diagonal blocks
-    alignas(16) float ld[2][36]; // current diagonal factors: strict lower triangle (28) + reciprocal pivots (8)
-};
-constexpr uint32_t WG_BYTES = OFF_MISC + ((sizeof(Misc) + 127) / 128) * 128;
-constexpr uint32_t SMEM_BYTES = NUM_WG * WG_BYTES + 128;     // + slot for the tensor-memory base address
-static_assert(SMEM_BYTES <= 227 * 1024, "shared memory of one CTA");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -187,8 +169,8 @@ __device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&r)[8])
 }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
-__device__ __forceinline__ void wg_barrier(int wg) { asm volatile("bar.sync %0, %1;" :: "r"(1 + wg), "r"(WG_THREADS) : "memory"); }
-__device__ __forceinline__ void pair_barrier(int wg, int x) { asm volatile("bar.sync %0, %1;" :: "r"(3 + 2 * wg + x), "r"(64) : "memory"); }
+// named barriers: 1 + wg = warps 0, 1 of a warpgroup (64 threads), 5 + wg = the whole warpgroup
+__device__ __forceinline__ void half_barrier(int wg) { asm volatile("bar.sync %0, %1;" :: "r"(1 + wg), "r"(64) : "memory"); }
 
 // ---- blocked Cholesky of S fused with the forward substitution Z' = Y' L^{-T} --------------------------------------
 __device__ __forceinline__ void mma_16x8x8(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
@@ -269,11 +251,11 @@ __device__ __forceinline__ void store_row8(unsigned char* grp, int slot, const f
     *reinterpret_cast<float4*>(grp + SC + (ROT ? ((slot + 4) & 7) : slot) * 16) = b;
 }
 
-// Gains (Eq. 4): K = -L^{-T} Z, i.e. row c of K' is -(row c of Z') L^{-1}.  Same two warps, same blocked scheme
-// run backwards: per 8-wide block kb = 7..0 every row owner solves x L_d = z for its row of Z' (in place in
+// Gains (Eq. 4): K = -L^{-T} Z, i.e. row c of K' is -(row c of Z') L^{-1}.  Warps 0, 1 of the warpgroup (pw = 0, 1) run
+// a blocked scheme backwards on L (fp32, rotated layout, at `Sm`) and Z' (at `Ym`): per 8-wide block kb = 7..0 every row owner solves x L_d = z for its row of Z' (in place in
 // `Ym`), then the columns left of the block get the update Z'[c][j] -= x[c][kb] . L[kb][j] as 3 x tf32 mma.
 // On return row c of Ym holds (Z' L^{-1})[c][:] = -K[:, c] (fp32).
-__device__ __forceinline__ void pair_gain_solve(const unsigned char* Sm, unsigned char* Ym, int wg, int x, int pw, int lane)
+__device__ __forceinline__ void pair_gain_solve(const unsigned char* Sm, unsigned char* Ym, int wg, int pw, int lane)
 {
     const int g = lane >> 2, t = lane & 3;
     const int tid2 = 32 * pw + lane;
@@ -305,7 +287,7 @@ __device__ __forceinline__ void pair_gain_solve(const unsigned char* Sm, unsigne
         store_row8<false, false>(py, own_slot, xr);
         if (kb == 0)
             break;
-        pair_barrier(wg, x);
+        half_barrier(wg);
         // B fragments: rows 8kb + t, 8kb + t + 4 of L, columns 8j + g (j < kb)
         uint32_t bh[7][2], bl[7][2];
         {
@@ -358,50 +340,11 @@ __device__ __forceinline__ void pair_gain_solve(const unsigned char* Sm, unsigne
                 *reinterpret_cast<float2*>(pc + 2 * j * SC + SR) = make_float2(acc[j][2], acc[j][3]);
             }
         }
-        pair_barrier(wg, x);
+        half_barrier(wg);
     }
 }
 
 // ---- global-memory helpers --------------------------------------------------------------------------------------
-// row j (64 values) of the Q matrix of one instance
-__device__ __forceinline__ void load_q_row(float (&q)[64], const OperandDev& Q, long long oq, int j)
-{
-    if (Q.dtype == TTC_BF16) {
-        const uint4* src = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(Q.ptr) + oq + (long long)j * N);
-#pragma unroll
-        for (int c = 0; c < 8; ++c) {
-            const uint4 v = __ldg(src + c);
-            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                q[8 * c + 2 * e] = __uint_as_float(w[e] << 16);
-                q[8 * c + 2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u);
-            }
-        }
-    } else {
-        const float4* src = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(Q.ptr) + oq + (long long)j * N);
-#pragma unroll
-        for (int c = 0; c < 16; ++c) {
-            const float4 v = __ldg(src + c);
-            q[4 * c] = v.x; q[4 * c + 1] = v.y; q[4 * c + 2] = v.z; q[4 * c + 3] = v.w;
-        }
-    }
-}
-// row `r` of a 128-row operand buffer <- 64 values rounded to tf32
-__device__ __forceinline__ void store_row_tf32(unsigned char* buf, int r, const float (&v)[64])
-{
-#pragma unroll
-    for (int c = 0; c < 16; ++c)
-        *reinterpret_cast<float4*>(buf + toff(r, 4 * c)) =
-            make_float4(round_tf32(v[4 * c]), round_tf32(v[4 * c + 1]), round_tf32(v[4 * c + 2]), round_tf32(v[4 * c + 3]));
-}
-__device__ __forceinline__ void store_row_global(float* dst, const float (&v)[64])
-{
-#pragma unroll
-    for (int c = 0; c < 16; ++c)
-        reinterpret_cast<float4*>(dst)[c] = make_float4(v[4 * c], v[4 * c + 1], v[4 * c + 2], v[4 * c + 3]);
-}
-
 __device__ __forceinline__ void wg_fail_instance(const SolveParams& p, long long inst, int code, int wt)
 {
     const float qn = quiet_nan();
@@ -426,8 +369,74 @@ __device__ __forceinline__ void wg_fail_instance(const SolveParams& p, long long
         p.info[inst] = code;
 }
 
-// Every output of the solve: K_t, P_t (or P_0), x_t, u_t (or u_0), info.  When the rollout needs gains that the
-// caller did not ask for they go to the workspace p.Kws.
+constexpr int NUM_WG = 4;
+constexpr int THREADS = NUM_WG * WG_THREADS;
+constexpr int TOK = 8;                                  // tokens per warpgroup and work item
+constexpr int CHUNK = NUM_WG * TOK;                   // tokens per work item of a CTA
+constexpr uint32_t OFF_X1 = 0;
+constexpr uint32_t OFF_X0 = MAT_BYTES;
+constexpr uint32_t OFF_PH = 2 * MAT_BYTES;
+constexpr uint32_t OFF_PL = 2 * MAT_BYTES + PAN_BYTES;
+constexpr uint32_t OFF_MISC = 2 * MAT_BYTES + 2 * PAN_BYTES;
+struct Misc {
+    unsigned long long mbar;     // MMA completion barrier (every thread waits on it)
+    unsigned long long mbar_w;   // completion of W = BA P': only the issuing thread waits on it
+    int dead;                    // set when a wait timed out
+    int flag;                    // first failed pivot (0 = none)
+    alignas(16) float x0[N];
+    alignas(16) float y0[N];     // Y x_0 / u_t of the rollout; during the factorisation: the 8 x 8 diagonal block
+    alignas(16) float ld[36];    // current diagonal factor: strict lower triangle (28) + reciprocal pivots (8)
+};
+constexpr uint32_t WG_BYTES = OFF_MISC + ((sizeof(Misc) + 127) / 128) * 128;
+struct CtaShared {
+    int chunk;                   // current work item
+    int dead;                    // some warpgroup gave up: the CTA stops taking work
+    uint32_t tmem_base;
+};
+constexpr uint32_t SMEM_BYTES = BUF_BYTES + NUM_WG * WG_BYTES + 128;
+static_assert(SMEM_BYTES <= 227 * 1024, "shared memory of one CTA");
+
+__device__ __forceinline__ void wg_barrier(int wg) { asm volatile("bar.sync %0, %1;" :: "r"(5 + wg), "r"(WG_THREADS) : "memory"); }
+
+// half a row (32 values) of the Q matrix of one instance
+__device__ __forceinline__ void load_q_half(float (&q)[32], const OperandDev& Q, long long oq, int j, int half)
+{
+    if (Q.dtype == TTC_BF16) {
+        const uint4* src = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(Q.ptr) + oq + (long long)j * N + 32 * half);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const uint4 v = __ldg(src + c);
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                q[8 * c + 2 * e] = __uint_as_float(w[e] << 16);
+                q[8 * c + 2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u);
+            }
+        }
+    } else {
+        const float4* src = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(Q.ptr) + oq + (long long)j * N + 32 * half);
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            const float4 v = __ldg(src + c);
+            q[4 * c] = v.x; q[4 * c + 1] = v.y; q[4 * c + 2] = v.z; q[4 * c + 3] = v.w;
+        }
+    }
+}
+// columns 32 half .. 32 half + 31 of row `r` of a 64-row operand <- values rounded to tf32
+__device__ __forceinline__ void store_half_tf32(unsigned char* buf, int r, int half, const float (&v)[32])
+{
+#pragma unroll
+    for (int c = 0; c < 8; ++c)
+        *reinterpret_cast<float4*>(buf + toff(r, 32 * half + 4 * c)) =
+            make_float4(round_tf32(v[4 * c]), round_tf32(v[4 * c + 1]), round_tf32(v[4 * c + 2]), round_tf32(v[4 * c + 3]));
+}
+__device__ __forceinline__ void store_half_global(float* dst, const float (&v)[32])
+{
+#pragma unroll
+    for (int c = 0; c < 8; ++c)
+        reinterpret_cast<float4*>(dst)[c] = make_float4(v[4 * c], v[4 * c + 1], v[4 * c + 2], v[4 * c + 3]);
+}
+
 // GAINS = the request needs every K_t (K, x or the full u wanted); the other instantiation carries none of that code.
 template <bool GAINS>
 __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams p, int* chunk_counter, int* error_flag)
@@ -438,39 +447,41 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
     const int wt = tid % WG_THREADS;
     const int warp = wt >> 5;                  // warp in warpgroup: owns tensor-memory lanes 32 warp .. 32 warp + 31
     const int lane = wt & 31;
-    unsigned char* wsm = smem_raw + (size_t)wg * WG_BYTES;
-    unsigned char* BA = wsm + OFF_BA;          // rows 0..63: B' (row j = column j of B), rows 64..127: A'
-    unsigned char* X0 = wsm + OFF_X0;          // [P_a; P_b] -> [Z_a'; Z_b'] -> next [P_a; P_b]
-    unsigned char* X1 = wsm + OFF_X1;          // [L_a; L_b], fp32 (kept only when the gains or u_0 need it)
-    unsigned char* PAN = wsm + OFF_PAN;        // panel operands: hi_a | lo_a | hi_b | lo_b
+    unsigned char* BA = smem_raw;              // rows 0..63: B' (row j = column j of B), rows 64..127: A'; shared by the CTA
+    unsigned char* wsm = smem_raw + BUF_BYTES + (size_t)wg * WG_BYTES;
+    unsigned char* X1 = wsm + OFF_X1;        // L, fp32 (kept only when the gains or u_0 need it)
+    unsigned char* X0 = wsm + OFF_X0;        // P -> Z' -> next P
+    unsigned char* PH = wsm + OFF_PH;        // panel operand, hi parts (128 x 8)
+    unsigned char* PL = wsm + OFF_PL;        // panel operand, lo parts
     Misc& misc = *reinterpret_cast<Misc*>(wsm + OFF_MISC);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_raw + (size_t)NUM_WG * WG_BYTES);
+    CtaShared& cta = *reinterpret_cast<CtaShared*>(smem_raw + BUF_BYTES + (size_t)NUM_WG * WG_BYTES);
     const uint32_t mbar = smem_u32(&misc.mbar);
+    const uint32_t mbar_w = smem_u32(&misc.mbar_w);
 
     if (wt == 0) {
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(mbar) : "memory");
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(mbar_w) : "memory");
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         misc.dead = 0;
     }
-    // rows 64..127 (Z') of the two low-part panel buffers stay zero: Z' is kept as tf32
-#pragma unroll
-    for (int x = 0; x < 2; ++x)
-        *reinterpret_cast<float4*>(PAN + (uint32_t)x * 2u * PAN_BYTES + PAN_BYTES + 8u * PSR + (uint32_t)wt * 16u) = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (tid == 0)
+        cta.dead = 0;
+    // rows 64..127 (Z') of the low-part panel buffer stay zero: Z' is kept as tf32
+    if (wt >= 64)
+        for (int e = wt - 64; e < 128; e += 64)
+            *reinterpret_cast<float4*>(PL + 8u * PSR + (uint32_t)e * 16u) = make_float4(0.f, 0.f, 0.f, 0.f);
     async_proxy_fence();
     if (tid < 32) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(smem_u32(tmem_slot)), "r"(512) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(smem_u32(&cta.tmem_base)), "r"(512) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tm = *tmem_slot + 256u * wg;
-    const uint32_t R0 = tm, R1 = tm + 64, R2 = tm + 128, R3 = tm + 192;
+    const uint32_t RW = cta.tmem_base + 128u * wg, RF = RW + 64u;
     const uint32_t lane_sel = (uint32_t)(32 * warp) << 16;
-    uint32_t parity = 0;
-    // one thread of warp 3 issues every MMA of the warpgroup (tensor-pipe order = its program order); the issue of
-    // a batch blocks that thread for about as long as the batch runs, and warps 0 and 1 factor the diagonal blocks
-    const bool issuer = wt == 96;
+    uint32_t parity = 0, parity_w = 0;
+    const bool issuer = wt == 96;              // one thread of warp 3 issues every MMA of the warpgroup
 
     const int H = p.H;
     const long long chunks_per_head = (p.tcount + CHUNK - 1) / CHUNK;
@@ -479,11 +490,10 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
     const bool want_u0 = (p.u != nullptr) && p.first_only && !need_K_all;
     const bool rollout = (p.x != nullptr) || (p.u != nullptr && need_K_all);
     float* Kbase = p.K ? p.K : p.Kws;
-    long long offA_loaded = -1, offB_loaded = -1, offR_loaded = -1;
+    long long offA_loaded = -1, offB_loaded = -1;
     const float* Rg = nullptr;
     bool dead = false;
 
-    // wait for the MMAs committed last; a timeout marks the warpgroup dead (checked after the next barrier)
     auto wait_mma = [&]() {
         if (!mbar_wait(mbar, parity)) {
             misc.dead = 1;
@@ -493,12 +503,15 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
         tc_fence_after();
     };
 
-    while (!dead) {
-        if (wt == 0)
-            misc.chunk = atomicAdd(chunk_counter, 1);
-        wg_barrier(wg);
-        const long long chunk = misc.chunk;
-        if (chunk >= nchunks)
+    for (;;) {
+        if (dead)
+            cta.dead = 1;
+        __syncthreads();                       // every warpgroup is done with BA and with the last work item
+        if (tid == 0)
+            cta.chunk = atomicAdd(chunk_counter, 1);
+        __syncthreads();
+        const long long chunk = cta.chunk;
+        if (chunk >= nchunks || cta.dead)
             break;
         const long long head = chunk / chunks_per_head;
         const long long tok0 = p.t0 + (chunk % chunks_per_head) * CHUNK;
@@ -507,110 +520,107 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
         {
             const long long oa = operand_offset(p.A, inst0, p.b1, p.b2);
             const long long ob = operand_offset(p.B, inst0, p.b1, p.b2);
-            const long long orr = operand_offset(p.R, inst0, p.b1, p.b2);
             if (oa != offA_loaded || ob != offB_loaded) {
                 const float* Ag = reinterpret_cast<const float*>(p.A.ptr) + oa;
                 const float* Bg = reinterpret_cast<const float*>(p.B.ptr) + ob;
-                for (int e = wt; e < N * N; e += WG_THREADS) {
+                for (int e = tid; e < N * N; e += THREADS) {
                     const int k = e >> 6, j = e & 63;
                     elem(BA, toff(j, k)) = round_tf32(__ldg(Bg + e));
                     elem(BA, toff(64 + j, k)) = round_tf32(__ldg(Ag + e));
                 }
                 offA_loaded = oa; offB_loaded = ob;
+                async_proxy_fence();
+                __syncthreads();
             }
-            offR_loaded = orr;
-            Rg = reinterpret_cast<const float*>(p.R.ptr) + orr;
+            Rg = reinterpret_cast<const float*>(p.R.ptr) + operand_offset(p.R, inst0, p.b1, p.b2);
         }
+        const int my0 = TOK * wg, my1 = min(ntok, TOK * wg + TOK);
 
-        for (int tk = 0; tk < ntok && !dead; tk += 2) {
-            const long long inst_x[2] = {inst0 + tk, inst0 + min(tk + 1, ntok - 1)};
-            const bool valid_b = tk + 1 < ntok;
-            const long long oq_x[2] = {operand_offset(p.Q, inst_x[0], p.b1, p.b2), operand_offset(p.Q, inst_x[1], p.b1, p.b2)};
-            // ---- P_H = Q: warps 2, 3 own the rows of the value matrices
+        for (int tk = my0; tk < my1 && !dead; ++tk) {
+            const long long inst = inst0 + tk;
+            const long long oq = operand_offset(p.Q, inst, p.b1, p.b2);
+            // ---- P_H = Q: warps 2, 3 own the rows of the value matrix
             if (warp >= 2) {
                 const int j = wt - 64;
 #pragma unroll 1
-                for (int x = 0; x < 2; ++x) {
-                    float q[64];
-                    load_q_row(q, p.Q, oq_x[x], j);
-                    store_row_tf32(X0, 64 * x + j, q);
-                    if (p.P && !p.first_only && (x == 0 || valid_b))
-                        store_row_global(p.P + (inst_x[x] * (long long)(H + 1) + H) * N * N + (long long)j * N, q);
+                for (int half = 0; half < 2; ++half) {
+                    float q[32];
+                    load_q_half(q, p.Q, oq, j, half);
+                    store_half_tf32(X0, j, half, q);
+                    if (p.P && !p.first_only)
+                        store_half_global(p.P + (inst * (long long)(H + 1) + H) * N * N + (long long)j * N + 32 * half, q);
                 }
-            } else if (p.x0.ptr) {
-                const int x = warp, j0 = 2 * lane;             // warp x stages x_0 of instance x
-                const long long ox = operand_offset(p.x0, inst_x[x], p.b1, p.b2);
-                misc.x0[x][j0] = load_elem(p.x0, ox + j0);
-                misc.x0[x][j0 + 1] = load_elem(p.x0, ox + j0 + 1);
+            } else if (p.x0.ptr && warp == 0) {
+                const long long ox = operand_offset(p.x0, inst, p.b1, p.b2);
+                misc.x0[2 * lane] = load_elem(p.x0, ox + 2 * lane);
+                misc.x0[2 * lane + 1] = load_elem(p.x0, ox + 2 * lane + 1);
             }
-            if (wt < 2)
-                misc.flag[wt] = 0;
+            if (wt == 0)
+                misc.flag = 0;
             async_proxy_fence();
             wg_barrier(wg);
 
             for (int ts = H - 1; ts >= 0 && !dead; --ts) {
-                // (1) W = BA [P_a P_b]' -> R0|R1 ; (2) F_a -> R2, F_b -> R3
+                // (1) W = BA P' -> R_W ; (2) F = W B -> R_F
                 if (issuer) {
                     tc_fence_after();
-                    gemm_ss(R0, smem_u32(BA), smem_u32(X0), 128, 0, false);
-                    gemm_ts(R2, R0, smem_u32(BA), 64);
-                    gemm_ts(R3, R1, smem_u32(BA), 64);
+                    gemm_ss(RW, smem_u32(BA), smem_u32(X0), 64, 0, false);
+                    // F reads W from tensor memory: an MMA whose A operand was written by the MMAs just before it is NOT
+                    // ordered after them by the pipe (measured: 7 % error in F when chained), so the issuing thread
+                    // waits for W on a barrier of its own before it issues F
+                    mma_commit(mbar_w);
+                    if (!mbar_wait(mbar_w, parity_w)) {
+                        misc.dead = 1;
+                        atomicExch(error_flag, 1);
+                    }
+                    parity_w ^= 1u;
+                    tc_fence_after();
+                    gemm_ts(RF, RW, smem_u32(BA), 64);
                     mma_commit(mbar);
                 }
                 wait_mma();
-                // (3) [S_x; Y_x'] = [L; Z'] L' panel by panel, thread wt owns row wt of both instances
+                // (3) [S; Y'] = [L; Z'] L' panel by panel, thread wt owns row wt
                 const bool keep_l = need_K_all || (ts == 0 && want_u0);
-                float* diag = &misc.y0[0][0];                  // [2][8][8]
-                float v[2][8];                                 // this row's columns of the current panel
-                // columns c0 .. c0 + 7 of row wt (+ R for the rows of S)
+                float* diag = &misc.y0[0];                     // [8][8]
+                float v[8];
                 auto load_cols = [&](int c0) {
-                    uint32_t raw[2][8];
-                    tmem_ld8(R2 + lane_sel + c0, raw[0]);
-                    tmem_ld8(R3 + lane_sel + c0, raw[1]);
+                    uint32_t raw[8];
+                    tmem_ld8(RF + lane_sel + c0, raw);
                     float4 r0 = make_float4(0.f, 0.f, 0.f, 0.f), r1 = r0;
                     if (warp < 2) {
                         r0 = __ldg(reinterpret_cast<const float4*>(Rg + (long long)wt * N + c0));
                         r1 = __ldg(reinterpret_cast<const float4*>(Rg + (long long)wt * N + c0 + 4));
                     }
                     tmem_wait_ld();
-#pragma unroll
-                    for (int x = 0; x < 2; ++x) {
-                        v[x][0] = __uint_as_float(raw[x][0]) + r0.x; v[x][1] = __uint_as_float(raw[x][1]) + r0.y;
-                        v[x][2] = __uint_as_float(raw[x][2]) + r0.z; v[x][3] = __uint_as_float(raw[x][3]) + r0.w;
-                        v[x][4] = __uint_as_float(raw[x][4]) + r1.x; v[x][5] = __uint_as_float(raw[x][5]) + r1.y;
-                        v[x][6] = __uint_as_float(raw[x][6]) + r1.z; v[x][7] = __uint_as_float(raw[x][7]) + r1.w;
-                    }
+                    v[0] = __uint_as_float(raw[0]) + r0.x; v[1] = __uint_as_float(raw[1]) + r0.y;
+                    v[2] = __uint_as_float(raw[2]) + r0.z; v[3] = __uint_as_float(raw[3]) + r0.w;
+                    v[4] = __uint_as_float(raw[4]) + r1.x; v[5] = __uint_as_float(raw[5]) + r1.y;
+                    v[6] = __uint_as_float(raw[6]) + r1.z; v[7] = __uint_as_float(raw[7]) + r1.w;
                 };
                 load_cols(0);
 #pragma unroll 1
                 for (int pnl = 0; pnl < 8; ++pnl) {
                     const int col = 8 * pnl;
                     if (warp == (pnl >> 2)) {
-                        // the 8 rows of the diagonal blocks belong to this warp: gather the blocks, factor them
-                        // (lanes 0..15 the block of instance a, lanes 16..31 that of b; redundantly within each
-                        // half) and publish L_d and the reciprocal pivots
+                        // the 8 rows of the diagonal block belong to this warp: gather the block, factor it (every
+                        // lane redundantly) and publish L_d and the reciprocal pivots
                         if ((unsigned)(wt - col) < 8u) {
-#pragma unroll
-                            for (int x = 0; x < 2; ++x) {
-                                float4* dst = reinterpret_cast<float4*>(diag + 64 * x + 8 * (wt - col));
-                                dst[0] = make_float4(v[x][0], v[x][1], v[x][2], v[x][3]);
-                                dst[1] = make_float4(v[x][4], v[x][5], v[x][6], v[x][7]);
-                            }
+                            float4* dst = reinterpret_cast<float4*>(diag + 8 * (wt - col));
+                            dst[0] = make_float4(v[0], v[1], v[2], v[3]);
+                            dst[1] = make_float4(v[4], v[5], v[6], v[7]);
                         }
                         __syncwarp();
-                        const int hx = lane >> 4, hl = lane & 15;
                         float l[8][8], rinv[8];
 #pragma unroll
                         for (int i = 0; i < 8; ++i) {
-                            const float4 a4 = *reinterpret_cast<const float4*>(diag + 64 * hx + 8 * i);
-                            const float4 b4 = *reinterpret_cast<const float4*>(diag + 64 * hx + 8 * i + 4);
+                            const float4 a4 = *reinterpret_cast<const float4*>(diag + 8 * i);
+                            const float4 b4 = *reinterpret_cast<const float4*>(diag + 8 * i + 4);
                             l[i][0] = a4.x; l[i][1] = a4.y; l[i][2] = a4.z; l[i][3] = a4.w;
                             l[i][4] = b4.x; l[i][5] = b4.y; l[i][6] = b4.z; l[i][7] = b4.w;
                         }
                         const int bad = chol8(l, rinv);
-                        if (hl == 0) {
-                            // strict lower triangle row by row (28 values), then the 8 reciprocal pivots
-                            float4* dst = reinterpret_cast<float4*>(&misc.ld[hx][0]);
+                        if (lane == 0) {
+                            float4* dst = reinterpret_cast<float4*>(&misc.ld[0]);
                             dst[0] = make_float4(l[1][0], l[2][0], l[2][1], l[3][0]);
                             dst[1] = make_float4(l[3][1], l[3][2], l[4][0], l[4][1]);
                             dst[2] = make_float4(l[4][2], l[4][3], l[5][0], l[5][1]);
@@ -620,9 +630,9 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
                             dst[6] = make_float4(l[7][3], l[7][4], l[7][5], l[7][6]);
                             dst[7] = make_float4(rinv[0], rinv[1], rinv[2], rinv[3]);
                             dst[8] = make_float4(rinv[4], rinv[5], rinv[6], rinv[7]);
+                            if (bad && misc.flag == 0)
+                                misc.flag = ts * N + col + bad;
                         }
-                        if (hl == 0 && bad && misc.flag[hx] == 0)
-                            misc.flag[hx] = ts * N + col + bad;
                     }
                     tc_fence_before();
                     wg_barrier(wg);
@@ -631,50 +641,48 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
                         break;
                     }
                     if (pnl == 7 && issuer) {
-                        // every row has read its last columns of F: (4x) DP_x = W_x A into the columns of F_x
+                        // every row has read its last columns of F: (4) DP = W A into the columns of F
                         tc_fence_after();
-                        gemm_ts(R2, R0, smem_u32(BA) + MAT_BYTES, 64);
-                        gemm_ts(R3, R1, smem_u32(BA) + MAT_BYTES, 64);
+                        gemm_ts(RF, RW, smem_u32(BA) + MAT_BYTES, 64);
                     }
-#pragma unroll
-                    for (int x = 0; x < 2; ++x) {
+                    {
                         float l[8][8], rinv[8];
-                        {
-                            const float4* src = reinterpret_cast<const float4*>(&misc.ld[x][0]);
-                            const float4 c0 = src[0], c1 = src[1], c2 = src[2], c3 = src[3], c4 = src[4], c5 = src[5],
-                                         c6 = src[6], c7 = src[7], c8 = src[8];
-                            l[1][0] = c0.x; l[2][0] = c0.y; l[2][1] = c0.z; l[3][0] = c0.w;
-                            l[3][1] = c1.x; l[3][2] = c1.y; l[4][0] = c1.z; l[4][1] = c1.w;
-                            l[4][2] = c2.x; l[4][3] = c2.y; l[5][0] = c2.z; l[5][1] = c2.w;
-                            l[5][2] = c3.x; l[5][3] = c3.y; l[5][4] = c3.z; l[6][0] = c3.w;
-                            l[6][1] = c4.x; l[6][2] = c4.y; l[6][3] = c4.z; l[6][4] = c4.w;
-                            l[6][5] = c5.x; l[7][0] = c5.y; l[7][1] = c5.z; l[7][2] = c5.w;
-                            l[7][3] = c6.x; l[7][4] = c6.y; l[7][5] = c6.z; l[7][6] = c6.w;
-                            rinv[0] = c7.x; rinv[1] = c7.y; rinv[2] = c7.z; rinv[3] = c7.w;
-                            rinv[4] = c8.x; rinv[5] = c8.y; rinv[6] = c8.z; rinv[7] = c8.w;
-                        }
-                        fsub8(v[x], l, rinv);
-                        unsigned char* ph = PAN + (uint32_t)x * 2u * PAN_BYTES + (uint32_t)(wt >> 3) * PSR + (uint32_t)(wt & 7) * 16u;
+                        const float4* src = reinterpret_cast<const float4*>(&misc.ld[0]);
+                        const float4 c0 = src[0], c1 = src[1], c2 = src[2], c3 = src[3], c4 = src[4], c5 = src[5],
+                                     c6 = src[6], c7 = src[7], c8 = src[8];
+                        l[1][0] = c0.x; l[2][0] = c0.y; l[2][1] = c0.z; l[3][0] = c0.w;
+                        l[3][1] = c1.x; l[3][2] = c1.y; l[4][0] = c1.z; l[4][1] = c1.w;
+                        l[4][2] = c2.x; l[4][3] = c2.y; l[5][0] = c2.z; l[5][1] = c2.w;
+                        l[5][2] = c3.x; l[5][3] = c3.y; l[5][4] = c3.z; l[6][0] = c3.w;
+                        l[6][1] = c4.x; l[6][2] = c4.y; l[6][3] = c4.z; l[6][4] = c4.w;
+                        l[6][5] = c5.x; l[7][0] = c5.y; l[7][1] = c5.z; l[7][2] = c5.w;
+                        l[7][3] = c6.x; l[7][4] = c6.y; l[7][5] = c6.z; l[7][6] = c6.w;
+                        rinv[0] = c7.x; rinv[1] = c7.y; rinv[2] = c7.z; rinv[3] = c7.w;
+                        rinv[4] = c8.x; rinv[5] = c8.y; rinv[6] = c8.z; rinv[7] = c8.w;
+                        fsub8(v, l, rinv);
+                    }
+                    {
+                        unsigned char* ph = PH + (uint32_t)(wt >> 3) * PSR + (uint32_t)(wt & 7) * 16u;
                         float hi[8];
                         if (warp < 2) {                        // row wt of L: lower triangular, ends at column wt
                             float lo[8];
 #pragma unroll
                             for (int j = 0; j < 8; ++j) {
                                 if (col + j > wt)
-                                    v[x][j] = 0.f;
-                                hi[j] = round_tf32(v[x][j]);
-                                lo[j] = v[x][j] - hi[j];
+                                    v[j] = 0.f;
+                                hi[j] = round_tf32(v[j]);
+                                lo[j] = v[j] - hi[j];
                             }
-                            *reinterpret_cast<float4*>(ph + PAN_BYTES) = make_float4(lo[0], lo[1], lo[2], lo[3]);
-                            *reinterpret_cast<float4*>(ph + PAN_BYTES + SC) = make_float4(lo[4], lo[5], lo[6], lo[7]);
+                            unsigned char* pl = PL + (uint32_t)(wt >> 3) * PSR + (uint32_t)(wt & 7) * 16u;
+                            *reinterpret_cast<float4*>(pl) = make_float4(lo[0], lo[1], lo[2], lo[3]);
+                            *reinterpret_cast<float4*>(pl + SC) = make_float4(lo[4], lo[5], lo[6], lo[7]);
                             if (keep_l)                        // fp32 copy for the gains / u_0
-                                store_row8<true, false>(X1 + (uint32_t)x * MAT_BYTES + (uint32_t)(wt >> 3) * SR + 2u * pnl * SC, wt & 7, v[x]);
-                        } else {                               // row wt - 64 of Z_x': kept as tf32 (operand of (5x)), low part zero
+                                store_row8<true, false>(X1 + (uint32_t)(wt >> 3) * SR + 2u * pnl * SC, wt & 7, v);
+                        } else {                               // row wt - 64 of Z': kept as tf32 (operand of (5)), low part zero
 #pragma unroll
                             for (int j = 0; j < 8; ++j)
-                                hi[j] = round_tf32(v[x][j]);
-                            unsigned char* pz = X0 + (uint32_t)x * MAT_BYTES + (uint32_t)((wt - 64) >> 3) * SR + 2u * pnl * SC +
-                                                (uint32_t)(wt & 7) * 16u;
+                                hi[j] = round_tf32(v[j]);
+                            unsigned char* pz = X0 + (uint32_t)((wt - 64) >> 3) * SR + 2u * pnl * SC + (uint32_t)(wt & 7) * 16u;
                             *reinterpret_cast<float4*>(pz) = make_float4(hi[0], hi[1], hi[2], hi[3]);
                             *reinterpret_cast<float4*>(pz + SC) = make_float4(hi[4], hi[5], hi[6], hi[7]);
                         }
@@ -685,18 +693,13 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
                         break;
                     async_proxy_fence();
                     wg_barrier(wg);
-                    if (issuer) {                              // G_x -= panel * panel[0:64]'  (hi*hi + lo*hi + hi*lo)
+                    if (issuer) {                              // G -= panel * panel[0:64]'  (hi*hi + lo*hi + hi*lo)
                         tc_fence_after();
                         const uint32_t idn = instr_desc(64, 1);
-#pragma unroll
-                        for (int x = 0; x < 2; ++x) {
-                            const uint32_t d = x ? R3 : R2;
-                            const uint64_t dh = panel_desc(smem_u32(PAN) + (uint32_t)x * 2u * PAN_BYTES);
-                            const uint64_t dl = panel_desc(smem_u32(PAN) + (uint32_t)x * 2u * PAN_BYTES + PAN_BYTES);
-                            mma_ss(d, dh, dh, idn, 1u);
-                            mma_ss(d, dl, dh, idn, 1u);
-                            mma_ss(d, dh, dl, idn, 1u);
-                        }
+                        const uint64_t dh = panel_desc(smem_u32(PH)), dl = panel_desc(smem_u32(PL));
+                        mma_ss(RF, dh, dh, idn, 1u);
+                        mma_ss(RF, dl, dh, idn, 1u);
+                        mma_ss(RF, dh, dl, idn, 1u);
                         mma_commit(mbar);
                     }
                     wait_mma();
@@ -706,110 +709,90 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
                 tc_fence_before();
                 wg_barrier(wg);
                 dead = dead || misc.dead != 0;
-                // (4x) was issued at the last panel (lanes 64..127 of R2 / R3 = A'P_x A); then
-                // (5a) DP_a -= Z_a' Z_a : A operand rows 64..127 = Z_a' (rows 0..63 = the A' rows of BA, unused)
-                // (5b) DP_b -= Z_b' Z_b : A operand = [Z_a'; Z_b']
+                // (5) DP -= Z' Z : A operand rows 64..127 = Z' (rows 0..63 = X1, unused lanes)
                 if (issuer && !dead) {
                     tc_fence_after();
-                    gemm_ss(R2, smem_u32(X0) - MAT_BYTES, smem_u32(X0), 64, 1, true);
-                    gemm_ss(R3, smem_u32(X0), smem_u32(X0) + MAT_BYTES, 64, 1, true);
+                    gemm_ss(RF, smem_u32(X0) - MAT_BYTES, smem_u32(X0), 64, 1, true);
                     mma_commit(mbar);
                 }
                 if (dead)
                     break;
-                {
-                    const int x = warp >> 1, pw = warp & 1;
-                    unsigned char* Sm = X1 + x * MAT_BYTES;
-                    unsigned char* Ym = X0 + x * MAT_BYTES;
-                    if (ts == 0 && want_u0) {
-                        // u_0 = K_0 x_0 = -L^{-T} (Z x_0), fp32, by the 64 threads of the pair
-                        const int i = 32 * pw + lane;
-                        pair_barrier(wg, x);
-                        float zi = 0.f;
+                if (ts == 0 && want_u0 && warp < 2) {
+                    // u_0 = K_0 x_0 = -L^{-T} (Z x_0), fp32, by the 64 threads of warps 0, 1
+                    const int i = wt;
+                    half_barrier(wg);
+                    float zi = 0.f;
 #pragma unroll 8
-                        for (int c = 0; c < N; ++c)
-                            zi = fmaf(elem(Ym, toff(c, i)), misc.x0[x][c], zi);          // Z[i][c] = Z'[c][i]
-                        misc.y0[x][i] = zi;
+                    for (int c = 0; c < N; ++c)
+                        zi = fmaf(elem(X0, toff(c, i)), misc.x0[c], zi);               // Z[i][c] = Z'[c][i]
+                    misc.y0[i] = zi;
 #pragma unroll 1
-                        for (int kb = 7; kb >= 0; --kb) {       // back substitution L' w = Z x_0 in 8-wide blocks
-                            pair_barrier(wg, x);
-                            const int c0 = 8 * kb;
-                            float l[8][8], w[8];
+                    for (int kb = 7; kb >= 0; --kb) {           // back substitution L' w = Z x_0 in 8-wide blocks
+                        half_barrier(wg);
+                        const int c0 = 8 * kb;
+                        float l[8][8], w[8];
 #pragma unroll
-                            for (int r = 0; r < 8; ++r) {
-                                load_row8<true>(l[r], Sm + toff(c0, c0), r);
-                                w[r] = misc.y0[x][c0 + r];
-                            }
+                        for (int r = 0; r < 8; ++r) {
+                            load_row8<true>(l[r], X1 + toff(c0, c0), r);
+                            w[r] = misc.y0[c0 + r];
+                        }
 #pragma unroll
-                            for (int r = 7; r >= 0; --r) {
-                                float v = w[r];
+                        for (int r = 7; r >= 0; --r) {
+                            float vv = w[r];
 #pragma unroll
-                                for (int j = r + 1; j < 8; ++j)
-                                    v = fmaf(-l[j][r], w[j], v);
-                                w[r] = v / l[r][r];
-                            }
-                            if (i < c0) {
-#pragma unroll
-                                for (int r = 0; r < 8; ++r)
-                                    zi = fmaf(-elem(Sm, toff_rot(c0 + r, i)), w[r], zi);
-                            }
-                            pair_barrier(wg, x);
-                            if (i < c0)
-                                misc.y0[x][i] = zi;
+                            for (int j = r + 1; j < 8; ++j)
+                                vv = fmaf(-l[j][r], w[j], vv);
+                            w[r] = vv / l[r][r];
+                        }
+                        if (i < c0) {
 #pragma unroll
                             for (int r = 0; r < 8; ++r)
-                                if (i == c0 + r && (x == 0 || valid_b))
-                                    p.u[inst_x[x] * (long long)N + i] = -w[r];
+                                zi = fmaf(-elem(X1, toff_rot(c0 + r, i)), w[r], zi);
                         }
+                        half_barrier(wg);
+                        if (i < c0)
+                            misc.y0[i] = zi;
+#pragma unroll
+                        for (int r = 0; r < 8; ++r)
+                            if (i == c0 + r)
+                                p.u[inst * (long long)N + i] = -w[r];
                     }
                 }
-                // P_t = Q + DP: warps 2, 3 own the rows (lanes 64..127)
-                float q[64];
-                if (!need_K_all && warp >= 2)
-                    load_q_row(q, p.Q, oq_x[0], wt - 64);
                 wait_mma();
                 if (need_K_all) {
                     // (5) has consumed Z': turn it into the gains in place, K_t[i][c] = -(Z' L^{-1})[c][i]
-                    const int x = warp >> 1, pw = warp & 1;
-                    unsigned char* Ym = X0 + x * MAT_BYTES;
-                    pair_gain_solve(X1 + x * MAT_BYTES, Ym, wg, x, pw, lane);
-                    const int cidx = 32 * pw + lane;
-                    if (x == 0 || valid_b) {
-                        float* kt = Kbase + (inst_x[x] * (long long)H + ts) * N * N + cidx;
-                        const unsigned char* row = Ym + (uint32_t)(cidx >> 3) * SR + (uint32_t)(cidx & 7) * 16u;
+                    if (warp < 2) {
+                        pair_gain_solve(X1, X0, wg, warp, lane);
+                        const int cidx = wt;
+                        float* kt = Kbase + (inst * (long long)H + ts) * N * N + cidx;
+                        const unsigned char* row = X0 + (uint32_t)(cidx >> 3) * SR + (uint32_t)(cidx & 7) * 16u;
 #pragma unroll
                         for (int q4 = 0; q4 < 16; ++q4) {
-                            const float4 v = *reinterpret_cast<const float4*>(row + q4 * SC);
-                            kt[(4 * q4 + 0) * N] = -v.x;
-                            kt[(4 * q4 + 1) * N] = -v.y;
-                            kt[(4 * q4 + 2) * N] = -v.z;
-                            kt[(4 * q4 + 3) * N] = -v.w;
+                            const float4 kv = *reinterpret_cast<const float4*>(row + q4 * SC);
+                            kt[(4 * q4 + 0) * N] = -kv.x;
+                            kt[(4 * q4 + 1) * N] = -kv.y;
+                            kt[(4 * q4 + 2) * N] = -kv.z;
+                            kt[(4 * q4 + 3) * N] = -kv.w;
                         }
                     }
-                    wg_barrier(wg);                    // X0 is free for the next value matrices
-                    if (warp >= 2)
-                        load_q_row(q, p.Q, oq_x[0], wt - 64);
+                    wg_barrier(wg);                   // X0 is free for the next value matrix
                 }
+                // P_t = Q + DP: warps 2, 3 own the rows (lanes 64..127)
                 if (warp >= 2) {
                     const int j = wt - 64;
 #pragma unroll 1
-                    for (int x = 0; x < 2; ++x) {
-                        if (x == 1)
-                            load_q_row(q, p.Q, oq_x[1], j);
-                        float h0[32], h1[32];
-                        const uint32_t src = (x == 0 ? R2 : R3) + lane_sel;
-                        tmem_ld32(src, h0);
-                        tmem_ld32(src + 32, h1);
+                    for (int half = 0; half < 2; ++half) {
+                        float q[32], hh[32];
+                        load_q_half(q, p.Q, oq, j, half);
+                        tmem_ld32(RF + lane_sel + 32 * half, hh);
 #pragma unroll
-                        for (int c = 0; c < 32; ++c) {
-                            q[c] += h0[c];
-                            q[32 + c] += h1[c];
-                        }
+                        for (int c = 0; c < 32; ++c)
+                            q[c] += hh[c];
                         if (ts > 0)
-                            store_row_tf32(X0, 64 * x + j, q);
-                        if (p.P && (x == 0 || valid_b) && (!p.first_only || ts == 0))
-                            store_row_global(p.P + (inst_x[x] * (long long)(p.first_only ? 1 : H + 1) + (p.first_only ? 0 : ts)) * N * N +
-                                                 (long long)j * N, q);
+                            store_half_tf32(X0, j, half, q);
+                        if (p.P && (!p.first_only || ts == 0))
+                            store_half_global(p.P + (inst * (long long)(p.first_only ? 1 : H + 1) + (p.first_only ? 0 : ts)) * N * N +
+                                                  (long long)j * N + 32 * half, q);
                     }
                 }
                 tc_fence_before();
@@ -819,17 +802,16 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
             }
             if (dead)
                 break;
-            if (rollout) {
-                // forward loop of Alg. 1 by the 64 threads of each instance: u_t = K_t x_t, x_{t+1} = A x_t + B u_t (fp32)
-                const int x = warp >> 1, i = 32 * (warp & 1) + lane;
-                const bool st = (x == 0 || valid_b) && misc.flag[x] == 0;
-                const long long inst = inst_x[x];
+            if (rollout && warp < 2) {
+                // forward loop of Alg. 1 by 64 threads: u_t = K_t x_t, x_{t+1} = A x_t + B u_t (fp32)
+                const int i = wt;
+                const bool st = misc.flag == 0;
                 float* xo = (p.x && st) ? p.x + inst * (long long)(H + 1) * N : nullptr;
                 float* uo = (p.u && st) ? p.u + inst * (long long)(p.first_only ? 1 : H) * N : nullptr;
                 const float4* Ar = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(p.A.ptr) + offA_loaded + (long long)i * N);
                 const float4* Br = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(p.B.ptr) + offB_loaded + (long long)i * N);
                 if (xo)
-                    xo[i] = misc.x0[x][i];
+                    xo[i] = misc.x0[i];
 #pragma unroll 1
                 for (int ts = 0; ts < H; ++ts) {
                     const float4* kr = reinterpret_cast<const float4*>(Kbase + (inst * (long long)H + ts) * N * N + (long long)i * N);
@@ -837,37 +819,37 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
 #pragma unroll
                     for (int c4 = 0; c4 < 16; ++c4) {
                         const float4 kv = kr[c4];
-                        const float4 xv = *reinterpret_cast<const float4*>(&misc.x0[x][4 * c4]);
+                        const float4 xv = *reinterpret_cast<const float4*>(&misc.x0[4 * c4]);
                         ui = fmaf(kv.x, xv.x, fmaf(kv.y, xv.y, fmaf(kv.z, xv.z, fmaf(kv.w, xv.w, ui))));
                     }
-                    misc.y0[x][i] = ui;
+                    misc.y0[i] = ui;
                     if (uo && (!p.first_only || ts == 0))
                         uo[(p.first_only ? 0 : (long long)ts * N) + i] = ui;
-                    pair_barrier(wg, x);
+                    half_barrier(wg);
                     float xi = 0.f;
 #pragma unroll
                     for (int c4 = 0; c4 < 16; ++c4) {
                         const float4 av = __ldg(Ar + c4), bv = __ldg(Br + c4);
-                        const float4 xv = *reinterpret_cast<const float4*>(&misc.x0[x][4 * c4]);
-                        const float4 uv = *reinterpret_cast<const float4*>(&misc.y0[x][4 * c4]);
+                        const float4 xv = *reinterpret_cast<const float4*>(&misc.x0[4 * c4]);
+                        const float4 uv = *reinterpret_cast<const float4*>(&misc.y0[4 * c4]);
                         xi = fmaf(av.x, xv.x, fmaf(av.y, xv.y, fmaf(av.z, xv.z, fmaf(av.w, xv.w, xi))));
                         xi = fmaf(bv.x, uv.x, fmaf(bv.y, uv.y, fmaf(bv.z, uv.z, fmaf(bv.w, uv.w, xi))));
                     }
-                    pair_barrier(wg, x);               // x_t and u_t consumed
-                    misc.x0[x][i] = xi;
+                    half_barrier(wg);               // x_t and u_t consumed
+                    misc.x0[i] = xi;
                     if (xo)
                         xo[(long long)(ts + 1) * N + i] = xi;
-                    pair_barrier(wg, x);
+                    half_barrier(wg);
                 }
             }
-            // ---- status / failed instances
-#pragma unroll 1
-            for (int x = 0; x < (valid_b ? 2 : 1); ++x) {
-                const int fl = misc.flag[x];
+            wg_barrier(wg);
+            // ---- status / failed instance
+            {
+                const int fl = misc.flag;
                 if (fl)
-                    wg_fail_instance(p, inst_x[x], fl, wt);
+                    wg_fail_instance(p, inst, fl, wt);
                 else if (p.info && wt == 0)
-                    p.info[inst_x[x]] = 0;
+                    p.info[inst] = 0;
             }
             wg_barrier(wg);
         }
@@ -875,8 +857,7 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
     tc_fence_before();
     __syncthreads();
     if (tid < 32)
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(*tmem_slot), "r"(512) : "memory");
-    (void)offR_loaded;
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(cta.tmem_base), "r"(512) : "memory");
 }
 
 inline size_t smem_bytes() { return SMEM_BYTES; }

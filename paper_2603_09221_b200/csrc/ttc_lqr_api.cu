@@ -11,7 +11,6 @@
 #include "common.cuh"
 #include "riccati_cta.cuh"
 #include "riccati_umma64.cuh"
-#include "riccati_umma64q.cuh"
 #include "riccati_warp.cuh"
 #include "ttc_layer.cuh"
 #include "scan_pair.cuh"
@@ -358,13 +357,13 @@ int solve_window(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, 
             if ((s = ensure(h->ws_E, sizeof(int) * 4))) return s;
             int* counter = static_cast<int*>(h->ws_E.ptr);
             TTC_CUDA(cudaMemsetAsync(counter, 0, 2 * sizeof(int), st));
-            const size_t smem = umma64::smem4_bytes();
-            auto kern = rollout_needs_all_K || K ? umma64::riccati_umma64q_kernel<true> : umma64::riccati_umma64q_kernel<false>;
+            const size_t smem = umma64::smem_bytes();
+            auto kern = rollout_needs_all_K || K ? umma64::riccati_umma64_kernel<true> : umma64::riccati_umma64_kernel<false>;
             TTC_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            const long long chunks = p.b0 * p.b1 * ((tcount + umma64::CHUNK4 - 1) / umma64::CHUNK4);
+            const long long chunks = p.b0 * p.b1 * ((tcount + umma64::CHUNK - 1) / umma64::CHUNK);
             long long grid = h->sm_count;
             if (grid > chunks) grid = chunks;
-            kern<<<(unsigned)grid, umma64::THREADS4, smem, st>>>(p, counter, counter + 1);
+            kern<<<(unsigned)grid, umma64::THREADS, smem, st>>>(p, counter, counter + 1);
             TTC_CUDA(cudaGetLastError());
             h->last_launches += 1;
             h->total_launches += 1;
