@@ -171,6 +171,7 @@ __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.
 
 // named barriers: 1 + wg = warps 0, 1 of a warpgroup (64 threads), 5 + wg = the whole warpgroup
 __device__ __forceinline__ void half_barrier(int wg) { asm volatile("bar.sync %0, %1;" :: "r"(1 + wg), "r"(64) : "memory"); }
+__device__ __forceinline__ void wg_barrier(int wg) { asm volatile("bar.sync %0, %1;" :: "r"(5 + wg), "r"(WG_THREADS) : "memory"); }
 
 // ---- blocked Cholesky of S fused with the forward substitution Z' = Y' L^{-T} --------------------------------------
 __device__ __forceinline__ void mma_16x8x8(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
@@ -251,43 +252,46 @@ __device__ __forceinline__ void store_row8(unsigned char* grp, int slot, const f
     *reinterpret_cast<float4*>(grp + SC + (ROT ? ((slot + 4) & 7) : slot) * 16) = b;
 }
 
-// Gains (Eq. 4): K = -L^{-T} Z, i.e. row c of K' is -(row c of Z') L^{-1}.  Warps 0, 1 of the warpgroup (pw = 0, 1) run
-// a blocked scheme backwards on L (fp32, rotated layout, at `Sm`) and Z' (at `Ym`): per 8-wide block kb = 7..0 every row owner solves x L_d = z for its row of Z' (in place in
-// `Ym`), then the columns left of the block get the update Z'[c][j] -= x[c][kb] . L[kb][j] as 3 x tf32 mma.
-// On return row c of Ym holds (Z' L^{-1})[c][:] = -K[:, c] (fp32).
-__device__ __forceinline__ void pair_gain_solve(const unsigned char* Sm, unsigned char* Ym, int wg, int pw, int lane)
+// Gains (Eq. 4): K = -L^{-T} Z, i.e. row c of K' is -(row c of Z') L^{-1}.  The four warps of the warpgroup run a
+// blocked scheme backwards on L (fp32, rotated layout, at `Sm`) and Z' (at `Ym`): per 8-wide block kb = 7..0 the
+// owner of row c (threads 0..63) solves x L_d = z for its row of Z' (in place in `Ym`), then the columns left of the
+// block get the update Z'[c][j] -= x[c][kb] . L[kb][j] as 3 x tf32 mma, one 16-row tile per warp.
+// On return row c of Ym holds (Z' L^{-1})[c][:] = -K[:, c] (fp32).  Ends with a warpgroup barrier.
+__device__ __forceinline__ void wg_gain_solve(const unsigned char* Sm, unsigned char* Ym, int wg, int warp, int lane)
 {
     const int g = lane >> 2, t = lane & 3;
-    const int tid2 = 32 * pw + lane;
+    const int wt = 32 * warp + lane;
     const uint32_t frag_ab = (uint32_t)g * 16u + (uint32_t)t * 4u;
     const uint32_t frag_c = (uint32_t)g * 16u + (uint32_t)(t >> 1) * SC + (uint32_t)((2 * t) & 3) * 4u;
     // (row t, col g) and (row t + 4, col g) of a tile of L (rotated layout: the chunk parity is g >> 2)
     const uint32_t frag_b = (uint32_t)((t + 4 * (g >> 2)) & 7) * 16u + (uint32_t)(g >> 2) * SC + (uint32_t)(g & 3) * 4u;
     const uint32_t frag_b4 = (uint32_t)((t + 4 + 4 * (g >> 2)) & 7) * 16u + (uint32_t)(g >> 2) * SC + (uint32_t)(g & 3) * 4u;
-    const uint32_t own_grp = (uint32_t)(tid2 >> 3) * SR;
-    const int own_slot = tid2 & 7;
+    const uint32_t own_grp = (uint32_t)((wt & 63) >> 3) * SR;
+    const int own_slot = wt & 7;
 #pragma unroll 1
     for (int kb = 7; kb >= 0; --kb) {
         const uint32_t kcol = 2u * kb * SC;
-        const unsigned char* dblk = Sm + (uint32_t)kb * SR + kcol;
-        float l[8][8], xr[8];
+        if (warp < 2) {
+            const unsigned char* dblk = Sm + (uint32_t)kb * SR + kcol;
+            float l[8][8], xr[8];
 #pragma unroll
-        for (int i = 0; i < 8; ++i)
-            load_row8<true>(l[i], dblk, i);
-        unsigned char* py = Ym + own_grp + kcol;
-        load_row8<false>(xr, py, own_slot);
+            for (int i = 0; i < 8; ++i)
+                load_row8<true>(l[i], dblk, i);
+            unsigned char* py = Ym + own_grp + kcol;
+            load_row8<false>(xr, py, own_slot);
 #pragma unroll
-        for (int j = 7; j >= 0; --j) {                 // x L_d = z, L_d lower triangular
-            float v = xr[j];
+            for (int j = 7; j >= 0; --j) {                 // x L_d = z, L_d lower triangular
+                float v = xr[j];
 #pragma unroll
-            for (int i = j + 1; i < 8; ++i)
-                v = fmaf(-xr[i], l[i][j], v);
-            xr[j] = __fdividef(v, l[j][j]);
+                for (int i = j + 1; i < 8; ++i)
+                    v = fmaf(-xr[i], l[i][j], v);
+                xr[j] = __fdividef(v, l[j][j]);
+            }
+            store_row8<false, false>(py, own_slot, xr);
         }
-        store_row8<false, false>(py, own_slot, xr);
+        wg_barrier(wg);
         if (kb == 0)
             break;
-        half_barrier(wg);
         // B fragments: rows 8kb + t, 8kb + t + 4 of L, columns 8j + g (j < kb)
         uint32_t bh[7][2], bl[7][2];
         {
@@ -299,9 +303,8 @@ __device__ __forceinline__ void pair_gain_solve(const unsigned char* Sm, unsigne
                     split_tf32(*reinterpret_cast<const float*>(pb + 2 * j * SC + frag_b4), bh[j][1], bl[j][1]);
                 }
         }
-#pragma unroll
-        for (int uu = 0; uu < 2; ++uu) {
-            const int mt = 2 * uu + pw;
+        {
+            const int mt = warp;                           // rows 16 mt .. 16 mt + 15 of Z'
             uint32_t ah[4], al[4];
             {
                 const unsigned char* pa = Ym + frag_ab + kcol + 2 * mt * SR;
@@ -340,7 +343,7 @@ __device__ __forceinline__ void pair_gain_solve(const unsigned char* Sm, unsigne
                 *reinterpret_cast<float2*>(pc + 2 * j * SC + SR) = make_float2(acc[j][2], acc[j][3]);
             }
         }
-        half_barrier(wg);
+        wg_barrier(wg);
     }
 }
 
@@ -396,7 +399,6 @@ struct CtaShared {
 constexpr uint32_t SMEM_BYTES = BUF_BYTES + NUM_WG * WG_BYTES + 128;
 static_assert(SMEM_BYTES <= 227 * 1024, "shared memory of one CTA");
 
-__device__ __forceinline__ void wg_barrier(int wg) { asm volatile("bar.sync %0, %1;" :: "r"(5 + wg), "r"(WG_THREADS) : "memory"); }
 
 // half a row (32 values) of the Q matrix of one instance
 __device__ __forceinline__ void load_q_half(float (&q)[32], const OperandDev& Q, long long oq, int j, int half)
@@ -488,7 +490,6 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
     const long long nchunks = p.b0 * p.b1 * chunks_per_head;
     constexpr bool need_K_all = GAINS;
     const bool want_u0 = (p.u != nullptr) && p.first_only && !need_K_all;
-    const bool rollout = (p.x != nullptr) || (p.u != nullptr && need_K_all);
     float* Kbase = p.K ? p.K : p.Kws;
     long long offA_loaded = -1, offB_loaded = -1;
     const float* Rg = nullptr;
@@ -761,8 +762,8 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
                 wait_mma();
                 if (need_K_all) {
                     // (5) has consumed Z': turn it into the gains in place, K_t[i][c] = -(Z' L^{-1})[c][i]
+                    wg_gain_solve(X1, X0, wg, warp, lane);
                     if (warp < 2) {
-                        pair_gain_solve(X1, X0, wg, warp, lane);
                         const int cidx = wt;
                         float* kt = Kbase + (inst * (long long)H + ts) * N * N + cidx;
                         const unsigned char* row = X0 + (uint32_t)(cidx >> 3) * SR + (uint32_t)(cidx & 7) * 16u;
@@ -802,52 +803,15 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
             }
             if (dead)
                 break;
-            if (rollout && warp < 2) {
-                // forward loop of Alg. 1 by 64 threads: u_t = K_t x_t, x_{t+1} = A x_t + B u_t (fp32)
-                const int i = wt;
-                const bool st = misc.flag == 0;
-                float* xo = (p.x && st) ? p.x + inst * (long long)(H + 1) * N : nullptr;
-                float* uo = (p.u && st) ? p.u + inst * (long long)(p.first_only ? 1 : H) * N : nullptr;
-                const float4* Ar = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(p.A.ptr) + offA_loaded + (long long)i * N);
-                const float4* Br = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(p.B.ptr) + offB_loaded + (long long)i * N);
-                if (xo)
-                    xo[i] = misc.x0[i];
-#pragma unroll 1
-                for (int ts = 0; ts < H; ++ts) {
-                    const float4* kr = reinterpret_cast<const float4*>(Kbase + (inst * (long long)H + ts) * N * N + (long long)i * N);
-                    float ui = 0.f;
-#pragma unroll
-                    for (int c4 = 0; c4 < 16; ++c4) {
-                        const float4 kv = kr[c4];
-                        const float4 xv = *reinterpret_cast<const float4*>(&misc.x0[4 * c4]);
-                        ui = fmaf(kv.x, xv.x, fmaf(kv.y, xv.y, fmaf(kv.z, xv.z, fmaf(kv.w, xv.w, ui))));
-                    }
-                    misc.y0[i] = ui;
-                    if (uo && (!p.first_only || ts == 0))
-                        uo[(p.first_only ? 0 : (long long)ts * N) + i] = ui;
-                    half_barrier(wg);
-                    float xi = 0.f;
-#pragma unroll
-                    for (int c4 = 0; c4 < 16; ++c4) {
-                        const float4 av = __ldg(Ar + c4), bv = __ldg(Br + c4);
-                        const float4 xv = *reinterpret_cast<const float4*>(&misc.x0[4 * c4]);
-                        const float4 uv = *reinterpret_cast<const float4*>(&misc.y0[4 * c4]);
-                        xi = fmaf(av.x, xv.x, fmaf(av.y, xv.y, fmaf(av.z, xv.z, fmaf(av.w, xv.w, xi))));
-                        xi = fmaf(bv.x, uv.x, fmaf(bv.y, uv.y, fmaf(bv.z, uv.z, fmaf(bv.w, uv.w, xi))));
-                    }
-                    half_barrier(wg);               // x_t and u_t consumed
-                    misc.x0[i] = xi;
-                    if (xo)
-                        xo[(long long)(ts + 1) * N + i] = xi;
-                    half_barrier(wg);
-                }
-            }
             wg_barrier(wg);
             // ---- status / failed instance
             {
                 const int fl = misc.flag;
-                if (fl)
+                if (fl) {
                     wg_fail_instance(p, inst, fl, wt);
+                    if (need_K_all && wt == 0)               // the rollout kernel skips instances whose first gain is NaN
+                        Kbase[inst * (long long)H * N * N] = quiet_nan();
+                }
                 else if (p.info && wt == 0)
                     p.info[inst] = 0;
             }
@@ -859,6 +823,110 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
     if (tid < 32)
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(cta.tmem_base), "r"(512) : "memory");
 }
+
+// ---- forward loop of Alg. 1 for n = m = 64: u_t = K_t x_t, x_{t+1} = A x_t + B u_t (fp32) ---------------------------
+// Separate kernel, launched after the backward pass: one warp per instance, 8 warps per CTA on consecutive tokens of
+// one head (A, B of the head in shared memory).  K_t (16 KB per step and instance) is streamed from memory exactly
+// once with fully coalesced 16-byte loads: lanes 0..15 and 16..31 each take one row per load and the 16 partial dot
+// products are reduced with shuffles.  Instances whose first gain is NaN (failed in the backward pass, outputs
+// already filled with NaN) are skipped.
+constexpr int ROLL_WARPS = 8;
+constexpr int ROLL_LD = N + 4;
+struct RollSmem {
+    float A[N * ROLL_LD], B[N * ROLL_LD];
+    float x[ROLL_WARPS][N], u[ROLL_WARPS][N];
+};
+__global__ void __launch_bounds__(32 * ROLL_WARPS, 5) rollout64_kernel(SolveParams p, const float* Kall)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    RollSmem& sm = *reinterpret_cast<RollSmem*>(smem_raw);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int H = p.H;
+    const long long chunks_per_head = (p.tcount + ROLL_WARPS - 1) / ROLL_WARPS;
+    const long long nchunks = p.b0 * p.b1 * chunks_per_head;
+    long long offA = -1, offB = -1;
+    for (long long chunk = blockIdx.x; chunk < nchunks; chunk += gridDim.x) {
+        const long long head = chunk / chunks_per_head;
+        const long long tok0 = p.t0 + (chunk % chunks_per_head) * ROLL_WARPS;
+        const long long inst0 = head * p.b2 + tok0;
+        const int ntok = (int)min((long long)ROLL_WARPS, p.t0 + p.tcount - tok0);
+        const long long oa = operand_offset(p.A, inst0, p.b1, p.b2), ob = operand_offset(p.B, inst0, p.b1, p.b2);
+        __syncthreads();
+        if (oa != offA || ob != offB) {
+            const float* Ag = reinterpret_cast<const float*>(p.A.ptr) + oa;
+            const float* Bg = reinterpret_cast<const float*>(p.B.ptr) + ob;
+            for (int e = threadIdx.x; e < N * N; e += 32 * ROLL_WARPS) {
+                sm.A[(e >> 6) * ROLL_LD + (e & 63)] = __ldg(Ag + e);
+                sm.B[(e >> 6) * ROLL_LD + (e & 63)] = __ldg(Bg + e);
+            }
+            offA = oa; offB = ob;
+        }
+        __syncthreads();
+        if (warp >= ntok)
+            continue;
+        const long long inst = inst0 + warp;
+        const float* Ki = Kall + inst * (long long)H * N * N;
+        if (isnan(__ldg(Ki)))
+            continue;
+        float* xs = sm.x[warp];
+        float* us = sm.u[warp];
+        float* xo = p.x ? p.x + inst * (long long)(H + 1) * N : nullptr;
+        float* uo = p.u ? p.u + inst * (long long)(p.first_only ? 1 : H) * N : nullptr;
+        {
+            const long long ox = operand_offset(p.x0, inst, p.b1, p.b2);
+            const float a = load_elem(p.x0, ox + lane), b = load_elem(p.x0, ox + lane + 32);
+            xs[lane] = a; xs[lane + 32] = b;
+            if (xo) { xo[lane] = a; xo[lane + 32] = b; }
+        }
+        __syncwarp();
+        const int half = lane >> 4, seg = lane & 15;
+#pragma unroll 1
+        for (int ts = 0; ts < H; ++ts) {
+            const float4 x4 = *reinterpret_cast<const float4*>(xs + 4 * seg);
+            const float4* Kt = reinterpret_cast<const float4*>(Ki + (long long)ts * N * N) + lane;     // row (lane >> 4), segment (lane & 15)
+#pragma unroll 8
+            for (int it = 0; it < 32; ++it) {                 // rows 2 it, 2 it + 1
+                const float4 k4 = __ldcs(Kt + 32 * it);
+                float s = fmaf(k4.x, x4.x, fmaf(k4.y, x4.y, fmaf(k4.z, x4.z, k4.w * x4.w)));
+                s += __shfl_xor_sync(0xffffffffu, s, 8);
+                s += __shfl_xor_sync(0xffffffffu, s, 4);
+                s += __shfl_xor_sync(0xffffffffu, s, 2);
+                s += __shfl_xor_sync(0xffffffffu, s, 1);
+                if (seg == 0)
+                    us[2 * it + half] = s;
+            }
+            __syncwarp();
+            if (uo && (!p.first_only || ts == 0)) {
+                float* ut = uo + (p.first_only ? 0 : (long long)ts * N);
+                ut[lane] = us[lane];
+                ut[lane + 32] = us[lane + 32];
+            }
+            float n0 = 0.f, n1 = 0.f;                         // rows lane and lane + 32 of A x + B u
+#pragma unroll
+            for (int c4 = 0; c4 < 16; ++c4) {
+                const float4 xv = *reinterpret_cast<const float4*>(xs + 4 * c4);
+                const float4 uv = *reinterpret_cast<const float4*>(us + 4 * c4);
+                const float4 a0 = *reinterpret_cast<const float4*>(sm.A + lane * ROLL_LD + 4 * c4);
+                const float4 a1 = *reinterpret_cast<const float4*>(sm.A + (lane + 32) * ROLL_LD + 4 * c4);
+                const float4 b0 = *reinterpret_cast<const float4*>(sm.B + lane * ROLL_LD + 4 * c4);
+                const float4 b1 = *reinterpret_cast<const float4*>(sm.B + (lane + 32) * ROLL_LD + 4 * c4);
+                n0 = fmaf(a0.x, xv.x, fmaf(a0.y, xv.y, fmaf(a0.z, xv.z, fmaf(a0.w, xv.w, n0))));
+                n0 = fmaf(b0.x, uv.x, fmaf(b0.y, uv.y, fmaf(b0.z, uv.z, fmaf(b0.w, uv.w, n0))));
+                n1 = fmaf(a1.x, xv.x, fmaf(a1.y, xv.y, fmaf(a1.z, xv.z, fmaf(a1.w, xv.w, n1))));
+                n1 = fmaf(b1.x, uv.x, fmaf(b1.y, uv.y, fmaf(b1.z, uv.z, fmaf(b1.w, uv.w, n1))));
+            }
+            __syncwarp();                                     // x_t and u_t consumed
+            xs[lane] = n0;
+            xs[lane + 32] = n1;
+            if (xo) {
+                xo[(long long)(ts + 1) * N + lane] = n0;
+                xo[(long long)(ts + 1) * N + lane + 32] = n1;
+            }
+            __syncwarp();
+        }
+    }
+}
+inline size_t rollout_smem_bytes() { return sizeof(RollSmem); }
 
 inline size_t smem_bytes() { return SMEM_BYTES; }
 

@@ -367,6 +367,18 @@ int solve_window(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, 
             TTC_CUDA(cudaGetLastError());
             h->last_launches += 1;
             h->total_launches += 1;
+            if (rollout_needs_all_K) {
+                // forward loop of Alg. 1 as a second, bandwidth-bound kernel: it streams every K_t once
+                const size_t rsmem = umma64::rollout_smem_bytes();
+                TTC_CUDA(cudaFuncSetAttribute(umma64::rollout64_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rsmem));
+                const long long rchunks = p.b0 * p.b1 * ((tcount + umma64::ROLL_WARPS - 1) / umma64::ROLL_WARPS);
+                long long rgrid = (long long)h->sm_count * 5;
+                if (rgrid > rchunks) rgrid = rchunks;
+                umma64::rollout64_kernel<<<(unsigned)rgrid, 32 * umma64::ROLL_WARPS, rsmem, st>>>(p, K ? K : p.Kws);
+                TTC_CUDA(cudaGetLastError());
+                h->last_launches += 1;
+                h->total_launches += 1;
+            }
             h->last_kernel = TTC_KERNEL_RICCATI_UMMA;
             return TTC_OK;
         }

@@ -147,7 +147,8 @@ def test_full_size_configuration_on_sampled_instances(cfg, expect):
     checks a stratified sample of instances (every sequence and head) one by one."""
     w = workloads.make_workload(cfg, device=DEV)
     gpu = pu.run_gpu(w)
-    assert lqr.KERNEL_NAMES[gpu["kernel"]] == expect and gpu["launches"] == 1
+    # one launch; the n = 64 path adds its streaming rollout kernel when x (or every u_t) is requested, as here
+    assert lqr.KERNEL_NAMES[gpu["kernel"]] == expect and gpu["launches"] == (2 if expect == "riccati_umma" else 1)
     S, Hd, T = w["batch"]
     toks = np.array([0, 1, T // 3, T - 2, T - 1])
     idx = (np.arange(S * Hd)[:, None] * T + toks[None, :]).reshape(-1)
