@@ -396,7 +396,9 @@ struct CtaShared {
     int dead;                    // some warpgroup gave up: the CTA stops taking work
     uint32_t tmem_base;
 };
-constexpr uint32_t SMEM_BYTES = BUF_BYTES + NUM_WG * WG_BYTES + 128;
+constexpr int R_LD = N + 4;                                // row stride of R in shared memory (conflict-free row owners)
+constexpr uint32_t R_BYTES = N * R_LD * 4;
+constexpr uint32_t SMEM_BYTES = BUF_BYTES + R_BYTES + NUM_WG * WG_BYTES + 128;
 static_assert(SMEM_BYTES <= 227 * 1024, "shared memory of one CTA");
 
 
@@ -450,13 +452,14 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
     const int warp = wt >> 5;                  // warp in warpgroup: owns tensor-memory lanes 32 warp .. 32 warp + 31
     const int lane = wt & 31;
     unsigned char* BA = smem_raw;              // rows 0..63: B' (row j = column j of B), rows 64..127: A'; shared by the CTA
-    unsigned char* wsm = smem_raw + BUF_BYTES + (size_t)wg * WG_BYTES;
+    float* Rs = reinterpret_cast<float*>(smem_raw + BUF_BYTES);   // R of the head, fp32, shared by the CTA
+    unsigned char* wsm = smem_raw + BUF_BYTES + R_BYTES + (size_t)wg * WG_BYTES;
     unsigned char* X1 = wsm + OFF_X1;        // L, fp32 (kept only when the gains or u_0 need it)
     unsigned char* X0 = wsm + OFF_X0;        // P -> Z' -> next P
     unsigned char* PH = wsm + OFF_PH;        // panel operand, hi parts (128 x 8)
     unsigned char* PL = wsm + OFF_PL;        // panel operand, lo parts
     Misc& misc = *reinterpret_cast<Misc*>(wsm + OFF_MISC);
-    CtaShared& cta = *reinterpret_cast<CtaShared*>(smem_raw + BUF_BYTES + (size_t)NUM_WG * WG_BYTES);
+    CtaShared& cta = *reinterpret_cast<CtaShared*>(smem_raw + BUF_BYTES + R_BYTES + (size_t)NUM_WG * WG_BYTES);
     const uint32_t mbar = smem_u32(&misc.mbar);
     const uint32_t mbar_w = smem_u32(&misc.mbar_w);
 
@@ -491,8 +494,7 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
     constexpr bool need_K_all = GAINS;
     const bool want_u0 = (p.u != nullptr) && p.first_only && !need_K_all;
     float* Kbase = p.K ? p.K : p.Kws;
-    long long offA_loaded = -1, offB_loaded = -1;
-    const float* Rg = nullptr;
+    long long offA_loaded = -1, offB_loaded = -1, offR_loaded = -1;
     bool dead = false;
 
     auto wait_mma = [&]() {
@@ -521,19 +523,21 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
         {
             const long long oa = operand_offset(p.A, inst0, p.b1, p.b2);
             const long long ob = operand_offset(p.B, inst0, p.b1, p.b2);
-            if (oa != offA_loaded || ob != offB_loaded) {
+            const long long orr = operand_offset(p.R, inst0, p.b1, p.b2);
+            if (oa != offA_loaded || ob != offB_loaded || orr != offR_loaded) {
                 const float* Ag = reinterpret_cast<const float*>(p.A.ptr) + oa;
                 const float* Bg = reinterpret_cast<const float*>(p.B.ptr) + ob;
+                const float* Rg = reinterpret_cast<const float*>(p.R.ptr) + orr;
                 for (int e = tid; e < N * N; e += THREADS) {
                     const int k = e >> 6, j = e & 63;
                     elem(BA, toff(j, k)) = round_tf32(__ldg(Bg + e));
                     elem(BA, toff(64 + j, k)) = round_tf32(__ldg(Ag + e));
+                    Rs[k * R_LD + j] = __ldg(Rg + e);
                 }
-                offA_loaded = oa; offB_loaded = ob;
+                offA_loaded = oa; offB_loaded = ob; offR_loaded = orr;
                 async_proxy_fence();
                 __syncthreads();
             }
-            Rg = reinterpret_cast<const float*>(p.R.ptr) + operand_offset(p.R, inst0, p.b1, p.b2);
         }
         const int my0 = TOK * wg, my1 = min(ntok, TOK * wg + TOK);
 
@@ -589,8 +593,8 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
                     tmem_ld8(RF + lane_sel + c0, raw);
                     float4 r0 = make_float4(0.f, 0.f, 0.f, 0.f), r1 = r0;
                     if (warp < 2) {
-                        r0 = __ldg(reinterpret_cast<const float4*>(Rg + (long long)wt * N + c0));
-                        r1 = __ldg(reinterpret_cast<const float4*>(Rg + (long long)wt * N + c0 + 4));
+                        r0 = *reinterpret_cast<const float4*>(Rs + wt * R_LD + c0);
+                        r1 = *reinterpret_cast<const float4*>(Rs + wt * R_LD + c0 + 4);
                     }
                     tmem_wait_ld();
                     v[0] = __uint_as_float(raw[0]) + r0.x; v[1] = __uint_as_float(raw[1]) + r0.y;
