@@ -842,7 +842,7 @@ struct RollSmem {
 };
 __global__ void __launch_bounds__(32 * ROLL_WARPS, 5) rollout64_kernel(SolveParams p, const float* Kall)
 {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
     RollSmem& sm = *reinterpret_cast<RollSmem*>(smem_raw);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int H = p.H;
