@@ -218,3 +218,21 @@ def test_host_buffer_entry_point_pipelined_slices(n, H, batch, bf16):
         assert torch.equal(out[k], gpu[k].cpu()), k
     ref = pu.run_oracle(w, idx=np.arange(0, N, max(1, N // 64)))
     pu.compare({k: out[k] for k in ("K", "P", "x", "u")}, ref, np.arange(0, N, max(1, N // 64)), w["tol"])
+
+
+@pytest.mark.parametrize("tokens", [13, 33, 71])
+def test_tensor_core_kernel_ragged_work_items(tokens):
+    """n = m = 64 on the tcgen05 kernel with token counts that leave warpgroups of a work item partly or wholly idle
+    (work items are 32 tokens of one head, 8 per warpgroup) and several heads per CTA; tighter bound than the
+    configuration tolerance so that an ordering or staging mistake cannot hide behind it."""
+    w = small_workload(64, 64, 5, (2, 3, tokens), seed=4242 + tokens, bf16=True)
+    N = 2 * 3 * tokens
+    ref = pu.run_oracle(w, first_only=False)
+    g = pu.run_gpu(w, want=("K", "P", "x", "u", "info"), first_only=False)
+    assert lqr.KERNEL_NAMES[g["kernel"]] == "riccati_umma" and g["launches"] == 2
+    errs = pu.compare(g, ref, np.arange(N), 5e-3)
+    g1 = pu.run_gpu(w, want=("P", "u", "info"), first_only=True)
+    assert g1["launches"] == 1
+    ref1 = pu.run_oracle(w, first_only=True)
+    errs1 = pu.compare(g1, ref1, np.arange(N), 1e-2)
+    print("ragged", tokens, errs, errs1)
