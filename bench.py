@@ -189,6 +189,12 @@ def run_layer(args):
     """--workload layer16 / layer32: one step = one ttc_lqr_solve_layer over the whole workload."""
     key = args.workload
     c = dict(workloads.LAYER_CONFIGS[key])
+    if args.horizon > 0:
+        c["T"] = args.horizon
+        c["name"] += "_T%d" % args.horizon
+    if args.batch:
+        c["batch"] = tuple(int(v) for v in args.batch.split("x"))
+        c["name"] += "_batch" + args.batch
     rank = int(os.environ.get("RANK", "0"))
     if args.impl == "reference":
         if rank != 0:
@@ -345,6 +351,8 @@ def main():
     ap.add_argument("--cpu-sample", type=int, default=256, help="instances the oracle is timed on")
     ap.add_argument("--ref-instances", type=int, default=256)
     ap.add_argument("--tokens", type=int, default=0, help="override the token count (small profiling captures)")
+    ap.add_argument("--horizon", type=int, default=0, help="layer workloads: override the planning horizon T (sweeps)")
+    ap.add_argument("--batch", default="", help="layer workloads: override the batch as SxHxT, e.g. 1x16x64 (sweeps)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
