@@ -532,6 +532,12 @@ static int launch_layer(ttc_lqr_handle* h, const ttc_layer_inputs* in, int32_t T
         smem = layer::smem_bytes<32>();
         chunks = (p.N + rwarp::Shape<32>::SLOTS - 1) / rwarp::Shape<32>::SLOTS;
         grid = (long long)h->sm_count * 3;
+    } else if (p.N <= (long long)h->sm_count * 2 * rwarp::Shape<16>::SLOTS) {
+        // the machine is less than half full: 16 lanes per instance walk the chain faster than 8 lanes with two columns each
+        kern = layer::ttc_layer_kernel<16>;
+        smem = layer::smem_bytes<16>();
+        chunks = (p.N + rwarp::Shape<16>::SLOTS - 1) / rwarp::Shape<16>::SLOTS;
+        grid = (long long)h->sm_count * 4;
     } else {
         kern = layer::ttc_layer_kernel_c2<16>;
         smem = layer::smem_bytes_c2<16>();
