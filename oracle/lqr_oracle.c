@@ -292,3 +292,121 @@ int lqr_oracle_solve_batch(int64_t N, int n, int m, int H,
     return lqr_oracle_solve_batch_tv(N, n, m, H, A, offA, 0, B, offB, 0, Q, offQ, 0, R, offR, 0, Q, offQ,
                                      x0, offx, K, P, x, u, info, first_only, nthreads);
 }
+
+/*
+ * Affine control cost (Definition A.1 with r_t; Prop. A.1): stage cost
+ *     1/2 (x_t'Q_t x_t + u_t'R_t u_t) + r_t'u_t,  terminal cost 1/2 x_H'Q_f x_H
+ * (with the linear term the factor 1/2 matters; P_t and K_t are those of lqr_oracle_solve_tv).
+ * Value function V_t(x) = 1/2 x'P_t x + p_t'x + c_t, p_H = 0, and for t = H-1..0 with
+ * S = R_t + B_t'P_{t+1}B_t, Y = B_t'P_{t+1}A_t:
+ *     K_t = -S^{-1} Y,                 k_t = -S^{-1} (B_t'p_{t+1} + r_t),
+ *     P_t = Q_t + A_t'P_{t+1}A_t + Y'K_t,   p_t = A_t'p_{t+1} + Y'k_t,
+ * then u_t = K_t x_t + k_t, x_{t+1} = A_t x_t + B_t u_t.
+ * r0: [H][m] with element stride sr between time indices (0 = the same vector at every t).
+ * Outputs (any may be NULL): K [H][m][n], kff [H][m], P [H+1][n][n], pvec [H+1][n], x [H+1][n], u [H][m].
+ * Returns as lqr_oracle_solve_tv.
+ */
+int lqr_oracle_solve_affine(int n, int m, int H, const double *A0, int64_t sA, const double *B0, int64_t sB,
+                            const double *Q0, int64_t sQ, const double *R0, int64_t sR, const double *r0, int64_t sr,
+                            const double *Qf, const double *x0, double *K, double *kff, double *P, double *pvec,
+                            double *x, double *u)
+{
+    if (n < 1 || m < 1 || H < 1)
+        return -1;
+    size_t nn = (size_t)n * n, nm = (size_t)n * m, mm = (size_t)m * m;
+    double *Pall = (double *)malloc(sizeof(double) * nn * (size_t)(H + 1));
+    double *pall = (double *)calloc((size_t)n * (size_t)(H + 1), sizeof(double));
+    double *Kall = (double *)malloc(sizeof(double) * nm * (size_t)H);
+    double *kall = (double *)malloc(sizeof(double) * (size_t)m * (size_t)H);
+    double *W = (double *)malloc(sizeof(double) * (3 * nn + 2 * nm + mm + 2 * (size_t)n + 2 * (size_t)m));
+    if (!Pall || !pall || !Kall || !kall || !W) {
+        free(Pall); free(pall); free(Kall); free(kall); free(W);
+        return -1;
+    }
+    double *PA = W, *AtPA = PA + nn, *YtK = AtPA + nn, *PB = YtK + nn, *Y = PB + nm, *S = Y + nm;
+    double *xt = S + mm, *xn = xt + n, *ut = xn + n, *g = ut + m;
+    int info = 0;
+
+    memcpy(Pall + nn * (size_t)H, Qf, sizeof(double) * nn);         /* P_H = Q_f, p_H = 0 */
+    for (int t = H - 1; t >= 0 && info == 0; --t) {
+        const double *Pn = Pall + nn * (size_t)(t + 1), *pn = pall + (size_t)n * (size_t)(t + 1);
+        double *Pt = Pall + nn * (size_t)t, *pt = pall + (size_t)n * (size_t)t;
+        double *Kt = Kall + nm * (size_t)t, *kt = kall + (size_t)m * (size_t)t;
+        const double *A = A0 + sA * t, *B = B0 + sB * t, *Q = Q0 + sQ * t, *R = R0 + sR * t, *r = r0 + sr * t;
+        mm_nn(n, m, n, Pn, B, PB);
+        mm_tn(m, m, n, B, PB, S);
+        for (size_t i = 0; i < mm; ++i)
+            S[i] += R[i];
+        mm_nn(n, n, n, Pn, A, PA);
+        mm_tn(m, n, n, B, PA, Y);
+        int bad = chol_lower(m, S);
+        if (bad) {
+            info = t * m + bad;
+            break;
+        }
+        memcpy(Kt, Y, sizeof(double) * nm);
+        chol_solve(m, n, S, Kt);
+        for (size_t i = 0; i < nm; ++i)
+            Kt[i] = -Kt[i];
+        for (int i = 0; i < m; ++i) {                               /* g = B'p_{t+1} + r_t */
+            double s = r[i];
+            for (int k = 0; k < n; ++k)
+                s += B[k * m + i] * pn[k];
+            g[i] = s;
+        }
+        memcpy(kt, g, sizeof(double) * (size_t)m);
+        chol_solve(m, 1, S, kt);
+        for (int i = 0; i < m; ++i)
+            kt[i] = -kt[i];                                         /* k_t = -S^{-1} g */
+        mm_tn(n, n, n, A, PA, AtPA);
+        mm_tn(n, n, m, Y, Kt, YtK);
+        for (int i = 0; i < n; ++i)
+            for (int j = 0; j < n; ++j)
+                Pt[i * n + j] = Q[i * n + j] + AtPA[i * n + j] + YtK[i * n + j];
+        for (int i = 0; i < n; ++i)
+            for (int j = i + 1; j < n; ++j) {
+                double s = 0.5 * (Pt[i * n + j] + Pt[j * n + i]);
+                Pt[i * n + j] = s;
+                Pt[j * n + i] = s;
+            }
+        for (int i = 0; i < n; ++i) {                               /* p_t = A'p_{t+1} + Y'k_t */
+            double s = 0.0;
+            for (int k = 0; k < n; ++k)
+                s += A[k * n + i] * pn[k];
+            for (int k = 0; k < m; ++k)
+                s += Y[k * n + i] * kt[k];
+            pt[i] = s;
+        }
+    }
+    if (info == 0) {
+        if (K) memcpy(K, Kall, sizeof(double) * nm * (size_t)H);
+        if (kff) memcpy(kff, kall, sizeof(double) * (size_t)m * (size_t)H);
+        if (P) memcpy(P, Pall, sizeof(double) * nn * (size_t)(H + 1));
+        if (pvec) memcpy(pvec, pall, sizeof(double) * (size_t)n * (size_t)(H + 1));
+        memcpy(xt, x0, sizeof(double) * (size_t)n);
+        if (x) memcpy(x, xt, sizeof(double) * (size_t)n);
+        for (int t = 0; t < H; ++t) {
+            const double *Kt = Kall + nm * (size_t)t, *kt = kall + (size_t)m * (size_t)t;
+            const double *A = A0 + sA * t, *B = B0 + sB * t;
+            for (int i = 0; i < m; ++i) {
+                double s = kt[i];
+                for (int j = 0; j < n; ++j)
+                    s += Kt[i * n + j] * xt[j];
+                ut[i] = s;
+            }
+            for (int i = 0; i < n; ++i) {
+                double s = 0.0;
+                for (int j = 0; j < n; ++j)
+                    s += A[i * n + j] * xt[j];
+                for (int j = 0; j < m; ++j)
+                    s += B[i * m + j] * ut[j];
+                xn[i] = s;
+            }
+            if (u) memcpy(u + (size_t)t * m, ut, sizeof(double) * (size_t)m);
+            if (x) memcpy(x + (size_t)(t + 1) * n, xn, sizeof(double) * (size_t)n);
+            memcpy(xt, xn, sizeof(double) * (size_t)n);
+        }
+    }
+    free(Pall); free(pall); free(Kall); free(kall); free(W);
+    return info;
+}

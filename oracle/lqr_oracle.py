@@ -51,6 +51,8 @@ def _load():
         )
         lib.lqr_oracle_solve_tv.restype = ctypes.c_int
         lib.lqr_oracle_solve_tv.argtypes = [ctypes.c_int] * 3 + [dp, ctypes.c_int64] * 4 + [dp] * 6 + [ctypes.c_int]
+        lib.lqr_oracle_solve_affine.restype = ctypes.c_int
+        lib.lqr_oracle_solve_affine.argtypes = [ctypes.c_int] * 3 + [dp, ctypes.c_int64] * 5 + [dp] * 8
         lib.lqr_oracle_solve_batch_tv.restype = ctypes.c_int
         lib.lqr_oracle_solve_batch_tv.argtypes = (
             [ctypes.c_int64, ctypes.c_int, ctypes.c_int, ctypes.c_int]
@@ -205,3 +207,23 @@ def solve_batch_tv(A, B, Q, R, Qf, x0, H, batch, tv=("A", "B", "Q", "R"), first_
     out["info"] = info
     out["threads"] = used
     return out
+
+
+def solve_affine(A, B, Q, R, r, Qf, x0, H):
+    """One instance with a linear control cost (Definition A.1 with ``r_t``; Prop. A.1): stage cost
+    ``1/2 (x_t'Q_t x_t + u_t'R_t u_t) + r_t'u_t``, terminal cost ``1/2 x_H'Qf x_H``.  Operands as for
+    :func:`solve_tv`; ``r`` is ``[H, m]`` or ``[m]``.  Returns a dict with ``K [H,m,n]``, ``k [H,m]`` (feed-forward:
+    ``u_t = K_t x_t + k_t``), ``P [H+1,n,n]``, ``p [H+1,n]``, ``x [H+1,n]``, ``u [H,m]``, ``info``."""
+    A, B, Q, R, r, Qf, x0 = map(_f64, (A, B, Q, R, r, Qf, x0))
+    n, m = B.shape[-2:]
+    strides = []
+    for a, tail in ((A, (n, n)), (B, (n, m)), (Q, (n, n)), (R, (m, m)), (r, (m,))):
+        assert a.shape in (tail, (H,) + tail), (a.shape, tail)
+        strides.append(0 if a.ndim == len(tail) else int(np.prod(tail)))
+    assert Qf.shape == (n, n) and x0.shape == (n,)
+    K = np.empty((H, m, n)); k = np.empty((H, m)); P = np.empty((H + 1, n, n)); p = np.empty((H + 1, n))
+    x = np.empty((H + 1, n)); u = np.empty((H, m))
+    info = _load().lqr_oracle_solve_affine(
+        n, m, H, _dptr(A), strides[0], _dptr(B), strides[1], _dptr(Q), strides[2], _dptr(R), strides[3],
+        _dptr(r), strides[4], _dptr(Qf), _dptr(x0), _dptr(K), _dptr(k), _dptr(P), _dptr(p), _dptr(x), _dptr(u))
+    return dict(K=K, k=k, P=P, p=p, x=x, u=u, info=info)
