@@ -165,6 +165,30 @@ int ttc_lqr_solve_tv(ttc_lqr_handle* h,
                      uint32_t flags, void* cuda_stream);
 
 /*
+ * Time-varying solve with a LINEAR CONTROL COST (Definition A.1 with r_t; Prop. A.1 / Alg. 1):
+ *     stage cost 1/2 (x_t'Q_t x_t + u_t'R_t u_t) + r_t'u_t,   terminal cost 1/2 x_H'Qf x_H
+ * (with the linear term the factor 1/2 matters; P_t and K_t are those of ttc_lqr_solve_tv).
+ * Value function V_t(x) = 1/2 x'P_t x + p_t'x + c_t, p_H = 0;
+ *     k_t = -(R_t + B_t'P_{t+1}B_t)^{-1} (B_t'p_{t+1} + r_t),   p_t = A_t'p_{t+1} + Y'k_t,  Y = B_t'P_{t+1}A_t,
+ *     u_t = K_t x_t + k_t,   x_{t+1} = A_t x_t + B_t u_t.
+ * In the paper's indexing r_t(here) = r_{t+1}(paper), like A, B and R.  This is the forward solve that the dual
+ * problem of Thm 3.2 needs.
+ *
+ * Arguments as for ttc_lqr_solve_tv, plus: r -- float32 vectors of length m, batch strides as for the
+ * other operands, r_tstride = element stride between consecutive time indices (0 = the same vector
+ * at every t); kff [N][H][m] receives k_t; pvec receives p_t, [N][H+1][n] or [N][n] = p_0 with
+ * TTC_OUT_FIRST_ONLY.  Each output may be NULL.  With TTC_OUT_FIRST_ONLY u = u_0 = K_0 x_0 + k_0.
+ * Failed instances: every requested output quiet NaN, info as for ttc_lqr_solve.  The scan method
+ * returns TTC_STATUS_UNSUPPORTED.
+ */
+int ttc_lqr_solve_affine(ttc_lqr_handle* h,
+                         const ttc_operand* A, const ttc_operand* B, const ttc_operand* Q, const ttc_operand* R,
+                         const int64_t tstride[4], const ttc_operand* Qf,
+                         const ttc_operand* r, int64_t r_tstride, const ttc_operand* x0, int32_t H,
+                         float* K, float* kff, float* P, float* pvec, float* x, float* u, int32_t* info,
+                         uint32_t flags, void* cuda_stream);
+
+/*
  * One Test-Time Control layer evaluation per instance with CONTEXTUALISED parameters
  * (Contextualization and Parameterization paragraphs of the TTC-Net section): the LQR parameters
  * of the planning horizon t = 1..T are synthesised inside the kernel from per-instance

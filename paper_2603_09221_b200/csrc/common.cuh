@@ -23,12 +23,15 @@ struct SolveParams {
     long long t0, tcount;      // token window [t0, t0 + tcount) of the last batch dimension solved by this launch
     OperandDev A, B, Q, R, x0;
     OperandDev Qf;             // terminal weight P_H (ptr null: P_H = Q)
+    OperandDev r;              // linear control cost r_t (vector of m; ptr null: none), Prop. A.1
     float* K;      // [N][H][m][n] or null
     float* P;      // [N][H+1][n][n] ([N][n][n] when first_only) or null
     float* x;      // [N][H+1][n] or null
     float* u;      // [N][H][m] ([N][m] when first_only) or null
     int* info;     // [N] or null
     float* Kws;    // workspace gains [N][H][m][n]: used when the rollout needs K_t but K is null
+    float* kff;    // feed-forward terms k_t [N][H][m] (caller's output or workspace) when r is given, else null
+    float* pvec;   // p_t [N][H+1][n] ([N][n] when first_only) or null
     int first_only;
 };
 

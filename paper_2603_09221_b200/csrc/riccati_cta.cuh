@@ -128,7 +128,8 @@ __device__ __forceinline__ float warp_dot(const float* row, const float* v, int 
 // memory (or, when only u_0 is wanted, the K_0 left in shared memory: pass Ksm and H_roll = 1).
 __device__ __forceinline__ void cta_rollout(const SolveParams& p, long long inst, float* sA,
                                             float* sB, const float* Kglob, const float* Ksm,
-                                            float* sx, float* sxn, float* su, int steps)
+                                            float* sx, float* sxn, float* su, int steps,
+                                            const float* kglob = nullptr, const float* ksm = nullptr)
 {
     const int n = p.n, m = p.m, H = p.H;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
@@ -146,10 +147,11 @@ __device__ __forceinline__ void cta_rollout(const SolveParams& p, long long inst
                 load_to_smem(sB, p.B, operand_offset(p.B, inst, p.b1, p.b2) + t * p.B.st, n * m);
             __syncthreads();
         }
+        const float* kt = ksm ? ksm : (kglob ? kglob + (long long)t * m : nullptr);     // u_t = K_t x_t + k_t
         for (int i = warp; i < m; i += nw) {
             const float s = warp_dot(Kt + i * n, sx, n);
             if (lane == 0)
-                su[i] = s;
+                su[i] = kt ? s + kt[i] : s;
         }
         __syncthreads();
         for (int i = warp; i < n; i += nw) {
@@ -191,14 +193,22 @@ __device__ __forceinline__ void cta_fail_instance(const SolveParams& p, long lon
         for (long long e = threadIdx.x; e < cnt; e += blockDim.x)
             p.u[inst * cnt + e] = qn;
     }
+    if (p.pvec) {
+        const long long cnt = (long long)(p.first_only ? 1 : H + 1) * n;
+        for (long long e = threadIdx.x; e < cnt; e += blockDim.x)
+            p.pvec[inst * cnt + e] = qn;
+    }
+    if (p.kff && p.r.ptr)
+        for (long long e = threadIdx.x; e < (long long)H * m; e += blockDim.x)
+            p.kff[inst * (long long)H * m + e] = qn;
     if (p.info && threadIdx.x == 0)
         p.info[inst] = code;
 }
 
 inline size_t riccati_cta_smem_bytes(int n, int m)
 {
-    // A, Q, P, T: n*n ; B, V, Y, K: n*m ; R, S: m*m ; x, xn: n ; u, col: m
-    return sizeof(float) * (size_t)(4 * n * n + 4 * n * m + 2 * m * m + 2 * n + 2 * m);
+    // A, Q, P, T: n*n ; B, V, Y, K: n*m ; R, S: m*m ; x, xn, p: n ; u, col, g: m
+    return sizeof(float) * (size_t)(4 * n * n + 4 * n * m + 2 * m * m + 3 * n + 3 * m);
 }
 
 __global__ void __launch_bounds__(256) riccati_cta_kernel(SolveParams p)
@@ -219,10 +229,14 @@ __global__ void __launch_bounds__(256) riccati_cta_kernel(SolveParams p)
     float* sxn = sx + n;
     float* su = sxn + n;
     float* scol = su + m;
+    float* sp = scol + m;      // p_{t+1} of the affine recursion (Prop. A.1)
+    float* sg = sp + n;        // B'p + r, then k_t
 
     for (long long widx = blockIdx.x; widx < p.b0 * p.b1 * p.tcount; widx += gridDim.x) {
         const long long inst = window_instance(p, widx);
         __syncthreads();
+        for (int e = threadIdx.x; e < n; e += blockDim.x)
+            sp[e] = 0.f;                                          // p_H = 0
         load_to_smem(sA, p.A, operand_offset(p.A, inst, p.b1, p.b2), n * n);
         load_to_smem(sB, p.B, operand_offset(p.B, inst, p.b1, p.b2), n * m);
         load_to_smem(sR, p.R, operand_offset(p.R, inst, p.b1, p.b2), m * m);
@@ -244,6 +258,9 @@ __global__ void __launch_bounds__(256) riccati_cta_kernel(SolveParams p)
         if (Pout && !p.first_only)
             for (int e = threadIdx.x; e < n * n; e += blockDim.x)
                 Pout[(long long)H * n * n + e] = sP[e];      // P_H
+        if (p.pvec && !p.first_only)
+            for (int e = threadIdx.x; e < n; e += blockDim.x)
+                p.pvec[inst * (long long)(H + 1) * n + (long long)H * n + e] = 0.f;
 
         int fail = 0;
         for (int t = H - 1; t >= 0; --t) {
@@ -289,6 +306,36 @@ __global__ void __launch_bounds__(256) riccati_cta_kernel(SolveParams p)
             if (Pout && (!p.first_only || t == 0))
                 for (int e = threadIdx.x; e < n * n; e += blockDim.x)
                     Pout[(long long)(p.first_only ? 0 : t) * n * n + e] = sP[e];
+            if (p.r.ptr) {
+                // linear control cost (Prop. A.1): k_t = -S^{-1}(B'p_{t+1} + r_t), p_t = A'p_{t+1} + Y'k_t
+                const long long orv = operand_offset(p.r, inst, p.b1, p.b2) + t * p.r.st;
+                for (int e = threadIdx.x; e < m; e += blockDim.x) {
+                    float g = load_elem(p.r, orv + e);
+                    for (int k = 0; k < n; ++k)
+                        g = fmaf(sB[k * m + e], sp[k], g);
+                    sg[e] = g;
+                }
+                __syncthreads();
+                smem_chol_solve_neg(m, 1, sS, sg);
+                __syncthreads();
+                float pn = 0.f;
+                const int i = threadIdx.x;
+                if (i < n) {
+                    for (int k = 0; k < n; ++k)
+                        pn = fmaf(sA[k * n + i], sp[k], pn);
+                    for (int k = 0; k < m; ++k)
+                        pn = fmaf(sY[k * n + i], sg[k], pn);
+                }
+                __syncthreads();
+                if (i < n) {
+                    sp[i] = pn;
+                    if (p.pvec && (!p.first_only || t == 0))
+                        p.pvec[inst * (long long)(p.first_only ? 1 : H + 1) * n + (long long)(p.first_only ? 0 : t) * n + i] = pn;
+                }
+                if (p.kff)
+                    for (int e = threadIdx.x; e < m; e += blockDim.x)
+                        p.kff[(inst * (long long)H + t) * m + e] = sg[e];
+            }
         }
         if (fail) {
             __syncthreads();
@@ -300,7 +347,9 @@ __global__ void __launch_bounds__(256) riccati_cta_kernel(SolveParams p)
         if (p.x || p.u) {
             __syncthreads();   // K_t written by this CTA are visible to it after the barrier
             const bool only_u0 = p.first_only && !p.x;
-            cta_rollout(p, inst, sA, sB, Kout, only_u0 ? sK : nullptr, sx, sxn, su, only_u0 ? 1 : H);
+            const float* kglob = (p.r.ptr && p.kff) ? p.kff + inst * (long long)H * m : nullptr;
+            cta_rollout(p, inst, sA, sB, Kout, only_u0 ? sK : nullptr, sx, sxn, su, only_u0 ? 1 : H, kglob,
+                        (only_u0 && p.r.ptr) ? sg : nullptr);
         }
     }
 }

@@ -51,6 +51,7 @@ struct ttc_lqr_handle {
     long long N;
     int sm_count;
     DevBuf ws_K, ws_P, ws_E;       // scratch used by kernels
+    DevBuf ws_k;                   // feed-forward terms k_t when the caller does not take them
     DevBuf st_in[5], st_out[5];    // device staging of ttc_lqr_solve_host
     DevBuf st_layer;               // device staging of ttc_lqr_solve_layer_host
     cudaStream_t host_stream;      // compute stream of ttc_lqr_solve_host
@@ -93,7 +94,7 @@ void release(DevBuf& b)
 
 size_t workspace_bytes(const ttc_lqr_handle* h)
 {
-    size_t s = h->ws_K.bytes + h->ws_P.bytes + h->ws_E.bytes + h->st_layer.bytes;
+    size_t s = h->ws_K.bytes + h->ws_P.bytes + h->ws_E.bytes + h->ws_k.bytes + h->st_layer.bytes;
     for (int i = 0; i < 5; ++i)
         s += h->st_in[i].bytes + h->st_out[i].bytes;
     return s;
@@ -243,6 +244,7 @@ int ttc_lqr_destroy(ttc_lqr_handle* h)
     release(h->ws_K);
     release(h->ws_P);
     release(h->ws_E);
+    release(h->ws_k);
     for (int i = 0; i < 5; ++i) {
         release(h->st_in[i]);
         release(h->st_out[i]);
@@ -296,7 +298,8 @@ namespace {
 int solve_window(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, const ttc_operand* Q,
                  const ttc_operand* R, const ttc_operand* x0, int32_t H, float* K, float* P, float* x,
                  float* u, int32_t* info, uint32_t flags, cudaStream_t st, long long t0, long long tcount,
-                 const int64_t* tstride = nullptr, const ttc_operand* Qf = nullptr)
+                 const int64_t* tstride = nullptr, const ttc_operand* Qf = nullptr,
+                 const ttc_operand* r = nullptr, int64_t r_tstride = 0, float* kff = nullptr, float* pvec = nullptr)
 {
     int s;
     const int n = h->cfg.n, m = h->cfg.m;
@@ -311,14 +314,18 @@ int solve_window(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, 
     if (tstride) {
         p.A.st = tstride[0]; p.B.st = tstride[1]; p.Q.st = tstride[2]; p.R.st = tstride[3];
     }
-    const bool time_varying = p.Qf.ptr != nullptr || (p.A.st | p.B.st | p.Q.st | p.R.st) != 0;
+    p.r = to_dev(r);
+    p.r.st = r_tstride;
+    const bool affine = p.r.ptr != nullptr;
+    const bool time_varying = affine || p.Qf.ptr != nullptr || (p.A.st | p.B.st | p.Q.st | p.R.st) != 0;
     p.K = K; p.P = P; p.x = x; p.u = u; p.info = info;
     p.Kws = nullptr;
+    p.kff = kff; p.pvec = pvec;
     p.first_only = (flags & TTC_OUT_FIRST_ONLY) ? 1 : 0;
 
     const int method = pick_method(h);
     if (method == TTC_SCAN && time_varying)
-        return fail(TTC_STATUS_UNSUPPORTED, "the scan method handles time-invariant problems only");
+        return fail(TTC_STATUS_UNSUPPORTED, "the scan method handles time-invariant problems without a linear cost only");
     // The rollout reads every K_t in forward order after the backward pass produced them in
     // reverse order; when the caller does not want K they live in the workspace.
     const bool rollout_needs_all_K = (x != nullptr) || (u != nullptr && !p.first_only);
@@ -348,6 +355,10 @@ int solve_window(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, 
         if (!K && rollout_needs_all_K) {
             if ((s = ensure(h->ws_K, sizeof(float) * (size_t)h->N * H * m * n))) return s;
             p.Kws = static_cast<float*>(h->ws_K.ptr);
+        }
+        if (affine && !kff && rollout_needs_all_K) {          // the rollout adds k_t at every step
+            if ((s = ensure(h->ws_k, sizeof(float) * (size_t)h->N * H * m))) return s;
+            p.kff = static_cast<float*>(h->ws_k.ptr);
         }
         const bool bf16_in = (Q->dtype == TTC_BF16) || (x0 && x0->ptr && x0->dtype == TTC_BF16);
         const bool want_tf32 = h->cfg.math == TTC_MATH_TF32 || (h->cfg.math == TTC_MATH_AUTO && bf16_in);
@@ -382,7 +393,7 @@ int solve_window(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, 
             h->last_kernel = TTC_KERNEL_RICCATI_UMMA;
             return TTC_OK;
         }
-        if (head_shared && n == m && (n == 16 || n == 32)) {
+        if (head_shared && n == m && (n == 16 || n == 32) && !affine) {
             // fp32 warp kernel: one instance per 16 / 32 lanes, chunks of tokens handed out by an atomic counter
             if ((s = ensure(h->ws_E, sizeof(int) * 4))) return s;
             int* counter = static_cast<int*>(h->ws_E.ptr);
@@ -442,6 +453,34 @@ int ttc_lqr_solve(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B,
     h->last_launches = 0;
     return solve_window(h, A, B, Q, R, x0, H, K, P, x, u, info, flags, static_cast<cudaStream_t>(cuda_stream), 0,
                         h->cfg.batch[2]);
+}
+
+int ttc_lqr_solve_affine(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, const ttc_operand* Q,
+                         const ttc_operand* R, const int64_t tstride[4], const ttc_operand* Qf,
+                         const ttc_operand* r, int64_t r_tstride, const ttc_operand* x0, int32_t H,
+                         float* K, float* kff, float* P, float* pvec, float* x, float* u, int32_t* info,
+                         uint32_t flags, void* cuda_stream)
+{
+    int s = validate_common(h, A, B, Q, R, x0, H, K, P, x, u, info, flags);
+    if (s)
+        return s;
+    if (!tstride)
+        return fail(TTC_STATUS_INVALID_ARGUMENT, "null tstride");
+    for (int i = 0; i < 4; ++i)
+        if (tstride[i] < 0)
+            return fail(TTC_STATUS_INVALID_ARGUMENT, "negative time stride");
+    if (r_tstride < 0)
+        return fail(TTC_STATUS_INVALID_ARGUMENT, "negative time stride of r");
+    if ((s = check_operand("Qf", Qf, true, tstride[2] == 0)))
+        return s;
+    if ((s = check_operand("r", r, false, false)))
+        return s;
+    if ((reinterpret_cast<uintptr_t>(kff) | reinterpret_cast<uintptr_t>(pvec)) & 15u)
+        return fail(TTC_STATUS_INVALID_ARGUMENT, "outputs must be 16-byte aligned");
+    TTC_CUDA(cudaSetDevice(h->cfg.device));
+    h->last_launches = 0;
+    return solve_window(h, A, B, Q, R, x0, H, K, P, x, u, info, flags, static_cast<cudaStream_t>(cuda_stream), 0,
+                        h->cfg.batch[2], tstride, (Qf && Qf->ptr) ? Qf : nullptr, r, r_tstride, kff, pvec);
 }
 
 // streams and events of the host-buffer entry points (created on first use)
@@ -839,8 +878,10 @@ extern "C" int ttc_lqr_solve_first_noalloc(int32_t n, int32_t m, const int64_t b
     p.t0 = 0; p.tcount = batch[2];
     p.A = to_dev(A); p.B = to_dev(B); p.Q = to_dev(Q); p.R = to_dev(R); p.x0 = to_dev(x0);
     p.Qf = to_dev(nullptr);
+    p.r = to_dev(nullptr);
     p.K = nullptr; p.P = P0; p.x = nullptr; p.u = u0; p.info = info;
     p.Kws = nullptr;
+    p.kff = nullptr; p.pvec = nullptr;
     p.first_only = 1;
     float* p1 = static_cast<float*>(scratch);
     int* flags = reinterpret_cast<int*>(static_cast<unsigned char*>(scratch) + p1_bytes);

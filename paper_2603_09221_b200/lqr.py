@@ -26,7 +26,7 @@ KERNEL_NAMES = {6: "ttc_layer", 0: "none", 1: "riccati_cta", 2: "riccati_warp", 
 EXPORTS = (
     "ttc_lqr_create", "ttc_lqr_solve", "ttc_lqr_solve_host", "ttc_lqr_destroy", "ttc_lqr_query",
     "ttc_lqr_status_string", "ttc_lqr_last_error", "ttc_lqr_solve_first_noalloc", "ttc_lqr_solve_tv",
-    "ttc_lqr_solve_layer", "ttc_lqr_solve_layer_host",
+    "ttc_lqr_solve_layer", "ttc_lqr_solve_layer_host", "ttc_lqr_solve_affine",
 )
 TTC_NOALLOC_SCRATCH_BYTES = 4 << 20
 
@@ -77,6 +77,9 @@ def load_library():
     lib.ttc_lqr_solve_tv.restype = ctypes.c_int
     lib.ttc_lqr_solve_tv.argtypes = [ctypes.c_void_p, opp, opp, opp, opp, P(ctypes.c_int64), opp, opp, ctypes.c_int32] + \
         [ctypes.c_void_p] * 5 + [ctypes.c_uint32, ctypes.c_void_p]
+    lib.ttc_lqr_solve_affine.restype = ctypes.c_int
+    lib.ttc_lqr_solve_affine.argtypes = [ctypes.c_void_p, opp, opp, opp, opp, P(ctypes.c_int64), opp, opp, ctypes.c_int64,
+                                         opp, ctypes.c_int32] + [ctypes.c_void_p] * 7 + [ctypes.c_uint32, ctypes.c_void_p]
     lib.ttc_lqr_solve_layer.restype = ctypes.c_int
     lib.ttc_lqr_solve_layer.argtypes = [ctypes.c_void_p, P(ttc_layer_inputs), ctypes.c_int32, ctypes.c_void_p,
                                         ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
@@ -218,6 +221,37 @@ class LqrSolver:
             self._h, ref(ops[0]), ref(ops[1]), ref(ops[2]), ref(ops[3]), tstride, ref(oqf), ref(ox), int(H),
             self._ptr(K), self._ptr(P), self._ptr(x), self._ptr(u), self._ptr(info), int(flags),
             ctypes.c_void_p(stream.cuda_stream)))
+
+    def solve_affine(self, A, B, Q, R, Qf, r, x0, H, tv=("A", "B", "Q", "R", "r"), K=None, kff=None, P=None, pvec=None,
+                     x=None, u=None, info=None, flags=0, stream=None):
+        """Enqueue ``ttc_lqr_solve_affine`` (linear control cost ``r_t'u_t``; Prop. A.1).  As :meth:`solve_tv`; ``r`` is
+        ``[..batch.., H, m]`` when ``"r"`` is in ``tv``, else ``[..batch.., m]``.  ``kff [N, H, m]`` receives the
+        feed-forward terms, ``pvec [N, H + 1, n]`` (``[N, n]`` with first-only) the linear value terms."""
+        ops, tstride = [], (ctypes.c_int64 * 4)()
+        for i, (name, t) in enumerate((("A", A), ("B", B), ("Q", Q), ("R", R))):
+            if name in tv:
+                if t.shape[-3] < H:
+                    raise ValueError("operand %s has %d time steps, H = %d" % (name, t.shape[-3], H))
+                ops.append(_operand(t[..., 0, :, :], 2, self.batch))
+                tstride[i] = t.stride(-3)
+            else:
+                ops.append(_operand(t, 2, self.batch))
+                tstride[i] = 0
+        if "r" in tv:
+            if r.shape[-2] < H:
+                raise ValueError("operand r has %d time steps, H = %d" % (r.shape[-2], H))
+            orr, rst = _operand(r[..., 0, :], 1, self.batch), r.stride(-2)
+        else:
+            orr, rst = _operand(r, 1, self.batch), 0
+        oqf = _operand(Qf, 2, self.batch)
+        ox = _operand(x0, 1, self.batch)
+        ref = lambda o: ctypes.byref(o) if o is not None else None
+        if stream is None:
+            stream = torch.cuda.current_stream(self.device)
+        _check(load_library().ttc_lqr_solve_affine(
+            self._h, ref(ops[0]), ref(ops[1]), ref(ops[2]), ref(ops[3]), tstride, ref(oqf), ref(orr), int(rst), ref(ox),
+            int(H), self._ptr(K), self._ptr(kff), self._ptr(P), self._ptr(pvec), self._ptr(x), self._ptr(u),
+            self._ptr(info), int(flags), ctypes.c_void_p(stream.cuda_stream)))
 
     def _layer_inputs(self, tensors, host):
         s_a, s_gamma_a, s_gamma_b, s_gamma_q, s_b, s_q, s_qf, r_inv, h0, B_basis, Q_basis = tensors
