@@ -43,6 +43,7 @@ struct Smem {
         float Lt[Shape<N>::MAT];       // rows of L' (columns of L); K_0 rows when only u_0 is wanted
         float rinv[N];                 // 1 / L[i][i]
         float x[N], u[N];
+        float pv[N], gv[N];            // affine recursion (Prop. A.1): p_{t+1}, B'p_{t+1} + r_t
     } slot[Shape<N>::SLOTS];
     int chunk;
 };
@@ -182,7 +183,8 @@ __device__ __forceinline__ void load_head_operands(Smem<N>& sm, const SolveParam
 }
 
 // TV = time-varying request (time strides or a terminal weight): the other instantiation carries none of that code.
-template <int N, bool TV>
+// AFF = linear control cost r_t'u_t (Prop. A.1: p_t, k_t); implies TV.
+template <int N, bool TV, bool AFF = false>
 __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kernel(SolveParams p, int* chunk_counter)
 {
     using S = Shape<N>;
@@ -197,6 +199,7 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
     const long long nchunks = p.b0 * p.b1 * chunks_per_head;
     const bool need_K_all = (p.K != nullptr) || (p.x != nullptr) || (p.u != nullptr && !p.first_only);
     const bool want_u0 = (p.u != nullptr) && p.first_only && !need_K_all;
+    const bool need_k_all = AFF && p.kff != nullptr;          // feed-forward terms wanted (output or rollout)
     float* Kbase = p.K ? p.K : p.Kws;
     long long offA = -1, offB = -1, offR = -1;
 
@@ -241,6 +244,13 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
         store_row<N>(sl.buf0 + c * LD, pcol);
         if (p.x0.ptr)
             sl.x[c] = load_elem(p.x0, operand_offset(p.x0, inst, p.b1, p.b2) + c);
+        float k0c = 0.f;                                      // k_0[c] when only u_0 is wanted
+        const long long orv = AFF ? operand_offset(p.r, inst, p.b1, p.b2) + c : 0;
+        if (AFF) {
+            sl.pv[c] = 0.f;                                   // p_H = 0
+            if (p.pvec && !p.first_only && active)
+                p.pvec[inst * (long long)(H + 1) * N + (long long)H * N + c] = 0.f;
+        }
         __syncwarp();
         int fail = 0;
 
@@ -313,6 +323,19 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
             float s[N], y[N];
             unpack_row<N>(s, s2);
             unpack_row<N>(y, y2);
+            float gz[N];                                      // B'p + r, then L^{-1}(.), then k_t = -S^{-1}(.) (every lane holds all of it)
+            float apc = 0.f;                                  // (A'p_{t+1})[c]
+            if (AFF) {
+                float pvv[N];
+                load_row<N>(pvv, sl.pv);
+                float gc = load_elem(p.r, orv + ts * p.r.st);
+#pragma unroll
+                for (int i = 0; i < N; ++i) {
+                    gc = fmaf(sm.B[i * LD + c], pvv[i], gc);
+                    apc = fmaf(sm.A[i * LD + c], pvv[i], apc);
+                }
+                sl.gv[c] = gc;
+            }
             float rs_own;
             const int bad = seg_chol<N>(s, rs_own, c);
             if (bad && !fail)
@@ -326,10 +349,17 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
             __syncwarp();
             float rinv[N];
             load_row<N>(rinv, sl.rinv);
+            if (AFF)
+                load_row<N>(gz, sl.gv);
 #pragma unroll
-            for (int k = 0; k < N; ++k) {                     // Z[:,c] = L^{-1} Y[:,c]
+            for (int k = 0; k < N; ++k) {                     // Z[:,c] = L^{-1} Y[:,c]  (and L^{-1}(B'p + r))
                 const float zk = y[k] * rinv[k];
                 y[k] = zk;
+                float zg = 0.f;
+                if (AFF) {
+                    zg = gz[k] * rinv[k];
+                    gz[k] = zg;
+                }
                 const float* lt = sl.Lt + k * LD;
 #pragma unroll
                 for (int i4 = (k + 1) & ~3; i4 < N; i4 += 4) {
@@ -338,7 +368,22 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
                     if (i4 + 1 > k) y[i4 + 1] = fmaf(-l4.y, zk, y[i4 + 1]);
                     if (i4 + 2 > k) y[i4 + 2] = fmaf(-l4.z, zk, y[i4 + 2]);
                     if (i4 + 3 > k) y[i4 + 3] = fmaf(-l4.w, zk, y[i4 + 3]);
+                    if (AFF) {
+                        if (i4 + 0 > k) gz[i4 + 0] = fmaf(-l4.x, zg, gz[i4 + 0]);
+                        if (i4 + 1 > k) gz[i4 + 1] = fmaf(-l4.y, zg, gz[i4 + 1]);
+                        if (i4 + 2 > k) gz[i4 + 2] = fmaf(-l4.z, zg, gz[i4 + 2]);
+                        if (i4 + 3 > k) gz[i4 + 3] = fmaf(-l4.w, zg, gz[i4 + 3]);
+                    }
                 }
+            }
+            if (AFF) {                                        // p_t[c] = (A'p_{t+1})[c] - Z[:,c] . L^{-1}(B'p_{t+1} + r_t)
+                float pc = apc;
+#pragma unroll
+                for (int q = 0; q < N; ++q)
+                    pc = fmaf(-y[q], gz[q], pc);
+                sl.pv[c] = pc;                                // every lane has read p_{t+1} before the barriers above
+                if (p.pvec && active && (!p.first_only || ts == 0))
+                    p.pvec[inst * (long long)(p.first_only ? 1 : H + 1) * N + (long long)(p.first_only ? 0 : ts) * N + c] = pc;
             }
 #pragma unroll
             for (int q = 0; q < N; ++q)
@@ -348,12 +393,17 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
             for (int q = 0; q < N; ++q)                       // Pn[:,c] -= Z' Z[:,c]
                 axpy_row<N>(p2, -sl.buf0[q * LD + c], sl.buf0 + q * LD);
             unpack_row<N>(pcol, p2);
-            const bool gains = need_K_all || (want_u0 && ts == 0);
-            if (gains) {                                      // K[:,c] = -L^{-T} Z[:,c]
+            const bool gains = need_K_all || need_k_all || (want_u0 && ts == 0);
+            if (gains) {                                      // K[:,c] = -L^{-T} Z[:,c]  (and k_t = -L^{-T} L^{-1}(B'p + r))
 #pragma unroll
                 for (int k = N - 1; k >= 0; --k) {
                     const float xk = y[k] * rinv[k];
                     y[k] = xk;
+                    float xg = 0.f;
+                    if (AFF) {
+                        xg = gz[k] * rinv[k];
+                        gz[k] = xg;
+                    }
                     const float* lr = sl.L + k * LD;
 #pragma unroll
                     for (int i4 = 0; i4 < k; i4 += 4) {
@@ -362,7 +412,24 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
                         if (i4 + 1 < k) y[i4 + 1] = fmaf(-l4.y, xk, y[i4 + 1]);
                         if (i4 + 2 < k) y[i4 + 2] = fmaf(-l4.z, xk, y[i4 + 2]);
                         if (i4 + 3 < k) y[i4 + 3] = fmaf(-l4.w, xk, y[i4 + 3]);
+                        if (AFF) {
+                            if (i4 + 0 < k) gz[i4 + 0] = fmaf(-l4.x, xg, gz[i4 + 0]);
+                            if (i4 + 1 < k) gz[i4 + 1] = fmaf(-l4.y, xg, gz[i4 + 1]);
+                            if (i4 + 2 < k) gz[i4 + 2] = fmaf(-l4.z, xg, gz[i4 + 2]);
+                            if (i4 + 3 < k) gz[i4 + 3] = fmaf(-l4.w, xg, gz[i4 + 3]);
+                        }
                     }
+                }
+                if (AFF) {
+                    float kc = 0.f;
+#pragma unroll
+                    for (int l = 0; l < N; ++l)
+                        if (l == c)
+                            kc = -gz[l];
+                    if (ts == 0)
+                        k0c = kc;
+                    if (need_k_all && active)
+                        p.kff[(inst * (long long)H + ts) * N + c] = kc;
                 }
                 if (need_K_all) {
                     if (active) {
@@ -371,7 +438,7 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
                         for (int l = 0; l < N; ++l)
                             kt[l * N] = -y[l];
                     }
-                } else {                                      // K_0 rows -> Lt (free after the forward substitution)
+                } else if (want_u0 && ts == 0) {              // K_0 rows -> Lt (free after the forward substitution)
 #pragma unroll
                     for (int l = 0; l < N; ++l)
                         sl.Lt[l * LD + c] = -y[l];
@@ -408,6 +475,14 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
                 for (long long e = c; e < cnt; e += N)
                     p.u[inst * cnt + e] = qn;
             }
+            if (AFF && p.pvec) {
+                const long long cnt = (long long)(p.first_only ? 1 : H + 1) * N;
+                for (long long e = c; e < cnt; e += N)
+                    p.pvec[inst * cnt + e] = qn;
+            }
+            if (need_k_all)
+                for (long long e = c; e < (long long)H * N; e += N)
+                    p.kff[inst * (long long)H * N + e] = qn;
         }
         if (p.info && active && c == 0)
             p.info[inst] = fail;
@@ -418,7 +493,7 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
             float kr[N], xv[N];
             load_row<N>(kr, sl.Lt + c * LD);
             load_row<N>(xv, sl.x);
-            float uc = 0.f;
+            float uc = AFF ? k0c : 0.f;                       // u_0 = K_0 x_0 + k_0
 #pragma unroll
             for (int j = 0; j < N; ++j)
                 uc = fmaf(kr[j], xv[j], uc);
@@ -449,7 +524,8 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
                 float xv[N];
                 load_row<N>(xv, sl.x);
                 const float4* kr = reinterpret_cast<const float4*>(Kout + (long long)ts * N * N + c * N);
-                float uc = 0.f;
+                float uc = need_k_all ? p.kff[(inst * (long long)H + ts) * N + c]        // own store of the backward pass
+                                      : (AFF && ts == 0) ? k0c : 0.f;
 #pragma unroll
                 for (int q = 0; q < N / 4; ++q) {
                     const float4 k4 = kr[q];

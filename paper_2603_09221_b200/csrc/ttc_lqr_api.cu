@@ -393,7 +393,7 @@ int solve_window(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, 
             h->last_kernel = TTC_KERNEL_RICCATI_UMMA;
             return TTC_OK;
         }
-        if (head_shared && n == m && (n == 16 || n == 32) && !affine) {
+        if (head_shared && n == m && (n == 16 || n == 32)) {
             // fp32 warp kernel: one instance per 16 / 32 lanes, chunks of tokens handed out by an atomic counter
             if ((s = ensure(h->ws_E, sizeof(int) * 4))) return s;
             int* counter = static_cast<int*>(h->ws_E.ptr);
@@ -402,12 +402,14 @@ int solve_window(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, 
             size_t smem;
             long long chunks, grid;
             if (n == 32) {
-                kern = time_varying ? rwarp::riccati_warp_kernel<32, true> : rwarp::riccati_warp_kernel<32, false>;
+                kern = affine ? rwarp::riccati_warp_kernel<32, true, true>
+                     : time_varying ? rwarp::riccati_warp_kernel<32, true> : rwarp::riccati_warp_kernel<32, false>;
                 smem = rwarp::smem_bytes<32>();
                 chunks = p.b0 * p.b1 * ((tcount + rwarp::Shape<32>::SLOTS - 1) / rwarp::Shape<32>::SLOTS);
                 grid = (long long)h->sm_count * 3;
             } else {
-                kern = time_varying ? rwarp::riccati_warp_kernel<16, true> : rwarp::riccati_warp_kernel<16, false>;
+                kern = affine ? rwarp::riccati_warp_kernel<16, true, true>
+                     : time_varying ? rwarp::riccati_warp_kernel<16, true> : rwarp::riccati_warp_kernel<16, false>;
                 smem = rwarp::smem_bytes<16>();
                 chunks = p.b0 * p.b1 * ((tcount + rwarp::Shape<16>::SLOTS - 1) / rwarp::Shape<16>::SLOTS);
                 grid = (long long)h->sm_count * 4;

@@ -23,7 +23,7 @@ def affine_workload(n, m, H, batch, seed, tv=("A", "B", "Q", "R", "r")):
     return w
 
 
-def run_both(w, first_only=False, want=("K", "kff", "P", "pvec", "x", "u", "info")):
+def run_both(w, first_only=False, want=("K", "kff", "P", "pvec", "x", "u", "info"), with_ref=True):
     n, m, H, batch = w["n"], w["m"], w["H"], w["batch"]
     N = int(np.prod(batch))
     s = lqr.LqrSolver(n, m, H, batch)
@@ -40,6 +40,8 @@ def run_both(w, first_only=False, want=("K", "kff", "P", "pvec", "x", "u", "info
     torch.cuda.synchronize()
     out["kernel"] = lqr.KERNEL_NAMES[s.query(lqr.TTC_QUERY_LAST_KERNEL)]
     s.close()
+    if not with_ref:
+        return out, None
     S, Hd, T = batch
     f64 = lambda t: t.to(torch.float64).cpu().numpy()
 
@@ -82,6 +84,7 @@ def test_affine_all_outputs(n, m, H):
     out, ref = run_both(w)
     errs = check(out, ref, False)
     print(n, m, H, out["kernel"], errs)
+    assert out["kernel"] == ("riccati_warp" if n == m and n in (16, 32) else "riccati_cta")
     for k in ("K", "kff", "P", "pvec", "x", "u"):
         assert not torch.any(out[k] == 123456.0), "canary left in %s" % k
 
@@ -101,3 +104,32 @@ def test_zero_linear_term_matches_the_time_varying_entry_point():
     out, ref = run_both(w)
     check(out, ref, False)
     assert float(out["kff"].abs().max()) == 0.0 and float(out["pvec"].abs().max()) == 0.0
+
+
+@pytest.mark.parametrize("n,T", [(16, 37), (32, 21)])
+def test_affine_warp_kernel_ragged_chunks_and_output_subsets(n, T):
+    """Several chunks of tokens per head with a ragged tail (idle segments), and the output combinations that take
+    different routes through the kernel: u_0 alone (k_0 kept in a register), K with u_0 (no feed-forward buffer),
+    the trajectory alone (k_t through the workspace), p_0 alone."""
+    w = affine_workload(n, n, 6, (2, 2, T), seed=4242 + n)
+    out, ref = run_both(w)
+    assert out["kernel"] == "riccati_warp"
+    check(out, ref, False)
+    for first_only, want in [(True, ("u", "info")), (True, ("K", "u", "info")), (False, ("x", "info")),
+                             (True, ("pvec", "info")), (True, ("kff", "u", "info"))]:
+        o, _ = run_both(w, first_only=first_only, want=want)
+        assert o["kernel"] == "riccati_warp"
+        check(o, ref, first_only)
+
+
+def test_affine_failure_fills_every_output_with_nan():
+    w = affine_workload(16, 16, 5, (1, 2, 9), seed=77)
+    w["R"] = w["R"].clone()
+    w["R"][0, 1, 0] = -50.0 * torch.eye(16, device=DEV)           # head 1: S_t loses positive definiteness
+    out, _ = run_both(w, with_ref=False)
+    info = out["info"].cpu().numpy().reshape(2, 9)
+    assert (info[0] == 0).all() and (info[1] != 0).all()
+    for k in ("K", "kff", "P", "pvec", "x", "u"):
+        t = out[k].reshape((2, 9) + out[k].shape[1:])
+        assert torch.isnan(t[1]).all(), k
+        assert torch.isfinite(t[0]).all(), k
