@@ -181,6 +181,31 @@ int ttc_lqr_solve_tv(ttc_lqr_handle* h,
  * Failed instances: every requested output quiet NaN, info as for ttc_lqr_solve.  The scan method
  * returns TTC_STATUS_UNSUPPORTED.
  */
+/*
+ * Gradients of a scalar loss l(o) of the layer output o = u_0* (Thm 3.2: primal and dual LQR), for the
+ * time-varying problem of ttc_lqr_solve_tv.  g [N][m] (float32, device) is dl/do.  The call runs
+ *   1. the backward Riccati pass (K_t) with the dual problem's linear cost on the first control riding along
+ *      (Prop. A.1 with r_0 = g: k_0 = -S_0^{-1} g; every later k_t is zero);
+ *   2. both rollouts: x_t, u_t = K_t x_t from x0 (primal), and xd_0 = 0, ud_0 = k_0, ud_t = K_t xd_t (dual);
+ *   3. both co-state sequences by  lam_H = Qf x_H,  lam_t = A_t' lam_{t+1} + Q_t x_t;
+ *   4. the outer products of the theorem, in this library's time indexing (A_t here = A_{t+1} of the paper):
+ *        dA [N][H][n][n]:  lam_{t+1} xd_t' + lamd_{t+1} x_t'      dB [N][H][n][m]:  lam_{t+1} ud_t' + lamd_{t+1} u_t'
+ *        dQ [N][H][n][n]:  1/2 (x_t xd_t' + xd_t x_t')            dQf [N][n][n]:    the same at t = H
+ *        dR [N][H][m][m]:  1/2 (u_t ud_t' + ud_t u_t')            dx0 [N][n]:       lamd_0
+ * and writes the forward output u0 [N][m].  Each output may be NULL (not computed).  Gradients are per instance
+ * and per time step: for an operand shared between instances or constant in time the caller sums the slices.
+ * dQ, dQf, dR are symmetric (derivatives along symmetric perturbations); Q_t and Qf must be symmetric.
+ * All outputs float32, device, 16-byte aligned, row-major; the call is asynchronous on cuda_stream.
+ * Failed instances (info != 0): every requested output quiet NaN.  Workspace: K_t, k_t and six vector sequences
+ * (N * (H m n + H m + 6 (H+1) max(n, m)) floats), grown on demand.
+ * Errors: as ttc_lqr_solve_tv; the scan method returns TTC_STATUS_UNSUPPORTED.
+ */
+int ttc_lqr_grad(ttc_lqr_handle* h,
+                 const ttc_operand* A, const ttc_operand* B, const ttc_operand* Q, const ttc_operand* R,
+                 const int64_t tstride[4], const ttc_operand* Qf, const ttc_operand* x0, const float* g, int32_t H,
+                 float* dA, float* dB, float* dQ, float* dQf, float* dR, float* dx0, float* u0, int32_t* info,
+                 void* cuda_stream);
+
 int ttc_lqr_solve_affine(ttc_lqr_handle* h,
                          const ttc_operand* A, const ttc_operand* B, const ttc_operand* Q, const ttc_operand* R,
                          const int64_t tstride[4], const ttc_operand* Qf,

@@ -24,6 +24,7 @@ struct SolveParams {
     OperandDev A, B, Q, R, x0;
     OperandDev Qf;             // terminal weight P_H (ptr null: P_H = Q)
     OperandDev r;              // linear control cost r_t (vector of m; ptr null: none), Prop. A.1
+    int r_count;               // r_t is given for t < r_count and zero from there on (the dual problem of Thm 3.2 has r_0 only)
     float* K;      // [N][H][m][n] or null
     float* P;      // [N][H+1][n][n] ([N][n][n] when first_only) or null
     float* x;      // [N][H+1][n] or null

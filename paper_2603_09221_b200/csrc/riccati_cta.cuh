@@ -310,7 +310,7 @@ __global__ void __launch_bounds__(256) riccati_cta_kernel(SolveParams p)
                 // linear control cost (Prop. A.1): k_t = -S^{-1}(B'p_{t+1} + r_t), p_t = A'p_{t+1} + Y'k_t
                 const long long orv = operand_offset(p.r, inst, p.b1, p.b2) + t * p.r.st;
                 for (int e = threadIdx.x; e < m; e += blockDim.x) {
-                    float g = load_elem(p.r, orv + e);
+                    float g = t < p.r_count ? load_elem(p.r, orv + e) : 0.f;
                     for (int k = 0; k < n; ++k)
                         g = fmaf(sB[k * m + e], sp[k], g);
                     sg[e] = g;

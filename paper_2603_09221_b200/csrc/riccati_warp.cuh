@@ -328,7 +328,7 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
             if (AFF) {
                 float pvv[N];
                 load_row<N>(pvv, sl.pv);
-                float gc = load_elem(p.r, orv + ts * p.r.st);
+                float gc = ts < p.r_count ? load_elem(p.r, orv + ts * p.r.st) : 0.f;
 #pragma unroll
                 for (int i = 0; i < N; ++i) {
                     gc = fmaf(sm.B[i * LD + c], pvv[i], gc);

@@ -13,6 +13,7 @@
 #include "riccati_umma64.cuh"
 #include "riccati_warp.cuh"
 #include "ttc_layer.cuh"
+#include "lqr_grad.cuh"
 #include "scan_pair.cuh"
 
 using namespace ttc;
@@ -52,6 +53,7 @@ struct ttc_lqr_handle {
     int sm_count;
     DevBuf ws_K, ws_P, ws_E;       // scratch used by kernels
     DevBuf ws_k;                   // feed-forward terms k_t when the caller does not take them
+    DevBuf ws_vec;                 // state, control and co-state sequences of the gradient entry point
     DevBuf st_in[5], st_out[5];    // device staging of ttc_lqr_solve_host
     DevBuf st_layer;               // device staging of ttc_lqr_solve_layer_host
     cudaStream_t host_stream;      // compute stream of ttc_lqr_solve_host
@@ -94,7 +96,7 @@ void release(DevBuf& b)
 
 size_t workspace_bytes(const ttc_lqr_handle* h)
 {
-    size_t s = h->ws_K.bytes + h->ws_P.bytes + h->ws_E.bytes + h->ws_k.bytes + h->st_layer.bytes;
+    size_t s = h->ws_K.bytes + h->ws_P.bytes + h->ws_E.bytes + h->ws_k.bytes + h->ws_vec.bytes + h->st_layer.bytes;
     for (int i = 0; i < 5; ++i)
         s += h->st_in[i].bytes + h->st_out[i].bytes;
     return s;
@@ -245,6 +247,7 @@ int ttc_lqr_destroy(ttc_lqr_handle* h)
     release(h->ws_P);
     release(h->ws_E);
     release(h->ws_k);
+    release(h->ws_vec);
     for (int i = 0; i < 5; ++i) {
         release(h->st_in[i]);
         release(h->st_out[i]);
@@ -299,7 +302,8 @@ int solve_window(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, 
                  const ttc_operand* R, const ttc_operand* x0, int32_t H, float* K, float* P, float* x,
                  float* u, int32_t* info, uint32_t flags, cudaStream_t st, long long t0, long long tcount,
                  const int64_t* tstride = nullptr, const ttc_operand* Qf = nullptr,
-                 const ttc_operand* r = nullptr, int64_t r_tstride = 0, float* kff = nullptr, float* pvec = nullptr)
+                 const ttc_operand* r = nullptr, int64_t r_tstride = 0, float* kff = nullptr, float* pvec = nullptr,
+                 int r_count = -1)
 {
     int s;
     const int n = h->cfg.n, m = h->cfg.m;
@@ -316,6 +320,7 @@ int solve_window(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, 
     }
     p.r = to_dev(r);
     p.r.st = r_tstride;
+    p.r_count = r_count < 0 ? H : r_count;
     const bool affine = p.r.ptr != nullptr;
     const bool time_varying = affine || p.Qf.ptr != nullptr || (p.A.st | p.B.st | p.Q.st | p.R.st) != 0;
     p.K = K; p.P = P; p.x = x; p.u = u; p.info = info;
@@ -483,6 +488,83 @@ int ttc_lqr_solve_affine(ttc_lqr_handle* h, const ttc_operand* A, const ttc_oper
     h->last_launches = 0;
     return solve_window(h, A, B, Q, R, x0, H, K, P, x, u, info, flags, static_cast<cudaStream_t>(cuda_stream), 0,
                         h->cfg.batch[2], tstride, (Qf && Qf->ptr) ? Qf : nullptr, r, r_tstride, kff, pvec);
+}
+
+int ttc_lqr_grad(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, const ttc_operand* Q,
+                 const ttc_operand* R, const int64_t tstride[4], const ttc_operand* Qf, const ttc_operand* x0,
+                 const float* g, int32_t H, float* dA, float* dB, float* dQ, float* dQf, float* dR, float* dx0,
+                 float* u0, int32_t* info, void* cuda_stream)
+{
+    int s = validate_common(h, A, B, Q, R, x0, H, nullptr, nullptr, nullptr, u0, info, 0);
+    if (s)
+        return s;
+    if (!x0 || !x0->ptr)
+        return fail(TTC_STATUS_INVALID_ARGUMENT, "operand x0 is null");
+    if (!tstride)
+        return fail(TTC_STATUS_INVALID_ARGUMENT, "null tstride");
+    for (int i = 0; i < 4; ++i)
+        if (tstride[i] < 0)
+            return fail(TTC_STATUS_INVALID_ARGUMENT, "negative time stride");
+    if ((s = check_operand("Qf", Qf, true, tstride[2] == 0)))
+        return s;
+    if (!g)
+        return fail(TTC_STATUS_INVALID_ARGUMENT, "null output gradient g");
+    const void* ptrs[8] = {g, dA, dB, dQ, dQf, dR, dx0, u0};
+    for (int i = 0; i < 8; ++i)
+        if (reinterpret_cast<uintptr_t>(ptrs[i]) & 15u)
+            return fail(TTC_STATUS_INVALID_ARGUMENT, "g and the gradient outputs must be 16-byte aligned");
+    if (pick_method(h) == TTC_SCAN)
+        return fail(TTC_STATUS_UNSUPPORTED, "the scan method has no gradient path");
+    TTC_CUDA(cudaSetDevice(h->cfg.device));
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const int n = h->cfg.n, m = h->cfg.m;
+    const int D = ((n > m ? n : m) + 3) & ~3;
+    if ((s = ensure(h->ws_K, sizeof(float) * (size_t)h->N * H * m * n))) return s;
+    if ((s = ensure(h->ws_k, sizeof(float) * (size_t)h->N * H * m))) return s;
+    if ((s = ensure(h->ws_vec, sizeof(float) * (size_t)h->N * 6 * (H + 1) * D))) return s;
+    float* Kws = static_cast<float*>(h->ws_K.ptr);
+    float* kws = static_cast<float*>(h->ws_k.ptr);
+    h->last_launches = 0;
+
+    // Backward pass of the primal problem (K_t) with the dual problem's linear cost riding along: r_0 = g, r_t = 0
+    // afterwards, so k_0 = -S_0^{-1} g is the dual's first control and every later k_t vanishes.
+    ttc_operand r;
+    r.ptr = g; r.dtype = TTC_F32; r.reserved = 0;
+    r.bstride[2] = m; r.bstride[1] = (int64_t)m * h->cfg.batch[2]; r.bstride[0] = r.bstride[1] * h->cfg.batch[1];
+    if ((s = solve_window(h, A, B, Q, R, x0, H, Kws, nullptr, nullptr, nullptr, info, 0, st, 0, h->cfg.batch[2], tstride,
+                          (Qf && Qf->ptr) ? Qf : nullptr, &r, 0, kws, nullptr, 1)))
+        return s;
+
+    grad::GradParams gp;
+    SolveParams& p = gp.sp;
+    p.n = n; p.m = m; p.H = H;
+    p.b0 = h->cfg.batch[0]; p.b1 = h->cfg.batch[1]; p.b2 = h->cfg.batch[2]; p.N = h->N;
+    p.t0 = 0; p.tcount = p.b2;
+    p.A = to_dev(A); p.B = to_dev(B); p.Q = to_dev(Q); p.R = to_dev(R); p.x0 = to_dev(x0);
+    p.Qf = to_dev((Qf && Qf->ptr) ? Qf : nullptr);
+    p.A.st = tstride[0]; p.B.st = tstride[1]; p.Q.st = tstride[2]; p.R.st = tstride[3];
+    p.r = to_dev(nullptr); p.r_count = 0;
+    p.K = nullptr; p.P = nullptr; p.x = nullptr; p.u = nullptr; p.info = info; p.Kws = nullptr;
+    p.kff = nullptr; p.pvec = nullptr; p.first_only = 0;
+    gp.K = Kws; gp.kff = kws; gp.vec = static_cast<float*>(h->ws_vec.ptr); gp.D = D;
+    gp.dA = dA; gp.dB = dB; gp.dQ = dQ; gp.dQf = dQf; gp.dR = dR; gp.dx0 = dx0; gp.u0 = u0;
+
+    long long grid = (h->N + grad::WARPS - 1) / grad::WARPS;
+    const long long cap = (long long)h->sm_count * 8;
+    if (grid > cap) grid = cap;
+    grad::grad_vectors_kernel<<<(unsigned)grid, 32 * grad::WARPS, 0, st>>>(gp);
+    TTC_CUDA(cudaGetLastError());
+    h->last_launches += 1;
+    h->total_launches += 1;
+    if (dA || dB || dQ || dQf || dR) {
+        grid = (h->N * (long long)(H + 1) + grad::WARPS - 1) / grad::WARPS;
+        if (grid > cap) grid = cap;
+        grad::grad_outer_kernel<<<(unsigned)grid, 32 * grad::WARPS, 0, st>>>(gp);
+        TTC_CUDA(cudaGetLastError());
+        h->last_launches += 1;
+        h->total_launches += 1;
+    }
+    return TTC_OK;
 }
 
 // streams and events of the host-buffer entry points (created on first use)
@@ -881,6 +963,7 @@ extern "C" int ttc_lqr_solve_first_noalloc(int32_t n, int32_t m, const int64_t b
     p.A = to_dev(A); p.B = to_dev(B); p.Q = to_dev(Q); p.R = to_dev(R); p.x0 = to_dev(x0);
     p.Qf = to_dev(nullptr);
     p.r = to_dev(nullptr);
+    p.r_count = 0;
     p.K = nullptr; p.P = P0; p.x = nullptr; p.u = u0; p.info = info;
     p.Kws = nullptr;
     p.kff = nullptr; p.pvec = nullptr;

@@ -26,7 +26,7 @@ KERNEL_NAMES = {6: "ttc_layer", 0: "none", 1: "riccati_cta", 2: "riccati_warp", 
 EXPORTS = (
     "ttc_lqr_create", "ttc_lqr_solve", "ttc_lqr_solve_host", "ttc_lqr_destroy", "ttc_lqr_query",
     "ttc_lqr_status_string", "ttc_lqr_last_error", "ttc_lqr_solve_first_noalloc", "ttc_lqr_solve_tv",
-    "ttc_lqr_solve_layer", "ttc_lqr_solve_layer_host", "ttc_lqr_solve_affine",
+    "ttc_lqr_solve_layer", "ttc_lqr_solve_layer_host", "ttc_lqr_solve_affine", "ttc_lqr_grad",
 )
 TTC_NOALLOC_SCRATCH_BYTES = 4 << 20
 
@@ -77,6 +77,9 @@ def load_library():
     lib.ttc_lqr_solve_tv.restype = ctypes.c_int
     lib.ttc_lqr_solve_tv.argtypes = [ctypes.c_void_p, opp, opp, opp, opp, P(ctypes.c_int64), opp, opp, ctypes.c_int32] + \
         [ctypes.c_void_p] * 5 + [ctypes.c_uint32, ctypes.c_void_p]
+    lib.ttc_lqr_grad.restype = ctypes.c_int
+    lib.ttc_lqr_grad.argtypes = [ctypes.c_void_p, opp, opp, opp, opp, P(ctypes.c_int64), opp, opp, ctypes.c_void_p,
+                                 ctypes.c_int32] + [ctypes.c_void_p] * 9
     lib.ttc_lqr_solve_affine.restype = ctypes.c_int
     lib.ttc_lqr_solve_affine.argtypes = [ctypes.c_void_p, opp, opp, opp, opp, P(ctypes.c_int64), opp, opp, ctypes.c_int64,
                                          opp, ctypes.c_int32] + [ctypes.c_void_p] * 7 + [ctypes.c_uint32, ctypes.c_void_p]
@@ -252,6 +255,34 @@ class LqrSolver:
             self._h, ref(ops[0]), ref(ops[1]), ref(ops[2]), ref(ops[3]), tstride, ref(oqf), ref(orr), int(rst), ref(ox),
             int(H), self._ptr(K), self._ptr(kff), self._ptr(P), self._ptr(pvec), self._ptr(x), self._ptr(u),
             self._ptr(info), int(flags), ctypes.c_void_p(stream.cuda_stream)))
+
+    def grad(self, A, B, Q, R, Qf, x0, g, H, tv=("A", "B", "Q", "R"), dA=None, dB=None, dQ=None, dQf=None, dR=None,
+             dx0=None, u0=None, info=None, stream=None):
+        """Enqueue ``ttc_lqr_grad`` (Thm 3.2): gradients of a loss of the first control ``u_0*`` given ``g = dl/du_0*``
+        (``[N, m]`` float32).  Operands as for :meth:`solve_tv`.  Outputs, each optional: ``dA [N, H, n, n]``,
+        ``dB [N, H, n, m]``, ``dQ [N, H, n, n]``, ``dQf [N, n, n]``, ``dR [N, H, m, m]``, ``dx0 [N, n]``, ``u0 [N, m]``,
+        ``info [N]`` (int32)."""
+        ops, tstride = [], (ctypes.c_int64 * 4)()
+        for i, (name, t) in enumerate((("A", A), ("B", B), ("Q", Q), ("R", R))):
+            if name in tv:
+                if t.shape[-3] < H:
+                    raise ValueError("operand %s has %d time steps, H = %d" % (name, t.shape[-3], H))
+                ops.append(_operand(t[..., 0, :, :], 2, self.batch))
+                tstride[i] = t.stride(-3)
+            else:
+                ops.append(_operand(t, 2, self.batch))
+                tstride[i] = 0
+        oqf = _operand(Qf, 2, self.batch)
+        ox = _operand(x0, 1, self.batch)
+        if tuple(g.shape) != (self.N, self.m) or g.dtype != torch.float32 or not g.is_contiguous():
+            raise ValueError("g must be a contiguous float32 tensor of shape (%d, %d)" % (self.N, self.m))
+        ref = lambda o: ctypes.byref(o) if o is not None else None
+        if stream is None:
+            stream = torch.cuda.current_stream(self.device)
+        _check(load_library().ttc_lqr_grad(
+            self._h, ref(ops[0]), ref(ops[1]), ref(ops[2]), ref(ops[3]), tstride, ref(oqf), ref(ox), self._ptr(g), int(H),
+            self._ptr(dA), self._ptr(dB), self._ptr(dQ), self._ptr(dQf), self._ptr(dR), self._ptr(dx0), self._ptr(u0),
+            self._ptr(info), ctypes.c_void_p(stream.cuda_stream)))
 
     def _layer_inputs(self, tensors, host):
         s_a, s_gamma_a, s_gamma_b, s_gamma_q, s_b, s_q, s_qf, r_inv, h0, B_basis, Q_basis = tensors
