@@ -166,6 +166,153 @@ def run_reference(args, cid, tv_key=None):
     print(json.dumps(line))
 
 
+GRAD_NAMES = ("dA", "dB", "dQ", "dQf", "dR", "dx0", "u0")
+
+
+def grad_oracle(w, g, idx, H):
+    """Thm 3.2 gradients of the sampled instances by the float64 oracle (one instance at a time)."""
+    from oracle import lqr_grad as og
+    S, Hd, T = w["batch"]
+    f64 = lambda t: t.to(torch.float64).cpu().numpy()
+    t0 = time.perf_counter()
+    refs = []
+    for i in idx:
+        head = (int(i) // T) % Hd
+        refs.append(og.grad(f64(w["A"][0, head, 0]), f64(w["B"][0, head, 0]), f64(w["Q"].reshape((-1,) + w["Q"].shape[3:])[i]),
+                            f64(w["R"][0, head, 0]), f64(w["Qf"].reshape((-1,) + w["Qf"].shape[3:])[i]),
+                            f64(w["x0"].reshape(-1, w["x0"].shape[-1])[i]), f64(g[i]), H))
+    ref = {k: np.stack([r[k] for r in refs]) for k in GRAD_NAMES}
+    return ref, time.perf_counter() - t0
+
+
+def run_grad(args):
+    """--workload grad16: one step = one ttc_lqr_grad over the whole workload (backward pass, both rollouts and
+    co-state sequences, outer products), every gradient written."""
+    key = args.workload
+    c = dict(workloads.TV_CONFIGS[key])
+    rank = int(os.environ.get("RANK", "0"))
+    n, m, H = c["n"], c["m"], c["H"]
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        S, Hd, Tk = c["batch"]
+        cnt = max(1, min(S * Hd * Tk, args.ref_instances // 8))
+        w = workloads.make_tv_workload(key, device="cpu", batch=(1, Hd, max(1, cnt // Hd)))
+        Nw = int(np.prod(w["batch"]))
+        g = torch.randn((Nw, m), generator=torch.Generator().manual_seed(7))
+        times = []
+        for it in range(args.warmup + args.steps):
+            _, dt = grad_oracle(w, g, range(Nw), H)
+            if it >= args.warmup:
+                times.append(dt)
+        ms = 1e3 * sum(times) / len(times)
+        val = Nw / (ms * 1e-3)
+        print(json.dumps({"impl": "reference", "metric": "lqr_instances_per_sec", "value": val, "unit": "instances/s",
+                          "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
+                          "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+                          "data": "synthetic",
+                          "config": {"workload": c["name"], "n": n, "m": m, "H": H, "instances_per_step": Nw,
+                                     "note": "bounded sample of the workload per step"},
+                          "cpu_baseline": {"value": val, "unit": "instances/s", "cores": 1, "kind": "oracle",
+                                           "sample": "%d instances per step, one at a time" % Nw},
+                          "e2e": {"value": val, "unit": "instances/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                          "gpu_launches": 0}))
+        return
+    args.warmup = max(args.warmup, 3)
+    from paper_2603_09221_b200 import lqr
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the solver has no CPU path")
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = world > 1
+    if dist:
+        import torch.distributed as td
+        td.init_process_group("nccl", device_id=torch.device("cuda", local))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    peaks = measured_peaks()
+    if args.tokens > 0:
+        c["batch"] = (c["batch"][0], c["batch"][1], args.tokens)
+        c["name"] += "_tokens%d" % args.tokens
+    w = workloads.make_tv_workload(key, device=dev, batch=c["batch"], seed=sharding.rank_seed(100, rank))
+    N = int(np.prod(c["batch"]))
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(sharding.rank_seed(300, rank))
+    g = torch.randn((N, m), generator=gen, device=dev)
+    solver = lqr.LqrSolver(n, m, H, c["batch"], device=local)
+    shp = dict(dA=(N, H, n, n), dB=(N, H, n, m), dQ=(N, H, n, n), dQf=(N, n, n), dR=(N, H, m, m), dx0=(N, n), u0=(N, m))
+    out = {k: torch.empty(v, device=dev) for k, v in shp.items()}
+    out["info"] = torch.empty((N,), dtype=torch.int32, device=dev)
+
+    def step():
+        solver.grad(w["A"], w["B"], w["Q"], w["R"], w["Qf"], w["x0"], g, H, tv=c["tv"], **out)
+
+    def barrier():
+        if dist:
+            td.barrier()
+        torch.cuda.synchronize(dev)
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    launches0 = solver.query(lqr.TTC_QUERY_TOTAL_LAUNCHES)
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    barrier()
+    evs[0].record()
+    for i in range(args.steps):
+        step()
+        evs[i + 1].record()
+    barrier()
+    launches = solver.query(lqr.TTC_QUERY_TOTAL_LAUNCHES) - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    per_step = [evs[i].elapsed_time(evs[i + 1]) for i in range(args.steps)]
+    value, ms_per_step, _ = sharding.aggregate_throughput(N, evs[0].elapsed_time(evs[-1]) / args.steps, device=dev)
+    if rank != 0:
+        if dist:
+            td.destroy_process_group()
+        return
+    # algorithmic bytes: Q_t, Q_f, x_0, g in (the per-head A_t, B_t, R_t are negligible); every gradient, u_0, info out
+    bin_i = 4 * (H * n * n + n * n + n + m)
+    bout_i = 4 * (H * (2 * n * n + n * m + m * m) + n * n + n + m + 1)
+    kernel_ms = statistics.median(per_step)
+    ach = N * (bin_i + bout_i) / (kernel_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
+                "traffic": None, "kernel": "whole step: backward pass + grad_vectors + grad_outer (3 launches)",
+                "kernel_ms": kernel_ms, "peak_note": "copy bandwidth, of %s" % peaks["source"],
+                "algorithmic_bytes_per_launch": N * (bin_i + bout_i)}
+    cpu = None
+    if not args.no_cpu_baseline and world == 1:
+        idx = np.unique(np.linspace(0, N - 1, max(8, args.cpu_sample // 8)).astype(np.int64))
+        ref, dt = grad_oracle(w, g, idx, H)
+        from tests import parity_util as pu
+        sel = torch.as_tensor(idx)
+        errs = {k: pu.block_rel_err(out[k].cpu()[sel].reshape(len(idx), -1).numpy(), ref[k].reshape(len(idx), -1), 1,
+                                    per_block=False) for k in GRAD_NAMES}
+        assert all(v <= c["tol"] for v in errs.values()), errs
+        assert int(out["info"].abs().max()) == 0
+        cpu = {"value": len(idx) / dt, "unit": "instances/s", "cores": 1, "kind": "oracle",
+               "sample": "%d instances spread over the workload, one at a time" % len(idx),
+               "seconds": dt, "parity_max_rel_err": errs, "speedup_gpu_over_cpu": value / (len(idx) / dt)}
+    print(json.dumps({"metric": "lqr_instances_per_sec", "value": value, "unit": "instances/s", "n_gpus": world,
+                      "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+                      "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                      "config": {"workload": c["name"], "n": n, "m": m, "H": H, "instances": N, "batch": list(c["batch"]),
+                                 "time_varying": list(c["tv"]), "outputs": list(GRAD_NAMES) + ["info"],
+                                 "l2": "inputs+outputs per step exceed L2 (%.2f GB)" % (N * (bin_i + bout_i) / 1e9)},
+                      "roofline": roofline, "cpu_baseline": cpu, "e2e": None,
+                      "e2e_note": "gradients stay on the device for the layers below; no host-buffer entry point",
+                      "gpu_launches": int(launches), "launches_per_step": launches / args.steps, "clocks": clocks,
+                      "ms_per_step_percentiles": {"p20": float(np.percentile(per_step, 20)),
+                                                  "p50": float(np.percentile(per_step, 50)),
+                                                  "p80": float(np.percentile(per_step, 80))}}))
+    solver.close()
+    if dist:
+        td.destroy_process_group()
+
+
 def layer_counts(c):
     """Per-instance algorithmic flops and HBM bytes of the contextualised layer solve: per step P Bbar (2 n^3),
     Bbar'V (n^3, S symmetric), Bbar'T (2 n^3), Cholesky (n^3 / 3), L^{-1}Y (n^3), Z'Z (n^3, symmetric); per
@@ -358,6 +505,9 @@ def main():
     args = ap.parse_args()
     if args.workload in workloads.LAYER_CONFIGS:
         run_layer(args)
+        return
+    if workloads.TV_CONFIGS.get(args.workload, {}).get("grad"):
+        run_grad(args)
         return
     tv_key = args.workload if args.workload in workloads.TV_CONFIGS else None
     cid = None if tv_key else int(args.workload.replace("cfg", ""))

@@ -547,12 +547,31 @@ int ttc_lqr_grad(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, 
     p.K = nullptr; p.P = nullptr; p.x = nullptr; p.u = nullptr; p.info = info; p.Kws = nullptr;
     p.kff = nullptr; p.pvec = nullptr; p.first_only = 0;
     gp.K = Kws; gp.kff = kws; gp.vec = static_cast<float*>(h->ws_vec.ptr); gp.D = D;
+    {
+        auto pow2 = [](int v) { return v > 0 && (v & (v - 1)) == 0; };
+        long long strides = p.A.st | p.B.st;
+        for (const OperandDev* o : {&p.A, &p.B})
+            strides |= o->s0 | o->s1 | o->s2;
+        gp.vec4 = (n % 4 == 0 && m % 4 == 0 && pow2(n / 4) && pow2(m / 4) && n <= 64 && m <= 64 && (strides & 3) == 0) ? 1 : 0;
+    }
     gp.dA = dA; gp.dB = dB; gp.dQ = dQ; gp.dQf = dQf; gp.dR = dR; gp.dx0 = dx0; gp.u0 = u0;
 
     long long grid = (h->N + grad::WARPS - 1) / grad::WARPS;
     const long long cap = (long long)h->sm_count * 8;
     if (grid > cap) grid = cap;
-    grad::grad_vectors_kernel<<<(unsigned)grid, 32 * grad::WARPS, 0, st>>>(gp);
+    {
+        long long qs = p.Q.st | p.Q.s0 | p.Q.s1 | p.Q.s2 | p.Qf.s0 | p.Qf.s1 | p.Qf.s2;
+        const bool small = gp.vec4 && n <= 16 && m <= 16 && p.Q.dtype == TTC_F32 && p.Qf.dtype == TTC_F32 && (qs & 3) == 0;
+        if (small) {
+            const size_t smem = grad::small_smem_bytes();
+            TTC_CUDA(cudaFuncSetAttribute(grad::grad_vectors_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            long long sgrid = (h->N + grad::WARPS - 1) / grad::WARPS;
+            if (sgrid > (long long)h->sm_count * 2) sgrid = (long long)h->sm_count * 2;      // two CTAs fit an SM
+            grad::grad_vectors_small_kernel<<<(unsigned)sgrid, 32 * grad::WARPS, smem, st>>>(gp);
+        }
+        else
+            grad::grad_vectors_kernel<<<(unsigned)grid, 32 * grad::WARPS, 0, st>>>(gp);
+    }
     TTC_CUDA(cudaGetLastError());
     h->last_launches += 1;
     h->total_launches += 1;
