@@ -586,12 +586,13 @@ __global__ void __launch_bounds__(32 * WARPS) grad_outer_kernel(GradParams g)
     float* ld = sm[warp][5];
     const long long items = p.N * (long long)(H + 1);
     const long long stride = (long long)gridDim.x * WARPS;
+    const bool small_items = items < (1ll << 31);             // 32-bit division is several times cheaper
     long long it = (long long)blockIdx.x * WARPS + warp;
 
     // the six vectors of one item, two elements per lane; fetched one item ahead of the stores
     float rv[6][2];
     auto fetch = [&](long long item) {
-        const long long inst = item / (H + 1);
+        const long long inst = small_items ? (long long)((unsigned)item / (unsigned)(H + 1)) : item / (H + 1);
         const int t = (int)(item - inst * (H + 1));
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
@@ -608,7 +609,7 @@ __global__ void __launch_bounds__(32 * WARPS) grad_outer_kernel(GradParams g)
     if (it < items)
         fetch(it);
     while (it < items) {
-        const long long inst = it / (H + 1);
+        const long long inst = small_items ? (long long)((unsigned)it / (unsigned)(H + 1)) : it / (H + 1);
         const int t = (int)(it - inst * (H + 1));
         __syncwarp();                                         // the previous item's reads of shared memory are done
 #pragma unroll
