@@ -88,6 +88,42 @@ def test_grad_all_outputs(n, m, H):
         assert torch.equal(out[k], out[k].transpose(-1, -2))
 
 
+@pytest.mark.parametrize("n,m,H", [(4, 4, 1), (4, 16, 2), (16, 4, 3), (16, 8, 5), (8, 16, 9), (16, 16, 1), (16, 16, 4), (32, 16, 3),
+                                   (16, 32, 3), (64, 64, 1), (20, 12, 1)])
+def test_grad_shapes_around_the_small_kernel(n, m, H):
+    """Rectangular B_t with n, m in {4, 8, 16} (the staged kernel: different float4 counts per row for K_t, A_t, B_t),
+    horizons shorter than, equal to and longer than its ring of stages, and sizes just outside it."""
+    batch = (1, 3, 11)
+    w = tv_workload(n, m, H, batch, seed=17 * n + 3 * m + H)
+    g = draw_g(33, m, 5)
+    out = run_gpu(w, g)
+    ref = run_oracle(w, g)
+    errs = errors(out, ref)
+    assert int(out["info"].abs().max()) == 0
+    assert all(v <= 1e-4 for v in errs.values()), errs
+    for k in NAMES:
+        assert not torch.any(out[k] == 123456.0), "canary left in %s" % k
+
+
+def test_grad_per_token_dynamics():
+    """A_t, B_t, R_t of every token its own (the contextualised layer's situation): no operand is shared."""
+    n, m, H, batch = 16, 16, 6, (2, 2, 7)
+    w = tv_workload(n, m, H, batch, seed=31)
+    S, Hd, T = batch
+    gen = torch.Generator(device=DEV)
+    gen.manual_seed(8)
+    for k in ("A", "B", "R"):
+        full = w[k].expand((S, Hd, T) + w[k].shape[3:]).clone()
+        if k != "R":
+            full = full + 0.05 * torch.randn(full.shape, generator=gen, device=DEV)
+        w[k] = full.contiguous()
+    g = draw_g(28, m, 6)
+    out = run_gpu(w, g)
+    ref = run_oracle(w, g)
+    assert out["kernel"] == "riccati_cta"                      # per-token dynamics: the generic backward pass
+    assert all(v <= 1e-4 for v in errors(out, ref).values())
+
+
 def test_grad_time_invariant_operands_and_output_subsets():
     w = tv_workload(16, 16, 9, (1, 3, 37), seed=5, tv=("Q",))                  # A, B, R constant in time, ragged chunks
     N = 111
