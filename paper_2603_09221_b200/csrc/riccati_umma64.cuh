@@ -799,6 +799,22 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
                             store_half_global(p.P + (inst * (long long)(p.first_only ? 1 : H + 1) + (p.first_only ? 0 : ts)) * N * N +
                                                   (long long)j * N + 32 * half, q);
                     }
+                    // Every eighth step the operand is replaced by (P + P') / 2.  Q and Z'Z are symmetric but the rounding
+                    // of A'(P A) is not, and the antisymmetric part E obeys E <- A'E A: along an open-loop unstable A it
+                    // grows however well the closed loop is damped, until S stops being positive definite.  Eight steps
+                    // of growth are harmless (the exchange costs about a sixth of a step).  X1 (Z', consumed by (5)) is free and takes the averaged rows.
+                    if (ts > 0 && (ts & 7) == 0) {
+                        half_barrier(wg);                     // both halves of every row are in X0
+#pragma unroll 8
+                        for (int c = 0; c < 64; ++c) {
+                            const int cj = (c + (j >> 2)) & 63;       // rotated per lane: the column reads hit 32 banks
+                            elem(X1, toff(j, cj)) = round_tf32(0.5f * (elem(X0, toff(j, cj)) + elem(X0, toff(cj, j))));
+                        }
+                        half_barrier(wg);                     // every column has been read
+#pragma unroll
+                        for (int c = 0; c < 16; ++c)
+                            *reinterpret_cast<float4*>(X0 + toff(j, 4 * c)) = *reinterpret_cast<const float4*>(X1 + toff(j, 4 * c));
+                    }
                 }
                 tc_fence_before();
                 async_proxy_fence();

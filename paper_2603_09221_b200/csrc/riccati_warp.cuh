@@ -444,14 +444,23 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
                         sl.Lt[l * LD + c] = -y[l];
                 }
             }
+            __syncwarp();                                     // rows of Z consumed
+            store_row<N>(sl.buf0 + c * LD, pcol);             // column c of P_t as row c
+            __syncwarp();
+            // P_t <- (P_t + P_t') / 2.  Q_t and Z'Z are symmetric, but the rounding of A'(P A) is not, and since the next
+            // step reads the rows above as columns, the antisymmetric part E obeys E <- -A'E A: it grows along an
+            // open-loop unstable A (|eig| > 1) however well the closed loop is damped, and takes over long horizons.
+#pragma unroll
+            for (int l = 0; l < N; ++l)
+                pcol[l] = 0.5f * (pcol[l] + sl.buf0[l * LD + c]);
             if (Pout && (!p.first_only || ts == 0)) {
                 float* pt = Pout + (long long)(p.first_only ? 0 : ts) * N * N + c;
 #pragma unroll
                 for (int l = 0; l < N; ++l)
                     pt[l * N] = pcol[l];
             }
-            __syncwarp();                                     // rows of Z consumed
-            store_row<N>(sl.buf0 + c * LD, pcol);             // rows of P_t (row c = column c)
+            __syncwarp();                                     // every lane has read its column
+            store_row<N>(sl.buf0 + c * LD, pcol);
             __syncwarp();
         }
 

@@ -50,12 +50,14 @@ TV_CONFIGS = {
 }
 
 
-def make_tv_workload(key="tv16", device="cpu", batch=None, seed=None, chunk=4096):
+def make_tv_workload(key="tv16", device="cpu", batch=None, seed=None, chunk=4096, horizon=None):
     """Inputs of a time-varying configuration: ``A, B, R [1,Hd,1,H,...]`` (float32, per head and time index),
     ``Q [S,Hd,T,H,n,n]``, ``Qf [S,Hd,T,n,n]``, ``x0 [S,Hd,T,n]`` plus the configuration fields."""
     c = dict(TV_CONFIGS[key])
     if batch is not None:
         c["batch"] = tuple(int(b) for b in batch)
+    if horizon is not None:
+        c["H"] = int(horizon)
     S, Hd, T = c["batch"]
     n, m, H = c["n"], c["m"], c["H"]
     seed = SEED0 + 100 if seed is None else seed
