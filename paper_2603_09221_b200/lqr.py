@@ -215,7 +215,7 @@ class LqrSolver:
             else:
                 ops.append(_operand(t, 2, self.batch))
                 tstride[i] = 0
-        oqf = _operand(Qf, 2, self.batch)
+        oqf = _operand(Qf, 2, self.batch) if Qf is not None else None      # NULL: Q_f = Q (Q constant in time)
         ox = _operand(x0, 1, self.batch)
         ref = lambda o: ctypes.byref(o) if o is not None else None
         if stream is None:
@@ -246,7 +246,7 @@ class LqrSolver:
             orr, rst = _operand(r[..., 0, :], 1, self.batch), r.stride(-2)
         else:
             orr, rst = _operand(r, 1, self.batch), 0
-        oqf = _operand(Qf, 2, self.batch)
+        oqf = _operand(Qf, 2, self.batch) if Qf is not None else None      # NULL: Q_f = Q (Q constant in time)
         ox = _operand(x0, 1, self.batch)
         ref = lambda o: ctypes.byref(o) if o is not None else None
         if stream is None:
@@ -272,7 +272,7 @@ class LqrSolver:
             else:
                 ops.append(_operand(t, 2, self.batch))
                 tstride[i] = 0
-        oqf = _operand(Qf, 2, self.batch)
+        oqf = _operand(Qf, 2, self.batch) if Qf is not None else None      # NULL: Q_f = Q (Q constant in time)
         ox = _operand(x0, 1, self.batch)
         if tuple(g.shape) != (self.N, self.m) or g.dtype != torch.float32 or not g.is_contiguous():
             raise ValueError("g must be a contiguous float32 tensor of shape (%d, %d)" % (self.N, self.m))

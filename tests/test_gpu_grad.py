@@ -188,3 +188,33 @@ def test_grad_full_size_sampled_instances():
         assert torch.equal(out[k], out[k].transpose(-1, -2))
     for k in NAMES:
         assert torch.isfinite(out[k]).all()
+
+
+@pytest.mark.parametrize("n", [8, 16, 24])
+def test_null_terminal_weight_means_the_constant_state_cost(n):
+    """Qf = NULL is allowed when Q is constant in time and then Q_f = Q, in all three time-varying entry points."""
+    H, batch = 7, (1, 2, 6)
+    w = tv_workload(n, n, H, batch, seed=70 + n, tv=("A", "B", "R"))
+    N = 12
+    g = draw_g(N, n, 11)
+    s = lqr.LqrSolver(n, n, H, batch)
+    mk = lambda *shape: torch.full(shape, 123456.0, device=DEV)
+    got, exp = {}, {}
+    for tag, Qf in (("null", None), ("given", w["Q"])):
+        o = dict(dA=mk(N, H, n, n), dQf=mk(N, n, n), dx0=mk(N, n), u0=mk(N, n))
+        s.grad(w["A"], w["B"], w["Q"], w["R"], Qf, w["x0"], g, H, tv=w["tv"], **o)
+        P, u = mk(N, H + 1, n, n), mk(N, H, n)
+        s.solve_tv(w["A"], w["B"], w["Q"], w["R"], Qf, w["x0"], H, tv=w["tv"], P=P, u=u)
+        pv, ua = mk(N, H + 1, n), mk(N, H, n)
+        r = torch.ones((1, 1, 1, n), device=DEV).expand(batch + (n,)).contiguous()
+        s.solve_affine(w["A"], w["B"], w["Q"], w["R"], Qf, r, w["x0"], H, tv=w["tv"], pvec=pv, u=ua)
+        torch.cuda.synchronize()
+        (got if tag == "null" else exp).update(o, P=P, u=u, pv=pv, ua=ua)
+    s.close()
+    for k in got:
+        assert not torch.any(got[k] == 123456.0), k
+        assert torch.equal(got[k], exp[k]), k
+    ww = dict(w, Qf=w["Q"])
+    ref = run_oracle(ww, g)
+    errs = errors({k: exp[k] for k in ("dA", "dQf", "dx0", "u0")}, ref)
+    assert all(v <= 1e-4 for v in errs.values()), errs
