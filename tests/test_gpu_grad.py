@@ -218,3 +218,33 @@ def test_null_terminal_weight_means_the_constant_state_cost(n):
     ref = run_oracle(ww, g)
     errs = errors({k: exp[k] for k in ("dA", "dQf", "dx0", "u0")}, ref)
     assert all(v <= 1e-4 for v in errs.values()), errs
+
+
+def test_grad_argument_errors():
+    n, m, H, batch = 8, 8, 4, (1, 1, 3)
+    w = tv_workload(n, m, H, batch, seed=1)
+    g = draw_g(3, m, 1)
+    s = lqr.LqrSolver(n, m, H, batch)
+    args = (w["A"], w["B"], w["Q"], w["R"], w["Qf"], w["x0"])
+    with pytest.raises(ValueError):                                            # g of the wrong shape: caught by the binding
+        s.grad(*args, g[:2], H, tv=w["tv"])
+    w5 = tv_workload(n, m, H + 1, batch, seed=2)
+    with pytest.raises(lqr.TtcError) as ei:                                    # horizon beyond the handle's maximum
+        s.grad(w5["A"], w5["B"], w5["Q"], w5["R"], w5["Qf"], w5["x0"], g, H + 1, tv=w5["tv"])
+    assert "INVALID_ARGUMENT" in str(ei.value)
+    with pytest.raises(lqr.TtcError) as ei:                                    # Q_t varies in time: Qf cannot be omitted
+        s.grad(w["A"], w["B"], w["Q"], w["R"], None, w["x0"], g, H, tv=w["tv"])
+    assert "INVALID_ARGUMENT" in str(ei.value)
+    mis = torch.empty(3 * n + 1, device=DEV)[1:].reshape(3, n)                 # 4-byte aligned only
+    with pytest.raises(lqr.TtcError) as ei:
+        s.grad(*args, g, H, tv=w["tv"], dx0=mis)
+    assert "INVALID_ARGUMENT" in str(ei.value)
+    s.close()
+    s = lqr.LqrSolver(n, m, H, batch, method=lqr.TTC_SCAN)
+    with pytest.raises(lqr.TtcError) as ei:
+        s.grad(*args, g, H, tv=w["tv"])
+    assert "UNSUPPORTED" in str(ei.value)
+    s.close()
+    # after the refused calls the handle still works
+    out = run_gpu(w, g)
+    assert all(v <= 1e-4 for v in errors(out, run_oracle(w, g)).values())
