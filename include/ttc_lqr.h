@@ -155,7 +155,8 @@ int ttc_lqr_solve(ttc_lqr_handle* h,
  * at every t); the matrix of step t of instance i starts at the operand's batch offset + t * tstride.
  * Qf [n][n] (F32 or BF16, batch strides like any operand) is the terminal weight; it may be NULL only when
  * tstride[2] == 0, and then Q_f = Q.  Everything else (outputs, info, flags, stream, errors) as ttc_lqr_solve.
- * Served by the fp32 kernels (n = m = 16 / 32 warp kernel, generic kernel otherwise); TTC_SCAN handles
+ * Served by the fp32 kernels (n = m = 16 / 32 warp kernel when A, B, R are all shared by the tokens of a head or all
+ * per token, generic kernel otherwise); TTC_SCAN handles
  * time-invariant problems only and returns TTC_STATUS_UNSUPPORTED here.
  */
 int ttc_lqr_solve_tv(ttc_lqr_handle* h,

@@ -182,9 +182,29 @@ __device__ __forceinline__ void load_head_operands(Smem<N>& sm, const SolveParam
     }
 }
 
+// Operands of ONE instance at time index t -> that instance's own copies (its N lanes; the caller synchronises the
+// segment).  Lane c takes column c of every row: N consecutive floats per request.
+template <int N>
+__device__ __forceinline__ void load_slot_operands(float* As, float* Bs, float* Rs, const SolveParams& p, long long oa,
+                                                   long long ob, long long orr, int t, bool la, bool lb, bool lr, int c)
+{
+    constexpr int LD = Shape<N>::LD;
+    const float* Ag = reinterpret_cast<const float*>(p.A.ptr) + oa + t * p.A.st;
+    const float* Bg = reinterpret_cast<const float*>(p.B.ptr) + ob + t * p.B.st;
+    const float* Rg = reinterpret_cast<const float*>(p.R.ptr) + orr + t * p.R.st;
+#pragma unroll 4
+    for (int k = 0; k < N; ++k) {
+        if (la) As[k * LD + c] = __ldg(Ag + k * N + c);
+        if (lb) Bs[k * LD + c] = __ldg(Bg + k * N + c);
+        if (lr) Rs[k * LD + c] = __ldg(Rg + k * N + c);
+    }
+}
+
 // TV = time-varying request (time strides or a terminal weight): the other instantiation carries none of that code.
 // AFF = linear control cost r_t'u_t (Prop. A.1: p_t, k_t); implies TV.
-template <int N, bool TV, bool AFF = false>
+// PT = A, B, R belong to the token, not to the head (the contextualised layer's situation): every instance keeps its own
+// copies behind the common part of shared memory and its lanes reload them; implies TV.
+template <int N, bool TV, bool AFF = false, bool PT = false>
 __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kernel(SolveParams p, int* chunk_counter)
 {
     using S = Shape<N>;
@@ -194,6 +214,10 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int sub = lane / N, c = lane % N;
     typename Smem<N>::Slot& sl = sm.slot[warp * S::IPW + sub];
+    float* own_ops = reinterpret_cast<float*>(smem_raw + ((sizeof(Smem<N>) + 15) & ~size_t(15))) + (warp * S::IPW + sub) * 3 * S::MAT;
+    float* const As = PT ? own_ops : sm.A;
+    float* const Bs = PT ? own_ops + S::MAT : sm.B;
+    float* const Rs = PT ? own_ops + 2 * S::MAT : sm.R;
     const int H = p.H;
     const long long chunks_per_head = (p.tcount + S::SLOTS - 1) / S::SLOTS;
     const long long nchunks = p.b0 * p.b1 * chunks_per_head;
@@ -218,8 +242,8 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
         const long long oa = operand_offset(p.A, inst0, p.b1, p.b2);
         const long long ob = operand_offset(p.B, inst0, p.b1, p.b2);
         const long long orr = operand_offset(p.R, inst0, p.b1, p.b2);
-        const bool tv_head = TV && (p.A.st | p.B.st | p.R.st) != 0;      // per-head operands change with the time index
-        if (tv_head || oa != offA || ob != offB || orr != offR) {
+        const bool tv_head = TV && (p.A.st | p.B.st | p.R.st) != 0;      // the operands change with the time index
+        if (!PT && (tv_head || oa != offA || ob != offB || orr != offR)) {
             load_head_operands<N>(sm, p, oa, ob, orr, TV ? H - 1 : 0, true, true, true);
             offA = oa; offB = ob; offR = orr;
         }
@@ -227,6 +251,11 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
         const int slot_idx = warp * S::IPW + sub;
         const bool active = slot_idx < ntok;                  // idle segments shadow the chunk's first instance
         const long long inst = inst0 + (active ? slot_idx : 0);
+        const long long oai = PT ? operand_offset(p.A, inst, p.b1, p.b2) : oa;
+        const long long obi = PT ? operand_offset(p.B, inst, p.b1, p.b2) : ob;
+        const long long ori = PT ? operand_offset(p.R, inst, p.b1, p.b2) : orr;
+        if (PT)
+            load_slot_operands<N>(As, Bs, Rs, p, oai, obi, ori, H - 1, true, true, true, c);    // ordered by the barrier below
         const long long oq = operand_offset(p.Q, inst, p.b1, p.b2) + (long long)c * N;
 
         float* Pout = (p.P && active) ? p.P + inst * (long long)(p.first_only ? 1 : H + 1) * N * N : nullptr;
@@ -256,10 +285,16 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
 
 #pragma unroll 1
         for (int ts = H - 1; ts >= 0; --ts) {
-            if (tv_head && ts != H - 1) {                     // A_t, B_t, R_t of this step (the whole CTA is in step)
-                __syncthreads();
-                load_head_operands<N>(sm, p, oa, ob, orr, ts, p.A.st != 0, p.B.st != 0, p.R.st != 0);
-                __syncthreads();
+            if (tv_head && ts != H - 1) {                     // A_t, B_t, R_t of this step
+                if (PT) {
+                    __syncwarp();
+                    load_slot_operands<N>(As, Bs, Rs, p, oai, obi, ori, ts, p.A.st != 0, p.B.st != 0, p.R.st != 0, c);
+                    __syncwarp();
+                } else {                                      // the whole CTA is in step
+                    __syncthreads();
+                    load_head_operands<N>(sm, p, oa, ob, orr, ts, p.A.st != 0, p.B.st != 0, p.R.st != 0);
+                    __syncthreads();
+                }
             }
             f32x2 vcol[N / 2], tcol[N / 2];
 #pragma unroll
@@ -269,7 +304,7 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
             }
 #pragma unroll 4
             for (int i = 0; i < N; ++i) {                     // V[:,c] = P B[:,c], T[:,c] = P A[:,c]
-                const float bic = sm.B[i * LD + c], aic = sm.A[i * LD + c];
+                const float bic = Bs[i * LD + c], aic = As[i * LD + c];
                 const f32x2 b2 = pack2(bic, bic), a2 = pack2(aic, aic);
                 const float* prow = sl.buf0 + i * LD;
 #pragma unroll
@@ -296,7 +331,7 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
             f32x2 s2[N / 2], y2[N / 2], p2[N / 2];
             {
                 float tmp[N];
-                load_row<N>(tmp, sm.R + c * LD);              // S[:,c] = R[:,c] + B' V[:,c]
+                load_row<N>(tmp, Rs + c * LD);              // S[:,c] = R[:,c] + B' V[:,c]
                 pack_row<N>(s2, tmp);
                 load_q_row<N>(tmp, p.Q, TV ? oq + ts * p.Q.st : oq);    // Pn[:,c] = Q_t[:,c] + A' T[:,c] ; Y[:,c] = B' T[:,c]
                 pack_row<N>(p2, tmp);
@@ -310,8 +345,8 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
                 const f32x2 vv = pack2(vk, vk), tt = pack2(tk, tk);
 #pragma unroll
                 for (int q = 0; q < N / 4; ++q) {             // each row of B and A is read once
-                    const ulonglong2 b4 = *reinterpret_cast<const ulonglong2*>(sm.B + k * LD + 4 * q);
-                    const ulonglong2 a4 = *reinterpret_cast<const ulonglong2*>(sm.A + k * LD + 4 * q);
+                    const ulonglong2 b4 = *reinterpret_cast<const ulonglong2*>(Bs + k * LD + 4 * q);
+                    const ulonglong2 a4 = *reinterpret_cast<const ulonglong2*>(As + k * LD + 4 * q);
                     fma2(s2[2 * q], vv, b4.x);
                     fma2(s2[2 * q + 1], vv, b4.y);
                     fma2(y2[2 * q], tt, b4.x);
@@ -331,8 +366,8 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
                 float gc = ts < p.r_count ? load_elem(p.r, orv + ts * p.r.st) : 0.f;
 #pragma unroll
                 for (int i = 0; i < N; ++i) {
-                    gc = fmaf(sm.B[i * LD + c], pvv[i], gc);
-                    apc = fmaf(sm.A[i * LD + c], pvv[i], apc);
+                    gc = fmaf(Bs[i * LD + c], pvv[i], gc);
+                    apc = fmaf(As[i * LD + c], pvv[i], apc);
                 }
                 sl.gv[c] = gc;
             }
@@ -513,8 +548,8 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
             float* uo = (p.u && store_ok) ? p.u + inst * (long long)(p.first_only ? N : H * N) : nullptr;
             float arow[N], brow[N];
             if (!tv_head) {
-                load_row<N>(arow, sm.A + c * LD);
-                load_row<N>(brow, sm.B + c * LD);
+                load_row<N>(arow, As + c * LD);
+                load_row<N>(brow, Bs + c * LD);
             }
             if (xo)
                 xo[c] = sl.x[c];
@@ -523,12 +558,18 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
             for (int ts = 0; ts < H; ++ts) {
                 if (tv_head) {                                // A_t, B_t of this step (after the backward pass they hold t = 0)
                     if (ts > 0) {
-                        __syncthreads();
-                        load_head_operands<N>(sm, p, oa, ob, orr, ts, p.A.st != 0, p.B.st != 0, false);
-                        __syncthreads();
+                        if (PT) {
+                            __syncwarp();
+                            load_slot_operands<N>(As, Bs, Rs, p, oai, obi, ori, ts, p.A.st != 0, p.B.st != 0, false, c);
+                            __syncwarp();
+                        } else {
+                            __syncthreads();
+                            load_head_operands<N>(sm, p, oa, ob, orr, ts, p.A.st != 0, p.B.st != 0, false);
+                            __syncthreads();
+                        }
                     }
-                    load_row<N>(arow, sm.A + c * LD);
-                    load_row<N>(brow, sm.B + c * LD);
+                    load_row<N>(arow, As + c * LD);
+                    load_row<N>(brow, Bs + c * LD);
                 }
                 float xv[N];
                 load_row<N>(xv, sl.x);
@@ -564,7 +605,11 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
 }
 
 template <int N>
-inline size_t smem_bytes() { return sizeof(Smem<N>); }
+inline size_t smem_bytes(bool per_token = false)
+{
+    // the per-token copies start on the next 16-byte boundary: their rows are read with 16-byte loads
+    return per_token ? ((sizeof(Smem<N>) + 15) & ~size_t(15)) + sizeof(float) * Shape<N>::SLOTS * 3 * Shape<N>::MAT : sizeof(Smem<N>);
+}
 
 } // namespace rwarp
 } // namespace ttc

@@ -398,7 +398,9 @@ int solve_window(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, 
             h->last_kernel = TTC_KERNEL_RICCATI_UMMA;
             return TTC_OK;
         }
-        if (head_shared && n == m && (n == 16 || n == 32)) {
+        // A, B, R either all per head or all per token (a mix goes to the generic kernel)
+        const bool per_token = A->bstride[2] != 0 && B->bstride[2] != 0 && R->bstride[2] != 0;
+        if ((head_shared || per_token) && n == m && (n == 16 || n == 32)) {
             // fp32 warp kernel: one instance per 16 / 32 lanes, chunks of tokens handed out by an atomic counter
             if ((s = ensure(h->ws_E, sizeof(int) * 4))) return s;
             int* counter = static_cast<int*>(h->ws_E.ptr);
@@ -407,15 +409,17 @@ int solve_window(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, 
             size_t smem;
             long long chunks, grid;
             if (n == 32) {
-                kern = affine ? rwarp::riccati_warp_kernel<32, true, true>
+                kern = per_token ? (affine ? rwarp::riccati_warp_kernel<32, true, true, true> : rwarp::riccati_warp_kernel<32, true, false, true>)
+                     : affine ? rwarp::riccati_warp_kernel<32, true, true>
                      : time_varying ? rwarp::riccati_warp_kernel<32, true> : rwarp::riccati_warp_kernel<32, false>;
-                smem = rwarp::smem_bytes<32>();
+                smem = rwarp::smem_bytes<32>(per_token);
                 chunks = p.b0 * p.b1 * ((tcount + rwarp::Shape<32>::SLOTS - 1) / rwarp::Shape<32>::SLOTS);
                 grid = (long long)h->sm_count * 3;
             } else {
-                kern = affine ? rwarp::riccati_warp_kernel<16, true, true>
+                kern = per_token ? (affine ? rwarp::riccati_warp_kernel<16, true, true, true> : rwarp::riccati_warp_kernel<16, true, false, true>)
+                     : affine ? rwarp::riccati_warp_kernel<16, true, true>
                      : time_varying ? rwarp::riccati_warp_kernel<16, true> : rwarp::riccati_warp_kernel<16, false>;
-                smem = rwarp::smem_bytes<16>();
+                smem = rwarp::smem_bytes<16>(per_token);
                 chunks = p.b0 * p.b1 * ((tcount + rwarp::Shape<16>::SLOTS - 1) / rwarp::Shape<16>::SLOTS);
                 grid = (long long)h->sm_count * 4;
             }

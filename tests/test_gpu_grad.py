@@ -120,7 +120,7 @@ def test_grad_per_token_dynamics():
     g = draw_g(28, m, 6)
     out = run_gpu(w, g)
     ref = run_oracle(w, g)
-    assert out["kernel"] == "riccati_cta"                      # per-token dynamics: the generic backward pass
+    assert out["kernel"] == "riccati_warp"                     # per-token dynamics: the warp kernel with per-instance copies
     assert all(v <= 1e-4 for v in errors(out, ref).values())
 
 
