@@ -176,10 +176,14 @@ def grad_oracle(w, g, idx, H):
     f64 = lambda t: t.to(torch.float64).cpu().numpy()
     t0 = time.perf_counter()
     refs = []
+    def head_or_token(t, i):                                 # A, B, R: [1, Hd, 1, ...] per head or [S, Hd, T, ...] per token
+        if t.shape[2] == 1:
+            return t[0, (int(i) // T) % Hd, 0]
+        return t.reshape((-1,) + t.shape[3:])[i]
+
     for i in idx:
-        head = (int(i) // T) % Hd
-        refs.append(og.grad(f64(w["A"][0, head, 0]), f64(w["B"][0, head, 0]), f64(w["Q"].reshape((-1,) + w["Q"].shape[3:])[i]),
-                            f64(w["R"][0, head, 0]), f64(w["Qf"].reshape((-1,) + w["Qf"].shape[3:])[i]),
+        refs.append(og.grad(f64(head_or_token(w["A"], i)), f64(head_or_token(w["B"], i)), f64(w["Q"].reshape((-1,) + w["Q"].shape[3:])[i]),
+                            f64(head_or_token(w["R"], i)), f64(w["Qf"].reshape((-1,) + w["Qf"].shape[3:])[i]),
                             f64(w["x0"].reshape(-1, w["x0"].shape[-1])[i]), f64(g[i]), H))
     ref = {k: np.stack([r[k] for r in refs]) for k in GRAD_NAMES}
     return ref, time.perf_counter() - t0
@@ -242,6 +246,12 @@ def run_grad(args):
         c["name"] += "_tokens%d" % args.tokens
     w = workloads.make_tv_workload(key, device=dev, batch=c["batch"], seed=sharding.rank_seed(100, rank), horizon=H)
     N = int(np.prod(c["batch"]))
+    if args.per_token:
+        # the contextualised layer's situation: every token its own A_t, B_t, R_t (here copies of the head's, which
+        # costs the same traffic and arithmetic as distinct ones)
+        for k in ("A", "B", "R"):
+            w[k] = w[k].expand(tuple(c["batch"]) + w[k].shape[3:]).contiguous()
+        c["name"] += "_per_token"
     gen = torch.Generator(device=dev)
     gen.manual_seed(sharding.rank_seed(300, rank))
     g = torch.randn((N, m), generator=gen, device=dev)
@@ -281,7 +291,7 @@ def run_grad(args):
             td.destroy_process_group()
         return
     # algorithmic bytes: Q_t, Q_f, x_0, g in (the per-head A_t, B_t, R_t are negligible); every gradient, u_0, info out
-    bin_i = 4 * (H * n * n + n * n + n + m)
+    bin_i = 4 * (H * n * n + n * n + n + m) + (4 * H * (n * n + n * m + m * m) if args.per_token else 0)
     bout_i = 4 * (H * (2 * n * n + n * m + m * m) + n * n + n + m + 1)
     kernel_ms = statistics.median(per_step)
     ach = N * (bin_i + bout_i) / (kernel_ms * 1e-3) / 1e9
@@ -511,6 +521,7 @@ def main():
     ap.add_argument("--tokens", type=int, default=0, help="override the token count (small profiling captures)")
     ap.add_argument("--horizon", type=int, default=0, help="layer workloads: override the planning horizon T (sweeps)")
     ap.add_argument("--batch", default="", help="layer and gradient workloads: override the batch as SxHxT, e.g. 1x16x64 (sweeps)")
+    ap.add_argument("--per-token", action="store_true", help="grad16: A_t, B_t, R_t per token instead of per head")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
