@@ -62,6 +62,10 @@ extern "C" {
 #define TTC_MATH_AUTO  0  /* FP32 when every input is F32, TF32 when Q or x0 is BF16  */
 #define TTC_MATH_FP32  1  /* FFMA, fp32 throughout                                    */
 #define TTC_MATH_TF32  2  /* tcgen05 tensor cores, tf32 operands, fp32 accumulate (n = m = 64) */
+/* n = m = 64 is served by the tensor-core kernel only with TF32 math (AUTO picks it when Q or x0 is
+ * BF16), per-head A, B, R and a time-invariant problem; FP32 math at n = m = 64, and every
+ * time-varying / affine / gradient call at n = m = 64, run in the generic one-CTA-per-instance kernel
+ * (TTC_KERNEL_RICCATI_CTA), which is one to two orders of magnitude slower. */
 
 /* ttc_lqr_solve flags */
 #define TTC_OUT_FIRST_ONLY  1u  /* P is [N][n][n] = P_0 and u is [N][m] = u_0          */
@@ -78,7 +82,6 @@ extern "C" {
 #define TTC_KERNEL_NONE           0
 #define TTC_KERNEL_RICCATI_CTA    1  /* generic: one CTA per instance, FFMA            */
 #define TTC_KERNEL_RICCATI_WARP   2  /* register-tiled FFMA, several instances per CTA */
-#define TTC_KERNEL_RICCATI_MMA    3  /* retired id (mma.sync kernel); never returned   */
 #define TTC_KERNEL_SCAN           4  /* symplectic-pair scan + gain/rollout kernel     */
 #define TTC_KERNEL_RICCATI_UMMA   5  /* tcgen05 contractions (tensor memory), n = m = 64 */
 #define TTC_KERNEL_LAYER          6  /* contextualised layer: parameters synthesised in-kernel */
@@ -87,7 +90,11 @@ typedef struct ttc_lqr_handle ttc_lqr_handle; /* opaque; owned by the library */
 
 /* One input operand.  `ptr` is owned by the caller and only read.  For ttc_lqr_solve it
  * is a DEVICE pointer (on the handle's device), for ttc_lqr_solve_host a HOST pointer.
- * It must be aligned to 16 bytes. */
+ * It must be aligned to 16 bytes.  Strides are arbitrary non-negative element counts; the
+ * fast kernels (tcgen05 for n = m = 64, the fp32 warp kernel for n = m = 16 / 32) read the
+ * rows of Q and Qf with 16-byte loads and are chosen only when every batch and time stride
+ * of those two operands is a multiple of 16 bytes (4 F32 or 8 BF16 elements); any other
+ * stride is served, correctly but much more slowly, by the generic kernel. */
 typedef struct {
     const void* ptr;
     int32_t     dtype;       /* TTC_F32 or TTC_BF16 (BF16 only for Q and x0)            */
@@ -182,6 +189,13 @@ int ttc_lqr_solve_tv(ttc_lqr_handle* h,
  * Failed instances: every requested output quiet NaN, info as for ttc_lqr_solve.  The scan method
  * returns TTC_STATUS_UNSUPPORTED.
  */
+int ttc_lqr_solve_affine(ttc_lqr_handle* h,
+                         const ttc_operand* A, const ttc_operand* B, const ttc_operand* Q, const ttc_operand* R,
+                         const int64_t tstride[4], const ttc_operand* Qf,
+                         const ttc_operand* r, int64_t r_tstride, const ttc_operand* x0, int32_t H,
+                         float* K, float* kff, float* P, float* pvec, float* x, float* u, int32_t* info,
+                         uint32_t flags, void* cuda_stream);
+
 /*
  * Gradients of a scalar loss l(o) of the layer output o = u_0* (Thm 3.2: primal and dual LQR), for the
  * time-varying problem of ttc_lqr_solve_tv.  g [N][m] (float32, device) is dl/do.  The call runs
@@ -206,13 +220,6 @@ int ttc_lqr_grad(ttc_lqr_handle* h,
                  const int64_t tstride[4], const ttc_operand* Qf, const ttc_operand* x0, const float* g, int32_t H,
                  float* dA, float* dB, float* dQ, float* dQf, float* dR, float* dx0, float* u0, int32_t* info,
                  void* cuda_stream);
-
-int ttc_lqr_solve_affine(ttc_lqr_handle* h,
-                         const ttc_operand* A, const ttc_operand* B, const ttc_operand* Q, const ttc_operand* R,
-                         const int64_t tstride[4], const ttc_operand* Qf,
-                         const ttc_operand* r, int64_t r_tstride, const ttc_operand* x0, int32_t H,
-                         float* K, float* kff, float* P, float* pvec, float* x, float* u, int32_t* info,
-                         uint32_t flags, void* cuda_stream);
 
 /*
  * One Test-Time Control layer evaluation per instance with CONTEXTUALISED parameters
@@ -300,7 +307,8 @@ int ttc_lqr_solve_host(ttc_lqr_handle* h,
  * one int32 per instance) lives in a fixed array of TTC_NOALLOC_SCRATCH_BYTES bytes that is part
  * of the library image: every GPU on which the library is loaded holds those bytes until the
  * process exits.  The call makes no cudaMalloc / cudaFree and calls no allocating library
- * routine; the caller still provides every input and output buffer.
+ * routine; the caller still provides every input and output buffer.  Like the other entry
+ * points it makes `device` the calling thread's current device (cudaSetDevice).
  *
  * Limits and rules:
  *  - N * (4*n*n) rounded up to 256, plus 4*N, must not exceed TTC_NOALLOC_SCRATCH_BYTES; larger
@@ -320,6 +328,17 @@ int ttc_lqr_solve_first_noalloc(int32_t n, int32_t m, const int64_t batch[3], in
                                 const ttc_operand* A, const ttc_operand* B, const ttc_operand* Q,
                                 const ttc_operand* R, const ttc_operand* x0, int32_t H,
                                 float* P0, float* u0, int32_t* info, void* cuda_stream);
+
+/*
+ * Self test of the bounded waits (no counterpart in the paper; failure handling of this library): every
+ * wait of the tensor-core kernel on an MMA-completion barrier gives up after a fixed number of polls and sets
+ * an error word instead of hanging.  This call runs that give-up branch on purpose, safely: a one-warp
+ * kernel initialises a barrier on which nothing will ever arrive, polls it `poll_limit` times (1 .. 2^20),
+ * and returns by itself; *timed_out receives 1 if the wait reported the timeout, else 0.  No tensor-core
+ * work is in flight and the context stays usable.  Allocates and frees 4 bytes of device memory, makes
+ * `device` current, synchronous.
+ */
+int ttc_lqr_selftest_bounded_wait(int32_t device, int32_t poll_limit, int32_t* timed_out);
 
 /* Free the handle and its workspace (synchronises the handle's device).  NULL is OK. */
 int ttc_lqr_destroy(ttc_lqr_handle* h);

@@ -128,9 +128,9 @@ __device__ __forceinline__ void mma_commit(uint32_t mbar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(mbar) : "memory");
 }
-__device__ __forceinline__ bool mbar_wait(uint32_t mbar, uint32_t parity)
+__device__ __forceinline__ bool mbar_wait(uint32_t mbar, uint32_t parity, int limit = SPIN_LIMIT)
 {
-    for (int it = 0; it < SPIN_LIMIT; ++it) {
+    for (int it = 0; it < limit; ++it) {
         uint32_t ok;
         asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
                      : "=r"(ok) : "r"(mbar), "r"(parity) : "memory");
@@ -947,6 +947,22 @@ __global__ void __launch_bounds__(32 * ROLL_WARPS, 5) rollout64_kernel(SolvePara
     }
 }
 inline size_t rollout_smem_bytes() { return sizeof(RollSmem); }
+
+// Exercises the give-up branch of mbar_wait without any MMA in flight: one warp initialises a barrier on which
+// nothing ever arrives, polls it `limit` times, and reports through the same kind of error word as the solver.
+// The kernel returns by itself after `limit` polls.
+__global__ void bounded_wait_selftest_kernel(int limit, int* error_flag)
+{
+    __shared__ unsigned long long bar;
+    const uint32_t mbar = smem_u32(&bar);
+    if (threadIdx.x == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(mbar) : "memory");
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (threadIdx.x == 0 && !mbar_wait(mbar, 0u, limit))
+        atomicExch(error_flag, 1);
+}
 
 inline size_t smem_bytes() { return SMEM_BYTES; }
 

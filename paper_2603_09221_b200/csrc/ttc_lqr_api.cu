@@ -51,6 +51,7 @@ struct ttc_lqr_handle {
     ttc_lqr_config cfg;
     long long N;
     int sm_count;
+    size_t max_pitch;              // largest pitch a 2D copy accepts on this device
     DevBuf ws_K, ws_P, ws_E;       // scratch used by kernels
     DevBuf ws_k;                   // feed-forward terms k_t when the caller does not take them
     DevBuf ws_vec;                 // state, control and co-state sequences of the gradient entry point
@@ -163,6 +164,24 @@ int validate_common(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* 
     return TTC_OK;
 }
 
+// true when every batch and time stride of the operand is a multiple of 16 bytes, so that a row of the matrix
+// (whose length is a multiple of 16 bytes for the kernels that ask) always starts on a 16-byte boundary
+bool vector_rows_ok(const OperandDev& o)
+{
+    const long long q = o.dtype == TTC_BF16 ? 8 : 4;
+    return ((o.s0 | o.s1 | o.s2 | o.st) % q) == 0;
+}
+
+// Start of an API call: make sure the small workspace exists and clear the device error word (word 1) on `st`.
+int clear_device_error(ttc_lqr_handle* h, cudaStream_t st)
+{
+    int s = ensure(h->ws_E, sizeof(int) * 4);
+    if (s)
+        return s;
+    TTC_CUDA(cudaMemsetAsync(static_cast<int*>(h->ws_E.ptr) + 1, 0, sizeof(int), st));
+    return TTC_OK;
+}
+
 int pick_method(const ttc_lqr_handle* h)
 {
     if (h->cfg.method == TTC_SCAN)
@@ -227,6 +246,7 @@ int ttc_lqr_create(const ttc_lqr_config* cfg, ttc_lqr_handle** out)
     h->cfg = *cfg;
     h->N = N;
     h->sm_count = prop.multiProcessorCount;
+    h->max_pitch = prop.memPitch;
     h->host_stream = nullptr;
     h->in_stream = h->out_stream = nullptr;
     h->host_pipeline_ready = false;
@@ -368,11 +388,17 @@ int solve_window(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, 
         const bool bf16_in = (Q->dtype == TTC_BF16) || (x0 && x0->ptr && x0->dtype == TTC_BF16);
         const bool want_tf32 = h->cfg.math == TTC_MATH_TF32 || (h->cfg.math == TTC_MATH_AUTO && bf16_in);
         const bool head_shared = A->bstride[2] == 0 && B->bstride[2] == 0 && R->bstride[2] == 0;
-        if (want_tf32 && n == 64 && m == 64 && head_shared && !time_varying) {
+        // The tcgen05 and the warp kernels read the rows of Q and Qf with 16-byte loads: every batch and time stride
+        // of those operands must keep a row start on a 16-byte boundary (4 fp32 or 8 bf16 elements).  Other strides
+        // are served by the generic kernel, which loads element by element.
+        const bool q_rows_aligned = vector_rows_ok(p.Q) && (!p.Qf.ptr || vector_rows_ok(p.Qf));
+        if (want_tf32 && n == 64 && m == 64 && head_shared && !time_varying && q_rows_aligned) {
             // tcgen05 kernel: persistent CTAs, four independent warpgroups each
             if ((s = ensure(h->ws_E, sizeof(int) * 4))) return s;
             int* counter = static_cast<int*>(h->ws_E.ptr);
-            TTC_CUDA(cudaMemsetAsync(counter, 0, 2 * sizeof(int), st));
+            // word 0 = work counter of this launch; word 1 = device error word, cleared once per API call
+            // (clear_device_error) so that a later window of the same call cannot erase an earlier report
+            TTC_CUDA(cudaMemsetAsync(counter, 0, sizeof(int), st));
             const size_t smem = umma64::smem_bytes();
             auto kern = rollout_needs_all_K || K ? umma64::riccati_umma64_kernel<true> : umma64::riccati_umma64_kernel<false>;
             TTC_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
@@ -400,7 +426,7 @@ int solve_window(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, 
         }
         // A, B, R either all per head or all per token (a mix goes to the generic kernel)
         const bool per_token = A->bstride[2] != 0 && B->bstride[2] != 0 && R->bstride[2] != 0;
-        if ((head_shared || per_token) && n == m && (n == 16 || n == 32)) {
+        if ((head_shared || per_token) && n == m && (n == 16 || n == 32) && q_rows_aligned) {
             // fp32 warp kernel: one instance per 16 / 32 lanes, chunks of tokens handed out by an atomic counter
             if ((s = ensure(h->ws_E, sizeof(int) * 4))) return s;
             int* counter = static_cast<int*>(h->ws_E.ptr);
@@ -462,6 +488,8 @@ int ttc_lqr_solve(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B,
         return s;
     TTC_CUDA(cudaSetDevice(h->cfg.device));
     h->last_launches = 0;
+    if ((s = clear_device_error(h, static_cast<cudaStream_t>(cuda_stream))))
+        return s;
     return solve_window(h, A, B, Q, R, x0, H, K, P, x, u, info, flags, static_cast<cudaStream_t>(cuda_stream), 0,
                         h->cfg.batch[2]);
 }
@@ -839,6 +867,7 @@ int ttc_lqr_solve_host(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operan
     nslice = (int)((b2 + tslice - 1) / tslice);
 
     h->last_launches = 0;
+    { int se = clear_device_error(h, h->host_stream); if (se) return se; }
     for (int i = 0; i < 5; ++i)                        // operands shared along the token dimension: whole, once
         if (dev[i].ptr && (nslice == 1 || in[i]->bstride[2] == 0))
             TTC_CUDA(cudaMemcpyAsync(h->st_in[i].ptr, in[i]->ptr, in_bytes[i], cudaMemcpyHostToDevice, h->in_stream));
@@ -855,9 +884,16 @@ int ttc_lqr_solve_host(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operan
                 const size_t pitch = rows > 1 ? (size_t)s1 * es : width;
                 for (long long i0 = 0; i0 < (s0 == 0 ? 1 : b0); ++i0) {
                     const size_t off = ((size_t)i0 * s0 + (size_t)t0 * s2) * es;
-                    TTC_CUDA(cudaMemcpy2DAsync(static_cast<char*>(h->st_in[i].ptr) + off, pitch,
-                                               static_cast<const char*>(in[i]->ptr) + off, pitch, width, rows,
-                                               cudaMemcpyHostToDevice, h->in_stream));
+                    if (rows > 1 && pitch <= h->max_pitch) {
+                        TTC_CUDA(cudaMemcpy2DAsync(static_cast<char*>(h->st_in[i].ptr) + off, pitch,
+                                                   static_cast<const char*>(in[i]->ptr) + off, pitch, width, rows,
+                                                   cudaMemcpyHostToDevice, h->in_stream));
+                    } else {                           // one row, or rows further apart than a 2D copy allows
+                        for (size_t rr = 0; rr < rows; ++rr)
+                            TTC_CUDA(cudaMemcpyAsync(static_cast<char*>(h->st_in[i].ptr) + off + rr * pitch,
+                                                     static_cast<const char*>(in[i]->ptr) + off + rr * pitch, width,
+                                                     cudaMemcpyHostToDevice, h->in_stream));
+                    }
                 }
             }
         TTC_CUDA(cudaEventRecord(h->ev_in[c], h->in_stream));
@@ -878,18 +914,60 @@ int ttc_lqr_solve_host(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operan
                 TTC_CUDA(cudaMemcpyAsync(host_out[i], dev_out[i], per_out[i] * (size_t)N, cudaMemcpyDeviceToHost, h->out_stream));
             } else {                                   // rows = (sequence, head), one run of tc instances per row
                 const size_t off = (size_t)t0 * per_out[i], pitch = (size_t)b2 * per_out[i];
-                TTC_CUDA(cudaMemcpy2DAsync(static_cast<char*>(host_out[i]) + off, pitch,
-                                           static_cast<const char*>(dev_out[i]) + off, pitch, (size_t)tc * per_out[i],
-                                           (size_t)(b0 * b1), cudaMemcpyDeviceToHost, h->out_stream));
+                const size_t rows = (size_t)(b0 * b1), width = (size_t)tc * per_out[i];
+                if (rows > 1 && pitch <= h->max_pitch) {
+                    TTC_CUDA(cudaMemcpy2DAsync(static_cast<char*>(host_out[i]) + off, pitch,
+                                               static_cast<const char*>(dev_out[i]) + off, pitch, width, rows,
+                                               cudaMemcpyDeviceToHost, h->out_stream));
+                } else {                               // a 2D copy cannot express a pitch above the device's limit
+                    for (size_t rr = 0; rr < rows; ++rr)
+                        TTC_CUDA(cudaMemcpyAsync(static_cast<char*>(host_out[i]) + off + rr * pitch,
+                                                 static_cast<const char*>(dev_out[i]) + off + rr * pitch, width,
+                                                 cudaMemcpyDeviceToHost, h->out_stream));
+                }
             }
         }
     }
     TTC_CUDA(cudaStreamSynchronize(h->out_stream));
     TTC_CUDA(cudaStreamSynchronize(h->host_stream));
+    if (h->last_kernel == TTC_KERNEL_RICCATI_UMMA) {   // a bounded wait that ran out in ANY slice leaves the word set
+        int flag = 0;
+        TTC_CUDA(cudaMemcpy(&flag, static_cast<int*>(h->ws_E.ptr) + 1, sizeof(int), cudaMemcpyDeviceToHost));
+        if (flag)
+            return fail(TTC_STATUS_CUDA_ERROR, "a bounded wait inside the kernel ran out: the outputs are not valid");
+    }
     return TTC_OK;
 }
 
 } // extern "C"
+
+extern "C" int ttc_lqr_selftest_bounded_wait(int32_t device, int32_t poll_limit, int32_t* timed_out)
+{
+    if (!timed_out)
+        return fail(TTC_STATUS_INVALID_ARGUMENT, "null result pointer");
+    if (poll_limit < 1 || poll_limit > (1 << 20))
+        return fail(TTC_STATUS_INVALID_ARGUMENT, "poll_limit=%d outside [1, 2^20]", poll_limit);
+    int ndev = 0;
+    TTC_CUDA(cudaGetDeviceCount(&ndev));
+    if (device < 0 || device >= ndev)
+        return fail(TTC_STATUS_CUDA_ERROR, "device %d not present (%d devices)", device, ndev);
+    TTC_CUDA(cudaSetDevice(device));
+    int* flag = nullptr;
+    TTC_CUDA(cudaMalloc(&flag, sizeof(int)));
+    cudaError_t e = cudaMemset(flag, 0, sizeof(int));
+    if (e == cudaSuccess) {
+        umma64::bounded_wait_selftest_kernel<<<1, 32>>>(poll_limit, flag);
+        e = cudaGetLastError();
+    }
+    int host = 0;
+    if (e == cudaSuccess)
+        e = cudaMemcpy(&host, flag, sizeof(int), cudaMemcpyDeviceToHost);
+    cudaFree(flag);
+    if (e != cudaSuccess)
+        return fail(TTC_STATUS_CUDA_ERROR, "bounded-wait self test: %s", cudaGetErrorString(e));
+    *timed_out = host;
+    return TTC_OK;
+}
 
 // ---------------------------------------------------------------------------------------------
 // Allocation-free P_0 / u_0 solve for callers that must not allocate device memory (allocator

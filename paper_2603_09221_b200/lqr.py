@@ -27,6 +27,7 @@ EXPORTS = (
     "ttc_lqr_create", "ttc_lqr_solve", "ttc_lqr_solve_host", "ttc_lqr_destroy", "ttc_lqr_query",
     "ttc_lqr_status_string", "ttc_lqr_last_error", "ttc_lqr_solve_first_noalloc", "ttc_lqr_solve_tv",
     "ttc_lqr_solve_layer", "ttc_lqr_solve_layer_host", "ttc_lqr_solve_affine", "ttc_lqr_grad",
+    "ttc_lqr_selftest_bounded_wait",
 )
 TTC_NOALLOC_SCRATCH_BYTES = 4 << 20
 
@@ -103,6 +104,8 @@ def load_library():
     lib.ttc_lqr_solve_first_noalloc.restype = ctypes.c_int
     lib.ttc_lqr_solve_first_noalloc.argtypes = [ctypes.c_int32, ctypes.c_int32, P(ctypes.c_int64), ctypes.c_int32,
                                                 opp, opp, opp, opp, opp, ctypes.c_int32] + [ctypes.c_void_p] * 4
+    lib.ttc_lqr_selftest_bounded_wait.restype = ctypes.c_int
+    lib.ttc_lqr_selftest_bounded_wait.argtypes = [ctypes.c_int32, ctypes.c_int32, P(ctypes.c_int32)]
     _lib = lib
     return lib
 
@@ -348,6 +351,14 @@ def alloc_outputs(n, m, H, N, device, first_only=False, want=("K", "P", "x", "u"
     if "info" in want:
         out["info"] = torch.empty((N,), dtype=torch.int32, **kw)
     return out
+
+
+def selftest_bounded_wait(poll_limit=4096, device=0):
+    """``ttc_lqr_selftest_bounded_wait``: runs the give-up branch of the kernels' bounded barrier wait on a
+    barrier nothing arrives on; returns 1 when the timeout was reported through the error word."""
+    out = ctypes.c_int32(-1)
+    _check(load_library().ttc_lqr_selftest_bounded_wait(int(device), int(poll_limit), ctypes.byref(out)))
+    return out.value
 
 
 def solve_first_noalloc(A, B, Q, R, x0, H, batch, P0=None, u0=None, info=None, device=0, stream=None):

@@ -1,15 +1,17 @@
 """Helpers shared by the GPU parity tests: run the CUDA library, run the oracle on the same
 inputs (all or a sample of instances), and the error measure.
 
-Error measure ("max relative error" of the target statement, made precise), per output tensor:
-  K, P : per instance and per time block t,
-         err = max|gpu - ref| / max( max|ref block|, 1e-6 * max over t of max|ref| )
-  x, u : per instance, err = max over t of max|gpu - ref| / max over t of max|ref|
-         (normalised by the trajectory, not by the block: the closed loop contracts the state by
-         orders of magnitude over the horizon and x_{t+1} = A x_t + B u_t cancels, so the error of
-         ANY fp32 result relative to a late, tiny block is >= 1e-5 even with exact gains rounded to
-         fp32; the block-wise figure is still computed and printed for information)
-and the reported figure is the maximum over instances (and t).
+Error measure ("max relative error" of the target statement, made precise), per output tensor, per
+instance and per time block t:
+    err = max|gpu - ref| / max( max|ref block|, floor * max over t of max|ref| )
+with floor = 1e-6 for K and P and floor = XU_FLOOR = 1e-4 for x and u; the reported figure is the maximum
+over instances and t.  The closed loop contracts the state by many orders of magnitude over the horizon
+(down to 3e-8 of |x_0| on the 16-state configuration, 1e-29 on the 32-state one) while
+x_{t+1} = A x_t + B u_t cancels, so the rounding of ANY float32 computation is an absolute error on the
+scale of the trajectory: tests/test_numerics_xu_error_measure.py shows a plain float32 recursion (LAPACK
+Cholesky) at 2.2e-4 with a floor of 1e-6 and at 2.8e-5 with 1e-4, which is therefore the smallest decade
+at which a 1e-4 bound is a property of the arithmetic and not of the sample.  The trajectory-normalised
+figure (floor = 1: max over t of the error / max over t of the reference) is computed and returned too.
 """
 import numpy as np
 import torch
@@ -18,7 +20,10 @@ from oracle import lqr_oracle as orc
 from paper_2603_09221_b200 import lqr
 
 
-def block_rel_err(gpu, ref, block_ndim, per_block=True):
+XU_FLOOR = 1e-4      # floor of the block-wise measure for x and u, relative to the largest block of the trajectory
+
+
+def block_rel_err(gpu, ref, block_ndim, per_block=True, floor=1e-6):
     """gpu/ref: [M, T, ...block...] (or [M, ...block...] when there is no time axis)."""
     gpu = np.asarray(gpu, dtype=np.float64)
     ref = np.asarray(ref, dtype=np.float64)
@@ -34,8 +39,8 @@ def block_rel_err(gpu, ref, block_ndim, per_block=True):
     blk = np.abs(r).max(axis=2)
     if not per_block:
         return float((diff.max(axis=1) / np.maximum(blk.max(axis=1), 1e-300)).max())
-    floor = 1e-6 * blk.max(axis=1, keepdims=True)
-    return float((diff / np.maximum(np.maximum(blk, floor), 1e-300)).max())
+    lo = floor * blk.max(axis=1, keepdims=True)
+    return float((diff / np.maximum(np.maximum(blk, lo), 1e-300)).max())
 
 
 def run_gpu(w, method=lqr.TTC_RICCATI, want=("K", "P", "x", "u", "info"), first_only=None, math=lqr.TTC_MATH_AUTO,
@@ -113,7 +118,8 @@ def run_oracle_tv(w, idx=None, first_only=None, H=None, nthreads=0):
 
 
 def compare(gpu, ref, idx, tol, names=("K", "P", "x", "u")):
-    """Returns {name: err}; asserts every requested output is within tol and info == 0."""
+    """Returns {name: err} with the block-wise figure of every requested output and, for x and u, the
+    trajectory-normalised one under "x_traj" / "u_traj"; asserts all of them within tol and info == 0."""
     n_dims = {"K": 2, "P": 2, "x": 1, "u": 1}
     errs = {}
     sel = torch.as_tensor(idx, dtype=torch.long)
@@ -121,7 +127,11 @@ def compare(gpu, ref, idx, tol, names=("K", "P", "x", "u")):
         if k not in gpu or k not in ref:
             continue
         g = gpu[k].cpu()[sel].numpy()
-        errs[k] = block_rel_err(g, ref[k], n_dims[k], per_block=k in ("K", "P"))
+        if k in ("x", "u"):
+            errs[k] = block_rel_err(g, ref[k], n_dims[k], floor=XU_FLOOR)
+            errs[k + "_traj"] = block_rel_err(g, ref[k], n_dims[k], per_block=False)
+        else:
+            errs[k] = block_rel_err(g, ref[k], n_dims[k])
     if "info" in gpu:
         assert int(gpu["info"].cpu()[sel].abs().max()) == 0, "GPU reported failures on valid inputs"
     assert int(np.abs(ref["info"]).max()) == 0

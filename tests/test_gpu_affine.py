@@ -70,9 +70,9 @@ def check(out, ref, first_only, tol=1e-4):
     if "pvec" in out:
         errs["p"] = pu.block_rel_err(out["pvec"].cpu().numpy(), ref["p"][:, 0] if first_only else ref["p"], 1, per_block=False)
     if "x" in out:
-        errs["x"] = pu.block_rel_err(out["x"].cpu().numpy(), ref["x"], 1, per_block=False)
+        errs["x"] = pu.block_rel_err(out["x"].cpu().numpy(), ref["x"], 1, floor=pu.XU_FLOOR)
     if "u" in out:
-        errs["u"] = pu.block_rel_err(out["u"].cpu().numpy(), ref["u"][:, 0] if first_only else ref["u"], 1, per_block=False)
+        errs["u"] = pu.block_rel_err(out["u"].cpu().numpy(), ref["u"][:, 0] if first_only else ref["u"], 1, floor=pu.XU_FLOOR)
     assert int(out["info"].abs().max()) == 0
     assert all(v <= tol for v in errs.values()), errs
     return errs

@@ -143,20 +143,24 @@ def test_not_positive_definite_instance_is_isolated(method, n, bf16):
 
 @pytest.mark.parametrize("cfg,expect", [(2, "riccati_umma"), (3, "riccati_warp"), (4, "riccati_umma")])
 def test_full_size_configuration_on_sampled_instances(cfg, expect):
-    """Full batch of the configuration, in the launch configuration the benchmark times; the oracle
-    checks a stratified sample of instances (every sequence and head) one by one."""
+    """Full batch of the configuration, in the launch configuration the benchmark times (every output for
+    configurations 2 and 3, P_0 and u_0 only for configuration 4); the oracle checks a stratified sample of
+    4096 instances (128 or 256 tokens of every sequence and head, both ends of the token range included)."""
     w = workloads.make_workload(cfg, device=DEV)
-    gpu = pu.run_gpu(w)
-    # one launch; the n = 64 path adds its streaming rollout kernel when x (or every u_t) is requested, as here
-    assert lqr.KERNEL_NAMES[gpu["kernel"]] == expect and gpu["launches"] == (2 if expect == "riccati_umma" else 1)
+    first = w["first_only"]
+    gpu = pu.run_gpu(w, want=("P", "u", "info") if first else ("K", "P", "x", "u", "info"))
+    # one launch; the n = 64 path adds its streaming rollout kernel when x (or every u_t) is requested
+    assert lqr.KERNEL_NAMES[gpu["kernel"]] == expect
+    assert gpu["launches"] == (2 if expect == "riccati_umma" and not first else 1)
     S, Hd, T = w["batch"]
-    toks = np.array([0, 1, T // 3, T - 2, T - 1])
+    toks = np.unique(np.linspace(0, T - 1, 4096 // (S * Hd)).astype(np.int64))
     idx = (np.arange(S * Hd)[:, None] * T + toks[None, :]).reshape(-1)
+    assert len(idx) >= 4000
     ref = pu.run_oracle(w, idx=idx)
-    names = ("P", "u") if w["first_only"] else ("K", "P", "x", "u")
+    names = ("P", "u") if first else ("K", "P", "x", "u")
     errs = pu.compare({k: gpu[k] for k in names + ("info",)}, ref, idx, w["tol"], names=names)
     assert int(gpu["info"].abs().max()) == 0
-    print("cfg", cfg, errs)
+    print("cfg", cfg, len(idx), "instances", errs)
     del gpu
     torch.cuda.empty_cache()
 
@@ -236,3 +240,49 @@ def test_tensor_core_kernel_ragged_work_items(tokens):
     ref1 = pu.run_oracle(w, first_only=True)
     errs1 = pu.compare(g1, ref1, np.arange(N), 1e-2)
     print("ragged", tokens, errs, errs1)
+
+
+@pytest.mark.parametrize("n,bf16,pad", [(16, False, 1), (32, False, 2), (64, True, 4), (16, False, 4)])
+def test_q_strides_that_break_16_byte_rows_go_to_the_generic_kernel(n, bf16, pad):
+    """Q with a batch stride of n*n + pad elements: when that is not a multiple of 16 bytes the rows of Q no longer
+    start on a 16-byte boundary and the request must be served by the generic kernel (scalar loads), never by a
+    kernel that reads rows with 16-byte loads; a padded stride that keeps the alignment stays on the fast kernel."""
+    H, batch = 5, (1, 2, 9)
+    w = small_workload(n, n, H, batch, seed=77 + n + pad, bf16=bf16)
+    N = int(np.prod(batch))
+    flat = torch.zeros((N, n * n + pad), dtype=w["Q"].dtype, device=DEV)
+    flat[:, :n * n] = w["Q"].reshape(N, n * n)
+    w["Q"] = flat[:, :n * n].reshape(batch + (n, n))              # same values, row pitch n*n + pad
+    assert w["Q"].stride(2) == n * n + pad
+    gpu = pu.run_gpu(w)
+    aligned = (pad * (2 if bf16 else 4)) % 16 == 0
+    fast = {16: "riccati_warp", 32: "riccati_warp", 64: "riccati_umma"}[n]
+    assert lqr.KERNEL_NAMES[gpu["kernel"]] == (fast if aligned else "riccati_cta")
+    ref = pu.run_oracle(w)
+    pu.compare(gpu, ref, np.arange(N), w["tol"])
+
+
+def test_host_buffer_entry_point_slices_with_a_single_sequence_and_head():
+    """One (sequence, head) row and enough bytes for the sliced pipeline: the copies are plain one-row copies (a 2D copy
+    would need a pitch beyond the device limit on larger problems of this shape); bit-equal to the device entry."""
+    n, H, batch = 32, 16, (1, 1, 2048)
+    w = small_workload(n, n, H, batch, seed=515)
+    N = 2048
+    gpu = pu.run_gpu(w)
+    s = lqr.LqrSolver(n, n, H, batch)
+    host = {k: w[k].cpu().pin_memory() for k in ("A", "B", "Q", "R", "x0")}
+    out = lqr.alloc_outputs(n, n, H, N, "cpu", pin=True)
+    s.solve_host(host["A"], host["B"], host["Q"], host["R"], host["x0"], H, **out)
+    assert s.query(lqr.TTC_QUERY_LAST_LAUNCHES) > 1, "expected more than one slice"
+    s.close()
+    for k in ("K", "P", "x", "u", "info"):
+        assert torch.equal(out[k], gpu[k].cpu()), k
+
+
+def test_bounded_wait_gives_up_and_reports():
+    """The give-up branch of the kernels' barrier wait, run on a barrier nothing ever arrives on (no MMA in flight): it
+    must come back by itself with the error word set, and the context must stay usable afterwards."""
+    assert lqr.selftest_bounded_wait(poll_limit=2000) == 1
+    w = small_workload(64, 64, 3, (1, 1, 9), seed=5, bf16=True)
+    g = pu.run_gpu(w)                      # run_gpu asserts that the solver's own error word is clear
+    pu.compare(g, pu.run_oracle(w), np.arange(9), 2e-2)

@@ -56,6 +56,27 @@ def test_noalloc_also_agrees_with_the_oracle():
     pu.compare({"P": P0, "u": u0, "info": info}, ref, np.arange(N), 1e-4, names=("P", "u"))
 
 
+def test_noalloc_leaves_the_device_memory_untouched_and_runs_on_a_side_stream():
+    """The property the entry point exists for: once the first call on the device has looked up the scratch address,
+    a call changes the amount of free device memory by nothing.  Run on a non-default stream."""
+    w, N = _first_call_inputs(1, (1, 8, 16))
+    P0 = torch.empty((N, 16, 16), device=DEV)
+    u0 = torch.empty((N, 16), device=DEV)
+    info = torch.empty((N,), dtype=torch.int32, device=DEV)
+    side = torch.cuda.Stream(device=DEV)
+    args = (w["A"], w["B"], w["Q"], w["R"], w["x0"], w["H"], w["batch"])
+    lqr.solve_first_noalloc(*args, P0=P0, u0=u0, info=info, stream=side)     # may be the address-resolving call
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info(0)[0]
+    P0.fill_(123456.0)
+    torch.cuda.synchronize()
+    lqr.solve_first_noalloc(*args, P0=P0, u0=u0, info=info, stream=side)
+    side.synchronize()
+    assert torch.cuda.mem_get_info(0)[0] == free_before
+    ref = pu.run_oracle(w, first_only=True)
+    pu.compare({"P": P0, "u": u0, "info": info}, ref, np.arange(N), 1e-4, names=("P", "u"))
+
+
 def test_noalloc_rejects_problems_beyond_its_scratch():
     w, N = _first_call_inputs(1, (4, 8, 128))        # 4096 instances x 16x16 floats = 4 MiB + status words
     P0 = torch.empty((N, 16, 16), device=DEV)
