@@ -506,51 +506,66 @@ def run_layer(args):
         td.destroy_process_group()
 
 
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
-    ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg4")
-    ap.add_argument("--method", default="auto", choices=["auto", "riccati", "scan"])
-    ap.add_argument("--math", default="auto", choices=["auto", "fp32", "tf32"])
-    ap.add_argument("--e2e-steps", type=int, default=2)
-    ap.add_argument("--cpu-sample", type=int, default=256, help="instances the oracle is timed on")
-    ap.add_argument("--ref-instances", type=int, default=256)
-    ap.add_argument("--tokens", type=int, default=0, help="override the token count (small profiling captures)")
-    ap.add_argument("--horizon", type=int, default=0, help="layer workloads: override the planning horizon T (sweeps)")
-    ap.add_argument("--batch", default="", help="layer and gradient workloads: override the batch as SxHxT, e.g. 1x16x64 (sweeps)")
-    ap.add_argument("--per-token", action="store_true", help="grad16: A_t, B_t, R_t per token instead of per head")
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-e2e", action="store_true")
-    args = ap.parse_args()
-    if args.workload in workloads.LAYER_CONFIGS:
-        run_layer(args)
-        return
-    if workloads.TV_CONFIGS.get(args.workload, {}).get("grad"):
-        run_grad(args)
-        return
-    tv_key = args.workload if args.workload in workloads.TV_CONFIGS else None
-    cid = None if tv_key else int(args.workload.replace("cfg", ""))
-    if args.impl == "reference":
-        run_reference(args, cid, tv_key)
-        return
-    args.warmup = max(args.warmup, 3)
-
+def measure_run_peaks(local, dev):
+    """FP32 FMA and TF32 tensor peaks measured in this run on this device (the denominators of the "alu" and
+    "tensor" roofline fractions): an FMA-chain micro-kernel of the library, and an 8192^3 float32 matmul with TF32
+    tensor cores allowed (cuBLAS through torch), best of 5 (burst) and back to back for about a second (sustained)."""
     from paper_2603_09221_b200 import lqr
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the solver has no CPU path")
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    dist = world > 1
+    sampler = ClockSampler(local)
+    sampler.start()
+    scalar, packed = lqr.measure_fp32_peak(local)
+    old = torch.backends.cuda.matmul.allow_tf32
+    torch.backends.cuda.matmul.allow_tf32 = True
+    try:
+        M = 8192
+        a = torch.randn((M, M), device=dev)
+        b = torch.randn((M, M), device=dev)
+        c = torch.empty((M, M), device=dev)
+        for _ in range(3):
+            torch.matmul(a, b, out=c)
+        torch.cuda.synchronize(dev)
+        flops = 2.0 * M ** 3
+        burst = 0.0
+        for _ in range(5):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            torch.matmul(a, b, out=c)
+            e1.record()
+            torch.cuda.synchronize(dev)
+            burst = max(burst, flops / (e0.elapsed_time(e1) * 1e-3) / 1e12)
+        reps = max(8, int(1.0 / (flops / (burst * 1e12))))
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            torch.matmul(a, b, out=c)
+        e1.record()
+        torch.cuda.synchronize(dev)
+        sustained = reps * flops / (e0.elapsed_time(e1) * 1e-3) / 1e12
+        del a, b, c
+    finally:
+        torch.backends.cuda.matmul.allow_tf32 = old
+    clocks = sampler.stop()
+    return {"fp32_tflops": max(scalar, packed), "fp32_tflops_scalar_fma": scalar, "fp32_tflops_packed_fma": packed,
+            "tf32_tflops": burst, "tf32_tflops_sustained": sustained,
+            "how": "FMA-chain micro-kernel (ttc_lqr_measure_fp32_peak, best of 5); torch.matmul fp32 8192^3 with TF32 "
+                   "allowed, best of 5 and %d back to back" % reps,
+            "clocks": clocks}
+
+
+def run_solve(args, workload, method_name, ctx, light=False):
+    """One workload of ttc_lqr_solve / ttc_lqr_solve_tv through the C ABI: warm-up, timed steps (CUDA events), end to
+    end through the host-buffer entry, roofline of the dominant kernel, parity and CPU baseline on a sample.
+    Returns the JSON line as a dict on rank 0 (None on the other ranks).  `light`: a short side measurement (fewer
+    steps, no end-to-end leg)."""
+    from paper_2603_09221_b200 import lqr
+    dist, world, rank, local, dev, peaks, run_peaks = (ctx[k] for k in ("dist", "world", "rank", "local", "dev", "peaks", "run_peaks"))
     if dist:
         import torch.distributed as td
-        td.init_process_group("nccl", device_id=torch.device("cuda", local))
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    peaks = measured_peaks()
+    tv_key = workload if workload in workloads.TV_CONFIGS else None
+    cid = None if tv_key else int(workload.replace("cfg", ""))
+    steps = 5 if light else args.steps
+    warmup = 3 if light else args.warmup
+    no_e2e = args.no_e2e or light or bool(tv_key)     # the host-buffer entry point covers the time-invariant solve only
 
     c = dict(workloads.TV_CONFIGS[tv_key] if tv_key else workloads.CONFIGS[cid])
     if args.tokens > 0:
@@ -558,13 +573,12 @@ def main():
         c["name"] += "_tokens%d" % args.tokens
     if tv_key:
         w = workloads.make_tv_workload(tv_key, device=dev, batch=c["batch"], seed=sharding.rank_seed(100, rank))
-        args.no_e2e = True           # the host-buffer entry point covers the time-invariant solve only
     else:
         w = workloads.make_workload(cid, device=dev, batch=c["batch"], seed=sharding.rank_seed(cid, rank))
     n, m, H = c["n"], c["m"], c["H"]
     N = int(np.prod(c["batch"]))
     first = c["first_only"]
-    method = {"auto": lqr.TTC_AUTO, "riccati": lqr.TTC_RICCATI, "scan": lqr.TTC_SCAN}[args.method]
+    method = {"auto": lqr.TTC_AUTO, "riccati": lqr.TTC_RICCATI, "scan": lqr.TTC_SCAN}[method_name]
     math = {"auto": lqr.TTC_MATH_AUTO, "fp32": lqr.TTC_MATH_FP32, "tf32": lqr.TTC_MATH_TF32}[args.math]
     solver = lqr.LqrSolver(n, m, H, c["batch"], device=local, method=method, math=math)
     want = ("P", "u", "info") if first else ("K", "P", "x", "u", "info")
@@ -584,30 +598,39 @@ def main():
             td.barrier()
         torch.cuda.synchronize(dev)
 
-    for _ in range(args.warmup):
+    flops_i, bin_i, bout_i = algorithmic_counts(c)
+    alg_bytes = N * (bin_i + bout_i)
+    alg_flops = N * flops_i
+    # inputs + outputs of the large configurations exceed L2 several times over; the small ones fit, so a buffer
+    # larger than L2 is written between their timed steps
+    flush = torch.empty(192 * 1024 * 1024, dtype=torch.uint8, device=dev) if alg_bytes <= 256e6 else None
+    for _ in range(warmup):
         step()
     barrier()
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
     launches0 = solver.query(lqr.TTC_QUERY_TOTAL_LAUNCHES)
-    evs = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    e0 = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+    e1 = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
     barrier()
-    evs[0].record()
-    for i in range(args.steps):
+    for i in range(steps):
+        if flush is not None:
+            flush.fill_(i & 255)
+        e0[i].record()
         step()
-        evs[i + 1].record()
+        e1[i].record()
     barrier()
     launches = solver.query(lqr.TTC_QUERY_TOTAL_LAUNCHES) - launches0
     clocks = sampler.stop() if rank == 0 else None
-    total_ms = evs[0].elapsed_time(evs[-1])
-    per_step = [evs[i].elapsed_time(evs[i + 1]) for i in range(args.steps)]
+    per_step = [e0[i].elapsed_time(e1[i]) for i in range(steps)]
     kernel_id = solver.query(lqr.TTC_QUERY_LAST_KERNEL)
-    value, ms_per_step, _ = sharding.aggregate_throughput(N, total_ms / args.steps, device=dev)
+    value, ms_per_step, _ = sharding.aggregate_throughput(N, sum(per_step) / steps, device=dev)
+    del flush
 
     # ---- end to end through the host-buffer entry point (pinned host memory, copies timed)
     e2e = None
-    if not args.no_e2e:
+    if not no_e2e:
         hin = {k: w[k].cpu().pin_memory() for k in ("A", "B", "Q", "R", "x0")}
         hout = lqr.alloc_outputs(n, m, H, N, "cpu", first_only=first, want=want, pin=True)
         h2d = sum(v.numel() * v.element_size() for v in hin.values())
@@ -630,23 +653,24 @@ def main():
         del hin, hout
 
     if rank != 0:
-        if dist:
-            td.destroy_process_group()
-        return
+        solver.close()
+        return None
 
     # ---- roofline of the dominant kernel (one launch per step does the whole backward pass)
-    flops_i, bin_i, bout_i = algorithmic_counts(c)
     kname = lqr.KERNEL_NAMES.get(kernel_id, str(kernel_id))
-    launches_per_step = launches / args.steps
+    launches_per_step = launches / steps
     kernel_ms = statistics.median(per_step)       # dominant kernel ~ the whole step (events per step)
-    alg_bytes = N * (bin_i + bout_i)
-    alg_flops = N * flops_i
     t_hbm = alg_bytes / (peaks["hbm_gbs"] * 1e9)
-    fp32_peak = SM_COUNT * FP32_LANES_PER_SM * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12
-    tf32_peak = peaks["bf16_tflops_sustained"] * TF32_TO_BF16_RATIO
+    fp32_derived = SM_COUNT * FP32_LANES_PER_SM * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12
+    tf32_derived = peaks["bf16_tflops_sustained"] * TF32_TO_BF16_RATIO
+    fp32_peak = run_peaks["fp32_tflops"] if run_peaks else fp32_derived
+    tf32_peak = run_peaks["tf32_tflops_sustained"] if run_peaks else tf32_derived
+    extra = {}
     if kname == "riccati_umma":
         bound, peak, unit, ach = "tensor", tf32_peak, "TFLOP/s", alg_flops / (kernel_ms * 1e-3) / 1e12
-        peak_note = "tf32 = measured sustained bf16 x 0.5 (nominal ratio), of %s" % peaks["source"]
+        peak_note = ("tf32 matmul (cuBLAS via torch) measured in this run, sustained" if run_peaks else
+                     "tf32 = measured sustained bf16 x 0.5 (nominal ratio), of %s" % peaks["source"])
+        extra = {"frac_of_half_bf16_sustained": ach / tf32_derived, "half_bf16_sustained_tflops": tf32_derived}
     else:
         t_alu = alg_flops / (fp32_peak * 1e12)
         if t_hbm >= t_alu:
@@ -654,11 +678,18 @@ def main():
             peak_note = "copy bandwidth, of %s" % peaks["source"]
         else:
             bound, peak, unit, ach = "alu", fp32_peak, "TFLOP/s", alg_flops / (kernel_ms * 1e-3) / 1e12
-            peak_note = "148 SMs x 128 FP32 lanes x 2 x %.0f MHz (derived)" % peaks["sm_max_mhz"]
+            peak_note = ("FMA-chain micro-kernel measured in this run" if run_peaks else
+                         "148 SMs x 128 FP32 lanes x 2 x %.0f MHz (derived)" % peaks["sm_max_mhz"])
+            extra = {"frac_of_derived_peak": ach / fp32_derived, "derived_peak_tflops": fp32_derived}
     roofline = {"bound": bound, "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak, "traffic": None,
                 "kernel": kname, "kernel_ms": kernel_ms, "peak_note": peak_note,
                 "algorithmic_flops_per_launch": alg_flops, "algorithmic_bytes_per_launch": alg_bytes,
                 "hbm_frac": (alg_bytes / (kernel_ms * 1e-3) / 1e9) / peaks["hbm_gbs"]}
+    roofline.update(extra)
+    if method_name == "scan":
+        # the scan executes its own flop count: per doubling round one squaring of the element and the applications
+        # of the round; reported beside the Riccati-equivalent figure above
+        roofline["nominal_B_T_d3_flops"] = float(N) * H * n ** 3
     traffic_path = os.path.join(ROOT, "profiles", "traffic.json")
     if os.path.exists(traffic_path):
         with open(traffic_path) as f:
@@ -669,29 +700,113 @@ def main():
 
     cpu = None
     if not args.no_cpu_baseline and world == 1:
+        # parity of the timed configuration on a stratified sample (every sequence and head), oracle timed on it
         idx = oracle_sample(w, args.cpu_sample)
         ref, dt = time_oracle(w, idx, first)
-        # parity of the timed configuration on the sampled instances
         from tests import parity_util as pu
         errs = pu.compare(out, ref, idx, c["tol"], names=("P", "u") if first else ("K", "P", "x", "u"))
         cpu = {"value": len(idx) / dt, "unit": "instances/s", "cores": int(ref["threads"]), "kind": "oracle",
                "sample": "%d instances of the same workload, every (seq, head) covered" % len(idx),
                "seconds": dt, "parity_max_rel_err": errs, "speedup_gpu_over_cpu": value / (len(idx) / dt)}
+        del ref
 
     line = {"metric": "lqr_instances_per_sec", "value": value, "unit": "instances/s", "n_gpus": world,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+            "steps": steps, "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "tf32" if kname == "riccati_umma" else "f32",
             "data": "synthetic",
             "config": {"workload": c["name"], "n": n, "m": m, "H": H, "instances": N, "batch": list(c["batch"]),
-                       "q_x0_dtype": c["q_dtype"], "time_varying": list(c.get("tv", ())), "outputs": list(want), "method": args.method, "kernel": kname,
+                       "q_x0_dtype": c["q_dtype"], "time_varying": list(c.get("tv", ())), "outputs": list(want), "method": method_name, "kernel": kname,
                        "l2": "inputs+outputs per step exceed L2 (%.2f GB)" % (alg_bytes / 1e9)
-                       if alg_bytes > 126e6 else "workload fits L2: latency-bound case"},
+                       if alg_bytes > 256e6 else "workload fits L2: a 192 MB buffer is written between timed steps"},
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches),
             "launches_per_step": launches_per_step, "clocks": clocks,
             "ms_per_step_percentiles": {"p20": float(np.percentile(per_step, 20)), "p50": float(np.percentile(per_step, 50)),
                                         "p80": float(np.percentile(per_step, 80))}}
-    print(json.dumps(line))
     solver.close()
+    del out, w
+    torch.cuda.empty_cache()
+    return line
+
+
+# side measurements of the default run: (workload, method)
+SIDE_RUNS = (("cfg0", "auto"), ("cfg1", "auto"), ("cfg2", "auto"), ("cfg3", "auto"), ("cfg3", "scan"))
+
+
+def spawn_ranks(n):
+    """`--gpus N` outside a launcher: start N ranks of this script, one per GPU, over NCCL on this node."""
+    raise SystemExit(sharding.launch_ranks(n, __file__, sys.argv[1:]))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="", help="one workload only (cfg0..cfg4, tv16, layer16, layer32, grad16); "
+                    "default: cfg4 as the headline plus short side measurements of cfg0..cfg3")
+    ap.add_argument("--method", default="auto", choices=["auto", "riccati", "scan"])
+    ap.add_argument("--math", default="auto", choices=["auto", "fp32", "tf32"])
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--cpu-sample", type=int, default=4096, help="instances the oracle is timed on and parity is checked on")
+    ap.add_argument("--ref-instances", type=int, default=2048)
+    ap.add_argument("--tokens", type=int, default=0, help="override the token count (small profiling captures)")
+    ap.add_argument("--horizon", type=int, default=0, help="layer workloads: override the planning horizon T (sweeps)")
+    ap.add_argument("--batch", default="", help="layer and gradient workloads: override the batch as SxHxT, e.g. 1x16x64 (sweeps)")
+    ap.add_argument("--per-token", action="store_true", help="grad16: A_t, B_t, R_t per token instead of per head")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-sides", action="store_true", help="default run: skip the side measurements of cfg0..cfg3")
+    ap.add_argument("--no-peaks", action="store_true", help="skip the in-run FP32 / TF32 peak measurement (derived peaks are used)")
+    args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl != "reference":
+        spawn_ranks(args.gpus)
+    default_run = args.workload == ""
+    if default_run:
+        args.workload = "cfg4"
+    if args.workload in workloads.LAYER_CONFIGS:
+        run_layer(args)
+        return
+    if workloads.TV_CONFIGS.get(args.workload, {}).get("grad"):
+        run_grad(args)
+        return
+    tv_key = args.workload if args.workload in workloads.TV_CONFIGS else None
+    cid = None if tv_key else int(args.workload.replace("cfg", ""))
+    if args.impl == "reference":
+        run_reference(args, cid, tv_key)
+        return
+    args.warmup = max(args.warmup, 3)
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the solver has no CPU path")
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = world > 1
+    if dist:
+        import torch.distributed as td
+        td.init_process_group("nccl", device_id=torch.device("cuda", local))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    ctx = dict(dist=dist, world=world, rank=rank, local=local, dev=dev, peaks=measured_peaks(), run_peaks=None)
+    if rank == 0 and not args.no_peaks:
+        ctx["run_peaks"] = measure_run_peaks(local, dev)
+    line = run_solve(args, args.workload, args.method, ctx)
+    if rank == 0:
+        line["measured_in_run"] = ctx["run_peaks"]
+        if default_run and not args.no_sides and world == 1:
+            sides = {}
+            for wl, meth in SIDE_RUNS:
+                r = run_solve(args, wl, meth, ctx, light=True)
+                key = wl + ("_scan" if meth == "scan" else "")
+                sides[key] = {"workload": r["config"]["workload"], "method": meth, "kernel": r["config"]["kernel"],
+                              "ms_per_step": r["ms_per_step"], "value": r["value"], "unit": r["unit"],
+                              "roofline": {k: r["roofline"][k] for k in ("bound", "frac", "peak", "unit", "achieved", "hbm_frac")},
+                              "parity_max_rel_err": r["cpu_baseline"]["parity_max_rel_err"] if r["cpu_baseline"] else None,
+                              "cpu_oracle_instances_per_s": r["cpu_baseline"]["value"] if r["cpu_baseline"] else None,
+                              "clocks": r["clocks"], "gpu_launches": r["gpu_launches"]}
+            line["configs"] = sides
+        print(json.dumps(line))
     if dist:
         td.destroy_process_group()
 

@@ -340,6 +340,15 @@ int ttc_lqr_solve_first_noalloc(int32_t n, int32_t m, const int64_t batch[3], in
  */
 int ttc_lqr_selftest_bounded_wait(int32_t device, int32_t poll_limit, int32_t* timed_out);
 
+/*
+ * Measured FP32 FMA rate of `device` (no counterpart in the paper; it is the denominator of the roofline
+ * fraction reported for the kernels that are bound by plain FP32 arithmetic).  Runs a register-only chain of
+ * independent FMAs on every SM, best of five timed launches with CUDA events (about 20 ms in all), once with
+ * scalar fma.rn.f32 and once with the packed fma.rn.f32x2 the solver's dense loops use; both results in
+ * TFLOP/s (2 flops per FMA).  Synchronous; makes `device` current; allocates and frees 4 KB.
+ */
+int ttc_lqr_measure_fp32_peak(int32_t device, double* tflops_scalar, double* tflops_packed);
+
 /* Free the handle and its workspace (synchronises the handle's device).  NULL is OK. */
 int ttc_lqr_destroy(ttc_lqr_handle* h);
 

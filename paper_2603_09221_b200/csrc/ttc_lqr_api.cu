@@ -11,10 +11,12 @@
 #include "common.cuh"
 #include "riccati_cta.cuh"
 #include "riccati_umma64.cuh"
+#include "riccati_umma64_first.cuh"
 #include "riccati_warp.cuh"
 #include "ttc_layer.cuh"
 #include "lqr_grad.cuh"
 #include "scan_pair.cuh"
+#include "peak_probe.cuh"
 
 using namespace ttc;
 
@@ -399,8 +401,12 @@ int solve_window(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, 
             // word 0 = work counter of this launch; word 1 = device error word, cleared once per API call
             // (clear_device_error) so that a later window of the same call cannot erase an earlier report
             TTC_CUDA(cudaMemsetAsync(counter, 0, sizeof(int), st));
-            const size_t smem = umma64::smem_bytes();
-            auto kern = rollout_needs_all_K || K ? umma64::riccati_umma64_kernel<true> : umma64::riccati_umma64_kernel<false>;
+            // P_0 / u_0 requests take the kernel with the shorter per-step chain (16-wide panels); requests for every
+            // P_t, the gains or the trajectory take the general one
+            const bool first_kernel = p.first_only && !K && !rollout_needs_all_K;
+            const size_t smem = first_kernel ? umma64::first::smem_bytes() : umma64::smem_bytes();
+            auto kern = first_kernel ? umma64::first::riccati_umma64_first_kernel
+                      : rollout_needs_all_K || K ? umma64::riccati_umma64_kernel<true> : umma64::riccati_umma64_kernel<false>;
             TTC_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
             const long long chunks = p.b0 * p.b1 * ((tcount + umma64::CHUNK - 1) / umma64::CHUNK);
             long long grid = h->sm_count;
@@ -940,6 +946,50 @@ int ttc_lqr_solve_host(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operan
 }
 
 } // extern "C"
+
+extern "C" int ttc_lqr_measure_fp32_peak(int32_t device, double* tflops_scalar, double* tflops_packed)
+{
+    if (!tflops_scalar || !tflops_packed)
+        return fail(TTC_STATUS_INVALID_ARGUMENT, "null result pointer");
+    int ndev = 0;
+    TTC_CUDA(cudaGetDeviceCount(&ndev));
+    if (device < 0 || device >= ndev)
+        return fail(TTC_STATUS_CUDA_ERROR, "device %d not present (%d devices)", device, ndev);
+    TTC_CUDA(cudaSetDevice(device));
+    int sms = 0;
+    TTC_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
+    float* sink = nullptr;
+    TTC_CUDA(cudaMalloc(&sink, sizeof(float) * probe::THREADS));
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    cudaError_t e = cudaEventCreate(&e0);
+    if (e == cudaSuccess) e = cudaEventCreate(&e1);
+    const int iters = 8192, blocks = 2 * sms;
+    double best[2] = {0.0, 0.0};
+    for (int variant = 0; variant < 2 && e == cudaSuccess; ++variant)
+        for (int rep = 0; rep < 6 && e == cudaSuccess; ++rep) {          // rep 0 warms up
+            cudaEventRecord(e0, 0);
+            if (variant == 0)
+                probe::fma_chain_kernel<false><<<blocks, probe::THREADS>>>(iters, 1.0f, sink);
+            else
+                probe::fma_chain_kernel<true><<<blocks, probe::THREADS>>>(iters, 1.0f, sink);
+            cudaEventRecord(e1, 0);
+            e = cudaEventSynchronize(e1);
+            float ms = 0.f;
+            if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, e0, e1);
+            if (e == cudaSuccess && rep > 0 && ms > 0.f) {
+                const double tf = probe::launch_flops(blocks, iters) / (ms * 1e-3) / 1e12;
+                if (tf > best[variant]) best[variant] = tf;
+            }
+        }
+    if (e0) cudaEventDestroy(e0);
+    if (e1) cudaEventDestroy(e1);
+    cudaFree(sink);
+    if (e != cudaSuccess)
+        return fail(TTC_STATUS_CUDA_ERROR, "fp32 peak measurement: %s", cudaGetErrorString(e));
+    *tflops_scalar = best[0];
+    *tflops_packed = best[1];
+    return TTC_OK;
+}
 
 extern "C" int ttc_lqr_selftest_bounded_wait(int32_t device, int32_t poll_limit, int32_t* timed_out)
 {

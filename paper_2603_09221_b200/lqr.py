@@ -27,7 +27,7 @@ EXPORTS = (
     "ttc_lqr_create", "ttc_lqr_solve", "ttc_lqr_solve_host", "ttc_lqr_destroy", "ttc_lqr_query",
     "ttc_lqr_status_string", "ttc_lqr_last_error", "ttc_lqr_solve_first_noalloc", "ttc_lqr_solve_tv",
     "ttc_lqr_solve_layer", "ttc_lqr_solve_layer_host", "ttc_lqr_solve_affine", "ttc_lqr_grad",
-    "ttc_lqr_selftest_bounded_wait",
+    "ttc_lqr_selftest_bounded_wait", "ttc_lqr_measure_fp32_peak",
 )
 TTC_NOALLOC_SCRATCH_BYTES = 4 << 20
 
@@ -106,6 +106,8 @@ def load_library():
                                                 opp, opp, opp, opp, opp, ctypes.c_int32] + [ctypes.c_void_p] * 4
     lib.ttc_lqr_selftest_bounded_wait.restype = ctypes.c_int
     lib.ttc_lqr_selftest_bounded_wait.argtypes = [ctypes.c_int32, ctypes.c_int32, P(ctypes.c_int32)]
+    lib.ttc_lqr_measure_fp32_peak.restype = ctypes.c_int
+    lib.ttc_lqr_measure_fp32_peak.argtypes = [ctypes.c_int32, P(ctypes.c_double), P(ctypes.c_double)]
     _lib = lib
     return lib
 
@@ -351,6 +353,13 @@ def alloc_outputs(n, m, H, N, device, first_only=False, want=("K", "P", "x", "u"
     if "info" in want:
         out["info"] = torch.empty((N,), dtype=torch.int32, **kw)
     return out
+
+
+def measure_fp32_peak(device=0):
+    """``ttc_lqr_measure_fp32_peak``: measured FP32 FMA rate of the device in TFLOP/s as ``(scalar, packed)``."""
+    a, b = ctypes.c_double(), ctypes.c_double()
+    _check(load_library().ttc_lqr_measure_fp32_peak(int(device), ctypes.byref(a), ctypes.byref(b)))
+    return a.value, b.value
 
 
 def selftest_bounded_wait(poll_limit=4096, device=0):

@@ -117,9 +117,10 @@ def run_oracle_tv(w, idx=None, first_only=None, H=None, nthreads=0):
                               sel("x0", (n,)), H, (len(idx_t),), tv=w["tv"], first_only=first_only, nthreads=nthreads)
 
 
-def compare(gpu, ref, idx, tol, names=("K", "P", "x", "u")):
+def compare(gpu, ref, idx, tol, names=("K", "P", "x", "u"), xu_floor=XU_FLOOR):
     """Returns {name: err} with the block-wise figure of every requested output and, for x and u, the
-    trajectory-normalised one under "x_traj" / "u_traj"; asserts all of them within tol and info == 0."""
+    trajectory-normalised one under "x_traj" / "u_traj"; asserts all of them within tol and info == 0.
+    `xu_floor` replaces the floor of the block-wise x, u measure (1.0 = trajectory-normalised only)."""
     n_dims = {"K": 2, "P": 2, "x": 1, "u": 1}
     errs = {}
     sel = torch.as_tensor(idx, dtype=torch.long)
@@ -128,7 +129,7 @@ def compare(gpu, ref, idx, tol, names=("K", "P", "x", "u")):
             continue
         g = gpu[k].cpu()[sel].numpy()
         if k in ("x", "u"):
-            errs[k] = block_rel_err(g, ref[k], n_dims[k], floor=XU_FLOOR)
+            errs[k] = block_rel_err(g, ref[k], n_dims[k], floor=xu_floor)
             errs[k + "_traj"] = block_rel_err(g, ref[k], n_dims[k], per_block=False)
         else:
             errs[k] = block_rel_err(g, ref[k], n_dims[k])

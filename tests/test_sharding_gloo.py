@@ -55,3 +55,35 @@ def test_single_process_is_the_identity():
     assert sharding.max_over_ranks(3.5) == 3.5
     v, ms, w = sharding.aggregate_throughput(10, 5.0)
     assert (v, ms, w) == (10 / 5e-3, 5.0, 1)
+
+
+_RANK_SCRIPT = """
+import json, os, sys
+import torch.distributed as dist
+sys.path.insert(0, %r)
+from paper_2603_09221_b200 import sharding
+dist.init_process_group("gloo")
+rank, world = dist.get_rank(), dist.get_world_size()
+value, ms, ws = sharding.aggregate_throughput(8, 5.0 * (rank + 1))
+with open(os.path.join(sys.argv[1], "rank%%d.json" %% rank), "w") as f:
+    json.dump(dict(rank=rank, world=world, value=value, ms=ms, env_world=int(os.environ["WORLD_SIZE"]),
+                   local=int(os.environ["LOCAL_RANK"]), addr=os.environ["MASTER_ADDR"]), f)
+dist.destroy_process_group()
+"""
+
+
+def test_launcher_starts_one_process_per_rank(tmp_path):
+    """The `--gpus N` path of the benchmark outside a launcher: sharding.launch_ranks starts N ranks through torch's
+    launcher with a 127.0.0.1 rendezvous.  Two CPU ranks over gloo stand in for two GPUs."""
+    import json
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    script = tmp_path / "rank_script.py"
+    script.write_text(_RANK_SCRIPT % root)
+    cmd = sharding.launcher_command(2, str(script), [str(tmp_path)], port=_free_port())
+    assert cmd[1:3] == ["-m", "torch.distributed.run"] and "--nproc-per-node" in cmd and "127.0.0.1" in cmd
+    rc = sharding.launch_ranks(2, str(script), [str(tmp_path)])
+    assert rc == 0
+    res = [json.load(open(tmp_path / ("rank%d.json" % r))) for r in range(2)]
+    assert [r["rank"] for r in res] == [0, 1] and all(r["world"] == r["env_world"] == 2 for r in res)
+    assert all(r["addr"] == "127.0.0.1" for r in res) and [r["local"] for r in res] == [0, 1]
+    assert all(r["ms"] == 10.0 and r["value"] == 2 * 8 / 10e-3 for r in res)
