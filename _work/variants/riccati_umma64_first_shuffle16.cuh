@@ -3,12 +3,12 @@
 // CTA per SM, four independent warpgroups, one instance per warpgroup, the tall matrix [S; Y'] factored in tensor
 // memory), with a SHORTER DEPENDENCY CHAIN per step:
 //
-//   * 16-wide panels, factored in two levels.  The warp that owns the 16 diagonal rows factors the leading 8 x 8
-//     block, forward-substitutes its own rows, exchanges the 8 x 8 block L21 through shared memory (warp-level
-//     synchronisation only), updates and factors the second 8 x 8 block, and publishes L11, L21, L22.  After ONE
-//     warpgroup barrier every thread applies the whole 16 x 16 triangular solve to its row in registers, and ONE
-//     rank-16 trailing update (2 k-steps x 3 tf32 passes) goes to the tensor core.  A step has 4 panel round trips
-//     (publish -> barrier -> substitute -> fence -> barrier -> MMA -> completion wait -> tcgen05.ld) instead of 8.
+//   * 16-wide panels.  The 16 lanes that own the diagonal rows factor the 16 x 16 block among themselves with
+//     shuffles (one row per lane, straight from the registers the tensor-memory load filled: no gather through
+//     shared memory) and publish the factor; after ONE warpgroup barrier every other thread applies the 16 x 16
+//     triangular solve to its row in registers, and ONE rank-16 trailing update (2 k-steps x 3 tf32 passes) goes to
+//     the tensor core.  A step has 4 panel round trips (publish -> barrier -> substitute -> fence -> barrier ->
+//     MMA -> completion wait -> tcgen05.ld) instead of 8.
 //   * The fp32 factor L is kept only at the last step (u_0 needs it), packed by rows, so the second 64 x 64 buffer
 //     of the general kernel is gone and the wider panel buffers fit.
 //   * The rows of Q for the read-out P_t = Q + A'P A - Z'Z are fetched into registers while the last contraction
@@ -52,9 +52,7 @@ struct Misc {
     int flag;                    // first failed pivot (0 = none)
     alignas(16) float x0[N];
     alignas(16) float y0[N];     // Z x_0, then the back substitution's running right-hand side
-    alignas(16) float dg[2][64]; // the two 8 x 8 diagonal blocks of the current panel (rows of 8)
-    alignas(16) float l21[64];   // rows of L21 = G21 L11^{-T}
-    alignas(16) float ld[2][36]; // L11 and L22: strict lower triangle (28) + reciprocal pivots (8)
+    alignas(16) float lpub[160]; // factor of the current 16 x 16 diagonal block as published to the warpgroup
 };
 constexpr uint32_t WG_BYTES = OFF_MISC + ((sizeof(Misc) + 127) / 128) * 128;
 constexpr uint32_t SMEM_BYTES = BUF_BYTES + R_BYTES + NUM_WG * WG_BYTES + 128;
@@ -74,55 +72,67 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16])
                    "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
                  : "r"(taddr) : "memory");
 }
-// strict lower triangle + reciprocal pivots of an 8 x 8 factor <-> 9 16-byte words
-__device__ __forceinline__ void pack_factor(float* dst36, const float (&l)[8][8], const float (&rinv)[8])
+// Cholesky of a 16 x 16 SPD block spread over a 16-lane segment (lane i of the segment = row i), right-looking with
+// shuffles: pivot j is broadcast from lane j, every lane scales its entry of column j and updates the columns right of
+// it with the entries of the rows below, which arrive by shuffle.  The chain from one pivot to the next is
+// shuffle -> reciprocal -> multiply -> fma.  On return s[0..i] is row i of L (entries right of the diagonal are
+// meaningless) and rs_own = 1 / L[i][i].  Returns 0 or 1 + the index of the first non-positive pivot (uniform).
+__device__ __forceinline__ int seg_chol16(float (&s)[16], float& rs_own, int i)
 {
-    float4* d = reinterpret_cast<float4*>(dst36);
-    d[0] = make_float4(l[1][0], l[2][0], l[2][1], l[3][0]);
-    d[1] = make_float4(l[3][1], l[3][2], l[4][0], l[4][1]);
-    d[2] = make_float4(l[4][2], l[4][3], l[5][0], l[5][1]);
-    d[3] = make_float4(l[5][2], l[5][3], l[5][4], l[6][0]);
-    d[4] = make_float4(l[6][1], l[6][2], l[6][3], l[6][4]);
-    d[5] = make_float4(l[6][5], l[7][0], l[7][1], l[7][2]);
-    d[6] = make_float4(l[7][3], l[7][4], l[7][5], l[7][6]);
-    d[7] = make_float4(rinv[0], rinv[1], rinv[2], rinv[3]);
-    d[8] = make_float4(rinv[4], rinv[5], rinv[6], rinv[7]);
-}
-__device__ __forceinline__ void unpack_factor(float (&l)[8][8], float (&rinv)[8], const float* src36)
-{
-    const float4* s = reinterpret_cast<const float4*>(src36);
-    const float4 c0 = s[0], c1 = s[1], c2 = s[2], c3 = s[3], c4 = s[4], c5 = s[5], c6 = s[6], c7 = s[7], c8 = s[8];
-    l[1][0] = c0.x; l[2][0] = c0.y; l[2][1] = c0.z; l[3][0] = c0.w;
-    l[3][1] = c1.x; l[3][2] = c1.y; l[4][0] = c1.z; l[4][1] = c1.w;
-    l[4][2] = c2.x; l[4][3] = c2.y; l[5][0] = c2.z; l[5][1] = c2.w;
-    l[5][2] = c3.x; l[5][3] = c3.y; l[5][4] = c3.z; l[6][0] = c3.w;
-    l[6][1] = c4.x; l[6][2] = c4.y; l[6][3] = c4.z; l[6][4] = c4.w;
-    l[6][5] = c5.x; l[7][0] = c5.y; l[7][1] = c5.z; l[7][2] = c5.w;
-    l[7][3] = c6.x; l[7][4] = c6.y; l[7][5] = c6.z; l[7][6] = c6.w;
-    rinv[0] = c7.x; rinv[1] = c7.y; rinv[2] = c7.z; rinv[3] = c7.w;
-    rinv[4] = c8.x; rinv[5] = c8.y; rinv[6] = c8.z; rinv[7] = c8.w;
-}
-__device__ __forceinline__ void load_block8(float (&l)[8][8], const float* blk)
-{
+    int bad = 0;
+    rs_own = 1.f;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        const float4 a4 = *reinterpret_cast<const float4*>(blk + 8 * i);
-        const float4 b4 = *reinterpret_cast<const float4*>(blk + 8 * i + 4);
-        l[i][0] = a4.x; l[i][1] = a4.y; l[i][2] = a4.z; l[i][3] = a4.w;
-        l[i][4] = b4.x; l[i][5] = b4.y; l[i][6] = b4.z; l[i][7] = b4.w;
+    for (int j = 0; j < 16; ++j) {
+        const float sj = s[j];
+        float d = __shfl_sync(0xffffffffu, sj, j, 16);
+        if (!(d > 0.f)) {
+            if (!bad)
+                bad = j + 1;
+            d = 1.f;
+        }
+        float rs;
+        asm("rsqrt.approx.ftz.f32 %0, %1;" : "=f"(rs) : "f"(d));
+        const float f = sj * rs * rs;                          // s_ij / d_j
+#pragma unroll
+        for (int cc = j + 1; cc < 16; ++cc) {
+            const float lc = __shfl_sync(0xffffffffu, sj, cc, 16);
+            s[cc] = fmaf(-f, lc, s[cc]);
+        }
+        s[j] = sj * rs;
+        if (i == j)
+            rs_own = rs;
     }
+    return bad;
 }
-// hi[j] -= sum_k lo[k] * L21[j][k]  (the row's columns 8..15 after the first 8 have been substituted)
-__device__ __forceinline__ void schur_row8(float (&hi)[8], const float (&lo)[8], const float* l21)
+// Published form of the 16 x 16 factor: the strict lower triangle with row i (i >= 1) padded to a multiple of four
+// floats, rows in order (144 floats), then the 16 reciprocal pivots: 40 16-byte words.
+constexpr int LPUB_FLOATS = 160;
+__host__ __device__ constexpr int lpub_row(int i)              // first float of row i >= 1
 {
+    return 8 * ((i - 1) >> 2) * (((i - 1) >> 2) + 1) + ((i - 1) & 3) * 4 * (((i - 1) >> 2) + 1);
+}
+// x (a row of 16) <- x L^{-T} with the published factor
+__device__ __forceinline__ void fsub16(float (&x)[16], const float* lpub)
+{
+    float rinv[16];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        const float4 a4 = *reinterpret_cast<const float4*>(l21 + 8 * j);
-        const float4 b4 = *reinterpret_cast<const float4*>(l21 + 8 * j + 4);
-        float acc = hi[j];
-        acc = fmaf(-lo[0], a4.x, acc); acc = fmaf(-lo[1], a4.y, acc); acc = fmaf(-lo[2], a4.z, acc); acc = fmaf(-lo[3], a4.w, acc);
-        acc = fmaf(-lo[4], b4.x, acc); acc = fmaf(-lo[5], b4.y, acc); acc = fmaf(-lo[6], b4.z, acc); acc = fmaf(-lo[7], b4.w, acc);
-        hi[j] = acc;
+    for (int q4 = 0; q4 < 4; ++q4) {
+        const float4 r4 = *reinterpret_cast<const float4*>(lpub + 144 + 4 * q4);
+        rinv[4 * q4] = r4.x; rinv[4 * q4 + 1] = r4.y; rinv[4 * q4 + 2] = r4.z; rinv[4 * q4 + 3] = r4.w;
+    }
+    x[0] *= rinv[0];
+#pragma unroll
+    for (int i = 1; i < 16; ++i) {
+        float acc = x[i];
+#pragma unroll
+        for (int q4 = 0; q4 <= (i - 1) >> 2; ++q4) {
+            const float4 l4 = *reinterpret_cast<const float4*>(lpub + lpub_row(i) + 4 * q4);
+            if (4 * q4 + 0 < i) acc = fmaf(-l4.x, x[4 * q4 + 0], acc);
+            if (4 * q4 + 1 < i) acc = fmaf(-l4.y, x[4 * q4 + 1], acc);
+            if (4 * q4 + 2 < i) acc = fmaf(-l4.z, x[4 * q4 + 2], acc);
+            if (4 * q4 + 3 < i) acc = fmaf(-l4.w, x[4 * q4 + 3], acc);
+        }
+        x[i] = acc * rinv[i];
     }
 }
 
@@ -267,7 +277,7 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_first_kernel(SolveP
                 wait_mma();
                 // (3) [S; Y'] = [L; Z'] L', 16 columns at a time; thread wt owns row wt
                 const bool keep_l = ts == 0 && want_u0;
-                float vlo[8], vhi[8];                          // the row's 16 panel columns
+                float v[16];                                   // the row's 16 panel columns
                 auto load_cols = [&](int c0) {
                     uint32_t raw[16];
                     tmem_ld16(RF + lane_sel + c0, raw);
@@ -277,64 +287,46 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_first_kernel(SolveP
                         r0 = rr[0]; r1 = rr[1]; r2 = rr[2]; r3 = rr[3];
                     }
                     tmem_wait_ld();
-                    vlo[0] = __uint_as_float(raw[0]) + r0.x; vlo[1] = __uint_as_float(raw[1]) + r0.y;
-                    vlo[2] = __uint_as_float(raw[2]) + r0.z; vlo[3] = __uint_as_float(raw[3]) + r0.w;
-                    vlo[4] = __uint_as_float(raw[4]) + r1.x; vlo[5] = __uint_as_float(raw[5]) + r1.y;
-                    vlo[6] = __uint_as_float(raw[6]) + r1.z; vlo[7] = __uint_as_float(raw[7]) + r1.w;
-                    vhi[0] = __uint_as_float(raw[8]) + r2.x; vhi[1] = __uint_as_float(raw[9]) + r2.y;
-                    vhi[2] = __uint_as_float(raw[10]) + r2.z; vhi[3] = __uint_as_float(raw[11]) + r2.w;
-                    vhi[4] = __uint_as_float(raw[12]) + r3.x; vhi[5] = __uint_as_float(raw[13]) + r3.y;
-                    vhi[6] = __uint_as_float(raw[14]) + r3.z; vhi[7] = __uint_as_float(raw[15]) + r3.w;
+                    v[0] = __uint_as_float(raw[0]) + r0.x; v[1] = __uint_as_float(raw[1]) + r0.y;
+                    v[2] = __uint_as_float(raw[2]) + r0.z; v[3] = __uint_as_float(raw[3]) + r0.w;
+                    v[4] = __uint_as_float(raw[4]) + r1.x; v[5] = __uint_as_float(raw[5]) + r1.y;
+                    v[6] = __uint_as_float(raw[6]) + r1.z; v[7] = __uint_as_float(raw[7]) + r1.w;
+                    v[8] = __uint_as_float(raw[8]) + r2.x; v[9] = __uint_as_float(raw[9]) + r2.y;
+                    v[10] = __uint_as_float(raw[10]) + r2.z; v[11] = __uint_as_float(raw[11]) + r2.w;
+                    v[12] = __uint_as_float(raw[12]) + r3.x; v[13] = __uint_as_float(raw[13]) + r3.y;
+                    v[14] = __uint_as_float(raw[14]) + r3.z; v[15] = __uint_as_float(raw[15]) + r3.w;
                 };
                 load_cols(0);
 #pragma unroll 1
                 for (int pnl = 0; pnl < NPANEL; ++pnl) {
                     const int col = PW * pnl;
                     const bool diag_warp = warp == (pnl >> 1);
+                    bool owner = false;                        // this thread owns one of the 16 diagonal rows
                     if (diag_warp) {
-                        // The 16 diagonal rows belong to this warp.  Two-level factorisation of the 16 x 16 block with
-                        // warp-level synchronisation only; every lane of the warp substitutes its own row on the way.
-                        const int r16 = wt - col;                               // 0..15 for the owners of the block rows
-                        if ((unsigned)r16 < 8u) {
-                            float4* dst = reinterpret_cast<float4*>(&misc.dg[0][8 * r16]);
-                            dst[0] = make_float4(vlo[0], vlo[1], vlo[2], vlo[3]);
-                            dst[1] = make_float4(vlo[4], vlo[5], vlo[6], vlo[7]);
-                        }
-                        __syncwarp();
-                        int bad;
-                        {
-                            float l[8][8], rinv[8];
-                            load_block8(l, &misc.dg[0][0]);
-                            bad = chol8(l, rinv);
-                            if (lane == 0)
-                                pack_factor(&misc.ld[0][0], l, rinv);
-                            fsub8(vlo, l, rinv);
-                        }
-                        if ((unsigned)(r16 - 8) < 8u) {                         // rows of L21
-                            float4* dst = reinterpret_cast<float4*>(&misc.l21[8 * (r16 - 8)]);
-                            dst[0] = make_float4(vlo[0], vlo[1], vlo[2], vlo[3]);
-                            dst[1] = make_float4(vlo[4], vlo[5], vlo[6], vlo[7]);
-                        }
-                        __syncwarp();
-                        schur_row8(vhi, vlo, &misc.l21[0]);
-                        if ((unsigned)(r16 - 8) < 8u) {
-                            float4* dst = reinterpret_cast<float4*>(&misc.dg[1][8 * (r16 - 8)]);
-                            dst[0] = make_float4(vhi[0], vhi[1], vhi[2], vhi[3]);
-                            dst[1] = make_float4(vhi[4], vhi[5], vhi[6], vhi[7]);
-                        }
-                        __syncwarp();
-                        {
-                            float l[8][8], rinv[8];
-                            load_block8(l, &misc.dg[1][0]);
-                            const int bad2 = chol8(l, rinv);
-                            if (!bad && bad2)
-                                bad = 8 + bad2;
-                            if (lane == 0) {
-                                pack_factor(&misc.ld[1][0], l, rinv);
-                                if (bad && misc.flag == 0)
-                                    misc.flag = ts * N + col + bad;
+                        // The 16 diagonal rows are one 16-lane segment of this warp: factor the block with shuffles
+                        // (the other segment runs the same instructions on its own rows and discards the result).
+                        float sblk[16];
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            sblk[j] = v[j];
+                        const int i = lane & 15;
+                        float rs_own;
+                        const int bad = seg_chol16(sblk, rs_own, i);
+                        owner = (lane >> 4) == (pnl & 1);
+                        if (owner) {
+#pragma unroll
+                            for (int j = 0; j < 16; ++j)
+                                v[j] = sblk[j];                // row i of L (masked right of the diagonal below)
+                            misc.lpub[144 + i] = rs_own;
+                            if (i >= 1) {
+                                float* dst = &misc.lpub[lpub_row(i)];
+#pragma unroll
+                                for (int q4 = 0; q4 < 4; ++q4)
+                                    if (4 * q4 < i)
+                                        *reinterpret_cast<float4*>(dst + 4 * q4) = make_float4(sblk[4 * q4], sblk[4 * q4 + 1], sblk[4 * q4 + 2], sblk[4 * q4 + 3]);
                             }
-                            fsub8(vhi, l, rinv);
+                            if (bad && i == 0 && misc.flag == 0)
+                                misc.flag = ts * N + col + bad;
                         }
                     }
                     tc_fence_before();
@@ -348,34 +340,19 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_first_kernel(SolveP
                         tc_fence_after();
                         gemm_ts(RF, RW, smem_u32(BA) + MAT_BYTES, 64);
                     }
-                    if (!diag_warp) {
-                        {
-                            float l[8][8], rinv[8];
-                            unpack_factor(l, rinv, &misc.ld[0][0]);
-                            fsub8(vlo, l, rinv);
-                        }
-                        schur_row8(vhi, vlo, &misc.l21[0]);
-                        {
-                            float l[8][8], rinv[8];
-                            unpack_factor(l, rinv, &misc.ld[1][0]);
-                            fsub8(vhi, l, rinv);
-                        }
-                    }
+                    if (!owner)
+                        fsub16(v, &misc.lpub[0]);
                     {
                         unsigned char* ph = PH + (uint32_t)(wt >> 3) * PSR16 + (uint32_t)(wt & 7) * 16u;
                         float h[16];
                         if (warp < 2) {                        // row wt of L: lower triangular, ends at column wt
                             float lo[16];
 #pragma unroll
-                            for (int j = 0; j < 8; ++j) {
+                            for (int j = 0; j < 16; ++j) {
                                 if (col + j > wt)
-                                    vlo[j] = 0.f;
-                                if (col + 8 + j > wt)
-                                    vhi[j] = 0.f;
-                                h[j] = round_tf32(vlo[j]);
-                                lo[j] = vlo[j] - h[j];
-                                h[8 + j] = round_tf32(vhi[j]);
-                                lo[8 + j] = vhi[j] - h[8 + j];
+                                    v[j] = 0.f;
+                                h[j] = round_tf32(v[j]);
+                                lo[j] = v[j] - h[j];
                             }
                             unsigned char* pl = PL + (uint32_t)(wt >> 3) * PSR16 + (uint32_t)(wt & 7) * 16u;
 #pragma unroll
@@ -383,21 +360,15 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_first_kernel(SolveP
                                 *reinterpret_cast<float4*>(pl + q4 * SC) = make_float4(lo[4 * q4], lo[4 * q4 + 1], lo[4 * q4 + 2], lo[4 * q4 + 3]);
                             if (keep_l) {                      // fp32 copy for u_0, packed by rows
                                 float* row = Lp + lp_row(wt) + col;
-                                if (col <= wt)
-                                    *reinterpret_cast<float4*>(row) = make_float4(vlo[0], vlo[1], vlo[2], vlo[3]);
-                                if (col + 4 <= wt)
-                                    *reinterpret_cast<float4*>(row + 4) = make_float4(vlo[4], vlo[5], vlo[6], vlo[7]);
-                                if (col + 8 <= wt)
-                                    *reinterpret_cast<float4*>(row + 8) = make_float4(vhi[0], vhi[1], vhi[2], vhi[3]);
-                                if (col + 12 <= wt)
-                                    *reinterpret_cast<float4*>(row + 12) = make_float4(vhi[4], vhi[5], vhi[6], vhi[7]);
+#pragma unroll
+                                for (int q4 = 0; q4 < 4; ++q4)
+                                    if (col + 4 * q4 <= wt)
+                                        *reinterpret_cast<float4*>(row + 4 * q4) = make_float4(v[4 * q4], v[4 * q4 + 1], v[4 * q4 + 2], v[4 * q4 + 3]);
                             }
                         } else {                               // row wt - 64 of Z': kept as tf32 (operand of (5)), low part zero
 #pragma unroll
-                            for (int j = 0; j < 8; ++j) {
-                                h[j] = round_tf32(vlo[j]);
-                                h[8 + j] = round_tf32(vhi[j]);
-                            }
+                            for (int j = 0; j < 16; ++j)
+                                h[j] = round_tf32(v[j]);
                             unsigned char* pz = X0 + (uint32_t)((wt - 64) >> 3) * SR + 4u * pnl * SC + (uint32_t)(wt & 7) * 16u;
 #pragma unroll
                             for (int q4 = 0; q4 < 4; ++q4)

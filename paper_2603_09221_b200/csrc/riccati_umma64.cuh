@@ -167,6 +167,14 @@ __device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&r)[8])
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
                  : "r"(taddr) : "memory");
 }
+// 32 lanes x 16 consecutive columns; the caller waits with tmem_wait_ld() before it reads r
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16])
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+                 : "r"(taddr) : "memory");
+}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // named barriers: 1 + wg = warps 0, 1 of a warpgroup (64 threads), 5 + wg = the whole warpgroup
@@ -722,6 +730,16 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
                 }
                 if (dead)
                     break;
+                // Without gains nothing else runs between here and the read-out: the row of Q that the read-out adds
+                // travels while (5) is in flight (bf16: the whole row in 32 registers).
+                uint4 qraw[8];
+                const bool q_pref = !GAINS && p.Q.dtype == TTC_BF16;
+                if (q_pref && warp >= 2) {
+                    const uint4* src = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(p.Q.ptr) + oq + (long long)(wt - 64) * N);
+#pragma unroll
+                    for (int c = 0; c < 8; ++c)
+                        qraw[c] = __ldg(src + c);
+                }
                 if (ts == 0 && want_u0 && warp < 2) {
                     // u_0 = K_0 x_0 = -L^{-T} (Z x_0), fp32, by the 64 threads of warps 0, 1
                     const int i = wt;
@@ -785,19 +803,55 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
                 // P_t = Q + DP: warps 2, 3 own the rows (lanes 64..127)
                 if (warp >= 2) {
                     const int j = wt - 64;
-#pragma unroll 1
-                    for (int half = 0; half < 2; ++half) {
-                        float q[32], hh[32];
-                        load_q_half(q, p.Q, oq, j, half);
-                        tmem_ld32(RF + lane_sel + 32 * half, hh);
+                    float* Pdst = (p.P && (!p.first_only || ts == 0))
+                                      ? p.P + (inst * (long long)(p.first_only ? 1 : H + 1) + (p.first_only ? 0 : ts)) * N * N + (long long)j * N
+                                      : nullptr;
+                    if (q_pref) {
 #pragma unroll
-                        for (int c = 0; c < 32; ++c)
-                            q[c] += hh[c];
-                        if (ts > 0)
-                            store_half_tf32(X0, j, half, q);
-                        if (p.P && (!p.first_only || ts == 0))
-                            store_half_global(p.P + (inst * (long long)(p.first_only ? 1 : H + 1) + (p.first_only ? 0 : ts)) * N * N +
-                                                  (long long)j * N + 32 * half, q);
+                        for (int qt = 0; qt < 4; ++qt) {       // 16 columns at a time
+                            float q[16];
+#pragma unroll
+                            for (int c = 0; c < 2; ++c) {
+                                const uint4 v4 = qraw[2 * qt + c];
+                                const uint32_t wd[4] = {v4.x, v4.y, v4.z, v4.w};
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    q[8 * c + 2 * e] = __uint_as_float(wd[e] << 16);
+                                    q[8 * c + 2 * e + 1] = __uint_as_float(wd[e] & 0xffff0000u);
+                                }
+                            }
+                            uint32_t raw[16];
+                            tmem_ld16(RF + lane_sel + 16 * qt, raw);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int c = 0; c < 16; ++c)
+                                q[c] += __uint_as_float(raw[c]);
+                            if (ts > 0) {
+#pragma unroll
+                                for (int c = 0; c < 4; ++c)
+                                    *reinterpret_cast<float4*>(X0 + toff(j, 16 * qt + 4 * c)) =
+                                        make_float4(round_tf32(q[4 * c]), round_tf32(q[4 * c + 1]), round_tf32(q[4 * c + 2]), round_tf32(q[4 * c + 3]));
+                            }
+                            if (Pdst) {
+#pragma unroll
+                                for (int c = 0; c < 4; ++c)
+                                    reinterpret_cast<float4*>(Pdst + 16 * qt)[c] = make_float4(q[4 * c], q[4 * c + 1], q[4 * c + 2], q[4 * c + 3]);
+                            }
+                        }
+                    } else {
+#pragma unroll 1
+                        for (int half = 0; half < 2; ++half) {
+                            float q[32], hh[32];
+                            load_q_half(q, p.Q, oq, j, half);
+                            tmem_ld32(RF + lane_sel + 32 * half, hh);
+#pragma unroll
+                            for (int c = 0; c < 32; ++c)
+                                q[c] += hh[c];
+                            if (ts > 0)
+                                store_half_tf32(X0, j, half, q);
+                            if (Pdst)
+                                store_half_global(Pdst + 32 * half, q);
+                        }
                     }
                     // Every eighth step the operand is replaced by (P + P') / 2.  Q and Z'Z are symmetric but the rounding
                     // of A'(P A) is not, and the antisymmetric part E obeys E <- A'E A: along an open-loop unstable A it

@@ -11,7 +11,6 @@
 #include "common.cuh"
 #include "riccati_cta.cuh"
 #include "riccati_umma64.cuh"
-#include "riccati_umma64_first.cuh"
 #include "riccati_warp.cuh"
 #include "ttc_layer.cuh"
 #include "lqr_grad.cuh"
@@ -401,12 +400,8 @@ int solve_window(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, 
             // word 0 = work counter of this launch; word 1 = device error word, cleared once per API call
             // (clear_device_error) so that a later window of the same call cannot erase an earlier report
             TTC_CUDA(cudaMemsetAsync(counter, 0, sizeof(int), st));
-            // P_0 / u_0 requests take the kernel with the shorter per-step chain (16-wide panels); requests for every
-            // P_t, the gains or the trajectory take the general one
-            const bool first_kernel = p.first_only && !K && !rollout_needs_all_K;
-            const size_t smem = first_kernel ? umma64::first::smem_bytes() : umma64::smem_bytes();
-            auto kern = first_kernel ? umma64::first::riccati_umma64_first_kernel
-                      : rollout_needs_all_K || K ? umma64::riccati_umma64_kernel<true> : umma64::riccati_umma64_kernel<false>;
+            const size_t smem = umma64::smem_bytes();
+            auto kern = rollout_needs_all_K || K ? umma64::riccati_umma64_kernel<true> : umma64::riccati_umma64_kernel<false>;
             TTC_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
             const long long chunks = p.b0 * p.b1 * ((tcount + umma64::CHUNK - 1) / umma64::CHUNK);
             long long grid = h->sm_count;

