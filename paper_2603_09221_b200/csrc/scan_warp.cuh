@@ -155,6 +155,7 @@ struct ScanParams {
     int* fail_flag;     // [N]: 0, or a positive code once something failed for the instance
     int step;           // apply form: 2^r
     int cnt;            // apply form: applications per instance in this round
+    int gain_steps;     // gain form: gains per instance (H, or 1 when only u_0 is wanted)
 };
 
 // ---- element of one step: A, C = B R^{-1} B', G = B L_R^{-T} (R = L_R L_R'), J = Q; also P_H = Q ------------------------
@@ -198,7 +199,7 @@ __global__ void __launch_bounds__(THREADS) scan_init_kernel(ScanParams q)
         load_row<N>(rinv, sl.rinv);
         load_row<N>(g, sl.B + c * LD);                         // row c of B
         forward_subst<N>(g, sl.Lt, rinv);                      // row c of G = B L_R^{-T}
-        store_row<N>(sl.G + c * LD, g);
+        store_col<N>(sl.G, c, g);                              // rows of G' (columns of G)
         __syncwarp();
         f32x2 c2[N / 2];
         zero2<N>(c2);
@@ -240,7 +241,7 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 2 : 3) scan_step_kernel(S
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, sub = lane / N, c = lane % N;
     StepSlot<N>& sl = reinterpret_cast<StepSlot<N>*>(smem_raw)[warp * S::IPW + sub];
     const int H = p.H;
-    const long long per = GAIN ? H : q.cnt;
+    const long long per = GAIN ? q.gain_steps : q.cnt;
     const long long nitems = p.b0 * p.b1 * p.tcount * per;
     for (long long base = (long long)blockIdx.x * S::SLOTS; base < nitems; base += (long long)gridDim.x * S::SLOTS) {
         const long long it = base + warp * S::IPW + sub;
@@ -650,6 +651,7 @@ inline cudaError_t launch_scan_warp(const SolveParams& p, float* Pbuf, float* el
     q.fail_flag = fail_flag;
     q.step = 1;
     q.cnt = 1;
+    q.gain_steps = 1;
     const long long nwin = p.b0 * p.b1 * p.tcount;
     const int H = p.H;
     int count = 0;
@@ -682,8 +684,9 @@ inline cudaError_t launch_scan_warp(const SolveParams& p, float* Pbuf, float* el
         }
     }
     const bool gains = p.K || p.x || p.u;
+    q.gain_steps = (p.K || p.x || (p.u && !p.first_only)) ? H : 1;
     if (gains) {
-        scan_step_kernel<N, true><<<blocks(nwin * H, 2), THREADS, sm_step, st>>>(q);
+        scan_step_kernel<N, true><<<blocks(nwin * q.gain_steps, 2), THREADS, sm_step, st>>>(q);
         if ((e = cudaGetLastError())) return e;
         ++count;
     }

@@ -15,6 +15,7 @@
 #include "ttc_layer.cuh"
 #include "lqr_grad.cuh"
 #include "scan_pair.cuh"
+#include "scan_warp.cuh"
 #include "peak_probe.cuh"
 
 using namespace ttc;
@@ -54,6 +55,7 @@ struct ttc_lqr_handle {
     int sm_count;
     size_t max_pitch;              // largest pitch a 2D copy accepts on this device
     DevBuf ws_K, ws_P, ws_E;       // scratch used by kernels
+    DevBuf ws_elem;                // scan elements (A_e, C_e, G_e, J_e per instance)
     DevBuf ws_k;                   // feed-forward terms k_t when the caller does not take them
     DevBuf ws_vec;                 // state, control and co-state sequences of the gradient entry point
     DevBuf st_in[5], st_out[5];    // device staging of ttc_lqr_solve_host
@@ -98,7 +100,7 @@ void release(DevBuf& b)
 
 size_t workspace_bytes(const ttc_lqr_handle* h)
 {
-    size_t s = h->ws_K.bytes + h->ws_P.bytes + h->ws_E.bytes + h->ws_k.bytes + h->ws_vec.bytes + h->st_layer.bytes;
+    size_t s = h->ws_K.bytes + h->ws_P.bytes + h->ws_E.bytes + h->ws_elem.bytes + h->ws_k.bytes + h->ws_vec.bytes + h->st_layer.bytes;
     for (int i = 0; i < 5; ++i)
         s += h->st_in[i].bytes + h->st_out[i].bytes;
     return s;
@@ -183,10 +185,21 @@ int clear_device_error(ttc_lqr_handle* h, cudaStream_t st)
     return TTC_OK;
 }
 
-int pick_method(const ttc_lqr_handle* h)
+// Method of one call.  TTC_AUTO means the sequential recursion except where the scan is measured to be faster:
+// time-invariant problems with n = m = 16 / 32 over long horizons with few instances.  The recursion then leaves most
+// of the GPU idle while it walks H dependent steps (4.4 us per step at n = 16, 12 us at n = 32), whereas the scan's
+// 2 log2(H) + 3 launches spread all N x H applications and gains over the machine (12 ns resp. 59 ns per instance
+// and step): the scan wins below about 300 (n = 16) and 180 (n = 32) instances.
+int pick_method(const ttc_lqr_handle* h, int H, bool time_varying, long long nwin)
 {
     if (h->cfg.method == TTC_SCAN)
         return TTC_SCAN;
+    const int n = h->cfg.n;
+    if (h->cfg.method == TTC_AUTO && !time_varying && n == h->cfg.m && (n == 16 || n == 32) && H >= 256) {
+        const long long in_flight = (long long)h->sm_count * (n == 32 ? 12 : 32);   // instances the recursion keeps resident
+        if (nwin * (n == 32 ? 10 : 16) <= in_flight)
+            return TTC_SCAN;
+    }
     return TTC_RICCATI;
 }
 
@@ -267,6 +280,7 @@ int ttc_lqr_destroy(ttc_lqr_handle* h)
     release(h->ws_K);
     release(h->ws_P);
     release(h->ws_E);
+    release(h->ws_elem);
     release(h->ws_k);
     release(h->ws_vec);
     for (int i = 0; i < 5; ++i) {
@@ -349,7 +363,7 @@ int solve_window(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, 
     p.kff = kff; p.pvec = pvec;
     p.first_only = (flags & TTC_OUT_FIRST_ONLY) ? 1 : 0;
 
-    const int method = pick_method(h);
+    const int method = pick_method(h, H, time_varying, nwin);
     if (method == TTC_SCAN && time_varying)
         return fail(TTC_STATUS_UNSUPPORTED, "the scan method handles time-invariant problems without a linear cost only");
     // The rollout reads every K_t in forward order after the backward pass produced them in
@@ -357,9 +371,11 @@ int solve_window(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, 
     const bool rollout_needs_all_K = (x != nullptr) || (u != nullptr && !p.first_only);
 
     if (method == TTC_SCAN) {
-        // Full mode keeps every P_t (in the caller's P or in the workspace); when only P_0 / u_0
-        // are wanted the scan keeps a single value matrix (P_1) per instance.
-        const int pfull = !(p.first_only && !K && !x);
+        // n = m = 16 / 32: the scan that is parallel in time; it keeps every P_t (in the caller's P or in the
+        // workspace).  Other shapes: the generic scan, which keeps every P_t, or a single value matrix (P_1) per
+        // instance when only P_0 / u_0 are wanted.
+        const bool warp_scan = n == m && (n == 16 || n == 32);
+        const int pfull = warp_scan || !(p.first_only && !K && !x);
         float* Pbuf;
         if (pfull && P && !p.first_only) {
             Pbuf = P;
@@ -370,7 +386,22 @@ int solve_window(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, 
         }
         if ((s = ensure(h->ws_E, sizeof(int) * (size_t)h->N))) return s;
         int launches = 0;
-        cudaError_t e = launch_scan_path(p, Pbuf, static_cast<int*>(h->ws_E.ptr), pfull, h->sm_count, st, &launches);
+        cudaError_t e;
+        if (warp_scan) {
+            // parallel in time: per doubling round one launch over every (instance, application) and one over the
+            // squarings, then one over every (instance, t) for the gains, then the rollout
+            if ((s = ensure(h->ws_elem, sizeof(float) * (size_t)h->N * scanw::ELEM_MATS * n * n))) return s;
+            if (!K && (x || u)) {
+                if ((s = ensure(h->ws_K, sizeof(float) * (size_t)h->N * H * m * n))) return s;
+                p.Kws = static_cast<float*>(h->ws_K.ptr);
+            }
+            float* elem = static_cast<float*>(h->ws_elem.ptr);
+            int* flags = static_cast<int*>(h->ws_E.ptr);
+            e = n == 16 ? scanw::launch_scan_warp<16>(p, Pbuf, elem, flags, h->sm_count, st, &launches)
+                        : scanw::launch_scan_warp<32>(p, Pbuf, elem, flags, h->sm_count, st, &launches);
+        } else {
+            e = launch_scan_path(p, Pbuf, static_cast<int*>(h->ws_E.ptr), pfull, h->sm_count, st, &launches);
+        }
         if (e != cudaSuccess)
             return fail(TTC_STATUS_CUDA_ERROR, "scan path launch: %s", cudaGetErrorString(e));
         h->last_launches += launches;
@@ -546,7 +577,7 @@ int ttc_lqr_grad(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, 
     for (int i = 0; i < 8; ++i)
         if (reinterpret_cast<uintptr_t>(ptrs[i]) & 15u)
             return fail(TTC_STATUS_INVALID_ARGUMENT, "g and the gradient outputs must be 16-byte aligned");
-    if (pick_method(h) == TTC_SCAN)
+    if (h->cfg.method == TTC_SCAN)
         return fail(TTC_STATUS_UNSUPPORTED, "the scan method has no gradient path");
     TTC_CUDA(cudaSetDevice(h->cfg.device));
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);

@@ -300,3 +300,20 @@ def test_bounded_wait_gives_up_and_reports():
     w = small_workload(64, 64, 3, (1, 1, 9), seed=5, bf16=True)
     g = pu.run_gpu(w)                      # run_gpu asserts that the solver's own error word is clear
     pu.compare(g, pu.run_oracle(w), np.arange(9), 2e-2)
+
+
+@pytest.mark.parametrize("n,H,batch,expect", [(16, 300, (1, 2, 8), "scan"), (32, 256, (1, 2, 5), "scan"),
+                                              (16, 300, (1, 8, 64), "riccati_warp"), (16, 64, (1, 2, 8), "riccati_warp")])
+def test_auto_method_takes_the_scan_for_few_instances_over_long_horizons(n, H, batch, expect):
+    """TTC_AUTO: the scan (parallel over the horizon) where the sequential recursion would leave the GPU idle -- few
+    instances, long horizon, n = m = 16 / 32 -- and the recursion elsewhere; same results either way."""
+    w = small_workload(n, n, H, batch, seed=911 + n + H, rho=0.98)
+    N = int(np.prod(batch))
+    idx = np.arange(0, N, max(1, N // 16))
+    gpu = pu.run_gpu(w, method=lqr.TTC_AUTO)
+    assert lqr.KERNEL_NAMES[gpu["kernel"]] == expect
+    ref = pu.run_oracle(w, idx=idx)
+    pu.compare(gpu, ref, idx, 1e-4)
+    g1 = pu.run_gpu(w, method=lqr.TTC_AUTO, want=("P", "u", "info"), first_only=True)
+    assert lqr.KERNEL_NAMES[g1["kernel"]] == expect
+    pu.compare(g1, pu.run_oracle(w, idx=idx, first_only=True), idx, 1e-4, names=("P", "u"))
