@@ -582,10 +582,19 @@ def run_solve(args, workload, method_name, ctx, light=False):
     math = {"auto": lqr.TTC_MATH_AUTO, "fp32": lqr.TTC_MATH_FP32, "tf32": lqr.TTC_MATH_TF32}[args.math]
     solver = lqr.LqrSolver(n, m, H, c["batch"], device=local, method=method, math=math)
     want = ("P", "u", "info") if first else ("K", "P", "x", "u", "info")
-    out = lqr.alloc_outputs(n, m, H, N, dev, first_only=first, want=want)
-    flags = lqr.TTC_OUT_FIRST_ONLY if first else 0
+    obf = args.out_dtype == "bf16" and not tv_key and not light
+    lowrank = args.lowrank_q and "U" in w and not light
+    out = lqr.alloc_outputs(n, m, H, N, dev, first_only=first, want=want, dtype=torch.bfloat16 if obf else torch.float32)
+    flags = (lqr.TTC_OUT_FIRST_ONLY if first else 0) | (lqr.TTC_OUT_BF16 if obf else 0)
+    if obf or lowrank:
+        no_e2e = True                      # the host-buffer entry point takes dense Q and returns float32
+        c["name"] += ("_outbf16" if obf else "") + ("_lowrankq" if lowrank else "")
 
     def step():
+        if lowrank:
+            solver.solve_lowrank_q(w["A"], w["B"], w["U"], w["d"], w["q_scale"], w["R"], w["x0"], H, K=out.get("K"),
+                                   P=out.get("P"), x=out.get("x"), u=out.get("u"), info=out.get("info"), flags=flags)
+            return
         if tv_key:
             solver.solve_tv(w["A"], w["B"], w["Q"], w["R"], w["Qf"], w["x0"], H, tv=c["tv"], K=out.get("K"),
                             P=out.get("P"), x=out.get("x"), u=out.get("u"), info=out.get("info"), flags=flags)
@@ -599,6 +608,10 @@ def run_solve(args, workload, method_name, ctx, light=False):
         torch.cuda.synchronize(dev)
 
     flops_i, bin_i, bout_i = algorithmic_counts(c)
+    if obf:
+        bout_i = bout_i // 2               # bfloat16 outputs
+    if lowrank:
+        bin_i = (n * 8 + n + n) * (2 if c["q_dtype"] == "bf16" else 4)      # U, d, x0
     alg_bytes = N * (bin_i + bout_i)
     alg_flops = N * flops_i
     # inputs + outputs of the large configurations exceed L2 several times over; the small ones fit, so a buffer
@@ -702,9 +715,21 @@ def run_solve(args, workload, method_name, ctx, light=False):
     if not args.no_cpu_baseline and world == 1:
         # parity of the timed configuration on a stratified sample (every sequence and head), oracle timed on it
         idx = oracle_sample(w, args.cpu_sample)
-        ref, dt = time_oracle(w, idx, first)
         from tests import parity_util as pu
-        errs = pu.compare(out, ref, idx, c["tol"], names=("P", "u") if first else ("K", "P", "x", "u"))
+        if lowrank:                        # the oracle gets the dense Q that the factors describe, formed in float64
+            from oracle import lqr_oracle as orc
+            A_, B_, _, R_, x0_ = pu.gather_inputs(w, idx)
+            sel = torch.as_tensor(idx, device=dev)
+            U_ = w["U"].reshape(N, n, 8)[sel].double().cpu().numpy()
+            d_ = w["d"].reshape(N, n)[sel].double().cpu().numpy()
+            Q_ = w["q_scale"] * U_ @ np.swapaxes(U_, 1, 2) + d_[:, :, None] * np.eye(n)
+            t0 = time.perf_counter()
+            ref = orc.solve_batch(A_, B_, Q_, R_, x0_, H, batch=(len(idx),), first_only=first)
+            dt = time.perf_counter() - t0
+        else:
+            ref, dt = time_oracle(w, idx, first)
+        got = {k: (v.float() if v.dtype == torch.bfloat16 else v) for k, v in out.items()}
+        errs = pu.compare(got, ref, idx, c["tol"] + (2.0 ** -8 if obf else 0.0), names=("P", "u") if first else ("K", "P", "x", "u"))
         cpu = {"value": len(idx) / dt, "unit": "instances/s", "cores": int(ref["threads"]), "kind": "oracle",
                "sample": "%d instances of the same workload, every (seq, head) covered" % len(idx),
                "seconds": dt, "parity_max_rel_err": errs, "speedup_gpu_over_cpu": value / (len(idx) / dt)}
@@ -715,7 +740,8 @@ def run_solve(args, workload, method_name, ctx, light=False):
             "scaling": "weak", "vs_baseline": None, "dtype": "tf32" if kname == "riccati_umma" else "f32",
             "data": "synthetic",
             "config": {"workload": c["name"], "n": n, "m": m, "H": H, "instances": N, "batch": list(c["batch"]),
-                       "q_x0_dtype": c["q_dtype"], "time_varying": list(c.get("tv", ())), "outputs": list(want), "method": method_name, "kernel": kname,
+                       "q_x0_dtype": c["q_dtype"], "output_dtype": "bf16" if obf else "f32",
+                       "q_operand": "U U'/8 + diag(d) factors" if lowrank else "dense", "time_varying": list(c.get("tv", ())), "outputs": list(want), "method": method_name, "kernel": kname,
                        "l2": "inputs+outputs per step exceed L2 (%.2f GB)" % (alg_bytes / 1e9)
                        if alg_bytes > 256e6 else "workload fits L2: a 192 MB buffer is written between timed steps"},
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches),
@@ -754,6 +780,8 @@ def main():
     ap.add_argument("--horizon", type=int, default=0, help="layer workloads: override the planning horizon T (sweeps)")
     ap.add_argument("--batch", default="", help="layer and gradient workloads: override the batch as SxHxT, e.g. 1x16x64 (sweeps)")
     ap.add_argument("--per-token", action="store_true", help="grad16: A_t, B_t, R_t per token instead of per head")
+    ap.add_argument("--out-dtype", default="f32", choices=["f32", "bf16"], help="bfloat16 K, P, x, u (TTC_OUT_BF16)")
+    ap.add_argument("--lowrank-q", action="store_true", help="cfg4: hand Q over as its factors (ttc_lqr_solve_lowrank_q)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-sides", action="store_true", help="default run: skip the side measurements of cfg0..cfg3")

@@ -69,6 +69,11 @@ extern "C" {
 
 /* ttc_lqr_solve flags */
 #define TTC_OUT_FIRST_ONLY  1u  /* P is [N][n][n] = P_0 and u is [N][m] = u_0          */
+#define TTC_OUT_BF16        2u  /* K, P, x, u are bfloat16 arrays (same shapes), rounded to
+                                   nearest even from the float32 results; halves the bytes the
+                                   write-bound requests store.  ttc_lqr_solve only, sequential
+                                   recursion, n = m in {16, 32, 64 with TF32 math}; other
+                                   requests return TTC_STATUS_UNSUPPORTED.  info stays int32. */
 
 /* ttc_lqr_query keys */
 #define TTC_QUERY_LAST_LAUNCHES    1  /* kernels launched by the last solve            */
@@ -132,7 +137,7 @@ int ttc_lqr_create(const ttc_lqr_config* cfg, ttc_lqr_handle** out);
  *
  * Inputs (device):  A [n][n], B [n][m], R [m][m] as F32;  Q [n][n], x0 [n] as F32 or BF16.
  *                   x0 may be NULL when neither x nor u is requested.
- * Outputs (device, F32, written completely, each may be NULL = not wanted):
+ * Outputs (device, F32 -- BF16 with TTC_OUT_BF16 --, written completely, each may be NULL = not wanted):
  *     K    [N][H][m][n]
  *     P    [N][H+1][n][n]    (or [N][n][n] = P_0   with TTC_OUT_FIRST_ONLY)
  *     x    [N][H+1][n]
@@ -150,6 +155,22 @@ int ttc_lqr_solve(ttc_lqr_handle* h,
                   const ttc_operand* R, const ttc_operand* x0, int32_t H,
                   float* K, float* P, float* x, float* u, int32_t* info,
                   uint32_t flags, void* cuda_stream);
+
+/*
+ * ttc_lqr_solve with the state cost handed over in factored form (Parameterization paragraph of the TTC-Net
+ * section: Q is a combination of a few basis directions plus a diagonal):
+ *     Q = scale * U U' + diag(d),      U [n][rank] and d [n] per instance (F32 or BF16, batch strides as any operand),
+ *     1 <= rank <= n, scale >= 0.  Q is symmetric positive semi-definite by construction when d >= 0.
+ * The library expands Q on the device into a float32 workspace it owns (N n^2 floats, one more kernel launch) and then
+ * runs exactly the ttc_lqr_solve path on it; the caller stores and transfers n (rank + 1) numbers per instance instead
+ * of n^2 (configuration 4: 1.2 KB instead of 8 KB).  With TTC_MATH_AUTO the tensor-core path is taken when U is BF16,
+ * as for a BF16 dense Q.  Everything else (outputs, info, flags, stream, errors) as ttc_lqr_solve.
+ */
+int ttc_lqr_solve_lowrank_q(ttc_lqr_handle* h,
+                            const ttc_operand* A, const ttc_operand* B, const ttc_operand* U, const ttc_operand* d,
+                            int32_t rank, float scale, const ttc_operand* R, const ttc_operand* x0, int32_t H,
+                            float* K, float* P, float* x, float* u, int32_t* info,
+                            uint32_t flags, void* cuda_stream);
 
 /*
  * Time-varying problem (Definition A.1 / Prop. A.1 with A_t, B_t, Q_t, R_t and a terminal weight Q_f;

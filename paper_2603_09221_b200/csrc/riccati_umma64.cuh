@@ -360,21 +360,22 @@ __device__ __forceinline__ void wg_fail_instance(const SolveParams& p, long long
 {
     const float qn = quiet_nan();
     const int H = p.H;
+    const int obf = p.out_bf16;
     if (p.K)
         for (long long e = wt; e < (long long)H * N * N; e += WG_THREADS)
-            p.K[inst * (long long)H * N * N + e] = qn;
+            store_out(p.K, inst * (long long)H * N * N + e, qn, obf);
     if (p.P) {
         const long long cnt = (long long)(p.first_only ? 1 : H + 1) * N * N;
         for (long long e = wt; e < cnt; e += WG_THREADS)
-            p.P[inst * cnt + e] = qn;
+            store_out(p.P, inst * cnt + e, qn, obf);
     }
     if (p.x)
         for (long long e = wt; e < (long long)(H + 1) * N; e += WG_THREADS)
-            p.x[inst * (long long)(H + 1) * N + e] = qn;
+            store_out(p.x, inst * (long long)(H + 1) * N + e, qn, obf);
     if (p.u) {
         const long long cnt = p.first_only ? N : (long long)H * N;
         for (long long e = wt; e < cnt; e += WG_THREADS)
-            p.u[inst * cnt + e] = qn;
+            store_out(p.u, inst * cnt + e, qn, obf);
     }
     if (p.info && wt == 0)
         p.info[inst] = code;
@@ -442,11 +443,12 @@ __device__ __forceinline__ void store_half_tf32(unsigned char* buf, int r, int h
         *reinterpret_cast<float4*>(buf + toff(r, 32 * half + 4 * c)) =
             make_float4(round_tf32(v[4 * c]), round_tf32(v[4 * c + 1]), round_tf32(v[4 * c + 2]), round_tf32(v[4 * c + 3]));
 }
-__device__ __forceinline__ void store_half_global(float* dst, const float (&v)[32])
+// 32 consecutive output elements starting at element `idx` of `base` (float32 or bfloat16 output)
+__device__ __forceinline__ void store_half_global(float* base, long long idx, const float (&v)[32], int bf16)
 {
 #pragma unroll
     for (int c = 0; c < 8; ++c)
-        reinterpret_cast<float4*>(dst)[c] = make_float4(v[4 * c], v[4 * c + 1], v[4 * c + 2], v[4 * c + 3]);
+        store_out4(base, idx + 4 * c, make_float4(v[4 * c], v[4 * c + 1], v[4 * c + 2], v[4 * c + 3]), bf16);
 }
 
 // GAINS = the request needs every K_t (K, x or the full u wanted); the other instantiation carries none of that code.
@@ -501,7 +503,10 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
     const long long nchunks = p.b0 * p.b1 * chunks_per_head;
     constexpr bool need_K_all = GAINS;
     const bool want_u0 = (p.u != nullptr) && p.first_only && !need_K_all;
-    float* Kbase = p.K ? p.K : p.Kws;
+    // With bfloat16 outputs the rollout kernel still reads float32 gains: they go to the workspace, and to K as
+    // bfloat16 too.
+    const int obf = p.out_bf16;
+    float* Kbase = (p.K && !obf) ? p.K : p.Kws;
     long long offA_loaded = -1, offB_loaded = -1, offR_loaded = -1;
     bool dead = false;
 
@@ -561,7 +566,7 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
                     load_q_half(q, p.Q, oq, j, half);
                     store_half_tf32(X0, j, half, q);
                     if (p.P && !p.first_only)
-                        store_half_global(p.P + (inst * (long long)(H + 1) + H) * N * N + (long long)j * N + 32 * half, q);
+                        store_half_global(p.P, (inst * (long long)(H + 1) + H) * N * N + (long long)j * N + 32 * half, q, obf);
                 }
             } else if (p.x0.ptr && warp == 0) {
                 const long long ox = operand_offset(p.x0, inst, p.b1, p.b2);
@@ -778,7 +783,7 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
 #pragma unroll
                         for (int r = 0; r < 8; ++r)
                             if (i == c0 + r)
-                                p.u[inst * (long long)N + i] = -w[r];
+                                store_out(p.u, inst * (long long)N + i, -w[r], obf);
                     }
                 }
                 wait_mma();
@@ -796,6 +801,13 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
                             kt[(4 * q4 + 1) * N] = -kv.y;
                             kt[(4 * q4 + 2) * N] = -kv.z;
                             kt[(4 * q4 + 3) * N] = -kv.w;
+                            if (obf && p.K) {
+                                const long long ko = (inst * (long long)H + ts) * N * N + cidx + (long long)(4 * q4) * N;
+                                store_out(p.K, ko, -kv.x, 1);
+                                store_out(p.K, ko + N, -kv.y, 1);
+                                store_out(p.K, ko + 2 * N, -kv.z, 1);
+                                store_out(p.K, ko + 3 * N, -kv.w, 1);
+                            }
                         }
                     }
                     wg_barrier(wg);                   // X0 is free for the next value matrix
@@ -803,9 +815,8 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
                 // P_t = Q + DP: warps 2, 3 own the rows (lanes 64..127)
                 if (warp >= 2) {
                     const int j = wt - 64;
-                    float* Pdst = (p.P && (!p.first_only || ts == 0))
-                                      ? p.P + (inst * (long long)(p.first_only ? 1 : H + 1) + (p.first_only ? 0 : ts)) * N * N + (long long)j * N
-                                      : nullptr;
+                    const bool Pdst = p.P && (!p.first_only || ts == 0);
+                    const long long Pidx = (inst * (long long)(p.first_only ? 1 : H + 1) + (p.first_only ? 0 : ts)) * N * N + (long long)j * N;
                     if (q_pref) {
 #pragma unroll
                         for (int qt = 0; qt < 4; ++qt) {       // 16 columns at a time
@@ -835,7 +846,7 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
                             if (Pdst) {
 #pragma unroll
                                 for (int c = 0; c < 4; ++c)
-                                    reinterpret_cast<float4*>(Pdst + 16 * qt)[c] = make_float4(q[4 * c], q[4 * c + 1], q[4 * c + 2], q[4 * c + 3]);
+                                    store_out4(p.P, Pidx + 16 * qt + 4 * c, make_float4(q[4 * c], q[4 * c + 1], q[4 * c + 2], q[4 * c + 3]), obf);
                             }
                         }
                     } else {
@@ -850,7 +861,7 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
                             if (ts > 0)
                                 store_half_tf32(X0, j, half, q);
                             if (Pdst)
-                                store_half_global(Pdst + 32 * half, q);
+                                store_half_global(p.P, Pidx + 32 * half, q, obf);
                         }
                     }
                     // Every eighth step the operand is replaced by (P + P') / 2.  Q and Z'Z are symmetric but the rounding
@@ -944,13 +955,14 @@ __global__ void __launch_bounds__(32 * ROLL_WARPS, 5) rollout64_kernel(SolvePara
             continue;
         float* xs = sm.x[warp];
         float* us = sm.u[warp];
-        float* xo = p.x ? p.x + inst * (long long)(H + 1) * N : nullptr;
-        float* uo = p.u ? p.u + inst * (long long)(p.first_only ? 1 : H) * N : nullptr;
+        const int obf = p.out_bf16;
+        const bool xo = p.x != nullptr, uo = p.u != nullptr;
+        const long long xoff = inst * (long long)(H + 1) * N, uoff = inst * (long long)(p.first_only ? 1 : H) * N;
         {
             const long long ox = operand_offset(p.x0, inst, p.b1, p.b2);
             const float a = load_elem(p.x0, ox + lane), b = load_elem(p.x0, ox + lane + 32);
             xs[lane] = a; xs[lane + 32] = b;
-            if (xo) { xo[lane] = a; xo[lane + 32] = b; }
+            if (xo) { store_out(p.x, xoff + lane, a, obf); store_out(p.x, xoff + lane + 32, b, obf); }
         }
         __syncwarp();
         const int half = lane >> 4, seg = lane & 15;
@@ -971,9 +983,9 @@ __global__ void __launch_bounds__(32 * ROLL_WARPS, 5) rollout64_kernel(SolvePara
             }
             __syncwarp();
             if (uo && (!p.first_only || ts == 0)) {
-                float* ut = uo + (p.first_only ? 0 : (long long)ts * N);
-                ut[lane] = us[lane];
-                ut[lane + 32] = us[lane + 32];
+                const long long ut = uoff + (p.first_only ? 0 : (long long)ts * N);
+                store_out(p.u, ut + lane, us[lane], obf);
+                store_out(p.u, ut + lane + 32, us[lane + 32], obf);
             }
             float n0 = 0.f, n1 = 0.f;                         // rows lane and lane + 32 of A x + B u
 #pragma unroll
@@ -993,8 +1005,8 @@ __global__ void __launch_bounds__(32 * ROLL_WARPS, 5) rollout64_kernel(SolvePara
             xs[lane] = n0;
             xs[lane + 32] = n1;
             if (xo) {
-                xo[(long long)(ts + 1) * N + lane] = n0;
-                xo[(long long)(ts + 1) * N + lane + 32] = n1;
+                store_out(p.x, xoff + (long long)(ts + 1) * N + lane, n0, obf);
+                store_out(p.x, xoff + (long long)(ts + 1) * N + lane + 32, n1, obf);
             }
             __syncwarp();
         }

@@ -224,7 +224,9 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
     const bool need_K_all = (p.K != nullptr) || (p.x != nullptr) || (p.u != nullptr && !p.first_only);
     const bool want_u0 = (p.u != nullptr) && p.first_only && !need_K_all;
     const bool need_k_all = AFF && p.kff != nullptr;          // feed-forward terms wanted (output or rollout)
-    float* Kbase = p.K ? p.K : p.Kws;
+    // With bfloat16 outputs the rollout still reads float32 gains: they go to the workspace, and to K as bfloat16 too.
+    const int obf = p.out_bf16;
+    float* Kbase = (p.K && !obf) ? p.K : p.Kws;
     long long offA = -1, offB = -1, offR = -1;
 
     for (;;) {
@@ -258,17 +260,18 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
             load_slot_operands<N>(As, Bs, Rs, p, oai, obi, ori, H - 1, true, true, true, c);    // ordered by the barrier below
         const long long oq = operand_offset(p.Q, inst, p.b1, p.b2) + (long long)c * N;
 
-        float* Pout = (p.P && active) ? p.P + inst * (long long)(p.first_only ? 1 : H + 1) * N * N : nullptr;
+        const bool wantP = p.P && active;
+        const long long Poff = inst * (long long)(p.first_only ? 1 : H + 1) * N * N;     // first element of this instance's P
         float* Kout = (Kbase && need_K_all) ? Kbase + inst * (long long)H * N * N : nullptr;
         float pcol[N];
         if (TV && p.Qf.ptr)
             load_q_row<N>(pcol, p.Qf, operand_offset(p.Qf, inst, p.b1, p.b2) + (long long)c * N);   // P_H = Q_f
         else
             load_q_row<N>(pcol, p.Q, oq);                     // P_H = Q
-        if (Pout && !p.first_only) {
+        if (wantP && !p.first_only) {
 #pragma unroll
             for (int l = 0; l < N; ++l)
-                Pout[(long long)H * N * N + l * N + c] = pcol[l];
+                store_out(p.P, Poff + (long long)H * N * N + l * N + c, pcol[l], obf);
         }
         store_row<N>(sl.buf0 + c * LD, pcol);
         if (p.x0.ptr)
@@ -472,6 +475,12 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
 #pragma unroll
                         for (int l = 0; l < N; ++l)
                             kt[l * N] = -y[l];
+                        if (obf && p.K) {
+                            const long long ko = (inst * (long long)H + ts) * N * N + c;
+#pragma unroll
+                            for (int l = 0; l < N; ++l)
+                                store_out(p.K, ko + l * N, -y[l], 1);
+                        }
                     }
                 } else if (want_u0 && ts == 0) {              // K_0 rows -> Lt (free after the forward substitution)
 #pragma unroll
@@ -488,11 +497,11 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
 #pragma unroll
             for (int l = 0; l < N; ++l)
                 pcol[l] = 0.5f * (pcol[l] + sl.buf0[l * LD + c]);
-            if (Pout && (!p.first_only || ts == 0)) {
-                float* pt = Pout + (long long)(p.first_only ? 0 : ts) * N * N + c;
+            if (wantP && (!p.first_only || ts == 0)) {
+                const long long po = Poff + (long long)(p.first_only ? 0 : ts) * N * N + c;
 #pragma unroll
                 for (int l = 0; l < N; ++l)
-                    pt[l * N] = pcol[l];
+                    store_out(p.P, po + l * N, pcol[l], obf);
             }
             __syncwarp();                                     // every lane has read its column
             store_row<N>(sl.buf0 + c * LD, pcol);
@@ -505,19 +514,19 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
             const float qn = quiet_nan();
             if (p.K)
                 for (long long e = c; e < (long long)H * N * N; e += N)
-                    p.K[inst * (long long)H * N * N + e] = qn;
+                    store_out(p.K, inst * (long long)H * N * N + e, qn, obf);
             if (p.P) {
                 const long long cnt = (long long)(p.first_only ? 1 : H + 1) * N * N;
                 for (long long e = c; e < cnt; e += N)
-                    p.P[inst * cnt + e] = qn;
+                    store_out(p.P, inst * cnt + e, qn, obf);
             }
             if (p.x)
                 for (long long e = c; e < (long long)(H + 1) * N; e += N)
-                    p.x[inst * (long long)(H + 1) * N + e] = qn;
+                    store_out(p.x, inst * (long long)(H + 1) * N + e, qn, obf);
             if (p.u) {
                 const long long cnt = p.first_only ? N : (long long)H * N;
                 for (long long e = c; e < cnt; e += N)
-                    p.u[inst * cnt + e] = qn;
+                    store_out(p.u, inst * cnt + e, qn, obf);
             }
             if (AFF && p.pvec) {
                 const long long cnt = (long long)(p.first_only ? 1 : H + 1) * N;
@@ -542,17 +551,17 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
             for (int j = 0; j < N; ++j)
                 uc = fmaf(kr[j], xv[j], uc);
             if (store_ok)
-                p.u[inst * (long long)N + c] = uc;
+                store_out(p.u, inst * (long long)N + c, uc, obf);
         } else if (p.x || p.u) {
-            float* xo = (p.x && store_ok) ? p.x + inst * (long long)(H + 1) * N : nullptr;
-            float* uo = (p.u && store_ok) ? p.u + inst * (long long)(p.first_only ? N : H * N) : nullptr;
+            const bool xo = p.x && store_ok, uo = p.u && store_ok;
+            const long long xoff = inst * (long long)(H + 1) * N, uoff = inst * (long long)(p.first_only ? N : H * N);
             float arow[N], brow[N];
             if (!tv_head) {
                 load_row<N>(arow, As + c * LD);
                 load_row<N>(brow, Bs + c * LD);
             }
             if (xo)
-                xo[c] = sl.x[c];
+                store_out(p.x, xoff + c, sl.x[c], obf);
             __syncwarp();                                     // K_t written by the other lanes are visible
 #pragma unroll 1
             for (int ts = 0; ts < H; ++ts) {
@@ -586,7 +595,7 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
                 }
                 sl.u[c] = uc;
                 if (uo && (!p.first_only || ts == 0))
-                    uo[(p.first_only ? 0 : ts * N) + c] = uc;
+                    store_out(p.u, uoff + (p.first_only ? 0 : ts * N) + c, uc, obf);
                 __syncwarp();
                 float uv[N];
                 load_row<N>(uv, sl.u);
@@ -597,7 +606,7 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
                 __syncwarp();                                 // x_t consumed by every lane
                 sl.x[c] = xc;
                 if (xo)
-                    xo[(long long)(ts + 1) * N + c] = xc;
+                    store_out(p.x, xoff + (long long)(ts + 1) * N + c, xc, obf);
                 __syncwarp();
             }
         }

@@ -55,6 +55,7 @@ struct ttc_lqr_handle {
     int sm_count;
     size_t max_pitch;              // largest pitch a 2D copy accepts on this device
     DevBuf ws_K, ws_P, ws_E;       // scratch used by kernels
+    DevBuf ws_Q;                   // dense Q expanded from a low-rank-plus-diagonal operand
     DevBuf ws_elem;                // scan elements (A_e, C_e, G_e, J_e per instance)
     DevBuf ws_k;                   // feed-forward terms k_t when the caller does not take them
     DevBuf ws_vec;                 // state, control and co-state sequences of the gradient entry point
@@ -100,7 +101,7 @@ void release(DevBuf& b)
 
 size_t workspace_bytes(const ttc_lqr_handle* h)
 {
-    size_t s = h->ws_K.bytes + h->ws_P.bytes + h->ws_E.bytes + h->ws_elem.bytes + h->ws_k.bytes + h->ws_vec.bytes + h->st_layer.bytes;
+    size_t s = h->ws_K.bytes + h->ws_P.bytes + h->ws_E.bytes + h->ws_elem.bytes + h->ws_Q.bytes + h->ws_k.bytes + h->ws_vec.bytes + h->st_layer.bytes;
     for (int i = 0; i < 5; ++i)
         s += h->st_in[i].bytes + h->st_out[i].bytes;
     return s;
@@ -150,7 +151,7 @@ int validate_common(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* 
         return fail(TTC_STATUS_INVALID_ARGUMENT, "null handle");
     if (H < 1 || H > h->cfg.max_horizon)
         return fail(TTC_STATUS_INVALID_ARGUMENT, "H=%d outside [1, max_horizon=%d]", H, h->cfg.max_horizon);
-    if (flags & ~TTC_OUT_FIRST_ONLY)
+    if (flags & ~(TTC_OUT_FIRST_ONLY | TTC_OUT_BF16))
         return fail(TTC_STATUS_INVALID_ARGUMENT, "unknown flag bits 0x%x", flags);
     int s;
     if ((s = check_operand("A", A, false, false))) return s;
@@ -281,6 +282,7 @@ int ttc_lqr_destroy(ttc_lqr_handle* h)
     release(h->ws_P);
     release(h->ws_E);
     release(h->ws_elem);
+    release(h->ws_Q);
     release(h->ws_k);
     release(h->ws_vec);
     for (int i = 0; i < 5; ++i) {
@@ -362,6 +364,8 @@ int solve_window(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, 
     p.Kws = nullptr;
     p.kff = kff; p.pvec = pvec;
     p.first_only = (flags & TTC_OUT_FIRST_ONLY) ? 1 : 0;
+    p.out_bf16 = (flags & TTC_OUT_BF16) ? 1 : 0;
+    const bool obf = p.out_bf16 != 0;
 
     const int method = pick_method(h, H, time_varying, nwin);
     if (method == TTC_SCAN && time_varying)
@@ -370,6 +374,8 @@ int solve_window(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, 
     // reverse order; when the caller does not want K they live in the workspace.
     const bool rollout_needs_all_K = (x != nullptr) || (u != nullptr && !p.first_only);
 
+    if (obf && (method == TTC_SCAN || time_varying))
+        return fail(TTC_STATUS_UNSUPPORTED, "bfloat16 outputs are served by the sequential recursion of ttc_lqr_solve only");
     if (method == TTC_SCAN) {
         // n = m = 16 / 32: the scan that is parallel in time; it keeps every P_t (in the caller's P or in the
         // workspace).  Other shapes: the generic scan, which keeps every P_t, or a single value matrix (P_1) per
@@ -409,7 +415,8 @@ int solve_window(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, 
         h->last_kernel = TTC_KERNEL_SCAN;
         return TTC_OK;
     } else {
-        if (!K && rollout_needs_all_K) {
+        // the rollout reads float32 gains: from K itself, or from the workspace when K is not wanted or is bfloat16
+        if ((!K && rollout_needs_all_K) || (obf && (K || rollout_needs_all_K))) {
             if ((s = ensure(h->ws_K, sizeof(float) * (size_t)h->N * H * m * n))) return s;
             p.Kws = static_cast<float*>(h->ws_K.ptr);
         }
@@ -448,7 +455,7 @@ int solve_window(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, 
                 const long long rchunks = p.b0 * p.b1 * ((tcount + umma64::ROLL_WARPS - 1) / umma64::ROLL_WARPS);
                 long long rgrid = (long long)h->sm_count * 5;
                 if (rgrid > rchunks) rgrid = rchunks;
-                umma64::rollout64_kernel<<<(unsigned)rgrid, 32 * umma64::ROLL_WARPS, rsmem, st>>>(p, K ? K : p.Kws);
+                umma64::rollout64_kernel<<<(unsigned)rgrid, 32 * umma64::ROLL_WARPS, rsmem, st>>>(p, (K && !obf) ? K : p.Kws);
                 TTC_CUDA(cudaGetLastError());
                 h->last_launches += 1;
                 h->total_launches += 1;
@@ -490,6 +497,9 @@ int solve_window(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, 
             h->last_kernel = TTC_KERNEL_RICCATI_WARP;
             return TTC_OK;
         }
+        if (obf)
+            return fail(TTC_STATUS_UNSUPPORTED, "bfloat16 outputs need n = m in {16, 32} or the tensor-core path at n = m = 64 "
+                                                "(per-head or per-token A, B, R; Q strides that keep 16-byte rows)");
         const size_t smem = riccati_cta_smem_bytes(n, m);
         TTC_CUDA(cudaFuncSetAttribute(riccati_cta_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         int per_sm = 1;
@@ -524,6 +534,57 @@ int ttc_lqr_solve(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B,
         return s;
     return solve_window(h, A, B, Q, R, x0, H, K, P, x, u, info, flags, static_cast<cudaStream_t>(cuda_stream), 0,
                         h->cfg.batch[2]);
+}
+
+int ttc_lqr_solve_lowrank_q(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, const ttc_operand* U,
+                            const ttc_operand* d, int32_t rank, float scale, const ttc_operand* R, const ttc_operand* x0,
+                            int32_t H, float* K, float* P, float* x, float* u, int32_t* info, uint32_t flags,
+                            void* cuda_stream)
+{
+    if (!h)
+        return fail(TTC_STATUS_INVALID_ARGUMENT, "null handle");
+    const int n = h->cfg.n;
+    if (rank < 1 || rank > n)
+        return fail(TTC_STATUS_INVALID_ARGUMENT, "rank=%d outside [1, n=%d]", rank, n);
+    if (!(scale >= 0.f))
+        return fail(TTC_STATUS_INVALID_ARGUMENT, "scale must be non-negative");
+    int s;
+    if ((s = check_operand("U", U, true, false))) return s;
+    if ((s = check_operand("d", d, true, false))) return s;
+    // the dense operand the solve will read: float32, one matrix per instance
+    ttc_operand Qd;
+    Qd.ptr = reinterpret_cast<const void*>(16);       // placeholder so that validation sees a non-null, aligned pointer
+    Qd.dtype = TTC_F32; Qd.reserved = 0;
+    Qd.bstride[2] = (int64_t)n * n;
+    Qd.bstride[1] = Qd.bstride[2] * h->cfg.batch[2];
+    Qd.bstride[0] = Qd.bstride[1] * h->cfg.batch[1];
+    if ((s = validate_common(h, A, B, &Qd, R, x0, H, K, P, x, u, info, flags))) return s;
+    TTC_CUDA(cudaSetDevice(h->cfg.device));
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if ((s = ensure(h->ws_Q, sizeof(float) * (size_t)h->N * n * n))) return s;
+    Qd.ptr = h->ws_Q.ptr;
+    h->last_launches = 0;
+    if ((s = clear_device_error(h, st))) return s;
+    {
+        SolveParams p;
+        p.n = n; p.m = h->cfg.m; p.H = H;
+        p.b0 = h->cfg.batch[0]; p.b1 = h->cfg.batch[1]; p.b2 = h->cfg.batch[2]; p.N = h->N;
+        p.t0 = 0; p.tcount = p.b2;
+        long long grid = h->N < (long long)h->sm_count * 8 ? h->N : (long long)h->sm_count * 8;
+        expand_lowrank_q_kernel<<<(unsigned)grid, 256, sizeof(float) * (size_t)(rank + 1) * n, st>>>(
+            p, to_dev(U), to_dev(d), rank, scale, static_cast<float*>(h->ws_Q.ptr));
+        TTC_CUDA(cudaGetLastError());
+        h->last_launches += 1;
+        h->total_launches += 1;
+    }
+    // AUTO math: tensor-core path when the factors were handed over in bfloat16, as for a bfloat16 dense Q
+    const bool bf16_factors = U->dtype == TTC_BF16;
+    const int math_saved = h->cfg.math;
+    if (math_saved == TTC_MATH_AUTO && bf16_factors && n == 64 && h->cfg.m == 64)
+        h->cfg.math = TTC_MATH_TF32;
+    s = solve_window(h, A, B, &Qd, R, x0, H, K, P, x, u, info, flags, st, 0, h->cfg.batch[2]);
+    h->cfg.math = math_saved;
+    return s;
 }
 
 int ttc_lqr_solve_affine(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, const ttc_operand* Q,
@@ -609,7 +670,7 @@ int ttc_lqr_grad(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operand* B, 
     p.A.st = tstride[0]; p.B.st = tstride[1]; p.Q.st = tstride[2]; p.R.st = tstride[3];
     p.r = to_dev(nullptr); p.r_count = 0;
     p.K = nullptr; p.P = nullptr; p.x = nullptr; p.u = nullptr; p.info = info; p.Kws = nullptr;
-    p.kff = nullptr; p.pvec = nullptr; p.first_only = 0;
+    p.kff = nullptr; p.pvec = nullptr; p.first_only = 0; p.out_bf16 = 0;
     gp.K = Kws; gp.kff = kws; gp.vec = static_cast<float*>(h->ws_vec.ptr); gp.D = D;
     {
         auto pow2 = [](int v) { return v > 0 && (v & (v - 1)) == 0; };
@@ -832,6 +893,8 @@ int ttc_lqr_solve_host(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operan
     // alignment of host pointers is irrelevant; validate the rest through a relaxed copy
     if (H < 1 || H > h->cfg.max_horizon)
         return fail(TTC_STATUS_INVALID_ARGUMENT, "H=%d outside [1, max_horizon=%d]", H, h->cfg.max_horizon);
+    if (flags & TTC_OUT_BF16)
+        return fail(TTC_STATUS_UNSUPPORTED, "the host-buffer entry point returns float32 outputs");
     if (flags & ~TTC_OUT_FIRST_ONLY)
         return fail(TTC_STATUS_INVALID_ARGUMENT, "unknown flag bits 0x%x", flags);
     TTC_CUDA(cudaSetDevice(h->cfg.device));
@@ -1145,6 +1208,7 @@ extern "C" int ttc_lqr_solve_first_noalloc(int32_t n, int32_t m, const int64_t b
     p.Kws = nullptr;
     p.kff = nullptr; p.pvec = nullptr;
     p.first_only = 1;
+    p.out_bf16 = 0;
     float* p1 = static_cast<float*>(scratch);
     int* flags = reinterpret_cast<int*>(static_cast<unsigned char*>(scratch) + p1_bytes);
     int launches = 0;

@@ -19,6 +19,7 @@ TTC_F32, TTC_BF16 = 0, 1
 TTC_AUTO, TTC_RICCATI, TTC_SCAN = 0, 1, 2
 TTC_MATH_AUTO, TTC_MATH_FP32, TTC_MATH_TF32 = 0, 1, 2
 TTC_OUT_FIRST_ONLY = 1
+TTC_OUT_BF16 = 2
 TTC_QUERY_LAST_LAUNCHES, TTC_QUERY_WORKSPACE_BYTES, TTC_QUERY_LAST_KERNEL, TTC_QUERY_TOTAL_LAUNCHES = 1, 2, 3, 4
 TTC_QUERY_DEVICE_ERROR = 5
 KERNEL_NAMES = {6: "ttc_layer", 0: "none", 1: "riccati_cta", 2: "riccati_warp", 4: "scan", 5: "riccati_umma"}
@@ -27,7 +28,7 @@ EXPORTS = (
     "ttc_lqr_create", "ttc_lqr_solve", "ttc_lqr_solve_host", "ttc_lqr_destroy", "ttc_lqr_query",
     "ttc_lqr_status_string", "ttc_lqr_last_error", "ttc_lqr_solve_first_noalloc", "ttc_lqr_solve_tv",
     "ttc_lqr_solve_layer", "ttc_lqr_solve_layer_host", "ttc_lqr_solve_affine", "ttc_lqr_grad",
-    "ttc_lqr_selftest_bounded_wait", "ttc_lqr_measure_fp32_peak",
+    "ttc_lqr_selftest_bounded_wait", "ttc_lqr_measure_fp32_peak", "ttc_lqr_solve_lowrank_q",
 )
 TTC_NOALLOC_SCRATCH_BYTES = 4 << 20
 
@@ -75,6 +76,9 @@ def load_library():
     lib.ttc_lqr_solve.restype = ctypes.c_int
     lib.ttc_lqr_solve.argtypes = [ctypes.c_void_p, opp, opp, opp, opp, opp, ctypes.c_int32] + \
         [ctypes.c_void_p] * 5 + [ctypes.c_uint32, ctypes.c_void_p]
+    lib.ttc_lqr_solve_lowrank_q.restype = ctypes.c_int
+    lib.ttc_lqr_solve_lowrank_q.argtypes = [ctypes.c_void_p, opp, opp, opp, opp, ctypes.c_int32, ctypes.c_float, opp, opp,
+                                            ctypes.c_int32] + [ctypes.c_void_p] * 5 + [ctypes.c_uint32, ctypes.c_void_p]
     lib.ttc_lqr_solve_tv.restype = ctypes.c_int
     lib.ttc_lqr_solve_tv.argtypes = [ctypes.c_void_p, opp, opp, opp, opp, P(ctypes.c_int64), opp, opp, ctypes.c_int32] + \
         [ctypes.c_void_p] * 5 + [ctypes.c_uint32, ctypes.c_void_p]
@@ -204,6 +208,19 @@ class LqrSolver:
         _check(load_library().ttc_lqr_solve(
             self._h, *refs, int(H), self._ptr(K), self._ptr(P), self._ptr(x), self._ptr(u), self._ptr(info),
             int(flags), ctypes.c_void_p(stream.cuda_stream)))
+
+    def solve_lowrank_q(self, A, B, U, d, scale, R, x0, H, K=None, P=None, x=None, u=None, info=None, flags=0, stream=None):
+        """Enqueue ``ttc_lqr_solve_lowrank_q``: as :meth:`solve` with ``Q = scale * U U' + diag(d)`` handed over as
+        ``U [..batch.., n, rank]`` and ``d [..batch.., n]``."""
+        ops = [_operand(A, 2, self.batch), _operand(B, 2, self.batch), _operand(U, 2, self.batch),
+               _operand(d, 1, self.batch), _operand(R, 2, self.batch), _operand(x0, 1, self.batch)]
+        ref = lambda o: ctypes.byref(o) if o is not None else None
+        if stream is None:
+            stream = torch.cuda.current_stream(self.device)
+        _check(load_library().ttc_lqr_solve_lowrank_q(
+            self._h, ref(ops[0]), ref(ops[1]), ref(ops[2]), ref(ops[3]), int(U.shape[-1]), ctypes.c_float(scale), ref(ops[4]),
+            ref(ops[5]), int(H), self._ptr(K), self._ptr(P), self._ptr(x), self._ptr(u), self._ptr(info), int(flags),
+            ctypes.c_void_p(stream.cuda_stream)))
 
     def solve_tv(self, A, B, Q, R, Qf, x0, H, tv=("A", "B", "Q", "R"), K=None, P=None, x=None, u=None, info=None,
                  flags=0, stream=None):
@@ -336,20 +353,22 @@ class LqrSolver:
             int(flags)))
 
 
-def alloc_outputs(n, m, H, N, device, first_only=False, want=("K", "P", "x", "u", "info"), pin=False):
-    """Allocate output tensors of the documented shapes (torch owns the memory)."""
+def alloc_outputs(n, m, H, N, device, first_only=False, want=("K", "P", "x", "u", "info"), pin=False,
+                  dtype=torch.float32):
+    """Allocate output tensors of the documented shapes (torch owns the memory); ``dtype=torch.bfloat16`` for calls
+    made with ``TTC_OUT_BF16``."""
     kw = dict(device=device)
     if pin and str(device) == "cpu":
         kw["pin_memory"] = True
     out = {}
     if "K" in want:
-        out["K"] = torch.empty((N, H, m, n), dtype=torch.float32, **kw)
+        out["K"] = torch.empty((N, H, m, n), dtype=dtype, **kw)
     if "P" in want:
-        out["P"] = torch.empty((N, n, n) if first_only else (N, H + 1, n, n), dtype=torch.float32, **kw)
+        out["P"] = torch.empty((N, n, n) if first_only else (N, H + 1, n, n), dtype=dtype, **kw)
     if "x" in want:
-        out["x"] = torch.empty((N, H + 1, n), dtype=torch.float32, **kw)
+        out["x"] = torch.empty((N, H + 1, n), dtype=dtype, **kw)
     if "u" in want:
-        out["u"] = torch.empty((N, m) if first_only else (N, H, m), dtype=torch.float32, **kw)
+        out["u"] = torch.empty((N, m) if first_only else (N, H, m), dtype=dtype, **kw)
     if "info" in want:
         out["info"] = torch.empty((N,), dtype=torch.int32, **kw)
     return out

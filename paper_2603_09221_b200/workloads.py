@@ -126,6 +126,9 @@ def make_workload(cfg_id, device="cpu", batch=None, seed=None, chunk=8192):
     N = S * Hd * T
     qdt = torch.bfloat16 if c["q_dtype"] == "bf16" else torch.float32
     Q = torch.empty((N, n, n), dtype=qdt, device=device)
+    low = c["q_kind"] != "full"
+    Uf = torch.empty((N, n, 8), dtype=qdt, device=device) if low else None       # the factors themselves, for callers that
+    df = torch.empty((N, n), dtype=qdt, device=device) if low else None          # hand Q over as U U'/8 + diag(d)
     eye = torch.eye(n, device=device)
     for s0 in range(0, N, chunk):
         cnt = min(chunk, N - s0)
@@ -136,11 +139,15 @@ def make_workload(cfg_id, device="cpu", batch=None, seed=None, chunk=8192):
             U = torch.randn((cnt, n, 8), generator=gen, device=device)
             d = 0.05 + 0.15 * torch.rand((cnt, n), generator=gen, device=device)
             q = U @ U.transpose(1, 2) / 8 + torch.diag_embed(d)
+            Uf[s0:s0 + cnt] = U.to(qdt)
+            df[s0:s0 + cnt] = d.to(qdt)
         q = 0.5 * (q + q.transpose(1, 2))
         Q[s0:s0 + cnt] = q.to(qdt)
     x0 = torch.randn((N, n), generator=gen, device=device).to(qdt)
     c.update(A=A, B=B, R=R, Q=Q.reshape(S, Hd, T, n, n), x0=x0.reshape(S, Hd, T, n),
              seed=seed, cfg_id=cfg_id)
+    if low:
+        c.update(U=Uf.reshape(S, Hd, T, n, 8), d=df.reshape(S, Hd, T, n), q_scale=1.0 / 8)
     return c
 
 
