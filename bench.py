@@ -414,8 +414,16 @@ def run_layer(args):
     info = torch.empty((N,), dtype=torch.int32, device=dev)
     ins = [w[k] for k in workloads.LAYER_KEYS]
 
+    baseline = args.method == "sigma"      # the row-normalised reverse symplectic product instead of the recursion
+    if baseline:
+        c["name"] += "_sigma_baseline"
+        args.no_e2e = True
+
     def step():
-        solver.solve_layer(*ins, T, u1=u1, P0=P0, info=info)
+        if baseline:
+            solver.solve_layer_sigma_baseline(*ins, T, u1=u1, P0=P0, info=info)
+        else:
+            solver.solve_layer(*ins, T, u1=u1, P0=P0, info=info)
 
     def barrier():
         if dist:
@@ -486,10 +494,18 @@ def run_layer(args):
         ref, dt = layer_oracle(w, idx, T)
         from tests import parity_util as pu
         sel = torch.as_tensor(idx)
-        errs = {"P0": pu.block_rel_err(P0.cpu()[sel].numpy(), ref["P0"], 2),
-                "u1": pu.block_rel_err(u1.cpu()[sel].numpy(), ref["u1"], 1)}
-        assert all(v <= c["tol"] for v in errs.values()), errs
-        assert int(info.abs().max()) == 0
+        if baseline:                       # a baseline whose float32 error grows with the horizon: reported, not gated
+            g_u, g_P = u1.cpu()[sel].double().numpy(), P0.cpu()[sel].double().numpy().reshape(len(idx), -1)
+            eu = np.abs(g_u - ref["u1"]).max(axis=1) / np.abs(ref["u1"]).max(axis=1)
+            eP = np.abs(g_P - ref["P0"].reshape(len(idx), -1)).max(axis=1) / np.abs(ref["P0"]).reshape(len(idx), -1).max(axis=1)
+            errs = {"u1_median": float(np.nanmedian(eu)), "u1_p90": float(np.nanpercentile(eu, 90)),
+                    "P0_median": float(np.nanmedian(eP)), "P0_p90": float(np.nanpercentile(eP, 90)),
+                    "singular_Y1": int((info.cpu()[sel] != 0).sum())}
+        else:
+            errs = {"P0": pu.block_rel_err(P0.cpu()[sel].numpy(), ref["P0"], 2),
+                    "u1": pu.block_rel_err(u1.cpu()[sel].numpy(), ref["u1"], 1)}
+            assert all(v <= c["tol"] for v in errs.values()), errs
+            assert int(info.abs().max()) == 0
         cpu = {"value": len(idx) / dt, "unit": "instances/s", "cores": int(ref["threads"]), "kind": "oracle",
                "sample": "%d instances spread over the workload (parameter synthesis in numpy + C recursion)" % len(idx),
                "seconds": dt, "parity_max_rel_err": errs, "speedup_gpu_over_cpu": value / (len(idx) / dt)}
@@ -497,7 +513,7 @@ def run_layer(args):
                       "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
                       "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
                       "config": {"workload": c["name"], "n": n, "r": r, "T": T, "instances": N, "batch": list(c["batch"]),
-                                 "outputs": ["u1", "P0", "info"], "kernel": "ttc_layer",
+                                 "outputs": ["u1", "P0", "info"], "kernel": "sigma_product (baseline)" if baseline else "ttc_layer",
                                  "l2": "working set fits L2: a 192 MB buffer is written between timed steps"},
                       "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches),
                       "launches_per_step": launches / args.steps, "clocks": clocks}))
@@ -771,7 +787,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="", help="one workload only (cfg0..cfg4, tv16, layer16, layer32, grad16); "
                     "default: cfg4 as the headline plus short side measurements of cfg0..cfg3")
-    ap.add_argument("--method", default="auto", choices=["auto", "riccati", "scan"])
+    ap.add_argument("--method", default="auto", choices=["auto", "riccati", "scan", "sigma"],
+                    help="sigma: layer workloads only, the row-normalised reverse symplectic product (baseline)")
     ap.add_argument("--math", default="auto", choices=["auto", "fp32", "tf32"])
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--cpu-sample", type=int, default=4096, help="instances the oracle is timed on and parity is checked on")

@@ -90,6 +90,7 @@ extern "C" {
 #define TTC_KERNEL_SCAN           4  /* symplectic-pair scan + gain/rollout kernel     */
 #define TTC_KERNEL_RICCATI_UMMA   5  /* tcgen05 contractions (tensor memory), n = m = 64 */
 #define TTC_KERNEL_LAYER          6  /* contextualised layer: parameters synthesised in-kernel */
+#define TTC_KERNEL_SIGMA_BASELINE 7 /* baseline: row-normalised reverse symplectic product   */
 
 typedef struct ttc_lqr_handle ttc_lqr_handle; /* opaque; owned by the library */
 
@@ -284,6 +285,21 @@ typedef struct ttc_layer_inputs {
 
 int ttc_lqr_solve_layer(ttc_lqr_handle* h, const ttc_layer_inputs* in, int32_t T,
                         float* u1, float* P0, int32_t* info, void* cuda_stream);
+
+/*
+ * BASELINE for comparison, not the recommended solver: the same layer evaluation by the reverse symplectic
+ * iteration of Thm 3.3 / Alg. 3 with the row normalisation of the paper's fused kernel (hardware co-design
+ * appendix): [Y1 Y2] = [I Q_T] Sigma_T ... Sigma_1 accumulated row by row in registers, each row divided by
+ * max(|y1|_1, |y2|_1) after every step, then P0 = Y1^{-1} Y2 by Gauss-Jordan elimination with partial pivoting,
+ * lambda_0 = P0 h0, u1 = -R_1^{-1} B_1' A_1^{-T} lambda_0.  Arguments, outputs and errors as ttc_lqr_solve_layer;
+ * info is 0 or 1 + the column at which Y1 had no non-zero pivot (outputs quiet NaN).  The product contains
+ * A_t^{-1} and propagates [state; co-state] like a shooting method: in float32 its error grows with the horizon
+ * (about 1e-5 at T = 2, percent level by T = 16 and no correct digit by T = 32 on the layer16 inputs) where the
+ * backward recursion of ttc_lqr_solve_layer stays near 1e-6.  It exists so that the efficiency sweep can time
+ * both formulations on the same inputs.
+ */
+int ttc_lqr_solve_layer_sigma_baseline(ttc_lqr_handle* h, const ttc_layer_inputs* in, int32_t T,
+                                       float* u1, float* P0, int32_t* info, void* cuda_stream);
 
 /*
  * ttc_lqr_solve_layer with HOST buffers: every pointer of `in` and u1 / P0 / info are host memory

@@ -13,6 +13,7 @@
 #include "riccati_umma64.cuh"
 #include "riccati_warp.cuh"
 #include "ttc_layer.cuh"
+#include "sigma_product.cuh"
 #include "lqr_grad.cuh"
 #include "scan_pair.cuh"
 #include "scan_warp.cuh"
@@ -830,6 +831,45 @@ int ttc_lqr_solve_layer(ttc_lqr_handle* h, const ttc_layer_inputs* in, int32_t T
     TTC_CUDA(cudaSetDevice(h->cfg.device));
     h->last_launches = 0;
     return launch_layer(h, in, T, u1, P0, info, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int ttc_lqr_solve_layer_sigma_baseline(ttc_lqr_handle* h, const ttc_layer_inputs* in, int32_t T, float* u1, float* P0,
+                                       int32_t* info, void* cuda_stream)
+{
+    int s = check_layer_call(h, in, T, true, u1, P0);
+    if (s)
+        return s;
+    TTC_CUDA(cudaSetDevice(h->cfg.device));
+    h->last_launches = 0;
+    const int n = h->cfg.n;
+    layer::LayerParams p;
+    p.N = h->N;
+    p.T = T;
+    p.r = in->r;
+    p.s_a = in->s_a; p.s_ga = in->s_gamma_a; p.s_gb = in->s_gamma_b; p.s_gq = in->s_gamma_q;
+    p.s_b = in->s_b; p.s_q = in->s_q; p.s_qf = in->s_qf;
+    p.r_inv = in->r_inv; p.h0 = in->h0;
+    p.B_basis = in->B_basis; p.Q_basis = in->Q_basis;
+    p.u1 = u1; p.P0 = P0; p.info = info;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const int slots = n == 32 ? rwarp::Shape<32>::SLOTS : rwarp::Shape<16>::SLOTS;
+    long long grid = (p.N + slots - 1) / slots;
+    const long long cap = (long long)h->sm_count * 8;
+    if (grid > cap) grid = cap;
+    if (n == 32) {
+        const size_t smem = sigma::smem_bytes<32>();
+        TTC_CUDA(cudaFuncSetAttribute(sigma::sigma_product_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        sigma::sigma_product_kernel<32><<<(unsigned)grid, rwarp::THREADS, smem, st>>>(p);
+    } else {
+        const size_t smem = sigma::smem_bytes<16>();
+        TTC_CUDA(cudaFuncSetAttribute(sigma::sigma_product_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        sigma::sigma_product_kernel<16><<<(unsigned)grid, rwarp::THREADS, smem, st>>>(p);
+    }
+    TTC_CUDA(cudaGetLastError());
+    h->last_launches += 1;
+    h->total_launches += 1;
+    h->last_kernel = TTC_KERNEL_SIGMA_BASELINE;
+    return TTC_OK;
 }
 
 int ttc_lqr_solve_layer_host(ttc_lqr_handle* h, const ttc_layer_inputs* in, int32_t T, float* u1, float* P0,

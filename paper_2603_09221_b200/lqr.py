@@ -22,13 +22,14 @@ TTC_OUT_FIRST_ONLY = 1
 TTC_OUT_BF16 = 2
 TTC_QUERY_LAST_LAUNCHES, TTC_QUERY_WORKSPACE_BYTES, TTC_QUERY_LAST_KERNEL, TTC_QUERY_TOTAL_LAUNCHES = 1, 2, 3, 4
 TTC_QUERY_DEVICE_ERROR = 5
-KERNEL_NAMES = {6: "ttc_layer", 0: "none", 1: "riccati_cta", 2: "riccati_warp", 4: "scan", 5: "riccati_umma"}
+KERNEL_NAMES = {7: "sigma_baseline", 6: "ttc_layer", 0: "none", 1: "riccati_cta", 2: "riccati_warp", 4: "scan", 5: "riccati_umma"}
 
 EXPORTS = (
     "ttc_lqr_create", "ttc_lqr_solve", "ttc_lqr_solve_host", "ttc_lqr_destroy", "ttc_lqr_query",
     "ttc_lqr_status_string", "ttc_lqr_last_error", "ttc_lqr_solve_first_noalloc", "ttc_lqr_solve_tv",
     "ttc_lqr_solve_layer", "ttc_lqr_solve_layer_host", "ttc_lqr_solve_affine", "ttc_lqr_grad",
     "ttc_lqr_selftest_bounded_wait", "ttc_lqr_measure_fp32_peak", "ttc_lqr_solve_lowrank_q",
+    "ttc_lqr_solve_layer_sigma_baseline",
 )
 TTC_NOALLOC_SCRATCH_BYTES = 4 << 20
 
@@ -91,6 +92,8 @@ def load_library():
     lib.ttc_lqr_solve_layer.restype = ctypes.c_int
     lib.ttc_lqr_solve_layer.argtypes = [ctypes.c_void_p, P(ttc_layer_inputs), ctypes.c_int32, ctypes.c_void_p,
                                         ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+    lib.ttc_lqr_solve_layer_sigma_baseline.restype = ctypes.c_int
+    lib.ttc_lqr_solve_layer_sigma_baseline.argtypes = lib.ttc_lqr_solve_layer.argtypes
     lib.ttc_lqr_solve_layer_host.restype = ctypes.c_int
     lib.ttc_lqr_solve_layer_host.argtypes = [ctypes.c_void_p, P(ttc_layer_inputs), ctypes.c_int32, ctypes.c_void_p,
                                              ctypes.c_void_p, ctypes.c_void_p]
@@ -335,6 +338,17 @@ class LqrSolver:
         if stream is None:
             stream = torch.cuda.current_stream(self.device)
         _check(load_library().ttc_lqr_solve_layer(
+            self._h, ctypes.byref(inp), int(T), self._ptr(u1), self._ptr(P0), self._ptr(info),
+            ctypes.c_void_p(stream.cuda_stream)))
+
+    def solve_layer_sigma_baseline(self, s_a, s_gamma_a, s_gamma_b, s_gamma_q, s_b, s_q, s_qf, r_inv, h0, B_basis, Q_basis, T,
+                                   u1=None, P0=None, info=None, stream=None):
+        """``ttc_lqr_solve_layer_sigma_baseline``: the same layer evaluation by the row-normalised reverse symplectic
+        product (a baseline whose float32 error grows with the horizon); arguments as :meth:`solve_layer`."""
+        inp = self._layer_inputs((s_a, s_gamma_a, s_gamma_b, s_gamma_q, s_b, s_q, s_qf, r_inv, h0, B_basis, Q_basis), False)
+        if stream is None:
+            stream = torch.cuda.current_stream(self.device)
+        _check(load_library().ttc_lqr_solve_layer_sigma_baseline(
             self._h, ctypes.byref(inp), int(T), self._ptr(u1), self._ptr(P0), self._ptr(info),
             ctypes.c_void_p(stream.cuda_stream)))
 
