@@ -779,6 +779,58 @@ def spawn_ranks(n):
     raise SystemExit(sharding.launch_ranks(n, __file__, sys.argv[1:]))
 
 
+def run_layer_sweep(args):
+    """--sweep with a layer workload: the horizon x batch grid of the paper's efficiency benchmark (d = 16,
+    T in 2^4..2^11, B in 2^4..2^13) for the layer solve and for the sigma-product baseline, forward pass only.
+    One JSON line with a row per grid point: median time of 5 solves, nominal B T d^3 throughput (the paper's
+    convention), and the error of u_1 against the float64 oracle on up to 64 instances."""
+    from paper_2603_09221_b200 import lqr
+    from oracle import ttc_layer as lay
+    key = args.workload
+    c = workloads.LAYER_CONFIGS[key]
+    n = c["n"]
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    grid_T = [16, 64, 256, 1024, 2048] if not args.horizon else [args.horizon]
+    grid_B = [16, 128, 1024, 8192]
+    flush = torch.empty(192 * 1024 * 1024, dtype=torch.uint8, device=dev)
+    rows = []
+    for B in grid_B:
+        batch = (1, 16, max(1, B // 16))
+        w = workloads.make_layer_workload(key, device=dev, batch=batch)
+        N = w["N"]
+        ins = [w[k] for k in workloads.LAYER_KEYS]
+        u1 = torch.empty((N, n), device=dev)
+        P0 = torch.empty((N, n, n), device=dev)
+        info = torch.empty((N,), dtype=torch.int32, device=dev)
+        idx = np.unique(np.linspace(0, N - 1, min(N, 64)).astype(np.int64))
+        f64 = lambda k, sel=None: (w[k] if sel is None else w[k][torch.as_tensor(sel, device=dev)]).to(torch.float64).cpu().numpy()
+        for T in grid_T:
+            solver = lqr.LqrSolver(n, n, T, batch, device=0)
+            ref = lay.solve_batch(*(f64(k, idx) for k in workloads.LAYER_KEYS[:9]), f64("B_basis"), f64("Q_basis"), T)
+            row = {"B": N, "T": T}
+            for name, fn in (("recursion", solver.solve_layer), ("sigma_baseline", solver.solve_layer_sigma_baseline)):
+                times = []
+                for it in range(8):
+                    flush.fill_(it)
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    fn(*ins, T, u1=u1, P0=P0, info=info)
+                    e1.record()
+                    torch.cuda.synchronize(dev)
+                    if it >= 3:
+                        times.append(e0.elapsed_time(e1))
+                ms = statistics.median(times)
+                err = np.abs(u1.cpu()[torch.as_tensor(idx)].double().numpy() - ref["u1"]).max(axis=1) / np.abs(ref["u1"]).max(axis=1)
+                row[name] = {"ms": ms, "nominal_BTd3_gflops": N * T * n ** 3 / (ms * 1e-3) / 1e9,
+                             "u1_rel_err_median": float(np.nanmedian(err)), "u1_rel_err_max": float(np.nanmax(err))}
+            rows.append(row)
+            solver.close()
+    print(json.dumps({"metric": "lqr_instances_per_sec", "sweep": key, "d": n, "data": "synthetic", "unit": "ms per solve",
+                      "note": "forward pass only; B x T grid of the paper's efficiency benchmark; a 192 MB buffer is written "
+                              "between timed solves", "rows": rows}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -799,6 +851,7 @@ def main():
     ap.add_argument("--per-token", action="store_true", help="grad16: A_t, B_t, R_t per token instead of per head")
     ap.add_argument("--out-dtype", default="f32", choices=["f32", "bf16"], help="bfloat16 K, P, x, u (TTC_OUT_BF16)")
     ap.add_argument("--lowrank-q", action="store_true", help="cfg4: hand Q over as its factors (ttc_lqr_solve_lowrank_q)")
+    ap.add_argument("--sweep", action="store_true", help="layer workloads: horizon x batch grid, recursion and sigma baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-sides", action="store_true", help="default run: skip the side measurements of cfg0..cfg3")
@@ -810,7 +863,10 @@ def main():
     if default_run:
         args.workload = "cfg4"
     if args.workload in workloads.LAYER_CONFIGS:
-        run_layer(args)
+        if args.sweep:
+            run_layer_sweep(args)
+        else:
+            run_layer(args)
         return
     if workloads.TV_CONFIGS.get(args.workload, {}).get("grad"):
         run_grad(args)

@@ -280,37 +280,65 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 2 : 3) scan_step_kernel(S
                 s[l] = (l == c) ? 1.f : 0.f;
         }
         __syncwarp();
-        float v[N], t[N];
+        // The dense loops run over k with four-fold unrolling and take their coefficients from the lane's own column
+        // of a shared-memory matrix (a fully unrolled body would be bound by instruction fetch).
+        float y[N];
+        f32x2 p2[N / 2];
         {
-            float bc[N], ac[N];
-            load_col<N>(bc, sl.B, c);
-            load_col<N>(ac, sl.A, c);
             f32x2 v2[N / 2], t2[N / 2];
             zero2<N>(v2);
             zero2<N>(t2);
-            mix<N>(v2, bc, sl.buf0);                           // V[:,c] = P B[:,c]
-            mix<N>(t2, ac, sl.buf0);                           // T[:,c] = P A[:,c]
+#pragma unroll 4
+            for (int i = 0; i < N; ++i) {                      // V[:,c] = P B[:,c], T[:,c] = P A[:,c]
+                const float bic = sl.B[i * LD + c], aic = sl.A[i * LD + c];
+                const f32x2 b2 = rwarp::pack2(bic, bic), a2 = rwarp::pack2(aic, aic);
+                const float* prow = sl.buf0 + i * LD;
+#pragma unroll
+                for (int q4 = 0; q4 < N / 4; ++q4) {
+                    const ulonglong2 t4 = *reinterpret_cast<const ulonglong2*>(prow + 4 * q4);
+                    rwarp::fma2(v2[2 * q4], t4.x, b2);
+                    rwarp::fma2(v2[2 * q4 + 1], t4.y, b2);
+                    rwarp::fma2(t2[2 * q4], t4.x, a2);
+                    rwarp::fma2(t2[2 * q4 + 1], t4.y, a2);
+                }
+            }
+            float v[N], t[N];
             unpack_row<N>(v, v2);
             unpack_row<N>(t, t2);
+            store_col<N>(sl.L, c, v);                          // own column only: no exchange
+            store_col<N>(sl.Lt, c, t);
         }
-        float y[N];
-        f32x2 p2[N / 2];
         {
             f32x2 s2[N / 2], y2[N / 2];
             pack_row<N>(s2, s);
             zero2<N>(y2);
-            mix<N>(s2, v, sl.B);                               // S[:,c] = R[:,c] + B'V[:,c]
-            mix<N>(y2, t, sl.B);                               // Y[:,c] = B'T[:,c]
-            unpack_row<N>(s, s2);
-            unpack_row<N>(y, y2);
             if (!GAIN) {
                 float jc[N];
 #pragma unroll
                 for (int l = 0; l < N; ++l)
                     jc[l] = __ldg(E + 3 * N * N + c * N + l);  // row c of J = column c
                 pack_row<N>(p2, jc);
-                mix<N>(p2, t, sl.A);                           // Pn[:,c] = J[:,c] + A'T[:,c]
             }
+#pragma unroll 4
+            for (int k = 0; k < N; ++k) {                      // S += B'V, Y = B'T, Pn = J + A'T: each row read once
+                const float vk = sl.L[k * LD + c], tk = sl.Lt[k * LD + c];
+                const f32x2 vv = rwarp::pack2(vk, vk), tt = rwarp::pack2(tk, tk);
+#pragma unroll
+                for (int q4 = 0; q4 < N / 4; ++q4) {
+                    const ulonglong2 b4 = *reinterpret_cast<const ulonglong2*>(sl.B + k * LD + 4 * q4);
+                    rwarp::fma2(s2[2 * q4], vv, b4.x);
+                    rwarp::fma2(s2[2 * q4 + 1], vv, b4.y);
+                    rwarp::fma2(y2[2 * q4], tt, b4.x);
+                    rwarp::fma2(y2[2 * q4 + 1], tt, b4.y);
+                    if (!GAIN) {
+                        const ulonglong2 a4 = *reinterpret_cast<const ulonglong2*>(sl.A + k * LD + 4 * q4);
+                        rwarp::fma2(p2[2 * q4], tt, a4.x);
+                        rwarp::fma2(p2[2 * q4 + 1], tt, a4.y);
+                    }
+                }
+            }
+            unpack_row<N>(s, s2);
+            unpack_row<N>(y, y2);
         }
         float rs_own;
         const int bad = rwarp::seg_chol<N>(s, rs_own, c);
@@ -338,11 +366,9 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 2 : 3) scan_step_kernel(S
         } else {
             store_col<N>(sl.buf0, c, y);                       // rows of Z
             __syncwarp();
-            float zn[N];
-#pragma unroll
-            for (int l = 0; l < N; ++l)
-                zn[l] = -y[l];
-            mix<N>(p2, zn, sl.buf0);                           // Pn[:,c] -= Z'Z[:,c]
+#pragma unroll 4
+            for (int k = 0; k < N; ++k)                        // Pn[:,c] -= Z'Z[:,c]
+                axpy_row<N>(p2, -sl.buf0[k * LD + c], sl.buf0 + k * LD);
             float pcol[N];
             unpack_row<N>(pcol, p2);
             __syncwarp();
