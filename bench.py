@@ -695,11 +695,15 @@ def run_solve(args, workload, method_name, ctx, light=False):
     fp32_peak = run_peaks["fp32_tflops"] if run_peaks else fp32_derived
     tf32_peak = run_peaks["tf32_tflops_sustained"] if run_peaks else tf32_derived
     extra = {}
-    if kname == "riccati_umma":
+    if kname == "riccati_umma" and alg_flops / (tf32_peak * 1e12) >= t_hbm:
         bound, peak, unit, ach = "tensor", tf32_peak, "TFLOP/s", alg_flops / (kernel_ms * 1e-3) / 1e12
         peak_note = ("tf32 matmul (cuBLAS via torch) measured in this run, sustained" if run_peaks else
                      "tf32 = measured sustained bf16 x 0.5 (nominal ratio), of %s" % peaks["source"])
         extra = {"frac_of_half_bf16_sustained": ach / tf32_derived, "half_bf16_sustained_tflops": tf32_derived}
+    elif kname == "riccati_umma":          # every K_t, P_t written: the bytes take longer than the flops at the tensor peak
+        bound, peak, unit, ach = "hbm", peaks["hbm_gbs"], "GB/s", alg_bytes / (kernel_ms * 1e-3) / 1e9
+        peak_note = "copy bandwidth, of %s (the tensor-core time at the measured tf32 peak is shorter)" % peaks["source"]
+        extra = {"tensor_frac": (alg_flops / (kernel_ms * 1e-3) / 1e12) / tf32_peak, "tf32_peak_tflops": tf32_peak}
     else:
         t_alu = alg_flops / (fp32_peak * 1e12)
         if t_hbm >= t_alu:
