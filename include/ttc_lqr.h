@@ -287,6 +287,38 @@ int ttc_lqr_solve_layer(ttc_lqr_handle* h, const ttc_layer_inputs* in, int32_t T
                         float* u1, float* P0, int32_t* info, void* cuda_stream);
 
 /*
+ * Gradients of a scalar loss l(u_1*) of the contextualised layer's output with respect to everything
+ * ttc_lqr_solve_layer is handed (Thm 3.2: primal and dual LQR; then the chain rule through the Contextualization /
+ * Parameterization paragraphs).  g [N][n] (device, float32) is dl/du_1*.  The per-step matrices dA_t, dB_t, dQ_t,
+ * dR_t of the theorem are never formed: their outer products are reduced as they appear onto
+ *     s_a, s_gamma_a, s_gamma_b, s_gamma_q, r_inv, h0   [N][n]         s_b, s_q, s_qf   [N][r]
+ * per instance, and onto B_basis, Q_basis [r][n][n], which are shared by all instances and therefore receive the SUM
+ * over the instances (accumulated with float atomics: the last bits depend on the order).  The Q_basis gradient is
+ * symmetric (derivative along symmetric perturbations, Q_basis[i] being symmetric).  Every member of `out` may be
+ * NULL (not computed); u1 (optional) receives the forward output, info as in ttc_lqr_solve_layer.  An instance whose
+ * backward pass failed (info != 0) gets quiet NaN in its per-instance gradients and adds nothing to the basis
+ * gradients.  All pointers device memory, float32, 16-byte aligned; asynchronous on cuda_stream.
+ * Workspace owned by the handle: N (T n^2 + (4 T + 5) n) floats, plus 3 N n^2 when a basis gradient is requested.
+ * Needs n == m in {16, 32}; 1 <= T <= max_horizon.
+ */
+typedef struct ttc_layer_grads {
+    float* s_a;
+    float* s_gamma_a;
+    float* s_gamma_b;
+    float* s_gamma_q;
+    float* s_b;
+    float* s_q;
+    float* s_qf;
+    float* r_inv;
+    float* h0;
+    float* B_basis;
+    float* Q_basis;
+} ttc_layer_grads;
+
+int ttc_lqr_layer_grad(ttc_lqr_handle* h, const ttc_layer_inputs* in, int32_t T, const float* g,
+                       const ttc_layer_grads* out, float* u1, int32_t* info, void* cuda_stream);
+
+/*
  * BASELINE for comparison, not the recommended solver: the same layer evaluation by the reverse symplectic
  * iteration of Thm 3.3 / Alg. 3 with the row normalisation of the paper's fused kernel (hardware co-design
  * appendix): [Y1 Y2] = [I Q_T] Sigma_T ... Sigma_1 accumulated row by row in registers, each row divided by

@@ -38,6 +38,10 @@ struct LayerParams {
     float* u1;                   // [N][n] or null
     float* P0;                   // [N][n][n] or null
     int* info;                   // [N] or null
+    // gradient path only (ttc_layer_kernel<N, true>): every gain and the dual problem's first control are kept
+    float* Kws;                  // [N][T][n][n]: K of step s = t - 1
+    const float* g;              // [N][n]: dl/du_1*
+    float* k0;                   // [N][n]: -S_0^{-1} g
 };
 
 using rwarp::Shape;
@@ -58,7 +62,9 @@ struct Smem {
     int chunk;
 };
 
-template <int N>
+// GRAD = the backward pass of the gradient entry point: the gain of EVERY step goes to p.Kws and, at the last step,
+// k_0 = -S_0^{-1} g (the first control of the dual problem of Thm 3.2) to p.k0.
+template <int N, bool GRAD = false>
 __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) ttc_layer_kernel(LayerParams p, int* chunk_counter)
 {
     using S = Shape<N>;
@@ -227,7 +233,7 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) ttc_layer_kernel(L
                     axpy_row<N>(p2, -sl.buf0[q * LD + c], sl.buf0 + q * LD);
                 unpack_row<N>(pcol, p2);
             }
-            if (s == 0 && p.u1) {                             // K[:,c] = -L^{-T} Z[:,c]; rows of K -> Lt
+            if (GRAD || (s == 0 && p.u1)) {                   // K[:,c] = -L^{-T} Z[:,c]; rows of K -> Lt
 #pragma unroll
                 for (int k = N - 1; k >= 0; --k) {
                     const float xk = y[k] * rinv[k];
@@ -242,9 +248,45 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) ttc_layer_kernel(L
                         if (i4 + 3 < k) y[i4 + 3] = fmaf(-l4.w, xk, y[i4 + 3]);
                     }
                 }
+                if (GRAD) {
+                    if (active) {
+                        float* kt = p.Kws + (inst * (long long)T + s) * N * N + c;
 #pragma unroll
-                for (int l = 0; l < N; ++l)
-                    sl.Lt[l * LD + c] = -y[l];
+                        for (int l = 0; l < N; ++l)
+                            kt[l * N] = -y[l];
+                    }
+                    if (s == 0) {
+                        // k_0 = -L^{-T} L^{-1} g with one component per lane: the pivot's value travels by shuffle,
+                        // lane i reads its own rows of L and L'
+                        float gz = __ldg(p.g + inst * N + c);
+                        const float rown = sl.rinv[c];
+#pragma unroll 4
+                        for (int k = 0; k < N; ++k) {
+                            const float zk = __shfl_sync(0xffffffffu, gz * rown, k, N);
+                            if (c > k)
+                                gz = fmaf(-sl.L[c * LD + k], zk, gz);
+                            else if (c == k)
+                                gz = zk;
+                        }
+#pragma unroll 4
+                        for (int k = N - 1; k >= 0; --k) {
+                            const float xk = __shfl_sync(0xffffffffu, gz * rown, k, N);
+                            if (c < k)
+                                gz = fmaf(-sl.Lt[c * LD + k], xk, gz);
+                            else if (c == k)
+                                gz = xk;
+                        }
+                        if (active)
+                            p.k0[inst * N + c] = -gz;
+                    }
+                }
+                if (s == 0) {
+                    if (GRAD)
+                        __syncwarp();                         // every lane is done with L' (the substitution of g)
+#pragma unroll
+                    for (int l = 0; l < N; ++l)
+                        sl.Lt[l * LD + c] = -y[l];
+                }
             }
             __syncwarp();                                     // rows of Z consumed
             store_row<N>(sl.buf0 + c * LD, pcol);             // rows of P_s (row c = column c)

@@ -14,6 +14,7 @@
 #include "riccati_warp.cuh"
 #include "ttc_layer.cuh"
 #include "sigma_product.cuh"
+#include "layer_grad.cuh"
 #include "lqr_grad.cuh"
 #include "scan_pair.cuh"
 #include "scan_warp.cuh"
@@ -56,6 +57,8 @@ struct ttc_lqr_handle {
     int sm_count;
     size_t max_pitch;              // largest pitch a 2D copy accepts on this device
     DevBuf ws_K, ws_P, ws_E;       // scratch used by kernels
+    DevBuf ws_info;                // status words of the layer-gradient backward pass when the caller takes none
+    DevBuf ws_G;                   // per-instance gradients of Bbar, Qbar, Q_T before the reduction onto the bases
     DevBuf ws_Q;                   // dense Q expanded from a low-rank-plus-diagonal operand
     DevBuf ws_elem;                // scan elements (A_e, C_e, G_e, J_e per instance)
     DevBuf ws_k;                   // feed-forward terms k_t when the caller does not take them
@@ -102,7 +105,7 @@ void release(DevBuf& b)
 
 size_t workspace_bytes(const ttc_lqr_handle* h)
 {
-    size_t s = h->ws_K.bytes + h->ws_P.bytes + h->ws_E.bytes + h->ws_elem.bytes + h->ws_Q.bytes + h->ws_k.bytes + h->ws_vec.bytes + h->st_layer.bytes;
+    size_t s = h->ws_K.bytes + h->ws_P.bytes + h->ws_E.bytes + h->ws_elem.bytes + h->ws_Q.bytes + h->ws_info.bytes + h->ws_G.bytes + h->ws_k.bytes + h->ws_vec.bytes + h->st_layer.bytes;
     for (int i = 0; i < 5; ++i)
         s += h->st_in[i].bytes + h->st_out[i].bytes;
     return s;
@@ -284,6 +287,8 @@ int ttc_lqr_destroy(ttc_lqr_handle* h)
     release(h->ws_E);
     release(h->ws_elem);
     release(h->ws_Q);
+    release(h->ws_info);
+    release(h->ws_G);
     release(h->ws_k);
     release(h->ws_vec);
     for (int i = 0; i < 5; ++i) {
@@ -792,6 +797,7 @@ static int launch_layer(ttc_lqr_handle* h, const ttc_layer_inputs* in, int32_t T
     p.r_inv = in->r_inv; p.h0 = in->h0;
     p.B_basis = in->B_basis; p.Q_basis = in->Q_basis;
     p.u1 = u1; p.P0 = P0; p.info = info;
+    p.Kws = nullptr; p.g = nullptr; p.k0 = nullptr;
     void (*kern)(layer::LayerParams, int*);
     size_t smem;
     long long chunks, grid;
@@ -851,6 +857,7 @@ int ttc_lqr_solve_layer_sigma_baseline(ttc_lqr_handle* h, const ttc_layer_inputs
     p.r_inv = in->r_inv; p.h0 = in->h0;
     p.B_basis = in->B_basis; p.Q_basis = in->Q_basis;
     p.u1 = u1; p.P0 = P0; p.info = info;
+    p.Kws = nullptr; p.g = nullptr; p.k0 = nullptr;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     const int slots = n == 32 ? rwarp::Shape<32>::SLOTS : rwarp::Shape<16>::SLOTS;
     long long grid = (p.N + slots - 1) / slots;
@@ -869,6 +876,106 @@ int ttc_lqr_solve_layer_sigma_baseline(ttc_lqr_handle* h, const ttc_layer_inputs
     h->last_launches += 1;
     h->total_launches += 1;
     h->last_kernel = TTC_KERNEL_SIGMA_BASELINE;
+    return TTC_OK;
+}
+
+int ttc_lqr_layer_grad(ttc_lqr_handle* h, const ttc_layer_inputs* in, int32_t T, const float* g,
+                       const ttc_layer_grads* out, float* u1, int32_t* info, void* cuda_stream)
+{
+    int s = check_layer_call(h, in, T, true, u1, nullptr);
+    if (s)
+        return s;
+    if (!g || !out)
+        return fail(TTC_STATUS_INVALID_ARGUMENT, "null output gradient g or null result struct");
+    const void* ptrs[13] = {g, out->s_a, out->s_gamma_a, out->s_gamma_b, out->s_gamma_q, out->s_b, out->s_q, out->s_qf,
+                            out->r_inv, out->h0, out->B_basis, out->Q_basis, info};
+    for (int i = 0; i < 13; ++i)
+        if (reinterpret_cast<uintptr_t>(ptrs[i]) & 15u)
+            return fail(TTC_STATUS_INVALID_ARGUMENT, "g and the gradient outputs must be 16-byte aligned");
+    TTC_CUDA(cudaSetDevice(h->cfg.device));
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const int n = h->cfg.n, r = in->r;
+    const size_t N = (size_t)h->N, nn = (size_t)n * n;
+    if ((s = ensure(h->ws_K, sizeof(float) * N * T * nn))) return s;
+    if ((s = ensure(h->ws_k, sizeof(float) * N * n))) return s;
+    if ((s = ensure(h->ws_vec, sizeof(float) * N * 4 * (T + 1) * n))) return s;
+    if ((s = ensure(h->ws_E, sizeof(int) * 4))) return s;
+    int* info_dev = info;
+    if (!info_dev) {
+        if ((s = ensure(h->ws_info, sizeof(int) * N))) return s;
+        info_dev = static_cast<int*>(h->ws_info.ptr);
+    }
+    const bool bases = out->B_basis || out->Q_basis;
+    if (bases && (s = ensure(h->ws_G, sizeof(float) * 3 * N * nn))) return s;
+    h->last_launches = 0;
+
+    // (1) backward Riccati pass on the synthesised parameters; every gain and k_0 = -S_0^{-1} g are kept
+    layer::LayerParams p;
+    p.N = h->N; p.T = T; p.r = r;
+    p.s_a = in->s_a; p.s_ga = in->s_gamma_a; p.s_gb = in->s_gamma_b; p.s_gq = in->s_gamma_q;
+    p.s_b = in->s_b; p.s_q = in->s_q; p.s_qf = in->s_qf;
+    p.r_inv = in->r_inv; p.h0 = in->h0;
+    p.B_basis = in->B_basis; p.Q_basis = in->Q_basis;
+    p.u1 = u1; p.P0 = nullptr; p.info = info_dev;
+    p.Kws = static_cast<float*>(h->ws_K.ptr); p.g = g; p.k0 = static_cast<float*>(h->ws_k.ptr);
+    int* counter = static_cast<int*>(h->ws_E.ptr);
+    TTC_CUDA(cudaMemsetAsync(counter, 0, sizeof(int), st));
+    {
+        void (*kern)(layer::LayerParams, int*) = n == 32 ? layer::ttc_layer_kernel<32, true> : layer::ttc_layer_kernel<16, true>;
+        const size_t smem = n == 32 ? layer::smem_bytes<32>() : layer::smem_bytes<16>();
+        const int slots = n == 32 ? rwarp::Shape<32>::SLOTS : rwarp::Shape<16>::SLOTS;
+        long long chunks = (p.N + slots - 1) / slots, grid = (long long)h->sm_count * (n == 32 ? 3 : 4);
+        if (grid > chunks) grid = chunks;
+        TTC_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        kern<<<(unsigned)grid, rwarp::THREADS, smem, st>>>(p, counter);
+        TTC_CUDA(cudaGetLastError());
+    }
+    // (2) rollouts, co-states and the reductions of Thm 3.2's outer products onto the coefficients
+    lgrad::LayerGradParams q;
+    q.lp = p;
+    q.vec = static_cast<float*>(h->ws_vec.ptr);
+    q.info = info_dev;
+    q.d_sa = out->s_a; q.d_ga = out->s_gamma_a; q.d_gb = out->s_gamma_b; q.d_gq = out->s_gamma_q;
+    q.d_ri = out->r_inv; q.d_h0 = out->h0;
+    q.d_sb = out->s_b; q.d_sq = out->s_q; q.d_sqf = out->s_qf;
+    float* G = bases ? static_cast<float*>(h->ws_G.ptr) : nullptr;
+    q.GB = G; q.GQ = G ? G + N * nn : nullptr; q.GF = G ? G + 2 * N * nn : nullptr;
+    {
+        const int slots = n == 32 ? rwarp::Shape<32>::SLOTS : rwarp::Shape<16>::SLOTS;
+        long long grid = (p.N + slots - 1) / slots;
+        const long long cap = (long long)h->sm_count * 8;
+        if (grid > cap) grid = cap;
+        if (n == 32) {
+            const size_t smem = sizeof(lgrad::Slot<32>) * slots;
+            TTC_CUDA(cudaFuncSetAttribute(lgrad::layer_grad_vectors_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            lgrad::layer_grad_vectors_kernel<32><<<(unsigned)grid, rwarp::THREADS, smem, st>>>(q);
+        } else {
+            const size_t smem = sizeof(lgrad::Slot<16>) * slots;
+            TTC_CUDA(cudaFuncSetAttribute(lgrad::layer_grad_vectors_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            lgrad::layer_grad_vectors_kernel<16><<<(unsigned)grid, rwarp::THREADS, smem, st>>>(q);
+        }
+        TTC_CUDA(cudaGetLastError());
+    }
+    h->last_launches += 2;
+    h->total_launches += 2;
+    // (3) the bases are shared by every instance: their gradients are sums over the instances
+    if (bases) {
+        long long grid = (long long)h->sm_count * 4;
+        if (grid > (long long)N) grid = (long long)N;
+        if (out->B_basis) {
+            TTC_CUDA(cudaMemsetAsync(out->B_basis, 0, sizeof(float) * (size_t)r * nn, st));
+            lgrad::basis_reduce_kernel<<<(unsigned)grid, 256, 0, st>>>(h->N, r, (int)nn, info_dev, in->s_b, q.GB, nullptr, nullptr, out->B_basis);
+            TTC_CUDA(cudaGetLastError());
+            h->last_launches += 1; h->total_launches += 1;
+        }
+        if (out->Q_basis) {
+            TTC_CUDA(cudaMemsetAsync(out->Q_basis, 0, sizeof(float) * (size_t)r * nn, st));
+            lgrad::basis_reduce_kernel<<<(unsigned)grid, 256, 0, st>>>(h->N, r, (int)nn, info_dev, in->s_q, q.GQ, in->s_qf, q.GF, out->Q_basis);
+            TTC_CUDA(cudaGetLastError());
+            h->last_launches += 1; h->total_launches += 1;
+        }
+    }
+    h->last_kernel = TTC_KERNEL_LAYER;
     return TTC_OK;
 }
 

@@ -29,7 +29,7 @@ EXPORTS = (
     "ttc_lqr_status_string", "ttc_lqr_last_error", "ttc_lqr_solve_first_noalloc", "ttc_lqr_solve_tv",
     "ttc_lqr_solve_layer", "ttc_lqr_solve_layer_host", "ttc_lqr_solve_affine", "ttc_lqr_grad",
     "ttc_lqr_selftest_bounded_wait", "ttc_lqr_measure_fp32_peak", "ttc_lqr_solve_lowrank_q",
-    "ttc_lqr_solve_layer_sigma_baseline",
+    "ttc_lqr_solve_layer_sigma_baseline", "ttc_lqr_layer_grad",
 )
 TTC_NOALLOC_SCRATCH_BYTES = 4 << 20
 
@@ -42,6 +42,13 @@ class ttc_operand(ctypes.Structure):
 class ttc_layer_inputs(ctypes.Structure):
     _fields_ = [(k, ctypes.c_void_p) for k in ("s_a", "s_gamma_a", "s_gamma_b", "s_gamma_q", "s_b", "s_q", "s_qf",
                                                "r_inv", "h0", "B_basis", "Q_basis")] + [("r", ctypes.c_int32)]
+
+
+LAYER_GRAD_KEYS = ("s_a", "s_gamma_a", "s_gamma_b", "s_gamma_q", "s_b", "s_q", "s_qf", "r_inv", "h0", "B_basis", "Q_basis")
+
+
+class ttc_layer_grads(ctypes.Structure):
+    _fields_ = [(k, ctypes.c_void_p) for k in LAYER_GRAD_KEYS]
 
 
 class ttc_lqr_config(ctypes.Structure):
@@ -94,6 +101,9 @@ def load_library():
                                         ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
     lib.ttc_lqr_solve_layer_sigma_baseline.restype = ctypes.c_int
     lib.ttc_lqr_solve_layer_sigma_baseline.argtypes = lib.ttc_lqr_solve_layer.argtypes
+    lib.ttc_lqr_layer_grad.restype = ctypes.c_int
+    lib.ttc_lqr_layer_grad.argtypes = [ctypes.c_void_p, P(ttc_layer_inputs), ctypes.c_int32, ctypes.c_void_p,
+                                       P(ttc_layer_grads), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
     lib.ttc_lqr_solve_layer_host.restype = ctypes.c_int
     lib.ttc_lqr_solve_layer_host.argtypes = [ctypes.c_void_p, P(ttc_layer_inputs), ctypes.c_int32, ctypes.c_void_p,
                                              ctypes.c_void_p, ctypes.c_void_p]
@@ -350,6 +360,26 @@ class LqrSolver:
             stream = torch.cuda.current_stream(self.device)
         _check(load_library().ttc_lqr_solve_layer_sigma_baseline(
             self._h, ctypes.byref(inp), int(T), self._ptr(u1), self._ptr(P0), self._ptr(info),
+            ctypes.c_void_p(stream.cuda_stream)))
+
+    def layer_grad(self, s_a, s_gamma_a, s_gamma_b, s_gamma_q, s_b, s_q, s_qf, r_inv, h0, B_basis, Q_basis, T, g,
+                   grads, u1=None, info=None, stream=None):
+        """Enqueue ``ttc_lqr_layer_grad``: gradients of a loss of the layer output ``u_1*`` given ``g = dl/du_1*``
+        (``[N, n]`` float32).  ``grads`` maps any of ``LAYER_GRAD_KEYS`` to an output tensor shaped like the input of
+        that name (the basis gradients are summed over the instances)."""
+        inp = self._layer_inputs((s_a, s_gamma_a, s_gamma_b, s_gamma_q, s_b, s_q, s_qf, r_inv, h0, B_basis, Q_basis), False)
+        out = ttc_layer_grads()
+        for k in LAYER_GRAD_KEYS:
+            t = grads.get(k)
+            if t is not None and (t.dtype != torch.float32 or not t.is_contiguous()):
+                raise ValueError("gradient output %s must be a contiguous float32 tensor" % k)
+            setattr(out, k, None if t is None else t.data_ptr())
+        if tuple(g.shape) != (self.N, self.n) or g.dtype != torch.float32 or not g.is_contiguous():
+            raise ValueError("g must be a contiguous float32 tensor of shape (%d, %d)" % (self.N, self.n))
+        if stream is None:
+            stream = torch.cuda.current_stream(self.device)
+        _check(load_library().ttc_lqr_layer_grad(
+            self._h, ctypes.byref(inp), int(T), self._ptr(g), ctypes.byref(out), self._ptr(u1), self._ptr(info),
             ctypes.c_void_p(stream.cuda_stream)))
 
     def solve_layer_host(self, s_a, s_gamma_a, s_gamma_b, s_gamma_q, s_b, s_q, s_qf, r_inv, h0, B_basis, Q_basis, T,
