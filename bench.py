@@ -419,8 +419,19 @@ def run_layer(args):
         c["name"] += "_sigma_baseline"
         args.no_e2e = True
 
+    gradient = args.grad                   # ttc_lqr_layer_grad: backward of the layer output w.r.t. every coefficient
+    if gradient:
+        c["name"] += "_grad"
+        args.no_e2e = True
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(sharding.rank_seed(400, rank))
+        gout = torch.randn((N, n), generator=gen, device=dev)
+        grads = {k: torch.empty_like(w[k]) for k in lqr.LAYER_GRAD_KEYS}
+
     def step():
-        if baseline:
+        if gradient:
+            solver.layer_grad(*ins, T, gout, grads, u1=u1, info=info)
+        elif baseline:
             solver.solve_layer_sigma_baseline(*ins, T, u1=u1, P0=P0, info=info)
         else:
             solver.solve_layer(*ins, T, u1=u1, P0=P0, info=info)
@@ -490,11 +501,26 @@ def run_layer(args):
                 "hbm_frac": (N * (bin_i + bout_i) / (kernel_ms * 1e-3) / 1e9) / peaks["hbm_gbs"]}
     cpu = None
     if not args.no_cpu_baseline and world == 1:
-        idx = np.unique(np.linspace(0, N - 1, args.cpu_sample).astype(np.int64))
-        ref, dt = layer_oracle(w, idx, T)
+        idx = np.unique(np.linspace(0, N - 1, args.cpu_sample if not gradient else max(8, args.cpu_sample // 64)).astype(np.int64))
         from tests import parity_util as pu
         sel = torch.as_tensor(idx)
-        if baseline:                       # a baseline whose float32 error grows with the horizon: reported, not gated
+        if gradient:                       # per-instance gradients against the float64 gradient oracle, one instance at a time
+            from oracle import ttc_layer_grad as og
+            f64 = lambda t: t.to(torch.float64).cpu().numpy()
+            t0 = time.perf_counter()
+            refs = [og.grad(*(f64(w[k][i]) for k in workloads.LAYER_KEYS[:9]), f64(w["B_basis"]), f64(w["Q_basis"]), T, f64(gout[i]))
+                    for i in idx]
+            dt = time.perf_counter() - t0
+            ref = {"threads": 1}
+            errs = {}
+            for k in lqr.LAYER_GRAD_KEYS[:9]:
+                got = grads[k].cpu()[sel].double().numpy()
+                exp = np.stack([r_[k] for r_ in refs])
+                errs[k] = float((np.abs(got - exp).max(axis=1) / np.maximum(np.abs(exp).max(axis=1), 1e-30)).max())
+            assert all(v <= c["tol"] for v in errs.values()), errs
+            assert int(info.abs().max()) == 0
+        elif baseline:
+            ref, dt = layer_oracle(w, idx, T)                       # a baseline whose float32 error grows with the horizon: reported, not gated
             g_u, g_P = u1.cpu()[sel].double().numpy(), P0.cpu()[sel].double().numpy().reshape(len(idx), -1)
             eu = np.abs(g_u - ref["u1"]).max(axis=1) / np.abs(ref["u1"]).max(axis=1)
             eP = np.abs(g_P - ref["P0"].reshape(len(idx), -1)).max(axis=1) / np.abs(ref["P0"]).reshape(len(idx), -1).max(axis=1)
@@ -502,6 +528,7 @@ def run_layer(args):
                     "P0_median": float(np.nanmedian(eP)), "P0_p90": float(np.nanpercentile(eP, 90)),
                     "singular_Y1": int((info.cpu()[sel] != 0).sum())}
         else:
+            ref, dt = layer_oracle(w, idx, T)
             errs = {"P0": pu.block_rel_err(P0.cpu()[sel].numpy(), ref["P0"], 2),
                     "u1": pu.block_rel_err(u1.cpu()[sel].numpy(), ref["u1"], 1)}
             assert all(v <= c["tol"] for v in errs.values()), errs
@@ -855,6 +882,7 @@ def main():
     ap.add_argument("--per-token", action="store_true", help="grad16: A_t, B_t, R_t per token instead of per head")
     ap.add_argument("--out-dtype", default="f32", choices=["f32", "bf16"], help="bfloat16 K, P, x, u (TTC_OUT_BF16)")
     ap.add_argument("--lowrank-q", action="store_true", help="cfg4: hand Q over as its factors (ttc_lqr_solve_lowrank_q)")
+    ap.add_argument("--grad", action="store_true", help="layer workloads: time ttc_lqr_layer_grad (every gradient requested)")
     ap.add_argument("--sweep", action="store_true", help="layer workloads: horizon x batch grid, recursion and sigma baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")

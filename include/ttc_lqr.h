@@ -298,7 +298,7 @@ int ttc_lqr_solve_layer(ttc_lqr_handle* h, const ttc_layer_inputs* in, int32_t T
  * NULL (not computed); u1 (optional) receives the forward output, info as in ttc_lqr_solve_layer.  An instance whose
  * backward pass failed (info != 0) gets quiet NaN in its per-instance gradients and adds nothing to the basis
  * gradients.  All pointers device memory, float32, 16-byte aligned; asynchronous on cuda_stream.
- * Workspace owned by the handle: N (T n^2 + (4 T + 5) n) floats, plus 3 N n^2 when a basis gradient is requested.
+ * Workspace owned by the handle: N (2 T n^2 + (4 T + 5) n) floats, plus 3 N n^2 when a basis gradient is requested.
  * Needs n == m in {16, 32}; 1 <= T <= max_horizon.
  */
 typedef struct ttc_layer_grads {

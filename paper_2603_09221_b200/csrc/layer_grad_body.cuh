@@ -131,6 +131,25 @@ __global__ void __launch_bounds__(THREADS, 2) layer_grad_vectors_kernel(LayerGra
             const float tt = (float)(s + 1), ts = (float)s;
             const float ea = __expf(-tt * ga_c), g_c = __expf(-tt * gb_c);
             const float a_c = fmaf(ea, sa_c, 1.f);
+            if (s + 1 < T) {
+                // co-states as lam_{s+1} = P_{s+1} x_{s+1} (and the same for the dual, whose linear term vanishes from
+                // s = 1 on): the recursion lam_s = a_s lam_{s+1} + Q_s x_s would amplify rounding by the open-loop a_s
+                float pr[N], xn[N], xdn[N];
+                load_vec_global<N>(pr, p.Pws + (inst * (long long)T + s + 1) * N * N + c * N);
+                load_vec_plain<N>(xn, X + (long long)(s + 1) * N);
+                load_vec_plain<N>(xdn, Xd + (long long)(s + 1) * N);
+                lam_c = 0.f;
+                lamd_c = 0.f;
+#pragma unroll
+                for (int j = 0; j < N; ++j) {
+                    lam_c = fmaf(pr[j], xn[j], lam_c);
+                    lamd_c = fmaf(pr[j], xdn[j], lamd_c);
+                }
+                __syncwarp();                                 // the previous step's reads of the co-state vectors are done
+                sl.lam[c] = lam_c;
+                sl.lamd[c] = lamd_c;
+                __syncwarp();
+            }
             float xv[N], xdv[N];
             load_vec_plain<N>(xv, X + (long long)s * N);       // written by this kernel: ordinary loads
             load_vec_plain<N>(xdv, Xd + (long long)s * N);
@@ -176,12 +195,8 @@ __global__ void __launch_bounds__(THREADS, 2) layer_grad_vectors_kernel(LayerGra
                 qxd = e_c * dot_row<N>(sl.Qb + c * LD, xdv);
                 d_gq = fmaf(-ts, fmaf(xc, qxd, xdc * qx), d_gq);
             }
-            lam_c = fmaf(a_c, lam_c, qx);
-            lamd_c = fmaf(a_c, lamd_c, qxd);
-            __syncwarp();                                     // lam_{s+1}, lamd_{s+1} (and the gq vector) consumed
-            sl.lam[c] = lam_c;
-            sl.lamd[c] = lamd_c;
-            __syncwarp();
+            if (s == 0)
+                lamd_c = a_c * lamd_c;                        // lamd_0 = A_1' lamd_1 (Q_0 = 0, xd_0 = 0): the gradient of h_0
         }
         d_ri /= ri_c * ri_c;
         // ---- outputs; contraction of the three matrices with the bases

@@ -40,6 +40,7 @@ struct LayerParams {
     int* info;                   // [N] or null
     // gradient path only (ttc_layer_kernel<N, true>): every gain and the dual problem's first control are kept
     float* Kws;                  // [N][T][n][n]: K of step s = t - 1
+    float* Pws;                  // [N][T][n][n]: P_s for 1 <= s <= T - 1 (slot 0 unused): the co-states are P_s x_s
     const float* g;              // [N][n]: dl/du_1*
     float* k0;                   // [N][n]: -S_0^{-1} g
 };
@@ -290,6 +291,12 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) ttc_layer_kernel(L
             }
             __syncwarp();                                     // rows of Z consumed
             store_row<N>(sl.buf0 + c * LD, pcol);             // rows of P_s (row c = column c)
+            if (GRAD && s >= 1 && active) {
+                float* pt = p.Pws + (inst * (long long)T + s) * N * N + c;
+#pragma unroll
+                for (int l = 0; l < N; ++l)
+                    pt[l * N] = pcol[l];
+            }
         }
         __syncwarp();
 

@@ -797,7 +797,7 @@ static int launch_layer(ttc_lqr_handle* h, const ttc_layer_inputs* in, int32_t T
     p.r_inv = in->r_inv; p.h0 = in->h0;
     p.B_basis = in->B_basis; p.Q_basis = in->Q_basis;
     p.u1 = u1; p.P0 = P0; p.info = info;
-    p.Kws = nullptr; p.g = nullptr; p.k0 = nullptr;
+    p.Kws = nullptr; p.Pws = nullptr; p.g = nullptr; p.k0 = nullptr;
     void (*kern)(layer::LayerParams, int*);
     size_t smem;
     long long chunks, grid;
@@ -857,7 +857,7 @@ int ttc_lqr_solve_layer_sigma_baseline(ttc_lqr_handle* h, const ttc_layer_inputs
     p.r_inv = in->r_inv; p.h0 = in->h0;
     p.B_basis = in->B_basis; p.Q_basis = in->Q_basis;
     p.u1 = u1; p.P0 = P0; p.info = info;
-    p.Kws = nullptr; p.g = nullptr; p.k0 = nullptr;
+    p.Kws = nullptr; p.Pws = nullptr; p.g = nullptr; p.k0 = nullptr;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     const int slots = n == 32 ? rwarp::Shape<32>::SLOTS : rwarp::Shape<16>::SLOTS;
     long long grid = (p.N + slots - 1) / slots;
@@ -896,7 +896,7 @@ int ttc_lqr_layer_grad(ttc_lqr_handle* h, const ttc_layer_inputs* in, int32_t T,
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     const int n = h->cfg.n, r = in->r;
     const size_t N = (size_t)h->N, nn = (size_t)n * n;
-    if ((s = ensure(h->ws_K, sizeof(float) * N * T * nn))) return s;
+    if ((s = ensure(h->ws_K, sizeof(float) * 2 * N * T * nn))) return s;           // every K_s, then every P_s
     if ((s = ensure(h->ws_k, sizeof(float) * N * n))) return s;
     if ((s = ensure(h->ws_vec, sizeof(float) * N * 4 * (T + 1) * n))) return s;
     if ((s = ensure(h->ws_E, sizeof(int) * 4))) return s;
@@ -918,6 +918,7 @@ int ttc_lqr_layer_grad(ttc_lqr_handle* h, const ttc_layer_inputs* in, int32_t T,
     p.B_basis = in->B_basis; p.Q_basis = in->Q_basis;
     p.u1 = u1; p.P0 = nullptr; p.info = info_dev;
     p.Kws = static_cast<float*>(h->ws_K.ptr); p.g = g; p.k0 = static_cast<float*>(h->ws_k.ptr);
+    p.Pws = p.Kws + N * T * nn;
     int* counter = static_cast<int*>(h->ws_E.ptr);
     TTC_CUDA(cudaMemsetAsync(counter, 0, sizeof(int), st));
     {
