@@ -165,6 +165,89 @@ __device__ __forceinline__ void axpy_row(f32x2 (&acc)[N / 2], float w, const flo
     }
 }
 
+// ---- 32 x 32 x 32 contractions on the tensor cores (n = 32): mma.sync m16n8k8, tf32 operands, fp32 accumulate, with the
+// operands split into tf32 high and low parts and three passes (lo*hi + hi*lo + hi*hi), which keeps float32-grade
+// accuracy (the 1e-4 tolerance of the float32 configurations rules out single-pass tf32).  One warp computes one
+// product; operands are float32 matrices in shared memory with row stride LD32 = 36 floats.
+//   acc[mt][nt][..] is the 16 x 8 tile (rows 16 mt.., columns 8 nt..) in the accumulator layout of the instruction:
+//   lane = 4 g + t holds (g, 2t), (g, 2t + 1), (g + 8, 2t), (g + 8, 2t + 1).
+__device__ __forceinline__ void mma_tf32(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1)
+{
+    asm("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void split_hi_lo(float x, uint32_t& hi, uint32_t& lo)
+{
+    hi = __float_as_uint(x) & 0xffffe000u;
+    lo = __float_as_uint(x - __uint_as_float(hi));
+}
+constexpr int LD32 = 36;
+// acc += A' * B with both operands stored k-major: A'[i][k] = Am[k * LD32 + i], B[k][j] = Bm[k * LD32 + j].
+// The instruction leaves the assignment of contraction indices to its k slots free as long as A and B agree, so
+// slot (t, half) of k-step ks takes k = 16 (ks / 2) + 8 half + 2 t + (ks % 2): with the row stride of 36 floats the
+// 32 lanes of a fragment load then fall into 32 different banks (bank = 8 t + g + 4 (ks % 2)).
+__device__ __forceinline__ void mma32_product(float (&acc)[2][4][4], const float* Am, const float* Bm, int lane)
+{
+    const int g = lane >> 2, t = lane & 3;
+#pragma unroll
+    for (int ks = 0; ks < 4; ++ks) {
+        const int k0 = 16 * (ks >> 1) + 2 * t + (ks & 1);
+        uint32_t ah[2][4], al[2][4], bh[4][2], bl[4][2];
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt) {
+            const int i0 = 16 * mt + g;
+            split_hi_lo(Am[k0 * LD32 + i0], ah[mt][0], al[mt][0]);
+            split_hi_lo(Am[k0 * LD32 + i0 + 8], ah[mt][1], al[mt][1]);
+            split_hi_lo(Am[(k0 + 8) * LD32 + i0], ah[mt][2], al[mt][2]);
+            split_hi_lo(Am[(k0 + 8) * LD32 + i0 + 8], ah[mt][3], al[mt][3]);
+        }
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) {
+            split_hi_lo(Bm[k0 * LD32 + 8 * nt + g], bh[nt][0], bl[nt][0]);
+            split_hi_lo(Bm[(k0 + 8) * LD32 + 8 * nt + g], bh[nt][1], bl[nt][1]);
+        }
+        // pass-major order: the eight accumulator tiles of a pass are independent of one another
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+            for (int mt = 0; mt < 2; ++mt)
+                mma_tf32(acc[mt][nt], al[mt][0], al[mt][1], al[mt][2], al[mt][3], bh[nt][0], bh[nt][1]);
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+            for (int mt = 0; mt < 2; ++mt)
+                mma_tf32(acc[mt][nt], ah[mt][0], ah[mt][1], ah[mt][2], ah[mt][3], bl[nt][0], bl[nt][1]);
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+            for (int mt = 0; mt < 2; ++mt)
+                mma_tf32(acc[mt][nt], ah[mt][0], ah[mt][1], ah[mt][2], ah[mt][3], bh[nt][0], bh[nt][1]);
+    }
+}
+__device__ __forceinline__ void mma32_zero(float (&acc)[2][4][4])
+{
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                acc[mt][nt][e] = 0.f;
+}
+// accumulator tiles -> row-major matrix in shared memory (8-byte stores)
+__device__ __forceinline__ void mma32_store(float* Dm, const float (&acc)[2][4][4], int lane)
+{
+    const int g = lane >> 2, t = lane & 3;
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) {
+            *reinterpret_cast<float2*>(Dm + (16 * mt + g) * LD32 + 8 * nt + 2 * t) = make_float2(acc[mt][nt][0], acc[mt][nt][1]);
+            *reinterpret_cast<float2*>(Dm + (16 * mt + g + 8) * LD32 + 8 * nt + 2 * t) = make_float2(acc[mt][nt][2], acc[mt][nt][3]);
+        }
+}
+
 // Per-head operands of time index t -> shared memory (all threads of the CTA; the caller synchronises).
 template <int N>
 __device__ __forceinline__ void load_head_operands(Smem<N>& sm, const SolveParams& p, long long oa, long long ob, long long orr,
@@ -209,6 +292,9 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
 {
     using S = Shape<N>;
     constexpr int LD = S::LD;
+    // n = 32, operands constant in time: the dense contractions of a step run on the tensor cores (mma.sync, three-pass
+    // tf32); the factorisation, the substitutions and the rollout stay on the FP32 pipe
+    constexpr bool MMA = (N == 32) && !TV;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     Smem<N>& sm = *reinterpret_cast<Smem<N>*>(smem_raw);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -299,68 +385,90 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
                     __syncthreads();
                 }
             }
-            f32x2 vcol[N / 2], tcol[N / 2];
-#pragma unroll
-            for (int k = 0; k < N / 2; ++k) {
-                vcol[k] = 0ull;
-                tcol[k] = 0ull;
-            }
-#pragma unroll 4
-            for (int i = 0; i < N; ++i) {                     // V[:,c] = P B[:,c], T[:,c] = P A[:,c]
-                const float bic = Bs[i * LD + c], aic = As[i * LD + c];
-                const f32x2 b2 = pack2(bic, bic), a2 = pack2(aic, aic);
-                const float* prow = sl.buf0 + i * LD;
-#pragma unroll
-                for (int q = 0; q < N / 4; ++q) {
-                    const ulonglong2 t = *reinterpret_cast<const ulonglong2*>(prow + 4 * q);
-                    fma2(vcol[2 * q], t.x, b2);
-                    fma2(vcol[2 * q + 1], t.y, b2);
-                    fma2(tcol[2 * q], t.x, a2);
-                    fma2(tcol[2 * q + 1], t.y, a2);
-                }
-            }
-            // stage the two columns in the instance's scratch (own column only: no exchange) so that the next loop
-            // can run over k without indexing registers dynamically
-#pragma unroll
-            for (int k = 0; k < N / 2; ++k) {
-                float v0, v1, t0, t1;
-                unpack2(vcol[k], v0, v1);
-                unpack2(tcol[k], t0, t1);
-                sl.L[(2 * k) * LD + c] = v0;
-                sl.L[(2 * k + 1) * LD + c] = v1;
-                sl.Lt[(2 * k) * LD + c] = t0;
-                sl.Lt[(2 * k + 1) * LD + c] = t1;
-            }
-            f32x2 s2[N / 2], y2[N / 2], p2[N / 2];
-            {
-                float tmp[N];
-                load_row<N>(tmp, Rs + c * LD);              // S[:,c] = R[:,c] + B' V[:,c]
-                pack_row<N>(s2, tmp);
-                load_q_row<N>(tmp, p.Q, TV ? oq + ts * p.Q.st : oq);    // Pn[:,c] = Q_t[:,c] + A' T[:,c] ; Y[:,c] = B' T[:,c]
-                pack_row<N>(p2, tmp);
-            }
-#pragma unroll
-            for (int l = 0; l < N / 2; ++l)
-                y2[l] = 0ull;
-#pragma unroll 4
-            for (int k = 0; k < N; ++k) {
-                const float vk = sl.L[k * LD + c], tk = sl.Lt[k * LD + c];
-                const f32x2 vv = pack2(vk, vk), tt = pack2(tk, tk);
-#pragma unroll
-                for (int q = 0; q < N / 4; ++q) {             // each row of B and A is read once
-                    const ulonglong2 b4 = *reinterpret_cast<const ulonglong2*>(Bs + k * LD + 4 * q);
-                    const ulonglong2 a4 = *reinterpret_cast<const ulonglong2*>(As + k * LD + 4 * q);
-                    fma2(s2[2 * q], vv, b4.x);
-                    fma2(s2[2 * q + 1], vv, b4.y);
-                    fma2(y2[2 * q], tt, b4.x);
-                    fma2(y2[2 * q + 1], tt, b4.y);
-                    fma2(p2[2 * q], tt, a4.x);
-                    fma2(p2[2 * q + 1], tt, a4.y);
-                }
-            }
             float s[N], y[N];
-            unpack_row<N>(s, s2);
-            unpack_row<N>(y, y2);
+            f32x2 p2[N / 2];
+            float pn[N];                                      // tensor-core path: column c of Q_t + A'T
+            // Tensor-core path: the six 32 x 32 x 32 products of a step (V = P B, T = P A, S - R = B'V, Y = B'T, A'T,
+            // Z'Z) share one copy of the product code: phases 0..4 run it on the way to the factorisation, phase 5 first
+            // factorises and substitutes, then runs it on Z.  Straight-line code for every product separately does not
+            // fit the instruction cache next to the unrolled factorisation.  Without tensor cores there is only phase 5.
+#pragma unroll 1
+            for (int ph = MMA ? 0 : 5; ph < 6; ++ph) {
+            if (!MMA || ph == 5) {
+            if constexpr (MMA) {
+                float tmp[N];
+                load_row<N>(s, Rs + c * LD);                  // S[:,c] = R[:,c] + (B'V)[c,:]  (symmetric)
+                load_row<N>(tmp, sl.buf0 + c * LD);
+                load_q_row<N>(pn, p.Q, oq);
+#pragma unroll
+                for (int l = 0; l < N; ++l) {
+                    s[l] += tmp[l];
+                    y[l] = sl.L[l * LD + c];
+                    pn[l] += sl.Lt[l * LD + c];
+                }
+            } else {
+                f32x2 vcol[N / 2], tcol[N / 2];
+#pragma unroll
+                for (int k = 0; k < N / 2; ++k) {
+                    vcol[k] = 0ull;
+                    tcol[k] = 0ull;
+                }
+#pragma unroll 4
+                for (int i = 0; i < N; ++i) {                     // V[:,c] = P B[:,c], T[:,c] = P A[:,c]
+                    const float bic = Bs[i * LD + c], aic = As[i * LD + c];
+                    const f32x2 b2 = pack2(bic, bic), a2 = pack2(aic, aic);
+                    const float* prow = sl.buf0 + i * LD;
+#pragma unroll
+                    for (int q = 0; q < N / 4; ++q) {
+                        const ulonglong2 t = *reinterpret_cast<const ulonglong2*>(prow + 4 * q);
+                        fma2(vcol[2 * q], t.x, b2);
+                        fma2(vcol[2 * q + 1], t.y, b2);
+                        fma2(tcol[2 * q], t.x, a2);
+                        fma2(tcol[2 * q + 1], t.y, a2);
+                    }
+                }
+                // stage the two columns in the instance's scratch (own column only: no exchange) so that the next loop
+                // can run over k without indexing registers dynamically
+#pragma unroll
+                for (int k = 0; k < N / 2; ++k) {
+                    float v0, v1, t0, t1;
+                    unpack2(vcol[k], v0, v1);
+                    unpack2(tcol[k], t0, t1);
+                    sl.L[(2 * k) * LD + c] = v0;
+                    sl.L[(2 * k + 1) * LD + c] = v1;
+                    sl.Lt[(2 * k) * LD + c] = t0;
+                    sl.Lt[(2 * k + 1) * LD + c] = t1;
+                }
+                f32x2 s2[N / 2], y2[N / 2];
+                {
+                    float tmp[N];
+                    load_row<N>(tmp, Rs + c * LD);              // S[:,c] = R[:,c] + B' V[:,c]
+                    pack_row<N>(s2, tmp);
+                    load_q_row<N>(tmp, p.Q, TV ? oq + ts * p.Q.st : oq);    // Pn[:,c] = Q_t[:,c] + A' T[:,c] ; Y[:,c] = B' T[:,c]
+                    pack_row<N>(p2, tmp);
+                }
+#pragma unroll
+                for (int l = 0; l < N / 2; ++l)
+                    y2[l] = 0ull;
+#pragma unroll 4
+                for (int k = 0; k < N; ++k) {
+                    const float vk = sl.L[k * LD + c], tk = sl.Lt[k * LD + c];
+                    const f32x2 vv = pack2(vk, vk), tt = pack2(tk, tk);
+#pragma unroll
+                    for (int q = 0; q < N / 4; ++q) {             // each row of B and A is read once
+                        const ulonglong2 b4 = *reinterpret_cast<const ulonglong2*>(Bs + k * LD + 4 * q);
+                        const ulonglong2 a4 = *reinterpret_cast<const ulonglong2*>(As + k * LD + 4 * q);
+                        fma2(s2[2 * q], vv, b4.x);
+                        fma2(s2[2 * q + 1], vv, b4.y);
+                        fma2(y2[2 * q], tt, b4.x);
+                        fma2(y2[2 * q + 1], tt, b4.y);
+                        fma2(p2[2 * q], tt, a4.x);
+                        fma2(p2[2 * q + 1], tt, a4.y);
+                    }
+                }
+                unpack_row<N>(s, s2);
+                unpack_row<N>(y, y2);
+            }
             float gz[N];                                      // B'p + r, then L^{-1}(.), then k_t = -S^{-1}(.) (every lane holds all of it)
             float apc = 0.f;                                  // (A'p_{t+1})[c]
             if (AFF) {
@@ -427,10 +535,12 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
             for (int q = 0; q < N; ++q)
                 sl.buf0[q * LD + c] = y[q];                   // rows of Z
             __syncwarp();
+            if constexpr (!MMA) {
 #pragma unroll 4
-            for (int q = 0; q < N; ++q)                       // Pn[:,c] -= Z' Z[:,c]
-                axpy_row<N>(p2, -sl.buf0[q * LD + c], sl.buf0 + q * LD);
-            unpack_row<N>(pcol, p2);
+                for (int q = 0; q < N; ++q)                   // Pn[:,c] -= Z' Z[:,c]
+                    axpy_row<N>(p2, -sl.buf0[q * LD + c], sl.buf0 + q * LD);
+                unpack_row<N>(pcol, p2);
+            }
             const bool gains = need_K_all || need_k_all || (want_u0 && ts == 0);
             if (gains) {                                      // K[:,c] = -L^{-T} Z[:,c]  (and k_t = -L^{-T} L^{-1}(B'p + r))
 #pragma unroll
@@ -488,6 +598,29 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
                         sl.Lt[l * LD + c] = -y[l];
                 }
             }
+            }                                                 // phase 5: factorisation, substitutions, gains
+            if constexpr (MMA) {
+                // phase:  0      1      2      3      4      5
+                // A'   :  P      P      B'     B'     A'     Z'          (P symmetric, so P B = P'B)
+                // B    :  B      A      V      T      T      Z
+                // to   :  L      L'     buf0   L      L'     L           (buf0: P, then B'V, then Z)
+                // The rows of L' may hold K_0 for the last step's u_0, so Z'Z goes to the rows of L.
+                const float* Am = ph < 2 ? sl.buf0 : ph == 4 ? As : ph == 5 ? sl.buf0 : Bs;
+                const float* Bm = ph == 0 ? Bs : ph == 1 ? As : ph == 2 ? sl.L : ph == 5 ? sl.buf0 : sl.Lt;
+                float* Dm = ph == 1 || ph == 4 ? sl.Lt : ph == 2 ? sl.buf0 : sl.L;
+                float acc[2][4][4];
+                mma32_zero(acc);
+                mma32_product(acc, Am, Bm, lane);
+                __syncwarp();                                 // every lane has read what the result overwrites
+                mma32_store(Dm, acc, lane);
+                __syncwarp();
+                if (ph == 5) {
+#pragma unroll
+                    for (int l = 0; l < N; ++l)
+                        pcol[l] = pn[l] - sl.L[l * LD + c];   // P_t[:,c] = Q[:,c] + A'T[:,c] - Z'Z[:,c]
+                }
+            }
+            }                                                 // phases
             __syncwarp();                                     // rows of Z consumed
             store_row<N>(sl.buf0 + c * LD, pcol);             // column c of P_t as row c
             __syncwarp();
