@@ -350,7 +350,7 @@ int ttc_lqr_solve_layer_host(ttc_lqr_handle* h, const ttc_layer_inputs* in, int3
  * pageable memory works but serialises them).  The call copies the inputs to device staging
  * buffers owned by the handle, solves on internal streams, copies the requested outputs back
  * and returns after everything has completed (synchronous).  Large problems are cut into up to
- * 8 slices of the last batch dimension so that the copy-in of one slice, the solve of the
+ * 32 slices of the last batch dimension so that the copy-in of one slice, the solve of the
  * previous one and the copy-out of the one before overlap; results are identical to
  * ttc_lqr_solve.  Strides have the same meaning.
  */

@@ -42,7 +42,7 @@ int fail(int status, const char* fmt, ...)
             return fail(TTC_STATUS_CUDA_ERROR, "%s: %s", #call, cudaGetErrorString(e_)); \
     } while (0)
 
-constexpr int kMaxSlices = 8;    // token slices of the pipelined host-buffer entry point
+constexpr int kMaxSlices = 32;   // token slices of the pipelined host-buffer entry point
 
 struct DevBuf {
     void* ptr = nullptr;
