@@ -868,7 +868,7 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="", help="one workload only (cfg0..cfg4, tv16, layer16, layer32, grad16); "
+    ap.add_argument("--workload", default="", help="one workload only (cfg0..cfg4, tv16, tv32, layer16, layer32, grad16); "
                     "default: cfg4 as the headline plus short side measurements of cfg0..cfg3")
     ap.add_argument("--method", default="auto", choices=["auto", "riccati", "scan", "sigma"],
                     help="sigma: layer workloads only, the row-normalised reverse symplectic product (baseline)")

@@ -292,9 +292,9 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
 {
     using S = Shape<N>;
     constexpr int LD = S::LD;
-    // n = 32, operands constant in time: the dense contractions of a step run on the tensor cores (mma.sync, three-pass
-    // tf32); the factorisation, the substitutions and the rollout stay on the FP32 pipe
-    constexpr bool MMA = (N == 32) && !TV;
+    // n = 32: the dense contractions of a step run on the tensor cores (mma.sync, three-pass tf32); the factorisation,
+    // the substitutions, the vector recursion of the affine term and the rollout stay on the FP32 pipe
+    constexpr bool MMA = (N == 32);
     extern __shared__ __align__(16) unsigned char smem_raw[];
     Smem<N>& sm = *reinterpret_cast<Smem<N>*>(smem_raw);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -399,7 +399,7 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) riccati_warp_kerne
                 float tmp[N];
                 load_row<N>(s, Rs + c * LD);                  // S[:,c] = R[:,c] + (B'V)[c,:]  (symmetric)
                 load_row<N>(tmp, sl.buf0 + c * LD);
-                load_q_row<N>(pn, p.Q, oq);
+                load_q_row<N>(pn, p.Q, TV ? oq + ts * p.Q.st : oq);
 #pragma unroll
                 for (int l = 0; l < N; ++l) {
                     s[l] += tmp[l];

@@ -44,6 +44,9 @@ CONFIGS = {
 TV_CONFIGS = {
     "tv16": dict(name="tv16_ttc_layer_d16_T32", batch=(4, 16, 1024), n=16, m=16, H=32, q_dtype="f32",
                  first_only=True, tol=1e-4, tv=("A", "B", "Q", "R")),
+    # the time-varying problem at d = 32 per head (a quarter of the tokens: the same bytes of Q_t)
+    "tv32": dict(name="tv32_ttc_layer_d32_T32", batch=(4, 16, 256), n=32, m=32, H=32, q_dtype="f32",
+                 first_only=True, tol=1e-4, tv=("A", "B", "Q", "R")),
     # the same problem, differentiated: gradients of a loss of u_0* with respect to every A_t, B_t, Q_t, R_t, Q_f, x_0
     "grad16": dict(name="grad16_ttc_layer_d16_T32", batch=(4, 16, 1024), n=16, m=16, H=32, q_dtype="f32",
                    first_only=True, tol=1e-4, tv=("A", "B", "Q", "R"), grad=True),
