@@ -71,6 +71,9 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) ttc_layer_kernel(L
     using S = Shape<N>;
     using namespace rwarp;
     constexpr int LD = S::LD;
+    // n = 32: the dense contractions run on the tensor cores (three-pass tf32 mma.sync, see riccati_warp.cuh).  With a
+    // diagonal A_t only three are left: V0 = P Bbar, Bbar'V0 and Z'Z; Y = G Bbar'P A_t is V0' scaled on both sides.
+    constexpr bool MMA = (N == 32);
     extern __shared__ __align__(16) unsigned char smem_raw[];
     Smem<N>& sm = *reinterpret_cast<Smem<N>*>(smem_raw);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -138,61 +141,82 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) ttc_layer_kernel(L
             sl.gb[c] = g_c;
             sl.gq[c] = q_c;
             __syncwarp();                                     // rows of P and the step's diagonals are in place
-            f32x2 vcol[N / 2];
-#pragma unroll
-            for (int k = 0; k < N / 2; ++k)
-                vcol[k] = 0ull;
-#pragma unroll 4
-            for (int i = 0; i < N; ++i) {                     // P Bbar[:,c]
-                const float bic = sl.Bb[i * LD + c];
-                axpy_row<N>(vcol, bic, sl.buf0 + i * LD);
-            }
-            // stage V[:,c] = g_c (P Bbar[:,c]) and T[:,c] = a_c P[:,c] (own column only) so that the next loop can
-            // run over k without indexing registers dynamically
-#pragma unroll
-            for (int k = 0; k < N / 2; ++k) {
-                float v0, v1;
-                unpack2(vcol[k], v0, v1);
-                sl.L[(2 * k) * LD + c] = g_c * v0;
-                sl.L[(2 * k + 1) * LD + c] = g_c * v1;
-                sl.Lt[(2 * k) * LD + c] = at_c * pcol[2 * k];
-                sl.Lt[(2 * k + 1) * LD + c] = at_c * pcol[2 * k + 1];
-            }
-            f32x2 s2[N / 2], y2[N / 2];
-#pragma unroll
-            for (int l = 0; l < N / 2; ++l) {
-                s2[l] = 0ull;
-                y2[l] = 0ull;
-            }
-#pragma unroll 4
-            for (int k = 0; k < N; ++k) {                     // Bbar' V[:,c] and Bbar' T[:,c]: each row of Bbar read once
-                const float vk = sl.L[k * LD + c], tk = sl.Lt[k * LD + c];
-                const f32x2 vv = pack2(vk, vk), t2 = pack2(tk, tk);
-#pragma unroll
-                for (int q = 0; q < N / 4; ++q) {
-                    const ulonglong2 b4 = *reinterpret_cast<const ulonglong2*>(sl.Bb + k * LD + 4 * q);
-                    fma2(s2[2 * q], vv, b4.x);
-                    fma2(s2[2 * q + 1], vv, b4.y);
-                    fma2(y2[2 * q], t2, b4.x);
-                    fma2(y2[2 * q + 1], t2, b4.y);
-                }
-            }
             float sv[N], y[N], pn[N];
-            unpack_row<N>(sv, s2);
-            unpack_row<N>(y, y2);
-            {
-                float gv[N], av[N], qv[N];
+            // Tensor-core path: one copy of the product code run in three phases (V0 = P Bbar -> rows of L, Bbar'V0 ->
+            // rows of L', then factorisation / substitutions / gains and Z'Z -> rows of L).  Otherwise only phase 2.
+#pragma unroll 1
+            for (int ph = MMA ? 0 : 2; ph < 3; ++ph) {
+            if (!MMA || ph == 2) {
+            if constexpr (MMA) {
+                float gv[N], av[N], qv[N], v0[N];
                 load_row<N>(gv, sl.gb);
                 load_row<N>(av, sl.at);
                 load_row<N>(qv, sl.gq);
+                load_row<N>(v0, sl.L + c * LD);               // row c of V0 = column c of Bbar'P
 #pragma unroll
                 for (int l = 0; l < N; ++l) {
-                    sv[l] *= gv[l];
-                    y[l] *= gv[l];
-                    // Pn[l][c] = q_l Qbar[l][c] q_c + a_l a_c P[l][c]
+                    sv[l] = gv[l] * g_c * sl.Lt[l * LD + c];  // S = G Bbar'P Bbar G + R
+                    y[l] = gv[l] * at_c * v0[l];              // Y = G Bbar'P A_t
                     pn[l] = fmaf(q_c * qv[l], qcol[l], av[l] * at_c * pcol[l]);
                     if (l == c)
                         sv[l] += r_c;
+                }
+            } else {
+                f32x2 vcol[N / 2];
+#pragma unroll
+                for (int k = 0; k < N / 2; ++k)
+                    vcol[k] = 0ull;
+#pragma unroll 4
+                for (int i = 0; i < N; ++i) {                     // P Bbar[:,c]
+                    const float bic = sl.Bb[i * LD + c];
+                    axpy_row<N>(vcol, bic, sl.buf0 + i * LD);
+                }
+                // stage V[:,c] = g_c (P Bbar[:,c]) and T[:,c] = a_c P[:,c] (own column only) so that the next loop can
+                // run over k without indexing registers dynamically
+#pragma unroll
+                for (int k = 0; k < N / 2; ++k) {
+                    float v0, v1;
+                    unpack2(vcol[k], v0, v1);
+                    sl.L[(2 * k) * LD + c] = g_c * v0;
+                    sl.L[(2 * k + 1) * LD + c] = g_c * v1;
+                    sl.Lt[(2 * k) * LD + c] = at_c * pcol[2 * k];
+                    sl.Lt[(2 * k + 1) * LD + c] = at_c * pcol[2 * k + 1];
+                }
+                f32x2 s2[N / 2], y2[N / 2];
+#pragma unroll
+                for (int l = 0; l < N / 2; ++l) {
+                    s2[l] = 0ull;
+                    y2[l] = 0ull;
+                }
+#pragma unroll 4
+                for (int k = 0; k < N; ++k) {                     // Bbar' V[:,c] and Bbar' T[:,c]: each row of Bbar read once
+                    const float vk = sl.L[k * LD + c], tk = sl.Lt[k * LD + c];
+                    const f32x2 vv = pack2(vk, vk), t2 = pack2(tk, tk);
+#pragma unroll
+                    for (int q = 0; q < N / 4; ++q) {
+                        const ulonglong2 b4 = *reinterpret_cast<const ulonglong2*>(sl.Bb + k * LD + 4 * q);
+                        fma2(s2[2 * q], vv, b4.x);
+                        fma2(s2[2 * q + 1], vv, b4.y);
+                        fma2(y2[2 * q], t2, b4.x);
+                        fma2(y2[2 * q + 1], t2, b4.y);
+                    }
+                }
+                unpack_row<N>(sv, s2);
+                unpack_row<N>(y, y2);
+                {
+                    float gv[N], av[N], qv[N];
+                    load_row<N>(gv, sl.gb);
+                    load_row<N>(av, sl.at);
+                    load_row<N>(qv, sl.gq);
+#pragma unroll
+                    for (int l = 0; l < N; ++l) {
+                        sv[l] *= gv[l];
+                        y[l] *= gv[l];
+                        // Pn[l][c] = q_l Qbar[l][c] q_c + a_l a_c P[l][c]
+                        pn[l] = fmaf(q_c * qv[l], qcol[l], av[l] * at_c * pcol[l]);
+                        if (l == c)
+                            sv[l] += r_c;
+                    }
                 }
             }
             float rs_own;
@@ -226,7 +250,7 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) ttc_layer_kernel(L
             for (int q = 0; q < N; ++q)
                 sl.buf0[q * LD + c] = y[q];                   // rows of Z
             __syncwarp();
-            {
+            if constexpr (!MMA) {
                 f32x2 p2[N / 2];
                 pack_row<N>(p2, pn);
 #pragma unroll 4
@@ -289,6 +313,34 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) ttc_layer_kernel(L
                         sl.Lt[l * LD + c] = -y[l];
                 }
             }
+            }                                                 // phase 2: factorisation, substitutions, gains
+            if constexpr (MMA) {
+                // phase:  0       1        2
+                // A'   :  P       Bbar'    Z'
+                // B    :  Bbar    V0       Z
+                // to   :  L       L'       L     (the rows of L' may hold K_1 by then)
+                const float* Am = ph == 1 ? sl.Bb : sl.buf0;
+                const float* Bm = ph == 0 ? sl.Bb : ph == 1 ? sl.L : sl.buf0;
+                float* Dm = ph == 1 ? sl.Lt : sl.L;
+                __syncwarp();                                 // every lane is done with what the operands replace
+                float acc[2][4][4];
+                mma32_zero(acc);
+                mma32_product(acc, Am, Bm, lane);
+                __syncwarp();
+                mma32_store(Dm, acc, lane);
+                __syncwarp();
+                if (ph == 2) {
+                    // P_s[:,c] = Pn[:,c] - Z'Z[:,c], with Z'Z averaged with its transpose: Pn is symmetric bit for bit
+                    // (the FP32 loops keep Z'Z so too), the three-pass product is only up to rounding, and an
+                    // antisymmetric part E obeys E <- A_t E A_t, which grows wherever the diagonal of A_t exceeds one
+                    float zr[N];
+                    load_row<N>(zr, sl.L + c * LD);
+#pragma unroll
+                    for (int l = 0; l < N; ++l)
+                        pcol[l] = pn[l] - 0.5f * (sl.L[l * LD + c] + zr[l]);
+                }
+            }
+            }                                                 // phases
             __syncwarp();                                     // rows of Z consumed
             store_row<N>(sl.buf0 + c * LD, pcol);             // rows of P_s (row c = column c)
             if (GRAD && s >= 1 && active) {

@@ -45,8 +45,10 @@ def check(u1, P0, info, ref, idx, tol):
 
 
 @pytest.mark.parametrize("key,batch,T", [("layer16", (1, 3, 7), 1), ("layer16", (2, 3, 9), 5), ("layer16", (1, 2, 33), 32),
-                                         ("layer32", (1, 2, 5), 3), ("layer32", (2, 2, 6), 17)])
+                                         ("layer32", (1, 2, 5), 3), ("layer32", (2, 2, 6), 17), ("layer32", (1, 2, 40), 32)])
 def test_layer_matches_oracle_on_every_instance(key, batch, T):
+    """The full horizon at n = 32 is the case that shows a value matrix drifting away from symmetry: its diagonal
+    A_t exceeds one, so an antisymmetric rounding residue doubles every few steps (1e-7 -> 1e-1 over 32 steps)."""
     w = workloads.make_layer_workload(key, device=DEV, batch=batch, seed=900 + T)
     u1, P0, info = run_gpu(w, T)
     idx = np.arange(w["N"])
