@@ -21,10 +21,18 @@
 //   (4)  DP = W * A = [ . ; A'P A]   (into the columns that held F)                         TS, N64
 //   (5)  DP -= Z' Z                                                                         SS, N64
 //   P <- Q + DP                  (P_t = Q + A'P A - Y'S^{-1}Y)
-// Tensor memory of a warpgroup (128 columns): R_W = W, R_F = F then DP.
-// Shared memory of a warpgroup: X1 (L in fp32, only when the gains or u_0 need it) | X0 (P, then Z') | panel hi |
-// panel lo | scratch.  X1 directly precedes X0: step (5) starts its A operand 64 rows before Z' so that Z' lands on
-// lanes 64..127 (what the first 64 rows multiply goes to lanes that are never read).
+//   Gains (every K_t wanted): rows 0..63 of the factorisation keep going after their diagonal block as the rows of
+//   X = L^{-T} (X L' = I is the same forward substitution as Z' L' = Y'; the tensor-memory row they reuse is the upper
+//   triangle of S, which its own panel's update brings to zero).  As rows of the B operand of the rank-8 updates they
+//   subtract Z'[n,p] X[r,p]' from column r of the rows of Z' once that column has been consumed, so that after the
+//   last panel columns 0..63 of lanes 64..127 hold -Z' L^{-1} = K_t': the gains fall out of the factorisation's own
+//   updates, in their error-compensated arithmetic (Z' keeps its low part for this), with no backward solve.
+//   (4) then follows the read-out of K_t'.
+// Tensor memory of a warpgroup (128 columns): R_W = W, R_F = F (then K_t' on lanes 64..127), then DP.
+// Shared memory of a warpgroup: X1 (L in fp32 at the last step when only u_0 is wanted; scratch of the periodic
+// symmetrisation) | X0 (P, then Z') | panel hi | panel lo | scratch.  X1 directly precedes X0: step (5) starts its A
+// operand 64 rows before Z' so that Z' lands on lanes 64..127 (what the first 64 rows multiply goes to lanes that are
+// never read).
 //
 // Shared-memory operands use the canonical K-major layout without swizzle: 8 x 4 (rows x k) core
 // matrices of 128 contiguous bytes, chunk stride 128 B along k, 2048 B between 8-row groups (256 B in the panel
@@ -176,28 +184,20 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16])
                  : "r"(taddr) : "memory");
 }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// 16 registers per thread -> 32 lanes x 16 consecutive columns; followed by tmem_wait_st() before anything depends on it
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16])
+{
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+                 :: "r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+                    "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]) : "memory");
+}
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 // named barriers: 1 + wg = warps 0, 1 of a warpgroup (64 threads), 5 + wg = the whole warpgroup
 __device__ __forceinline__ void half_barrier(int wg) { asm volatile("bar.sync %0, %1;" :: "r"(1 + wg), "r"(64) : "memory"); }
 __device__ __forceinline__ void wg_barrier(int wg) { asm volatile("bar.sync %0, %1;" :: "r"(5 + wg), "r"(WG_THREADS) : "memory"); }
 
 // ---- blocked Cholesky of S fused with the forward substitution Z' = Y' L^{-T} --------------------------------------
-__device__ __forceinline__ void mma_16x8x8(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                           uint32_t b0, uint32_t b1)
-{
-    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
-                 "{%0,%1,%2,%3};"
-                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-// x = hi + lo with hi exactly representable in tf32 (truncation); the tensor core ignores the low 13 bits
-// of lo, an error of 2^-21 |x|.  hi*hi + hi*lo + lo*hi then has fp32-grade accuracy.
-__device__ __forceinline__ void split_tf32(float x, uint32_t& hi, uint32_t& lo)
-{
-    hi = __float_as_uint(x) & 0xffffe000u;
-    lo = __float_as_uint(x - __uint_as_float(hi));
-}
-
 // In-thread Cholesky of an 8 x 8 SPD block: l (lower triangle) is overwritten by L, rinv[i] = 1 / L[i][i].
 // Right-looking; the chain from one pivot to the next is rsqrt -> multiply -> fma.
 // Returns 0 or 1 + the index of the first non-positive pivot.
@@ -258,101 +258,6 @@ __device__ __forceinline__ void store_row8(unsigned char* grp, int slot, const f
     }
     *reinterpret_cast<float4*>(grp + slot * 16) = a;
     *reinterpret_cast<float4*>(grp + SC + (ROT ? ((slot + 4) & 7) : slot) * 16) = b;
-}
-
-// Gains (Eq. 4): K = -L^{-T} Z, i.e. row c of K' is -(row c of Z') L^{-1}.  The four warps of the warpgroup run a
-// blocked scheme backwards on L (fp32, rotated layout, at `Sm`) and Z' (at `Ym`): per 8-wide block kb = 7..0 the
-// owner of row c (threads 0..63) solves x L_d = z for its row of Z' (in place in `Ym`), then the columns left of the
-// block get the update Z'[c][j] -= x[c][kb] . L[kb][j] as 3 x tf32 mma, one 16-row tile per warp.
-// On return row c of Ym holds (Z' L^{-1})[c][:] = -K[:, c] (fp32).  Ends with a warpgroup barrier.
-__device__ __forceinline__ void wg_gain_solve(const unsigned char* Sm, unsigned char* Ym, int wg, int warp, int lane)
-{
-    const int g = lane >> 2, t = lane & 3;
-    const int wt = 32 * warp + lane;
-    const uint32_t frag_ab = (uint32_t)g * 16u + (uint32_t)t * 4u;
-    const uint32_t frag_c = (uint32_t)g * 16u + (uint32_t)(t >> 1) * SC + (uint32_t)((2 * t) & 3) * 4u;
-    // (row t, col g) and (row t + 4, col g) of a tile of L (rotated layout: the chunk parity is g >> 2)
-    const uint32_t frag_b = (uint32_t)((t + 4 * (g >> 2)) & 7) * 16u + (uint32_t)(g >> 2) * SC + (uint32_t)(g & 3) * 4u;
-    const uint32_t frag_b4 = (uint32_t)((t + 4 + 4 * (g >> 2)) & 7) * 16u + (uint32_t)(g >> 2) * SC + (uint32_t)(g & 3) * 4u;
-    const uint32_t own_grp = (uint32_t)((wt & 63) >> 3) * SR;
-    const int own_slot = wt & 7;
-#pragma unroll 1
-    for (int kb = 7; kb >= 0; --kb) {
-        const uint32_t kcol = 2u * kb * SC;
-        if (warp < 2) {
-            const unsigned char* dblk = Sm + (uint32_t)kb * SR + kcol;
-            float l[8][8], xr[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i)
-                load_row8<true>(l[i], dblk, i);
-            unsigned char* py = Ym + own_grp + kcol;
-            load_row8<false>(xr, py, own_slot);
-#pragma unroll
-            for (int j = 7; j >= 0; --j) {                 // x L_d = z, L_d lower triangular
-                float v = xr[j];
-#pragma unroll
-                for (int i = j + 1; i < 8; ++i)
-                    v = fmaf(-xr[i], l[i][j], v);
-                xr[j] = __fdividef(v, l[j][j]);
-            }
-            store_row8<false, false>(py, own_slot, xr);
-        }
-        wg_barrier(wg);
-        if (kb == 0)
-            break;
-        // B fragments: rows 8kb + t, 8kb + t + 4 of L, columns 8j + g (j < kb)
-        uint32_t bh[7][2], bl[7][2];
-        {
-            const unsigned char* pb = Sm + (uint32_t)kb * SR;
-#pragma unroll
-            for (int j = 0; j < 7; ++j)
-                if (j < kb) {
-                    split_tf32(*reinterpret_cast<const float*>(pb + 2 * j * SC + frag_b), bh[j][0], bl[j][0]);
-                    split_tf32(*reinterpret_cast<const float*>(pb + 2 * j * SC + frag_b4), bh[j][1], bl[j][1]);
-                }
-        }
-        {
-            const int mt = warp;                           // rows 16 mt .. 16 mt + 15 of Z'
-            uint32_t ah[4], al[4];
-            {
-                const unsigned char* pa = Ym + frag_ab + kcol + 2 * mt * SR;
-                split_tf32(-*reinterpret_cast<const float*>(pa), ah[0], al[0]);
-                split_tf32(-*reinterpret_cast<const float*>(pa + SR), ah[1], al[1]);
-                split_tf32(-*reinterpret_cast<const float*>(pa + SC), ah[2], al[2]);
-                split_tf32(-*reinterpret_cast<const float*>(pa + SR + SC), ah[3], al[3]);
-            }
-            unsigned char* pc = Ym + frag_c + 2 * mt * SR;
-            float acc[7][4];
-#pragma unroll
-            for (int j = 0; j < 7; ++j) {
-                if (j >= kb)
-                    continue;
-                const float2 lo = *reinterpret_cast<const float2*>(pc + 2 * j * SC);
-                const float2 hi = *reinterpret_cast<const float2*>(pc + 2 * j * SC + SR);
-                acc[j][0] = lo.x; acc[j][1] = lo.y; acc[j][2] = hi.x; acc[j][3] = hi.y;
-            }
-#pragma unroll
-            for (int j = 0; j < 7; ++j)
-                if (j < kb)
-                    mma_16x8x8(acc[j], al[0], al[1], al[2], al[3], bh[j][0], bh[j][1]);
-#pragma unroll
-            for (int j = 0; j < 7; ++j)
-                if (j < kb)
-                    mma_16x8x8(acc[j], ah[0], ah[1], ah[2], ah[3], bl[j][0], bl[j][1]);
-#pragma unroll
-            for (int j = 0; j < 7; ++j)
-                if (j < kb)
-                    mma_16x8x8(acc[j], ah[0], ah[1], ah[2], ah[3], bh[j][0], bh[j][1]);
-#pragma unroll
-            for (int j = 0; j < 7; ++j) {
-                if (j >= kb)
-                    continue;
-                *reinterpret_cast<float2*>(pc + 2 * j * SC) = make_float2(acc[j][0], acc[j][1]);
-                *reinterpret_cast<float2*>(pc + 2 * j * SC + SR) = make_float2(acc[j][2], acc[j][3]);
-            }
-        }
-        wg_barrier(wg);
-    }
 }
 
 // ---- global-memory helpers --------------------------------------------------------------------------------------
@@ -598,7 +503,7 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
                 }
                 wait_mma();
                 // (3) [S; Y'] = [L; Z'] L' panel by panel, thread wt owns row wt
-                const bool keep_l = need_K_all || (ts == 0 && want_u0);
+                const bool keep_l = ts == 0 && want_u0;        // fp32 copy of L for the back substitution of u_0
                 float* diag = &misc.y0[0];                     // [8][8]
                 float v[8];
                 auto load_cols = [&](int c0) {
@@ -615,6 +520,38 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
                     v[4] = __uint_as_float(raw[4]) + r1.x; v[5] = __uint_as_float(raw[5]) + r1.y;
                     v[6] = __uint_as_float(raw[6]) + r1.z; v[7] = __uint_as_float(raw[7]) + r1.w;
                 };
+                if (GAINS && warp < 2) {
+                    // The rows of L^{-T} start from the upper triangle of S, the factorisation reads the lower one, and
+                    // the two differ by the rounding of the tf32 contractions (and of a P that is only symmetrised now
+                    // and then): at 1e-3 of |S| that would be the error of the gains.  Mirror the lower triangle into
+                    // the upper one first: every row through X1 (free here), element (r, c) at word 64 r + (c ^ r) so
+                    // that both the row stores and the column reads touch 32 banks.
+                    float* tr = reinterpret_cast<float*>(X1);
+#pragma unroll
+                    for (int qt = 0; qt < 4; ++qt) {
+                        uint32_t raw[16];
+                        tmem_ld16(RF + lane_sel + 16 * qt, raw);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int c = 0; c < 16; ++c)
+                            tr[64 * wt + ((16 * qt + c) ^ wt)] = __uint_as_float(raw[c]);
+                    }
+                    half_barrier(wg);
+#pragma unroll
+                    for (int qt = 0; qt < 4; ++qt) {
+                        uint32_t raw[16];
+                        tmem_ld16(RF + lane_sel + 16 * qt, raw);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int c = 0; c < 16; ++c) {
+                            const int cc = 16 * qt + c;
+                            if (cc > wt)
+                                raw[c] = __float_as_uint(tr[64 * cc + (wt ^ cc)]);
+                        }
+                        tmem_st16(RF + lane_sel + 16 * qt, raw);
+                    }
+                    tmem_wait_st();
+                }
                 load_cols(0);
 #pragma unroll 1
                 for (int pnl = 0; pnl < 8; ++pnl) {
@@ -658,11 +595,22 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
                         dead = true;
                         break;
                     }
-                    if (pnl == 7 && issuer) {
+                    if (!GAINS && pnl == 7 && issuer) {
                         // every row has read its last columns of F: (4) DP = W A into the columns of F
+                        // (with gains the columns of F still collect K_t': (4) follows their read-out)
                         tc_fence_after();
                         gemm_ts(RF, RW, smem_u32(BA) + MAT_BYTES, 64);
                     }
+                    // GAINS: rows 0..63 carry X = L^{-T} behind L.  Row r of L ends in its diagonal block; from there on the
+                    // same tensor-memory row (the unused upper triangle of S, which the trailing updates have brought to
+                    // L[r,p] L[c,p]' = what this panel's update removes) is continued as row r of X (X L' = I is the
+                    // substitution the rows of Z' go through): in the diagonal panel the operand row is
+                    // L[r,p] + e_r L_d^{-T}, afterwards it is the row read back from tensor memory, substituted.
+                    // These rows are also rows of the B operand, so the trailing updates keep subtracting
+                    // Z'[n,p] X[r,p]' from column r of the rows of Z' after that column has been consumed (and brought to
+                    // zero by its own panel): when the last panel is done, columns 0..63 of lanes 64..127 hold
+                    // -Z' X' = -Z' L^{-1} = K_t', in the error-compensated arithmetic of the updates.  No backward solve.
+                    float xi[8];                               // diagonal panel: row wt - col of L_d^{-T} (GAINS, warps 0, 1)
                     {
                         float l[8][8], rinv[8];
                         const float4* src = reinterpret_cast<const float4*>(&misc.ld[0]);
@@ -678,28 +626,58 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
                         rinv[0] = c7.x; rinv[1] = c7.y; rinv[2] = c7.z; rinv[3] = c7.w;
                         rinv[4] = c8.x; rinv[5] = c8.y; rinv[6] = c8.z; rinv[7] = c8.w;
                         fsub8(v, l, rinv);
+                        if (GAINS && warp < 2) {
+#pragma unroll
+                            for (int j = 0; j < 8; ++j)
+                                xi[j] = 0.f;
+                            if (warp == (pnl >> 2)) {          // the warp of the diagonal block: row (wt - col) of L_d^{-T}
+#pragma unroll
+                                for (int j = 0; j < 8; ++j)
+                                    xi[j] = (col + j == wt) ? 1.f : 0.f;
+                                fsub8(xi, l, rinv);
+                            }
+                        }
                     }
                     {
                         unsigned char* ph = PH + (uint32_t)(wt >> 3) * PSR + (uint32_t)(wt & 7) * 16u;
                         float hi[8];
                         if (warp < 2) {                        // row wt of L: lower triangular, ends at column wt
                             float lo[8];
+                            if (GAINS) {
+                                const bool done = wt < col;    // finished row: v is its row of L^{-T}
 #pragma unroll
-                            for (int j = 0; j < 8; ++j) {
-                                if (col + j > wt)
-                                    v[j] = 0.f;
-                                hi[j] = round_tf32(v[j]);
-                                lo[j] = v[j] - hi[j];
+                                for (int j = 0; j < 8; ++j)
+                                    if (!done && col + j > wt)
+                                        v[j] = 0.f;
+#pragma unroll
+                                for (int j = 0; j < 8; ++j) {
+                                    const float a = done ? v[j] : v[j] + xi[j];
+                                    hi[j] = round_tf32(a);
+                                    lo[j] = a - hi[j];
+                                }
+                            } else {
+#pragma unroll
+                                for (int j = 0; j < 8; ++j) {
+                                    if (col + j > wt)
+                                        v[j] = 0.f;
+                                    hi[j] = round_tf32(v[j]);
+                                    lo[j] = v[j] - hi[j];
+                                }
                             }
                             unsigned char* pl = PL + (uint32_t)(wt >> 3) * PSR + (uint32_t)(wt & 7) * 16u;
                             *reinterpret_cast<float4*>(pl) = make_float4(lo[0], lo[1], lo[2], lo[3]);
                             *reinterpret_cast<float4*>(pl + SC) = make_float4(lo[4], lo[5], lo[6], lo[7]);
-                            if (keep_l)                        // fp32 copy for the gains / u_0
+                            if (keep_l)                        // fp32 copy for u_0
                                 store_row8<true, false>(X1 + (uint32_t)(wt >> 3) * SR + 2u * pnl * SC, wt & 7, v);
-                        } else {                               // row wt - 64 of Z': kept as tf32 (operand of (5)), low part zero
+                        } else {                               // row wt - 64 of Z': tf32 as operand of (5)
 #pragma unroll
                             for (int j = 0; j < 8; ++j)
                                 hi[j] = round_tf32(v[j]);
+                            if (GAINS) {                       // the gains collect in the updates: keep the low part too
+                                unsigned char* pl = PL + (uint32_t)(wt >> 3) * PSR + (uint32_t)(wt & 7) * 16u;
+                                *reinterpret_cast<float4*>(pl) = make_float4(v[0] - hi[0], v[1] - hi[1], v[2] - hi[2], v[3] - hi[3]);
+                                *reinterpret_cast<float4*>(pl + SC) = make_float4(v[4] - hi[4], v[5] - hi[5], v[6] - hi[6], v[7] - hi[7]);
+                            }
                             unsigned char* pz = X0 + (uint32_t)((wt - 64) >> 3) * SR + 2u * pnl * SC + (uint32_t)(wt & 7) * 16u;
                             *reinterpret_cast<float4*>(pz) = make_float4(hi[0], hi[1], hi[2], hi[3]);
                             *reinterpret_cast<float4*>(pz + SC) = make_float4(hi[4], hi[5], hi[6], hi[7]);
@@ -707,7 +685,7 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
                         *reinterpret_cast<float4*>(ph) = make_float4(hi[0], hi[1], hi[2], hi[3]);
                         *reinterpret_cast<float4*>(ph + SC) = make_float4(hi[4], hi[5], hi[6], hi[7]);
                     }
-                    if (pnl == 7)
+                    if (pnl == 7 && !GAINS)
                         break;
                     async_proxy_fence();
                     wg_barrier(wg);
@@ -721,7 +699,27 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
                         mma_commit(mbar);
                     }
                     wait_mma();
+                    if (pnl == 7)
+                        break;
                     load_cols(col + 8);
+                }
+                if (GAINS && warp >= 2 && !dead && misc.dead == 0) {
+                    // K_t' from the columns of F (lanes 64..127): thread 64 + n holds K_t[:, n]
+                    const int nn = wt - 64;
+                    const long long ko = (inst * (long long)H + ts) * N * N + nn;
+#pragma unroll
+                    for (int qt = 0; qt < 4; ++qt) {
+                        uint32_t raw[16];
+                        tmem_ld16(RF + lane_sel + 16 * qt, raw);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int c = 0; c < 16; ++c) {
+                            const float kv = __uint_as_float(raw[c]);
+                            Kbase[ko + (long long)(16 * qt + c) * N] = kv;
+                            if (obf && p.K)
+                                store_out(p.K, ko + (long long)(16 * qt + c) * N, kv, 1);
+                        }
+                    }
                 }
                 async_proxy_fence();
                 tc_fence_before();
@@ -730,6 +728,8 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
                 // (5) DP -= Z' Z : A operand rows 64..127 = Z' (rows 0..63 = X1, unused lanes)
                 if (issuer && !dead) {
                     tc_fence_after();
+                    if (GAINS)                                 // (4), once K_t' has been read out of the columns of F
+                        gemm_ts(RF, RW, smem_u32(BA) + MAT_BYTES, 64);
                     gemm_ss(RF, smem_u32(X0) - MAT_BYTES, smem_u32(X0), 64, 1, true);
                     mma_commit(mbar);
                 }
@@ -787,31 +787,6 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
                     }
                 }
                 wait_mma();
-                if (need_K_all) {
-                    // (5) has consumed Z': turn it into the gains in place, K_t[i][c] = -(Z' L^{-1})[c][i]
-                    wg_gain_solve(X1, X0, wg, warp, lane);
-                    if (warp < 2) {
-                        const int cidx = wt;
-                        float* kt = Kbase + (inst * (long long)H + ts) * N * N + cidx;
-                        const unsigned char* row = X0 + (uint32_t)(cidx >> 3) * SR + (uint32_t)(cidx & 7) * 16u;
-#pragma unroll
-                        for (int q4 = 0; q4 < 16; ++q4) {
-                            const float4 kv = *reinterpret_cast<const float4*>(row + q4 * SC);
-                            kt[(4 * q4 + 0) * N] = -kv.x;
-                            kt[(4 * q4 + 1) * N] = -kv.y;
-                            kt[(4 * q4 + 2) * N] = -kv.z;
-                            kt[(4 * q4 + 3) * N] = -kv.w;
-                            if (obf && p.K) {
-                                const long long ko = (inst * (long long)H + ts) * N * N + cidx + (long long)(4 * q4) * N;
-                                store_out(p.K, ko, -kv.x, 1);
-                                store_out(p.K, ko + N, -kv.y, 1);
-                                store_out(p.K, ko + 2 * N, -kv.z, 1);
-                                store_out(p.K, ko + 3 * N, -kv.w, 1);
-                            }
-                        }
-                    }
-                    wg_barrier(wg);                   // X0 is free for the next value matrix
-                }
                 // P_t = Q + DP: warps 2, 3 own the rows (lanes 64..127)
                 if (warp >= 2) {
                     const int j = wt - 64;
