@@ -280,65 +280,89 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 2 : 3) scan_step_kernel(S
                 s[l] = (l == c) ? 1.f : 0.f;
         }
         __syncwarp();
-        // The dense loops run over k with four-fold unrolling and take their coefficients from the lane's own column
-        // of a shared-memory matrix (a fully unrolled body would be bound by instruction fetch).
         float y[N];
         f32x2 p2[N / 2];
-        {
-            f32x2 v2[N / 2], t2[N / 2];
-            zero2<N>(v2);
-            zero2<N>(t2);
-#pragma unroll 4
-            for (int i = 0; i < N; ++i) {                      // V[:,c] = P B[:,c], T[:,c] = P A[:,c]
-                const float bic = sl.B[i * LD + c], aic = sl.A[i * LD + c];
-                const f32x2 b2 = rwarp::pack2(bic, bic), a2 = rwarp::pack2(aic, aic);
-                const float* prow = sl.buf0 + i * LD;
+        float pn[N];                                           // tensor-core path: column c of J + A'T
+        // n = 32: the dense products run on the tensor cores (three-pass tf32 mma.sync, rwarp::mma32_product), one copy
+        // of the product code in phases as in riccati_warp_kernel: V = P B -> L, T = P A -> L', B'V -> buf0, Y = B'T -> L,
+        // A'T -> L' (applications only); the last phase factorises, substitutes and, for an application, runs Z'Z -> L.
+        constexpr bool MMA = (N == 32);
+        constexpr int LAST = GAIN ? 4 : 5;
+#pragma unroll 1
+        for (int ph = MMA ? 0 : LAST; ph <= LAST; ++ph) {
+        if (!MMA || ph == LAST) {
+        if constexpr (MMA) {
+            float tmp[N];
+            load_row<N>(tmp, sl.buf0 + c * LD);                // (B'V)[c,:] = (B'V)[:,c]
 #pragma unroll
-                for (int q4 = 0; q4 < N / 4; ++q4) {
-                    const ulonglong2 t4 = *reinterpret_cast<const ulonglong2*>(prow + 4 * q4);
-                    rwarp::fma2(v2[2 * q4], t4.x, b2);
-                    rwarp::fma2(v2[2 * q4 + 1], t4.y, b2);
-                    rwarp::fma2(t2[2 * q4], t4.x, a2);
-                    rwarp::fma2(t2[2 * q4 + 1], t4.y, a2);
-                }
+            for (int l = 0; l < N; ++l) {
+                s[l] += tmp[l];
+                y[l] = sl.L[l * LD + c];
             }
-            float v[N], t[N];
-            unpack_row<N>(v, v2);
-            unpack_row<N>(t, t2);
-            store_col<N>(sl.L, c, v);                          // own column only: no exchange
-            store_col<N>(sl.Lt, c, t);
-        }
-        {
-            f32x2 s2[N / 2], y2[N / 2];
-            pack_row<N>(s2, s);
-            zero2<N>(y2);
             if (!GAIN) {
-                float jc[N];
 #pragma unroll
                 for (int l = 0; l < N; ++l)
-                    jc[l] = __ldg(E + 3 * N * N + c * N + l);  // row c of J = column c
-                pack_row<N>(p2, jc);
+                    pn[l] = __ldg(E + 3 * N * N + c * N + l) + sl.Lt[l * LD + c];
             }
+        } else {
+            // The dense loops run over k with four-fold unrolling and take their coefficients from the lane's own column
+            // of a shared-memory matrix (a fully unrolled body would be bound by instruction fetch).
+            {
+                f32x2 v2[N / 2], t2[N / 2];
+                zero2<N>(v2);
+                zero2<N>(t2);
 #pragma unroll 4
-            for (int k = 0; k < N; ++k) {                      // S += B'V, Y = B'T, Pn = J + A'T: each row read once
-                const float vk = sl.L[k * LD + c], tk = sl.Lt[k * LD + c];
-                const f32x2 vv = rwarp::pack2(vk, vk), tt = rwarp::pack2(tk, tk);
+                for (int i = 0; i < N; ++i) {                      // V[:,c] = P B[:,c], T[:,c] = P A[:,c]
+                    const float bic = sl.B[i * LD + c], aic = sl.A[i * LD + c];
+                    const f32x2 b2 = rwarp::pack2(bic, bic), a2 = rwarp::pack2(aic, aic);
+                    const float* prow = sl.buf0 + i * LD;
 #pragma unroll
-                for (int q4 = 0; q4 < N / 4; ++q4) {
-                    const ulonglong2 b4 = *reinterpret_cast<const ulonglong2*>(sl.B + k * LD + 4 * q4);
-                    rwarp::fma2(s2[2 * q4], vv, b4.x);
-                    rwarp::fma2(s2[2 * q4 + 1], vv, b4.y);
-                    rwarp::fma2(y2[2 * q4], tt, b4.x);
-                    rwarp::fma2(y2[2 * q4 + 1], tt, b4.y);
-                    if (!GAIN) {
-                        const ulonglong2 a4 = *reinterpret_cast<const ulonglong2*>(sl.A + k * LD + 4 * q4);
-                        rwarp::fma2(p2[2 * q4], tt, a4.x);
-                        rwarp::fma2(p2[2 * q4 + 1], tt, a4.y);
+                    for (int q4 = 0; q4 < N / 4; ++q4) {
+                        const ulonglong2 t4 = *reinterpret_cast<const ulonglong2*>(prow + 4 * q4);
+                        rwarp::fma2(v2[2 * q4], t4.x, b2);
+                        rwarp::fma2(v2[2 * q4 + 1], t4.y, b2);
+                        rwarp::fma2(t2[2 * q4], t4.x, a2);
+                        rwarp::fma2(t2[2 * q4 + 1], t4.y, a2);
                     }
                 }
+                float v[N], t[N];
+                unpack_row<N>(v, v2);
+                unpack_row<N>(t, t2);
+                store_col<N>(sl.L, c, v);                          // own column only: no exchange
+                store_col<N>(sl.Lt, c, t);
             }
-            unpack_row<N>(s, s2);
-            unpack_row<N>(y, y2);
+            {
+                f32x2 s2[N / 2], y2[N / 2];
+                pack_row<N>(s2, s);
+                zero2<N>(y2);
+                if (!GAIN) {
+                    float jc[N];
+#pragma unroll
+                    for (int l = 0; l < N; ++l)
+                        jc[l] = __ldg(E + 3 * N * N + c * N + l);  // row c of J = column c
+                    pack_row<N>(p2, jc);
+                }
+#pragma unroll 4
+                for (int k = 0; k < N; ++k) {                      // S += B'V, Y = B'T, Pn = J + A'T: each row read once
+                    const float vk = sl.L[k * LD + c], tk = sl.Lt[k * LD + c];
+                    const f32x2 vv = rwarp::pack2(vk, vk), tt = rwarp::pack2(tk, tk);
+#pragma unroll
+                    for (int q4 = 0; q4 < N / 4; ++q4) {
+                        const ulonglong2 b4 = *reinterpret_cast<const ulonglong2*>(sl.B + k * LD + 4 * q4);
+                        rwarp::fma2(s2[2 * q4], vv, b4.x);
+                        rwarp::fma2(s2[2 * q4 + 1], vv, b4.y);
+                        rwarp::fma2(y2[2 * q4], tt, b4.x);
+                        rwarp::fma2(y2[2 * q4 + 1], tt, b4.y);
+                        if (!GAIN) {
+                            const ulonglong2 a4 = *reinterpret_cast<const ulonglong2*>(sl.A + k * LD + 4 * q4);
+                            rwarp::fma2(p2[2 * q4], tt, a4.x);
+                            rwarp::fma2(p2[2 * q4 + 1], tt, a4.y);
+                        }
+                    }
+                }
+                unpack_row<N>(s, s2);
+                unpack_row<N>(y, y2);
+            }
         }
         float rs_own;
         const int bad = rwarp::seg_chol<N>(s, rs_own, c);
@@ -366,11 +390,22 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 2 : 3) scan_step_kernel(S
         } else {
             store_col<N>(sl.buf0, c, y);                       // rows of Z
             __syncwarp();
-#pragma unroll 4
-            for (int k = 0; k < N; ++k)                        // Pn[:,c] -= Z'Z[:,c]
-                axpy_row<N>(p2, -sl.buf0[k * LD + c], sl.buf0 + k * LD);
             float pcol[N];
-            unpack_row<N>(pcol, p2);
+            if constexpr (MMA) {
+                float acc[2][4][4];
+                rwarp::mma32_zero(acc);
+                rwarp::mma32_product(acc, sl.buf0, sl.buf0, lane);
+                rwarp::mma32_store(sl.L, acc, lane);           // nobody reads the rows of L in this form
+                __syncwarp();
+#pragma unroll
+                for (int l = 0; l < N; ++l)
+                    pcol[l] = pn[l] - sl.L[l * LD + c];        // Pn[:,c] - Z'Z[:,c]
+            } else {
+#pragma unroll 4
+                for (int k = 0; k < N; ++k)                    // Pn[:,c] -= Z'Z[:,c]
+                    axpy_row<N>(p2, -sl.buf0[k * LD + c], sl.buf0 + k * LD);
+                unpack_row<N>(pcol, p2);
+            }
             __syncwarp();
             store_row<N>(sl.buf0 + c * LD, pcol);              // column c as row c, then average with the transpose
             __syncwarp();
@@ -384,6 +419,22 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 2 : 3) scan_step_kernel(S
                     dst[l4] = make_float4(pcol[4 * l4], pcol[4 * l4 + 1], pcol[4 * l4 + 2], pcol[4 * l4 + 3]);
             }
         }
+        } else if constexpr (MMA) {
+            // phase:  0      1      2      3      4
+            // A'   :  P      P      B'     B'     A'          (P symmetric, so P B = P'B)
+            // B    :  B      A      V      T      T
+            // to   :  L      L'     buf0   L      L'          (buf0: P, then B'V)
+            const float* Am = ph < 2 ? sl.buf0 : ph == 4 ? sl.A : sl.B;
+            const float* Bm = ph == 0 ? sl.B : ph == 1 ? sl.A : ph == 2 ? sl.L : sl.Lt;
+            float* Dm = ph == 1 || ph == 4 ? sl.Lt : ph == 2 ? sl.buf0 : sl.L;
+            float acc[2][4][4];
+            rwarp::mma32_zero(acc);
+            rwarp::mma32_product(acc, Am, Bm, lane);
+            __syncwarp();                                      // every lane has read what the result overwrites
+            rwarp::mma32_store(Dm, acc, lane);
+            __syncwarp();
+        }
+        }                                                      // phases
     }
 }
 
