@@ -338,7 +338,9 @@ int ttc_lqr_solve_layer_sigma_baseline(ttc_lqr_handle* h, const ttc_layer_inputs
  * (pinned memory lets the copies run at full speed; pageable memory works).  The call copies the
  * inputs to a device staging buffer owned by the handle, runs the same kernel on an internal
  * stream, copies the requested outputs back and returns after everything has completed
- * (synchronous).  No alignment requirement on host pointers.  Results are identical to
+ * (synchronous).  Large batches are cut into up to 32 slices of the instance dimension so that
+ * the copy-in of one slice, the solve of the previous one and the copy-out of the one before
+ * overlap.  No alignment requirement on host pointers.  Results are identical to
  * ttc_lqr_solve_layer.
  */
 int ttc_lqr_solve_layer_host(ttc_lqr_handle* h, const ttc_layer_inputs* in, int32_t T,

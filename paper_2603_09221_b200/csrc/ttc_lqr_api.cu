@@ -780,8 +780,9 @@ static int check_layer_call(ttc_lqr_handle* h, const ttc_layer_inputs* in, int32
 }
 
 // all pointers are device memory here
+// Instances [i0, i0 + cnt) of the handle's batch (the arrays are instance-major, the bases shared).
 static int launch_layer(ttc_lqr_handle* h, const ttc_layer_inputs* in, int32_t T, float* u1, float* P0, int32_t* info,
-                        cudaStream_t st)
+                        cudaStream_t st, long long i0 = 0, long long cnt = -1)
 {
     const int n = h->cfg.n;
     int s;
@@ -789,14 +790,15 @@ static int launch_layer(ttc_lqr_handle* h, const ttc_layer_inputs* in, int32_t T
     int* counter = static_cast<int*>(h->ws_E.ptr);
     TTC_CUDA(cudaMemsetAsync(counter, 0, sizeof(int), st));
     layer::LayerParams p;
-    p.N = h->N;
+    p.N = cnt < 0 ? h->N : cnt;
     p.T = T;
     p.r = in->r;
-    p.s_a = in->s_a; p.s_ga = in->s_gamma_a; p.s_gb = in->s_gamma_b; p.s_gq = in->s_gamma_q;
-    p.s_b = in->s_b; p.s_q = in->s_q; p.s_qf = in->s_qf;
-    p.r_inv = in->r_inv; p.h0 = in->h0;
+    const long long on = i0 * n, orr = i0 * in->r;
+    p.s_a = in->s_a + on; p.s_ga = in->s_gamma_a + on; p.s_gb = in->s_gamma_b + on; p.s_gq = in->s_gamma_q + on;
+    p.s_b = in->s_b + orr; p.s_q = in->s_q + orr; p.s_qf = in->s_qf + orr;
+    p.r_inv = in->r_inv + on; p.h0 = in->h0 + on;
     p.B_basis = in->B_basis; p.Q_basis = in->Q_basis;
-    p.u1 = u1; p.P0 = P0; p.info = info;
+    p.u1 = u1 ? u1 + on : nullptr; p.P0 = P0 ? P0 + on * n : nullptr; p.info = info ? info + i0 : nullptr;
     p.Kws = nullptr; p.Pws = nullptr; p.g = nullptr; p.k0 = nullptr;
     void (*kern)(layer::LayerParams, int*);
     size_t smem;
@@ -1005,30 +1007,61 @@ int ttc_lqr_solve_layer_host(ttc_lqr_handle* h, const ttc_layer_inputs* in, int3
         return s;
     cudaStream_t st = h->host_stream;
     unsigned char* base = static_cast<unsigned char*>(h->st_layer.ptr);
-    const float* dptr[11];
+    unsigned char* dptr[11];
     size_t off = 0;
     for (int i = 0; i < 11; ++i) {
-        dptr[i] = reinterpret_cast<const float*>(base + off);
-        TTC_CUDA(cudaMemcpyAsync(base + off, src[i], in_bytes[i], cudaMemcpyHostToDevice, st));
+        dptr[i] = base + off;
         off += pad(in_bytes[i]);
     }
-    void* dev_out[3] = {nullptr, nullptr, nullptr};
+    unsigned char* dev_out[3] = {nullptr, nullptr, nullptr};
     for (int i = 0; i < 3; ++i)
         if (host_out[i]) {
             dev_out[i] = base + off;
             off += pad(out_bytes[i]);
         }
     ttc_layer_inputs din = *in;
-    din.s_a = dptr[0]; din.s_gamma_a = dptr[1]; din.s_gamma_b = dptr[2]; din.s_gamma_q = dptr[3];
-    din.s_b = dptr[4]; din.s_q = dptr[5]; din.s_qf = dptr[6]; din.r_inv = dptr[7]; din.h0 = dptr[8];
-    din.B_basis = dptr[9]; din.Q_basis = dptr[10];
-    if ((s = launch_layer(h, &din, T, static_cast<float*>(dev_out[0]), static_cast<float*>(dev_out[1]),
-                          static_cast<int32_t*>(dev_out[2]), st)))
-        return s;
-    for (int i = 0; i < 3; ++i)
-        if (host_out[i])
-            TTC_CUDA(cudaMemcpyAsync(host_out[i], dev_out[i], out_bytes[i], cudaMemcpyDeviceToHost, st));
+    din.s_a = reinterpret_cast<const float*>(dptr[0]); din.s_gamma_a = reinterpret_cast<const float*>(dptr[1]);
+    din.s_gamma_b = reinterpret_cast<const float*>(dptr[2]); din.s_gamma_q = reinterpret_cast<const float*>(dptr[3]);
+    din.s_b = reinterpret_cast<const float*>(dptr[4]); din.s_q = reinterpret_cast<const float*>(dptr[5]);
+    din.s_qf = reinterpret_cast<const float*>(dptr[6]); din.r_inv = reinterpret_cast<const float*>(dptr[7]);
+    din.h0 = reinterpret_cast<const float*>(dptr[8]);
+    din.B_basis = reinterpret_cast<const float*>(dptr[9]); din.Q_basis = reinterpret_cast<const float*>(dptr[10]);
+
+    // Slices of the instance dimension: copy in, solve and copy out overlap across slices (as in ttc_lqr_solve_host).
+    // The bases are shared and go first.
+    int nslice = 1;
+    if (total >= ((size_t)16 << 20) && N >= 8192)
+        nslice = (int)(N / 4096 < (size_t)kMaxSlices ? N / 4096 : (size_t)kMaxSlices);
+    size_t per = (N + nslice - 1) / nslice;
+    per = (per + 63) / 64 * 64;
+    nslice = (int)((N + per - 1) / per);
+    const size_t per_inst_in[9] = {4 * n, 4 * n, 4 * n, 4 * n, 4 * r, 4 * r, 4 * r, 4 * n, 4 * n};
+    const size_t per_inst_out[3] = {4 * n, 4 * n * n, 4};
+    for (int i = 9; i < 11; ++i)
+        TTC_CUDA(cudaMemcpyAsync(dptr[i], src[i], in_bytes[i], cudaMemcpyHostToDevice, h->in_stream));
+    for (int c = 0; c < nslice; ++c) {
+        const size_t i0 = (size_t)c * per, cnt = (N - i0 < per) ? N - i0 : per;
+        for (int i = 0; i < 9; ++i)
+            TTC_CUDA(cudaMemcpyAsync(dptr[i] + i0 * per_inst_in[i], static_cast<const unsigned char*>(src[i]) + i0 * per_inst_in[i],
+                                     cnt * per_inst_in[i], cudaMemcpyHostToDevice, h->in_stream));
+        TTC_CUDA(cudaEventRecord(h->ev_in[c], h->in_stream));
+        TTC_CUDA(cudaStreamWaitEvent(st, h->ev_in[c], 0));
+        if ((s = launch_layer(h, &din, T, reinterpret_cast<float*>(dev_out[0]), reinterpret_cast<float*>(dev_out[1]),
+                              reinterpret_cast<int32_t*>(dev_out[2]), st, (long long)i0, (long long)cnt))) {
+            cudaDeviceSynchronize();
+            return s;
+        }
+        TTC_CUDA(cudaEventRecord(h->ev_done[c], st));
+        TTC_CUDA(cudaStreamWaitEvent(h->out_stream, h->ev_done[c], 0));
+        for (int i = 0; i < 3; ++i)
+            if (host_out[i])
+                TTC_CUDA(cudaMemcpyAsync(static_cast<unsigned char*>(host_out[i]) + i0 * per_inst_out[i],
+                                         dev_out[i] + i0 * per_inst_out[i], cnt * per_inst_out[i], cudaMemcpyDeviceToHost,
+                                         h->out_stream));
+    }
+    TTC_CUDA(cudaStreamSynchronize(h->out_stream));
     TTC_CUDA(cudaStreamSynchronize(st));
+    TTC_CUDA(cudaStreamSynchronize(h->in_stream));
     return TTC_OK;
 }
 

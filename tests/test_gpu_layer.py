@@ -115,6 +115,24 @@ def test_layer_full_size_on_sampled_instances():
     assert float((Ps - Ps.transpose(-1, -2)).abs().max() / Ps.abs().max()) < 1e-5
 
 
+def test_host_buffer_entry_point_pipelined_slices():
+    """Enough instances for the host-buffer entry point to cut the batch into slices whose copies and solves overlap
+    (ragged last slice): bit-equal to the device entry point, every output element written."""
+    w = workloads.make_layer_workload("layer16", device=DEV, batch=(1, 5, 4001), seed=13)
+    T, n, N = 6, w["n"], w["N"]
+    u_d, P_d, info_d = run_gpu(w, T)
+    s = lqr.LqrSolver(n, n, T, w["batch"])
+    hin = [w[k].cpu().pin_memory() for k in workloads.LAYER_KEYS]
+    u_h = torch.full((N, n), 7.0).pin_memory()
+    P_h = torch.full((N, n, n), 7.0).pin_memory()
+    info_h = torch.full((N,), -3, dtype=torch.int32).pin_memory()
+    for _ in range(2):                                     # the staging buffers and events are reused
+        s.solve_layer_host(*hin, T, u1=u_h, P0=P_h, info=info_h)
+        assert s.query(lqr.TTC_QUERY_LAST_LAUNCHES) > 1, "expected more than one slice"
+        assert torch.equal(u_h, u_d.cpu()) and torch.equal(P_h, P_d.cpu()) and torch.equal(info_h, info_d.cpu())
+    s.close()
+
+
 def test_layer_rejects_unsupported_shapes():
     s = lqr.LqrSolver(8, 8, 4, (1, 1, 4))
     w = workloads.make_layer_workload("layer16", device=DEV, batch=(1, 1, 4))
