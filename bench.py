@@ -629,8 +629,9 @@ def run_solve(args, workload, method_name, ctx, light=False):
     lowrank = args.lowrank_q and "U" in w and not light
     out = lqr.alloc_outputs(n, m, H, N, dev, first_only=first, want=want, dtype=torch.bfloat16 if obf else torch.float32)
     flags = (lqr.TTC_OUT_FIRST_ONLY if first else 0) | (lqr.TTC_OUT_BF16 if obf else 0)
+    if lowrank:
+        no_e2e = True                      # the host-buffer entry point takes dense Q
     if obf or lowrank:
-        no_e2e = True                      # the host-buffer entry point takes dense Q and returns float32
         c["name"] += ("_outbf16" if obf else "") + ("_lowrankq" if lowrank else "")
 
     def step():
@@ -688,7 +689,8 @@ def run_solve(args, workload, method_name, ctx, light=False):
     e2e = None
     if not no_e2e:
         hin = {k: w[k].cpu().pin_memory() for k in ("A", "B", "Q", "R", "x0")}
-        hout = lqr.alloc_outputs(n, m, H, N, "cpu", first_only=first, want=want, pin=True)
+        hout = lqr.alloc_outputs(n, m, H, N, "cpu", first_only=first, want=want, pin=True,
+                                 dtype=torch.bfloat16 if obf else torch.float32)
         h2d = sum(v.numel() * v.element_size() for v in hin.values())
         d2h = sum(v.numel() * v.element_size() for v in hout.values())
 

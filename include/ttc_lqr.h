@@ -354,7 +354,8 @@ int ttc_lqr_solve_layer_host(ttc_lqr_handle* h, const ttc_layer_inputs* in, int3
  * and returns after everything has completed (synchronous).  Large problems are cut into up to
  * 32 slices of the last batch dimension so that the copy-in of one slice, the solve of the
  * previous one and the copy-out of the one before overlap; results are identical to
- * ttc_lqr_solve.  Strides have the same meaning.
+ * ttc_lqr_solve.  Strides have the same meaning.  Flags as for ttc_lqr_solve: with TTC_OUT_BF16
+ * K, P, x, u are bfloat16 host arrays, which halves the bytes copied back.
  */
 int ttc_lqr_solve_host(ttc_lqr_handle* h,
                        const ttc_operand* A, const ttc_operand* B, const ttc_operand* Q,

@@ -3,6 +3,7 @@
 // convenience entry point.  No torch types, no CPU fallback: without a CUDA device of
 // compute capability 10.x every call fails with TTC_STATUS_CUDA_ERROR.
 #include <cstdarg>
+#include <cmath>
 #include <cstdio>
 #include <cstring>
 #include <mutex>
@@ -1074,9 +1075,7 @@ int ttc_lqr_solve_host(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operan
     // alignment of host pointers is irrelevant; validate the rest through a relaxed copy
     if (H < 1 || H > h->cfg.max_horizon)
         return fail(TTC_STATUS_INVALID_ARGUMENT, "H=%d outside [1, max_horizon=%d]", H, h->cfg.max_horizon);
-    if (flags & TTC_OUT_BF16)
-        return fail(TTC_STATUS_UNSUPPORTED, "the host-buffer entry point returns float32 outputs");
-    if (flags & ~TTC_OUT_FIRST_ONLY)
+    if (flags & ~(TTC_OUT_FIRST_ONLY | TTC_OUT_BF16))
         return fail(TTC_STATUS_INVALID_ARGUMENT, "unknown flag bits 0x%x", flags);
     TTC_CUDA(cudaSetDevice(h->cfg.device));
     { int sp = ensure_host_pipeline(h); if (sp) return sp; }
@@ -1111,9 +1110,10 @@ int ttc_lqr_solve_host(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operan
         dev[i].ptr = h->st_in[i].ptr;
     }
     void* host_out[5] = {K, P, x, u, info};
+    const size_t esz = (flags & TTC_OUT_BF16) ? 2 : sizeof(float);     // K, P, x, u as bfloat16 halve the copy-out
     const size_t per_out[5] = {                        // bytes per instance
-        sizeof(float) * (size_t)H * m * n, sizeof(float) * (size_t)(first ? 1 : H + 1) * n * n,
-        sizeof(float) * (size_t)(H + 1) * n, sizeof(float) * (size_t)(first ? 1 : H) * m, sizeof(int32_t)};
+        esz * (size_t)H * m * n, esz * (size_t)(first ? 1 : H + 1) * n * n,
+        esz * (size_t)(H + 1) * n, esz * (size_t)(first ? 1 : H) * m, sizeof(int32_t)};
     void* dev_out[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
     size_t total_bytes = 0;
     for (int i = 0; i < 5; ++i) {
@@ -1140,6 +1140,35 @@ int ttc_lqr_solve_host(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operan
     }
     long long tslice = (b2 + nslice - 1) / nslice;
     tslice = (tslice + 15) / 16 * 16;
+    // few bytes per instance and step: the solve, not the link, sets the pace (a problem bound by its copies is better
+    // off with the shortest slices, whose first copy-in and last copy-out are all that stays exposed)
+    const bool solve_bound = (double)total_bytes < 64.0 * n * (double)N * H;
+    if (nslice > 1 && solve_bound && n == m && (n == 16 || n == 32 || n == 64)) {
+        // The kernels behind these shapes run a persistent grid over work items of a few tokens of one head.  A slice
+        // whose items do not fill a whole number of rounds of that grid leaves SMs idle in its last round (a slice
+        // of 128 tokens x 32 heads is 128 items for 148 CTAs of the n = 64 kernel), so prefer the slice length that
+        // fills its rounds best, among those that are at least 128 tokens and keep the slice count within the limit.
+        const int item_tokens = n == 64 ? 32 : n == 32 ? 4 : 8;
+        const long long grid = (long long)h->sm_count * (n == 64 ? 1 : n == 32 ? 3 : 4);
+        const double round_tokens = (double)(grid * item_tokens) / (double)(b0 * b1);      // tokens per head in one round
+        auto fill = [&](long long t) {
+            const double rounds = std::ceil((double)((t + item_tokens - 1) / item_tokens * item_tokens) / round_tokens - 1e-9);
+            return (double)t / (rounds * round_tokens);
+        };
+        long long best = tslice;
+        double best_fill = fill(tslice);
+        for (int j = 1; j <= 8; ++j) {
+            const long long step = item_tokens > 16 ? item_tokens : 16;
+            const long long t = (long long)(j * round_tokens) / step * step;
+            if (t < 128 || t >= b2 || (b2 + t - 1) / t > kMaxSlices)
+                continue;
+            if (fill(t) > best_fill + 0.03) {
+                best = t;
+                best_fill = fill(t);
+            }
+        }
+        tslice = best;
+    }
     nslice = (int)((b2 + tslice - 1) / tslice);
 
     h->last_launches = 0;

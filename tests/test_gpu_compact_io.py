@@ -90,3 +90,26 @@ def test_low_rank_plus_diagonal_state_cost(n, rank, H, batch, bf16):
     f64 = lambda t: t.double().cpu().numpy()
     ref = orc.solve_batch(f64(w["A"]), f64(w["B"]), Q64, f64(w["R"]), f64(w["x0"]), H, batch=batch)
     pu.compare(out, ref, np.arange(N), w["tol"])
+
+
+@pytest.mark.parametrize("n,H,batch,bf16_in,first_only", [(32, 6, (1, 2, 9), False, True), (64, 4, (1, 2, 512), True, False)])
+def test_host_buffer_entry_point_with_bfloat16_outputs(n, H, batch, bf16_in, first_only):
+    """TTC_OUT_BF16 through ttc_lqr_solve_host (one slice, and the sliced pipeline at n = 64): the host arrays hold
+    bfloat16 and equal the device entry point's bfloat16 outputs bit for bit."""
+    w = small_workload(n, n, H, batch, seed=400 + n, bf16=bf16_in)
+    N = int(np.prod(batch))
+    want = ("P", "u", "info") if first_only else ("K", "P", "x", "u", "info")
+    dev = solve(w, H, first_only, want, torch.bfloat16)
+    s = lqr.LqrSolver(n, n, H, batch)
+    host = {k: w[k].cpu().pin_memory() for k in ("A", "B", "Q", "R", "x0")}
+    out = lqr.alloc_outputs(n, n, H, N, "cpu", first_only=first_only, want=want, pin=True, dtype=torch.bfloat16)
+    for k, v in out.items():
+        v.fill_(-7 if k == "info" else 12345.0)
+    flags = (lqr.TTC_OUT_FIRST_ONLY if first_only else 0) | lqr.TTC_OUT_BF16
+    s.solve_host(host["A"], host["B"], host["Q"], host["R"], host["x0"], H, K=out.get("K"), P=out.get("P"), x=out.get("x"),
+                 u=out.get("u"), info=out.get("info"), flags=flags)
+    if n == 64:
+        assert s.query(lqr.TTC_QUERY_LAST_LAUNCHES) > 1, "expected more than one slice"
+    s.close()
+    for k in want:
+        assert torch.equal(out[k], dev[k].cpu()), k
