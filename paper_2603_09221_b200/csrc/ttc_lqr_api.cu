@@ -1143,6 +1143,7 @@ int ttc_lqr_solve_host(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operan
     // few bytes per instance and step: the solve, not the link, sets the pace (a problem bound by its copies is better
     // off with the shortest slices, whose first copy-in and last copy-out are all that stays exposed)
     const bool solve_bound = (double)total_bytes < 64.0 * n * (double)N * H;
+    long long edge = 0;                                // tokens of one round of the grid (0: unknown)
     if (nslice > 1 && solve_bound && n == m && (n == 16 || n == 32 || n == 64)) {
         // The kernels behind these shapes run a persistent grid over work items of a few tokens of one head.  A slice
         // whose items do not fill a whole number of rounds of that grid leaves SMs idle in its last round (a slice
@@ -1168,8 +1169,27 @@ int ttc_lqr_solve_host(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operan
             }
         }
         tslice = best;
+        const long long step = item_tokens > 16 ? item_tokens : 16;
+        edge = (long long)round_tokens / step * step;
     }
     nslice = (int)((b2 + tslice - 1) / tslice);
+    // slice boundaries; a solve-bound pipeline starts and ends with a short slice (one round of the grid, 128 tokens
+    // at least): the first copy-in and the last copy-out are the only copies that nothing overlaps
+    long long cut[kMaxSlices + 1];
+    for (int c = 0; c <= nslice; ++c)
+        cut[c] = (c * tslice < b2) ? c * tslice : b2;
+    if (nslice > 2 && edge >= 128 && tslice >= 2 * edge) {
+        const long long mid = b2 - 2 * edge;
+        const int nmid = (int)((mid + tslice - 1) / tslice);
+        if (mid > 0 && nmid + 2 <= kMaxSlices) {
+            nslice = nmid + 2;
+            cut[0] = 0;
+            for (int c = 0; c < nmid; ++c)
+                cut[c + 1] = edge + c * tslice;
+            cut[nmid + 1] = b2 - edge;
+            cut[nmid + 2] = b2;
+        }
+    }
 
     h->last_launches = 0;
     { int se = clear_device_error(h, h->host_stream); if (se) return se; }
@@ -1177,7 +1197,7 @@ int ttc_lqr_solve_host(ttc_lqr_handle* h, const ttc_operand* A, const ttc_operan
         if (dev[i].ptr && (nslice == 1 || in[i]->bstride[2] == 0))
             TTC_CUDA(cudaMemcpyAsync(h->st_in[i].ptr, in[i]->ptr, in_bytes[i], cudaMemcpyHostToDevice, h->in_stream));
     for (int c = 0; c < nslice; ++c) {
-        const long long t0 = c * tslice, tc = (b2 - t0 < tslice) ? b2 - t0 : tslice;
+        const long long t0 = cut[c], tc = cut[c + 1] - cut[c];
         if (nslice > 1)
             for (int i = 0; i < 5; ++i) {
                 if (!dev[i].ptr || in[i]->bstride[2] == 0)
