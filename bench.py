@@ -336,10 +336,11 @@ def run_grad(args):
 
 def layer_counts(c):
     """Per-instance algorithmic flops and HBM bytes of the contextualised layer solve: per step P Bbar (2 n^3),
-    Bbar'V (n^3, S symmetric), Bbar'T (2 n^3), Cholesky (n^3 / 3), L^{-1}Y (n^3), Z'Z (n^3, symmetric); per
-    instance the synthesis of Bbar, Qbar, Q_T (6 r n^2).  Bytes: coefficient vectors in, u_1* and P_0 out."""
+    Bbar'V (n^3, S symmetric), Cholesky (n^3 / 3), L^{-1}Y (n^3), Z'Z (n^3, symmetric); Y = G Bbar'P A_t is the
+    transpose of P Bbar scaled on both sides (A_t diagonal) and costs no contraction; per instance the synthesis of
+    Bbar, Qbar, Q_T (6 r n^2).  Bytes: coefficient vectors in, u_1* and P_0 out."""
     n, r, T = c["n"], c["r"], c["T"]
-    flops = (7.0 + 1.0 / 3.0) * n**3 * T + 6.0 * r * n * n
+    flops = (5.0 + 1.0 / 3.0) * n**3 * T + 6.0 * r * n * n
     return flops, 4 * (6 * n + 3 * r), 4 * (n + n * n)
 
 

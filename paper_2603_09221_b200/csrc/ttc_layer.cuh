@@ -171,38 +171,26 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) ttc_layer_kernel(L
                     const float bic = sl.Bb[i * LD + c];
                     axpy_row<N>(vcol, bic, sl.buf0 + i * LD);
                 }
-                // stage V[:,c] = g_c (P Bbar[:,c]) and T[:,c] = a_c P[:,c] (own column only) so that the next loop can
-                // run over k without indexing registers dynamically
+                // stage V[:,c] = g_c (P Bbar[:,c]) so that the next loop can run over k without indexing registers
+                // dynamically.  With a diagonal A_t, Y = G Bbar'P A_t is the transpose of V scaled by a_c: column c of Y
+                // is row c of the staged matrix, and the contraction Bbar'T is not needed.
 #pragma unroll
                 for (int k = 0; k < N / 2; ++k) {
                     float v0, v1;
                     unpack2(vcol[k], v0, v1);
                     sl.L[(2 * k) * LD + c] = g_c * v0;
                     sl.L[(2 * k + 1) * LD + c] = g_c * v1;
-                    sl.Lt[(2 * k) * LD + c] = at_c * pcol[2 * k];
-                    sl.Lt[(2 * k + 1) * LD + c] = at_c * pcol[2 * k + 1];
                 }
-                f32x2 s2[N / 2], y2[N / 2];
+                __syncwarp();
+                f32x2 s2[N / 2];
 #pragma unroll
-                for (int l = 0; l < N / 2; ++l) {
+                for (int l = 0; l < N / 2; ++l)
                     s2[l] = 0ull;
-                    y2[l] = 0ull;
-                }
 #pragma unroll 4
-                for (int k = 0; k < N; ++k) {                     // Bbar' V[:,c] and Bbar' T[:,c]: each row of Bbar read once
-                    const float vk = sl.L[k * LD + c], tk = sl.Lt[k * LD + c];
-                    const f32x2 vv = pack2(vk, vk), t2 = pack2(tk, tk);
-#pragma unroll
-                    for (int q = 0; q < N / 4; ++q) {
-                        const ulonglong2 b4 = *reinterpret_cast<const ulonglong2*>(sl.Bb + k * LD + 4 * q);
-                        fma2(s2[2 * q], vv, b4.x);
-                        fma2(s2[2 * q + 1], vv, b4.y);
-                        fma2(y2[2 * q], t2, b4.x);
-                        fma2(y2[2 * q + 1], t2, b4.y);
-                    }
-                }
+                for (int k = 0; k < N; ++k)                       // Bbar' V[:,c]
+                    axpy_row<N>(s2, sl.L[k * LD + c], sl.Bb + k * LD);
                 unpack_row<N>(sv, s2);
-                unpack_row<N>(y, y2);
+                load_row<N>(y, sl.L + c * LD);                    // g_l (Bbar'P)[l][c]
                 {
                     float gv[N], av[N], qv[N];
                     load_row<N>(gv, sl.gb);
@@ -211,7 +199,7 @@ __global__ void __launch_bounds__(THREADS, (N == 32) ? 3 : 4) ttc_layer_kernel(L
 #pragma unroll
                     for (int l = 0; l < N; ++l) {
                         sv[l] *= gv[l];
-                        y[l] *= gv[l];
+                        y[l] *= at_c;
                         // Pn[l][c] = q_l Qbar[l][c] q_c + a_l a_c P[l][c]
                         pn[l] = fmaf(q_c * qv[l], qcol[l], av[l] * at_c * pcol[l]);
                         if (l == c)
@@ -542,15 +530,21 @@ __global__ void __launch_bounds__(THREADS, 2) ttc_layer_kernel_c2(LayerParams p,
                 unpack_row<N>(v0, a0);
                 unpack_row<N>(v1, a1);
             }
-            f32x2 s20[N / 2], s21[N / 2], y20[N / 2], y21[N / 2];
+            // V[:, c] = g_c (P Bbar)[:, c] goes to the rows of L (free until the factor is published): with a diagonal A_t,
+            // Y = G Bbar'P A_t is the transpose of V scaled by a_c, so column c of Y is row c of that buffer and the
+            // contraction Bbar'T is not needed
+#pragma unroll
+            for (int k = 0; k < N; ++k)
+                *reinterpret_cast<float2*>(sl.L + k * LD + c0) = make_float2(g0 * v0[k], g1 * v1[k]);
+            __syncwarp();
+            f32x2 s20[N / 2], s21[N / 2];
 #pragma unroll
             for (int l = 0; l < N / 2; ++l)
-                s20[l] = s21[l] = y20[l] = y21[l] = 0ull;
-            // fully unrolled: V[k][c] = g_c v[k] and T[k][c] = a_c P[k][c] come straight from registers
+                s20[l] = s21[l] = 0ull;
+            // fully unrolled: V[k][c] = g_c v[k] comes straight from registers
 #pragma unroll
-            for (int k = 0; k < N; ++k) {                     // Bbar' V and Bbar' T for both columns: each row of Bbar read once
+            for (int k = 0; k < N; ++k) {                     // Bbar' V for both columns: each row of Bbar read once
                 const f32x2 w0 = pack2(g0 * v0[k], g0 * v0[k]), w1 = pack2(g1 * v1[k], g1 * v1[k]);
-                const f32x2 u0 = pack2(at0 * p0[k], at0 * p0[k]), u1 = pack2(at1 * p1[k], at1 * p1[k]);
 #pragma unroll
                 for (int q = 0; q < N / 4; ++q) {
                     const ulonglong2 b4 = *reinterpret_cast<const ulonglong2*>(sl.Bb + k * LD + 4 * q);
@@ -558,17 +552,13 @@ __global__ void __launch_bounds__(THREADS, 2) ttc_layer_kernel_c2(LayerParams p,
                     fma2(s20[2 * q + 1], w0, b4.y);
                     fma2(s21[2 * q], w1, b4.x);
                     fma2(s21[2 * q + 1], w1, b4.y);
-                    fma2(y20[2 * q], u0, b4.x);
-                    fma2(y20[2 * q + 1], u0, b4.y);
-                    fma2(y21[2 * q], u1, b4.x);
-                    fma2(y21[2 * q + 1], u1, b4.y);
                 }
             }
             float s0[N], s1[N], y0[N], y1[N], pn0[N], pn1[N];
             unpack_row<N>(s0, s20);
             unpack_row<N>(s1, s21);
-            unpack_row<N>(y0, y20);
-            unpack_row<N>(y1, y21);
+            load_row<N>(y0, sl.L + c0 * LD);                  // g_l (Bbar'P)[l][c0]
+            load_row<N>(y1, sl.L + c1 * LD);
             {
                 float gv[N], av[N], qv[N];
                 load_row<N>(gv, sl.gb);
@@ -578,8 +568,8 @@ __global__ void __launch_bounds__(THREADS, 2) ttc_layer_kernel_c2(LayerParams p,
                 for (int l = 0; l < N; ++l) {
                     s0[l] *= gv[l];
                     s1[l] *= gv[l];
-                    y0[l] *= gv[l];
-                    y1[l] *= gv[l];
+                    y0[l] *= at0;
+                    y1[l] *= at1;
                     pn0[l] = fmaf(qq0 * qv[l], q0[l], av[l] * at0 * p0[l]);
                     pn1[l] = fmaf(qq1 * qv[l], q1[l], av[l] * at1 * p1[l]);
                     if (l == c0)
