@@ -437,7 +437,8 @@ __device__ __forceinline__ void axpy_row2(rwarp::f32x2 (&acc0)[N / 2], rwarp::f3
     }
 }
 
-template <int N>
+// GRAD: as in ttc_layer_kernel (every K_s, every P_s with s >= 1 and k_0 = -S_0^{-1} g are kept).
+template <int N, bool GRAD = false>
 __global__ void __launch_bounds__(THREADS, 2) ttc_layer_kernel_c2(LayerParams p, int* chunk_counter)
 {
     using S = Shape2<N>;
@@ -621,7 +622,7 @@ __global__ void __launch_bounds__(THREADS, 2) ttc_layer_kernel_c2(LayerParams p,
                 unpack_row<N>(p0, p20);
                 unpack_row<N>(p1, p21);
             }
-            if (s == 0 && p.u1) {                             // K[:, c] = -L^{-T} Z[:, c]; rows of K -> Lt
+            if (GRAD || (s == 0 && p.u1)) {                   // K[:, c] = -L^{-T} Z[:, c]; rows of K -> Lt
 #pragma unroll
                 for (int k = N - 1; k >= 0; --k) {
                     const float x0 = y0[k] * rinv[k], x1 = y1[k] * rinv[k];
@@ -637,13 +638,51 @@ __global__ void __launch_bounds__(THREADS, 2) ttc_layer_kernel_c2(LayerParams p,
                         if (i4 + 3 < k) { y0[i4 + 3] = fmaf(-l4.w, x0, y0[i4 + 3]); y1[i4 + 3] = fmaf(-l4.w, x1, y1[i4 + 3]); }
                     }
                 }
+                if (GRAD) {
+                    if (active) {
+                        float* kt = p.Kws + (inst * (long long)T + s) * N * N + c0;
 #pragma unroll
-                for (int l = 0; l < N; ++l)
-                    *reinterpret_cast<float2*>(sl.Lt + l * LD + c0) = make_float2(-y0[l], -y1[l]);
+                        for (int l = 0; l < N; ++l)
+                            *reinterpret_cast<float2*>(kt + l * N) = make_float2(-y0[l], -y1[l]);
+                    }
+                    if (s == 0) {
+                        // k_0 = -L^{-T} L^{-1} g, two components per lane: the pivot's value travels by shuffle, a lane
+                        // reads its own rows of L and L'
+                        const float2 gg = __ldg(reinterpret_cast<const float2*>(p.g + inst * N + c0));
+                        float gz0 = gg.x, gz1 = gg.y;
+                        const float r0 = sl.rinv[c0], r1 = sl.rinv[c1];
+#pragma unroll 4
+                        for (int k = 0; k < N; ++k) {
+                            const float zk = __shfl_sync(0xffffffffu, (k & 1) ? gz1 * r1 : gz0 * r0, k >> 1, G);
+                            if (c0 > k) gz0 = fmaf(-sl.L[c0 * LD + k], zk, gz0); else if (c0 == k) gz0 = zk;
+                            if (c1 > k) gz1 = fmaf(-sl.L[c1 * LD + k], zk, gz1); else if (c1 == k) gz1 = zk;
+                        }
+#pragma unroll 4
+                        for (int k = N - 1; k >= 0; --k) {
+                            const float xk = __shfl_sync(0xffffffffu, (k & 1) ? gz1 * r1 : gz0 * r0, k >> 1, G);
+                            if (c0 < k) gz0 = fmaf(-sl.Lt[c0 * LD + k], xk, gz0); else if (c0 == k) gz0 = xk;
+                            if (c1 < k) gz1 = fmaf(-sl.Lt[c1 * LD + k], xk, gz1); else if (c1 == k) gz1 = xk;
+                        }
+                        if (active)
+                            *reinterpret_cast<float2*>(p.k0 + inst * N + c0) = make_float2(-gz0, -gz1);
+                        __syncwarp();                         // every lane is done with L' (the substitution of g)
+                    }
+                }
+                if (s == 0) {
+#pragma unroll
+                    for (int l = 0; l < N; ++l)
+                        *reinterpret_cast<float2*>(sl.Lt + l * LD + c0) = make_float2(-y0[l], -y1[l]);
+                }
             }
             __syncwarp();                                     // rows of Z consumed
             store_row<N>(sl.buf0 + c0 * LD, p0);              // rows of P_s (row c = column c)
             store_row<N>(sl.buf0 + c1 * LD, p1);
+            if (GRAD && s >= 1 && active) {
+                float* pt = p.Pws + (inst * (long long)T + s) * N * N + c0;
+#pragma unroll
+                for (int l = 0; l < N; ++l)
+                    *reinterpret_cast<float2*>(pt + l * N) = make_float2(p0[l], p1[l]);
+            }
         }
         __syncwarp();
 

@@ -925,10 +925,13 @@ int ttc_lqr_layer_grad(ttc_lqr_handle* h, const ttc_layer_inputs* in, int32_t T,
     int* counter = static_cast<int*>(h->ws_E.ptr);
     TTC_CUDA(cudaMemsetAsync(counter, 0, sizeof(int), st));
     {
-        void (*kern)(layer::LayerParams, int*) = n == 32 ? layer::ttc_layer_kernel<32, true> : layer::ttc_layer_kernel<16, true>;
-        const size_t smem = n == 32 ? layer::smem_bytes<32>() : layer::smem_bytes<16>();
-        const int slots = n == 32 ? rwarp::Shape<32>::SLOTS : rwarp::Shape<16>::SLOTS;
-        long long chunks = (p.N + slots - 1) / slots, grid = (long long)h->sm_count * (n == 32 ? 3 : 4);
+        // n = 16 with the machine at least half full: two columns per lane, as in the forward call
+        const bool c2 = n == 16 && p.N > (long long)h->sm_count * 2 * rwarp::Shape<16>::SLOTS;
+        void (*kern)(layer::LayerParams, int*) = n == 32 ? layer::ttc_layer_kernel<32, true>
+                                               : c2 ? layer::ttc_layer_kernel_c2<16, true> : layer::ttc_layer_kernel<16, true>;
+        const size_t smem = n == 32 ? layer::smem_bytes<32>() : c2 ? layer::smem_bytes_c2<16>() : layer::smem_bytes<16>();
+        const int slots = n == 32 ? rwarp::Shape<32>::SLOTS : c2 ? layer::Shape2<16>::SLOTS : rwarp::Shape<16>::SLOTS;
+        long long chunks = (p.N + slots - 1) / slots, grid = (long long)h->sm_count * (n == 32 ? 3 : c2 ? 2 : 4);
         if (grid > chunks) grid = chunks;
         TTC_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         kern<<<(unsigned)grid, rwarp::THREADS, smem, st>>>(p, counter);

@@ -58,6 +58,46 @@ def test_every_gradient_matches_the_oracle(key, batch, T):
     assert float((Qg - Qg.transpose(1, 2)).abs().max()) <= 1e-5 * float(Qg.abs().max())
 
 
+def test_two_column_backward_pass_at_a_batch_that_fills_the_machine():
+    """More than 2368 instances at n = 16: the backward pass runs with two columns per lane (the kernel the benchmark's
+    layer16 gradients use).  Sampled instances against the oracle; the basis gradients, which sum over every instance,
+    against a second call in which the same instances go through the one-column kernel in two halves."""
+    key, batch, T = "layer16", (1, 4, 640), 5
+    w = workloads.make_layer_workload(key, device=DEV, batch=batch, seed=77)
+    n, N = w["n"], w["N"]
+    gen = torch.Generator(device=DEV)
+    gen.manual_seed(99)
+    g = torch.randn((N, n), generator=gen, device=DEV)
+
+    def call(lo, hi):
+        s = lqr.LqrSolver(n, n, T, (1, 1, hi - lo))
+        grads = {k: torch.full_like(w[k] if k in ("B_basis", "Q_basis") else w[k][lo:hi], 777.0) for k in lqr.LAYER_GRAD_KEYS}
+        u1 = torch.full((hi - lo, n), 777.0, device=DEV)
+        info = torch.full((hi - lo,), -5, dtype=torch.int32, device=DEV)
+        ins = [w[k] if k in ("B_basis", "Q_basis") else w[k][lo:hi].contiguous() for k in workloads.LAYER_KEYS]
+        s.layer_grad(*ins, T, g[lo:hi].contiguous(), grads, u1=u1, info=info)
+        torch.cuda.synchronize()
+        s.close()
+        return grads, u1, info
+
+    full, u_full, info = call(0, N)
+    assert int(info.abs().max()) == 0
+    halves = [call(0, N // 2), call(N // 2, N)]
+    f64 = lambda t: t.to(torch.float64).cpu().numpy()
+    for i in range(0, N, 107):
+        ref = og.grad(*(f64(w[k][i]) for k in workloads.LAYER_KEYS[:9]), f64(w["B_basis"]), f64(w["Q_basis"]), T, f64(g[i]))
+        assert rel(u_full[i].cpu().numpy(), ref["u1"]) <= 1e-4
+        for k in PER_INSTANCE:
+            got = full[k][i].double().cpu().numpy()
+            assert np.abs(got - ref[k]).max() <= 1e-4 * max(np.abs(ref[k]).max(), 1e-7), (k, i)
+    for k in PER_INSTANCE:
+        both = torch.cat([halves[0][0][k], halves[1][0][k]])
+        assert float((full[k] - both).abs().max()) <= 1e-4 * float(both.abs().max()), k
+    for k in ("B_basis", "Q_basis"):
+        both = halves[0][0][k].double() + halves[1][0][k].double()
+        assert float((full[k].double() - both).abs().max()) <= 1e-4 * float(both.abs().max()), k
+
+
 def test_partial_requests_and_no_info():
     w, grads, u1, info, refs, launches = run_both("layer16", (1, 2, 6), 5, want=("s_a", "h0", "s_q"), with_info=False)
     assert launches == 2 and set(grads) == {"s_a", "h0", "s_q"}
