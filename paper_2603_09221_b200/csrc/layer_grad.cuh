@@ -88,7 +88,7 @@ __device__ __forceinline__ void load_vec_plain(float (&v)[N], const float* src)
 
 // the kernel body is in layer_grad_body.cuh
 template <int N>
-__global__ void __launch_bounds__(THREADS, 2) layer_grad_vectors_kernel(LayerGradParams q);
+__global__ void __launch_bounds__(THREADS, (N == 32) ? 2 : 4) layer_grad_vectors_kernel(LayerGradParams q);
 
 // dBasis[k][e] += sum over a slice of instances of coef[i][k] * G[i][e]; one CTA per slice, atomics at the end.
 // Up to two (coefficient, matrix) pairs go to the same destination (Q^(k) collects s_Q[k] dQbar and s_Qf[k] dQ_T).

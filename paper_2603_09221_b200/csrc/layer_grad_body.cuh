@@ -5,7 +5,7 @@ namespace ttc {
 namespace lgrad {
 
 template <int N>
-__global__ void __launch_bounds__(THREADS, 2) layer_grad_vectors_kernel(LayerGradParams q)
+__global__ void __launch_bounds__(THREADS, (N == 32) ? 2 : 4) layer_grad_vectors_kernel(LayerGradParams q)
 {
     using S = Shape<N>;
     constexpr int LD = S::LD;
