@@ -178,6 +178,22 @@ def test_full_size_configuration_on_sampled_instances(cfg, expect):
     torch.cuda.empty_cache()
 
 
+@pytest.mark.parametrize("first", [False, True])
+def test_tensor_core_kernel_on_float32_inputs_when_asked_for(first):
+    """float32 Q and x0 at n = m = 64 go to the generic kernel by default; with TTC_MATH_TF32 the tensor-core kernel takes
+    them (the rows of Q are then read as float32).  Checked at the tf32 bounds of the bfloat16 configurations."""
+    w = small_workload(64, 64, 6, (1, 2, 21), seed=640, bf16=False)
+    N = 42
+    want = ("P", "u", "info") if first else ("K", "P", "x", "u", "info")
+    g = pu.run_gpu(w, want=want, first_only=first, math=lqr.TTC_MATH_TF32)
+    assert lqr.KERNEL_NAMES[g["kernel"]] == "riccati_umma"
+    ref = pu.run_oracle(w, first_only=first)
+    names = want[:-1]
+    pu.compare(g, ref, np.arange(N), 5e-3, names=names, xu_floor=1.0)
+    pu.compare(g, ref, np.arange(N), 2e-2, names=names)
+    assert int(g["info"].abs().max()) == 0
+
+
 def test_invalid_arguments_are_rejected():
     w = small_workload(8, 8, 4, (1, 1, 4), seed=3)
     with pytest.raises(lqr.TtcError):
