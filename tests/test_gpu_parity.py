@@ -292,6 +292,28 @@ def test_q_strides_that_break_16_byte_rows_go_to_the_generic_kernel(n, bf16, pad
     pu.compare(gpu, ref, np.arange(N), w["tol"])
 
 
+def test_host_buffer_entry_point_slices_sized_to_the_grid():
+    """A request that moves few bytes per instance and step (P_0, u_0 only) with many heads: the host-buffer entry point
+    sizes its slices to whole rounds of the persistent grid and starts and ends with a short slice; the results must
+    still equal the device entry point's bit for bit, every element written."""
+    n, H, batch = 64, 8, (1, 32, 1024)
+    w = small_workload(n, n, H, batch, seed=808, bf16=True)
+    N = int(np.prod(batch))
+    gpu = pu.run_gpu(w, want=("P", "u", "info"), first_only=True)
+    s = lqr.LqrSolver(n, n, H, batch)
+    host = {k: w[k].cpu().pin_memory() for k in ("A", "B", "Q", "R", "x0")}
+    out = lqr.alloc_outputs(n, n, H, N, "cpu", first_only=True, want=("P", "u", "info"), pin=True)
+    for k, v in out.items():
+        v.fill_(-7 if k == "info" else 12345.0)
+    s.solve_host(host["A"], host["B"], host["Q"], host["R"], host["x0"], H, P=out["P"], u=out["u"], info=out["info"],
+                 flags=lqr.TTC_OUT_FIRST_ONLY)
+    launches = s.query(lqr.TTC_QUERY_LAST_LAUNCHES)
+    s.close()
+    assert 3 < launches < 32, launches                     # neither one launch nor the 128-token default
+    for k in ("P", "u", "info"):
+        assert torch.equal(out[k], gpu[k].cpu()), k
+
+
 def test_host_buffer_entry_point_slices_with_a_single_sequence_and_head():
     """One (sequence, head) row and enough bytes for the sliced pipeline: the copies are plain one-row copies (a 2D copy
     would need a pitch beyond the device limit on larger problems of this shape); bit-equal to the device entry."""
