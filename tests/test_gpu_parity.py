@@ -178,6 +178,23 @@ def test_full_size_configuration_on_sampled_instances(cfg, expect):
     torch.cuda.empty_cache()
 
 
+def test_first_control_request_on_a_batch_that_fills_the_machine():
+    """ttc_lqr_solve at n = 16 with P_0 and u_0 only on 5200 instances (several work items per CTA, ragged last item
+    per head): every instance against the oracle, and a failed instance (indefinite Q) gets NaN and its pivot code."""
+    w = small_workload(16, 16, 9, (1, 8, 650), seed=1616)
+    N = 5200
+    w["Q"] = w["Q"].clone()
+    w["Q"][0, 3, 17] = -50.0 * torch.eye(16, device=DEV)
+    g = pu.run_gpu(w, want=("P", "u", "info"), first_only=True)
+    assert lqr.KERNEL_NAMES[g["kernel"]] == "riccati_warp"
+    bad = 3 * 650 + 17
+    assert int(g["info"][bad]) > 0 and torch.isnan(g["P"][bad]).all() and torch.isnan(g["u"][bad]).all()
+    ok = np.array([i for i in range(N) if i != bad])
+    assert int(g["info"][torch.from_numpy(ok).to(DEV)].abs().max()) == 0
+    ref = pu.run_oracle(w, idx=ok, first_only=True)
+    pu.compare(g, ref, ok, 1e-4, names=("P", "u"))
+
+
 @pytest.mark.parametrize("first", [False, True])
 def test_tensor_core_kernel_on_float32_inputs_when_asked_for(first):
     """float32 Q and x0 at n = m = 64 go to the generic kernel by default; with TTC_MATH_TF32 the tensor-core kernel takes

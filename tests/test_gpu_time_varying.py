@@ -136,3 +136,20 @@ def test_ttc_layer_shaped_workload_full_size_on_sampled_instances():
     # symmetry of P_0 holds at any size
     P = out["P"][:: 97]
     assert float((P - P.transpose(-1, -2)).abs().max() / P.abs().max()) < 1e-5
+
+
+@pytest.mark.parametrize("tv,first_only,want,bf16", [(("A", "B", "Q", "R"), True, ("P", "u", "info"), False),
+                                                     ((), True, ("P", "u", "info"), True),
+                                                     (("Q",), False, ("P", "info"), False)])
+def test_value_matrix_and_first_control_on_batches_that_fill_the_machine(tv, first_only, want, bf16):
+    """n = 16, 5600 instances, P and the first control only (the shape of request the time-varying benchmark workload
+    makes): several work items per CTA, 700 tokens per head leave the last work item of every head ragged.  Every
+    instance against the oracle."""
+    w = tv_workload(16, 16, 7, (2, 4, 700), seed=1600 + len(tv), tv=tv, bf16=bf16)
+    out, ref = run_both(w, want=want, first_only=first_only)
+    assert lqr.KERNEL_NAMES[out["kernel"]] == "riccati_warp"
+    names = tuple(k for k in want if k != "info")
+    pu.compare(out, ref, np.arange(5600), 2e-2 if bf16 else 1e-4, names=names)
+    for k in names:
+        assert not torch.any(out[k] == 123456.0), "canary left in %s" % k
+    assert int(out["info"].abs().max()) == 0
