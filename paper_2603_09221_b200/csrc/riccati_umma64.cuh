@@ -369,7 +369,7 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
     unsigned char* BA = smem_raw;              // rows 0..63: B' (row j = column j of B), rows 64..127: A'; shared by the CTA
     float* Rs = reinterpret_cast<float*>(smem_raw + BUF_BYTES);   // R of the head, fp32, shared by the CTA
     unsigned char* wsm = smem_raw + BUF_BYTES + R_BYTES + (size_t)wg * WG_BYTES;
-    unsigned char* X1 = wsm + OFF_X1;        // L, fp32 (kept only when the gains or u_0 need it)
+    unsigned char* X1 = wsm + OFF_X1;        // L in fp32 for u_0 at the last step; scratch of the mirror and of the symmetrisation
     unsigned char* X0 = wsm + OFF_X0;        // P -> Z' -> next P
     unsigned char* PH = wsm + OFF_PH;        // panel operand, hi parts (128 x 8)
     unsigned char* PL = wsm + OFF_PL;        // panel operand, lo parts
@@ -842,7 +842,7 @@ __global__ void __launch_bounds__(THREADS, 1) riccati_umma64_kernel(SolveParams 
                     // Every eighth step the operand is replaced by (P + P') / 2.  Q and Z'Z are symmetric but the rounding
                     // of A'(P A) is not, and the antisymmetric part E obeys E <- A'E A: along an open-loop unstable A it
                     // grows however well the closed loop is damped, until S stops being positive definite.  Eight steps
-                    // of growth are harmless (the exchange costs about a sixth of a step).  X1 (Z', consumed by (5)) is free and takes the averaged rows.
+                    // of growth are harmless (the exchange costs about a sixth of a step).  X1 is free here and takes the averaged rows.
                     if (ts > 0 && (ts & 7) == 0) {
                         half_barrier(wg);                     // both halves of every row are in X0
 #pragma unroll 8
